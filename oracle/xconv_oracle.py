@@ -1,0 +1,244 @@
+"""Float64 CPU oracle for the XConv layer (test infrastructure, not product code).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may use this
+module.  It shares no code with the CUDA path and imports nothing from it.
+
+Everything is plain numpy in float64 on logical (batch, channel, y, x) arrays.
+Where a step is a dense contraction, ``numpy.matmul`` / ``numpy.einsum`` serves as
+that step; there is no blocking, fusion or reordering beyond what the formulas
+state.
+
+Notation (Section 3, "Single channel case" and "Multi-channel case"):
+  B batch, Cin/Cout channels, N = H*W pixels, r probing vectors,
+  X  [B, Cin, H, W]     layer input
+  dY [B, Cout, H, W]    back-propagated residual (delta Y)
+  W  [Cout, Cin, KH, KW] weights; the i-th weight has offset k(i) = (ky-ph, kx-pw)
+  Z  [r, Cin, H, W]     probing vectors (column j of the paper's Z, reshaped)
+  S  [r, B]             the sketch, the paper's X-bar = Z^T X   (text after Eq. 4, Algorithm 1 forward step 3)
+  L  [r, Cout, H, W]    backward probe L = X-bar dY^T           (Algorithm 1 backward step 3)
+
+Shift operator.  The paper's T_k is a circular shift; every layer this library is
+used on is a zero-padded convolution, for which the matching operator is the
+truncating shift (out-of-range pixels read as zero).  ``circular=True`` selects the
+paper's literal operator and is used as a second self-check.  In both cases
+  (shift(A, dy, dx))[..., y, x] = A[..., y+dy, x+dx].
+
+Direction of the shift in the gradient.  From Y = sum_i w_i T_k(i) X with
+(T_k X)[q] = X[q + k], the exact weight gradient is
+  dw_i = sum_{b,q} dY[q, b] X[q + k(i), b] = tr(X dY^T S_k),  (S_k z)[q] = z[q + k],
+so the paper's T_{-k(i)} in Eq. (2) acts on a probing vector as z -> z[. + k(i)]:
+output pixel q pairs with the probe value at input pixel q + k(i).
+
+Pinned by tests/test_oracle_pins.py: brute-force loops and finite differences
+(conv_forward, dw_exact, dx_exact), exact recovery with an orthogonal probe basis,
+unbiasedness, the closed-form Hutchinson variance, Proposition 1's bound and the
+literal block-matrix estimator of Eq. (6) (sketch, backprobe, wgrad_estimate).
+No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _pads(KH, KW, pad):
+    if pad is None:
+        return (KH - 1) // 2, (KW - 1) // 2
+    return pad
+
+
+def shift(A: np.ndarray, dy: int, dx: int, circular: bool = False) -> np.ndarray:
+    """(shift A)[..., y, x] = A[..., y+dy, x+dx]; zero outside the image unless ``circular``.
+
+    Section 3, text after Eq. (1): the i-th weight applies a shift with offset k(i).
+    """
+    A = np.asarray(A, dtype=F64)
+    if circular:
+        return np.roll(A, shift=(-dy, -dx), axis=(-2, -1))
+    H, W = A.shape[-2], A.shape[-1]
+    out = np.zeros_like(A)
+    y0, y1 = max(0, -dy), min(H, H - dy)
+    x0, x1 = max(0, -dx), min(W, W - dx)
+    if y0 < y1 and x0 < x1:
+        out[..., y0:y1, x0:x1] = A[..., y0 + dy:y1 + dy, x0 + dx:x1 + dx]
+    return out
+
+
+def conv_forward(X, W, pad=None, circular=False):
+    """Y^m = sum_n W^{n,m} X^n with W^{n,m} = sum_i w_i^{n,m} T_k(i)   (Eq. 5; Algorithm 1 forward step 1).
+
+    Y[b,m,y,x] = sum_{n,ky,kx} W[m,n,ky,kx] X[b,n,y+ky-ph,x+kx-pw]  (cross-correlation, stride 1).
+    """
+    X = np.asarray(X, F64)
+    W = np.asarray(W, F64)
+    Cout, Cin, KH, KW = W.shape
+    ph, pw = _pads(KH, KW, pad)
+    Y = np.zeros((X.shape[0], Cout) + X.shape[2:], F64)
+    for ky in range(KH):
+        for kx in range(KW):
+            Xs = shift(X, ky - ph, kx - pw, circular)
+            Y += np.einsum("mn,bnyx->bmyx", W[:, :, ky, kx], Xs)
+    return Y
+
+
+def dw_exact(X, dY, KH=3, KW=3, pad=None, circular=False):
+    """Exact weight gradient dw_i^{n,m} = tr(X^n (dY^m)^T T_{-k(i)})   (Eq. 2 and the sentence after Eq. 5).
+
+    dW[m,n,ky,kx] = sum_{b,y,x} dY[b,m,y,x] X[b,n,y+ky-ph,x+kx-pw].
+    """
+    X = np.asarray(X, F64)
+    dY = np.asarray(dY, F64)
+    ph, pw = _pads(KH, KW, pad)
+    dW = np.zeros((dY.shape[1], X.shape[1], KH, KW), F64)
+    for ky in range(KH):
+        for kx in range(KW):
+            Xs = shift(X, ky - ph, kx - pw, circular)
+            dW[:, :, ky, kx] = np.einsum("bmyx,bnyx->mn", dY, Xs)
+    return dW
+
+
+def dx_exact(dY, W, pad=None, circular=False):
+    """Exact input gradient: the adjoint of ``conv_forward`` in X (standard back-propagation,
+    which the method leaves untouched -- abstract and Section 1).
+
+    dX[b,n,u,v] = sum_{m,ky,kx} W[m,n,ky,kx] dY[b,m,u-ky+ph,v-kx+pw].
+    """
+    dY = np.asarray(dY, F64)
+    W = np.asarray(W, F64)
+    Cout, Cin, KH, KW = W.shape
+    ph, pw = _pads(KH, KW, pad)
+    dX = np.zeros((dY.shape[0], Cin) + dY.shape[2:], F64)
+    for ky in range(KH):
+        for kx in range(KW):
+            dYs = shift(dY, -(ky - ph), -(kx - pw), circular)
+            dX += np.einsum("mn,bmyx->bnyx", W[:, :, ky, kx], dYs)
+    return dX
+
+
+def sketch(X, Z):
+    """X-bar = Z^T X in R^{r x B}: step (i) of the three-step procedure after Eq. (6);
+    Algorithm 1 forward step 3.   S[j,b] = sum_{n,y,x} Z[j,n,y,x] X[b,n,y,x]."""
+    X = np.asarray(X, F64)
+    Z = np.asarray(Z, F64)
+    return Z.reshape(Z.shape[0], -1) @ X.reshape(X.shape[0], -1).T
+
+
+def backprobe(S, dY):
+    """L = X-bar dY^T (Algorithm 1 backward step 3), reshaped per output channel (step ii).
+
+    L[j,m,y,x] = sum_b S[j,b] dY[b,m,y,x]."""
+    S = np.asarray(S, F64)
+    dY = np.asarray(dY, F64)
+    L = S @ dY.reshape(dY.shape[0], -1)
+    return L.reshape((S.shape[0],) + dY.shape[1:])
+
+
+def channel_scale(Z):
+    """Scale of the estimator per input channel: 1/nnz(Z_n), nnz = number of probing vectors
+    whose block n is not identically zero (Eq. 8).  For dense probes this is 1/r (Eq. 6).
+    A channel with no non-zero block gets scale 0 (its estimate is then 0)."""
+    Z = np.asarray(Z, F64)
+    nnz = np.count_nonzero(np.any(Z.reshape(Z.shape[0], Z.shape[1], -1) != 0, axis=2), axis=0)
+    return np.where(nnz > 0, 1.0 / np.maximum(nnz, 1), 0.0)
+
+
+def wgrad_contract(L, Z, KH=3, KW=3, pad=None, circular=False, scale=None):
+    """Step (iii): probe each block from the left, dw_i = (1/r) tr(L T_{-k(i)} Z)
+    (Eq. 6 block by block; Algorithm 1 backward step 4).
+
+    dW[m,n,ky,kx] = scale[n] * sum_{j,y,x} L[j,m,y,x] Z[j,n,y+ky-ph,x+kx-pw],
+    scale = 1/r unless given (Eq. 8 uses 1/nnz(Z_n))."""
+    L = np.asarray(L, F64)
+    Z = np.asarray(Z, F64)
+    r = Z.shape[0]
+    ph, pw = _pads(KH, KW, pad)
+    if scale is None:
+        scale = np.full(Z.shape[1], 1.0 / r)
+    dW = np.zeros((L.shape[1], Z.shape[1], KH, KW), F64)
+    for ky in range(KH):
+        for kx in range(KW):
+            Zs = shift(Z, ky - ph, kx - pw, circular)
+            dW[:, :, ky, kx] = np.einsum("jmyx,jnyx->mn", L, Zs) * scale[None, :]
+    return dW
+
+
+def wgrad_estimate(S, dY, Z, KH=3, KW=3, pad=None, circular=False, scale=None):
+    """Algorithm 1 backward steps 3-4 in the paper's order: L first, then the offset traces."""
+    return wgrad_contract(backprobe(S, dY), Z, KH, KW, pad, circular, scale)
+
+
+def xconv_layer(X, W, dY, Z, pad=None, circular=False, scale=None):
+    """Algorithm 1 end to end for one layer: returns Y, the sketch, the dW estimate and exact dX."""
+    KH, KW = W.shape[2], W.shape[3]
+    Y = conv_forward(X, W, pad, circular)
+    S = sketch(X, Z)
+    dW = wgrad_estimate(S, dY, Z, KH, KW, pad, circular, scale)
+    dX = dx_exact(dY, W, pad, circular)
+    return Y, S, dW, dX
+
+
+# --- the literal block-matrix form of Eq. (6), for tiny layers only ---------------------------
+
+def shift_matrix(H, W, dy, dx, circular=False):
+    """Dense N x N matrix S_k with (S_k z)[q] = z[q + k], q = y*W + x, built entry by entry."""
+    N = H * W
+    M = np.zeros((N, N), F64)
+    for y in range(H):
+        for x in range(W):
+            yy, xx = y + dy, x + dx
+            if circular:
+                yy %= H
+                xx %= W
+            elif not (0 <= yy < H and 0 <= xx < W):
+                continue
+            M[y * W + x, yy * W + xx] = 1.0
+    return M
+
+
+def wgrad_estimate_literal(X, dY, Z, KH=3, KW=3, pad=None, circular=False):
+    """Eq. (6) as printed: form every block A^{m,n} = (X^n (dY^m)^T T_{-k(i)})^T, stack them into A,
+    probe A from the right with the r columns of Z and each block row from the left.
+    G^{m,n} = (1/r) sum_j z_{n,j}^T (A z_j)_m.  O(N^2) memory: tiny inputs only."""
+    X = np.asarray(X, F64)
+    dY = np.asarray(dY, F64)
+    Z = np.asarray(Z, F64)
+    B, Cin, H, W = X.shape
+    Cout = dY.shape[1]
+    r = Z.shape[0]
+    N = H * W
+    ph, pw = _pads(KH, KW, pad)
+    Xm = X.reshape(B, Cin, N)
+    dYm = dY.reshape(B, Cout, N)
+    Zc = Z.reshape(r, Cin * N).T          # the paper's Z in R^{N Cin x r}
+    dW = np.zeros((Cout, Cin, KH, KW), F64)
+    for ky in range(KH):
+        for kx in range(KW):
+            Tk = shift_matrix(H, W, ky - ph, kx - pw, circular)
+            A = np.zeros((Cout * N, Cin * N), F64)
+            for m in range(Cout):
+                for n in range(Cin):
+                    outer = Xm[:, n, :].T @ dYm[:, m, :]          # X^n (dY^m)^T, N x N
+                    A[m * N:(m + 1) * N, n * N:(n + 1) * N] = (outer @ Tk).T
+            AZ = A @ Zc                                            # (i) probe from the right
+            for m in range(Cout):
+                for n in range(Cin):
+                    acc = 0.0
+                    for j in range(r):
+                        acc += Zc[n * N:(n + 1) * N, j] @ AZ[m * N:(m + 1) * N, j]   # (iii)
+                    dW[m, n, ky, kx] = acc / r
+    return dW
+
+
+def memory_factor(Cin, H, W, r):
+    """Stored elements, exact (X) over sketched (X-bar), per sample: N*Cin / r (Section 3 and 4.1)."""
+    return (H * W * Cin) / r
+
+
+def rel_fro(a, b):
+    """||a - b||_F / ||b||_F."""
+    a = np.asarray(a, F64)
+    b = np.asarray(b, F64)
+    d = np.linalg.norm((a - b).ravel())
+    n = np.linalg.norm(b.ravel())
+    return d / n if n > 0 else d

@@ -1,0 +1,374 @@
+"""Pins for the float64 oracle: each check ties it to something other than itself --
+brute-force loops, closed forms, invariants, special cases that reduce to a plain
+matrix product, values and bounds the paper prints.  CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import xconv_oracle as O
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def _tiny(seed=0, B=2, Cin=3, Cout=2, H=5, W=4, KH=3, KW=3):
+    g = _rng(seed)
+    X = g.standard_normal((B, Cin, H, W))
+    Wt = g.standard_normal((Cout, Cin, KH, KW))
+    dY = g.standard_normal((B, Cout, H, W))
+    return X, Wt, dY
+
+
+# ---------------------------------------------------------------- P1: brute force (Eq. 1, 2, 5)
+
+def _loops_conv(X, Wt, circular):
+    B, Cin, H, W = X.shape
+    Cout, _, KH, KW = Wt.shape
+    ph, pw = (KH - 1) // 2, (KW - 1) // 2
+    Y = np.zeros((B, Cout, H, W))
+    for b in range(B):
+        for m in range(Cout):
+            for y in range(H):
+                for x in range(W):
+                    acc = 0.0
+                    for n in range(Cin):
+                        for ky in range(KH):
+                            for kx in range(KW):
+                                yy, xx = y + ky - ph, x + kx - pw
+                                if circular:
+                                    yy, xx = yy % H, xx % W
+                                elif not (0 <= yy < H and 0 <= xx < W):
+                                    continue
+                                acc += Wt[m, n, ky, kx] * X[b, n, yy, xx]
+                    Y[b, m, y, x] = acc
+    return Y
+
+
+def _loops_dw(X, dY, KH, KW, circular):
+    B, Cin, H, W = X.shape
+    Cout = dY.shape[1]
+    ph, pw = (KH - 1) // 2, (KW - 1) // 2
+    dW = np.zeros((Cout, Cin, KH, KW))
+    for m in range(Cout):
+        for n in range(Cin):
+            for ky in range(KH):
+                for kx in range(KW):
+                    acc = 0.0
+                    for b in range(B):
+                        for y in range(H):
+                            for x in range(W):
+                                yy, xx = y + ky - ph, x + kx - pw
+                                if circular:
+                                    yy, xx = yy % H, xx % W
+                                elif not (0 <= yy < H and 0 <= xx < W):
+                                    continue
+                                acc += dY[b, m, y, x] * X[b, n, yy, xx]
+                    dW[m, n, ky, kx] = acc
+    return dW
+
+
+def _loops_dx(dY, Wt, circular):
+    B, Cout, H, W = dY.shape
+    _, Cin, KH, KW = Wt.shape
+    ph, pw = (KH - 1) // 2, (KW - 1) // 2
+    dX = np.zeros((B, Cin, H, W))
+    # scatter form: every term W*dY of the forward sum sends its gradient to the pixel it read
+    for b in range(B):
+        for m in range(Cout):
+            for y in range(H):
+                for x in range(W):
+                    for n in range(Cin):
+                        for ky in range(KH):
+                            for kx in range(KW):
+                                yy, xx = y + ky - ph, x + kx - pw
+                                if circular:
+                                    yy, xx = yy % H, xx % W
+                                elif not (0 <= yy < H and 0 <= xx < W):
+                                    continue
+                                dX[b, n, yy, xx] += Wt[m, n, ky, kx] * dY[b, m, y, x]
+    return dX
+
+
+@pytest.mark.parametrize("circular", [False, True])
+@pytest.mark.parametrize("K", [1, 3, 5])
+def test_p1_brute_force_loops(circular, K):
+    X, Wt, dY = _tiny(seed=K, H=5, W=6 if K == 5 else 4, KH=K, KW=K)
+    np.testing.assert_allclose(O.conv_forward(X, Wt, circular=circular), _loops_conv(X, Wt, circular), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O.dw_exact(X, dY, K, K, circular=circular), _loops_dw(X, dY, K, K, circular), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(O.dx_exact(dY, Wt, circular=circular), _loops_dx(dY, Wt, circular), rtol=0, atol=1e-12)
+
+
+def test_p1_gradients_by_finite_difference():
+    """f(W, X) = <conv(X, W), G> is bilinear, so one-sided differences are exact up to rounding."""
+    X, Wt, G = _tiny(seed=11)
+    f0 = np.sum(O.conv_forward(X, Wt) * G)
+    dW = O.dw_exact(X, G)
+    dX = O.dx_exact(G, Wt)
+    g = _rng(5)
+    for _ in range(12):
+        idx = tuple(g.integers(0, s) for s in Wt.shape)
+        Wp = Wt.copy(); Wp[idx] += 1.0
+        assert abs((np.sum(O.conv_forward(X, Wp) * G) - f0) - dW[idx]) < 1e-10
+        idx = tuple(g.integers(0, s) for s in X.shape)
+        Xp = X.copy(); Xp[idx] += 1.0
+        assert abs((np.sum(O.conv_forward(Xp, Wt) * G) - f0) - dX[idx]) < 1e-10
+
+
+def test_conv_is_cross_correlation_of_a_unit_impulse():
+    """A unit impulse in X reproduces the flipped kernel around it: fixes the sign of k(i)."""
+    H = W = 5
+    X = np.zeros((1, 1, H, W)); X[0, 0, 2, 2] = 1.0
+    Wt = np.arange(9, dtype=float).reshape(1, 1, 3, 3)
+    Y = O.conv_forward(X, Wt)
+    # Y[y,x] = W[ky,kx] with y+ky-1 = 2, x+kx-1 = 2
+    for ky in range(3):
+        for kx in range(3):
+            assert Y[0, 0, 3 - ky, 3 - kx] == Wt[0, 0, ky, kx]
+
+
+# ---------------------------------------------------------------- P2: exact recovery
+
+def _orth_probes(Cin, H, W, seed):
+    D = Cin * H * W
+    Q, _ = np.linalg.qr(_rng(seed).standard_normal((D, D)))
+    return (math.sqrt(D) * Q).reshape(D, Cin, H, W)      # rows j: Z2d^T Z2d = D * I
+
+
+@pytest.mark.parametrize("circular", [False, True])
+def test_p2_exact_recovery_with_orthogonal_basis(circular):
+    """With r = Cin*N probes and (1/r) Z Z^T = I the estimator is the exact gradient
+    ("recovers the exact gradient in the limit", Section 2)."""
+    X, Wt, dY = _tiny(seed=3, B=3, Cin=2, Cout=3, H=4, W=3)
+    Z = _orth_probes(2, 4, 3, seed=9)
+    S = O.sketch(X, Z)
+    est = O.wgrad_estimate(S, dY, Z, circular=circular)
+    np.testing.assert_allclose(est, _loops_dw(X, dY, 3, 3, circular), rtol=0, atol=1e-11)
+
+
+def test_p2_exact_recovery_with_hadamard_rademacher_basis():
+    from scipy.linalg import hadamard
+    Cin, H, W = 2, 4, 4                      # Cin*N = 32, a power of two
+    X, Wt, dY = _tiny(seed=4, B=3, Cin=Cin, Cout=2, H=H, W=W)
+    Z = hadamard(Cin * H * W).astype(float).reshape(-1, Cin, H, W)   # +-1 entries, Z^T Z = r I
+    est = O.wgrad_estimate(O.sketch(X, Z), dY, Z)
+    np.testing.assert_allclose(est, _loops_dw(X, dY, 3, 3, False), rtol=0, atol=1e-11)
+
+
+def test_p2_wrong_shift_sign_would_fail():
+    """The exact gradient is not symmetric under k -> -k on generic data, so P2 pins the direction."""
+    X, Wt, dY = _tiny(seed=3, B=3, Cin=2, Cout=3, H=4, W=3)
+    dW = _loops_dw(X, dY, 3, 3, False)
+    assert O.rel_fro(dW[:, :, ::-1, ::-1], dW) > 0.5
+
+
+# ---------------------------------------------------------------- literal Eq. (6) vs the three steps
+
+@pytest.mark.parametrize("circular", [False, True])
+def test_three_steps_equal_literal_block_estimator(circular):
+    X, Wt, dY = _tiny(seed=6, B=2, Cin=2, Cout=2, H=3, W=4)
+    Z = _rng(7).standard_normal((5, 2, 3, 4))
+    lit = O.wgrad_estimate_literal(X, dY, Z, circular=circular)
+    est = O.wgrad_estimate(O.sketch(X, Z), dY, Z, circular=circular)
+    np.testing.assert_allclose(est, lit, rtol=0, atol=1e-11)
+
+
+def test_shift_matrix_is_the_shift():
+    g = _rng(2)
+    A = g.standard_normal((4, 5))
+    for dy in (-1, 0, 1):
+        for dx in (-2, 0, 1):
+            for circ in (False, True):
+                M = O.shift_matrix(4, 5, dy, dx, circ)
+                np.testing.assert_array_equal((M @ A.ravel()).reshape(4, 5), O.shift(A, dy, dx, circ))
+    # circular shifts are permutations (the paper's T_k), truncating ones are not
+    assert np.allclose(O.shift_matrix(4, 5, 1, -1, True).sum(0), 1)
+    assert O.shift_matrix(4, 5, 1, -1, False).sum() < 20
+
+
+# ---------------------------------------------------------------- P8: special cases
+
+def test_p8_single_channel_reduces_to_eq4():
+    """Cin = Cout = 1: dw_i ~ (1/r) sum_j (z_j^T X)(dY^T T_{-k(i)} z_j)   (Eq. 4)."""
+    H, W, B, r = 4, 5, 3, 6
+    g = _rng(8)
+    X = g.standard_normal((B, 1, H, W)); dY = g.standard_normal((B, 1, H, W))
+    Z = g.standard_normal((r, 1, H, W))
+    est = O.wgrad_estimate(O.sketch(X, Z), dY, Z)
+    Xm = X.reshape(B, -1).T; dYm = dY.reshape(B, -1).T; Zm = Z.reshape(r, -1).T   # N x B, N x B, N x r
+    for ky in range(3):
+        for kx in range(3):
+            Tk = O.shift_matrix(H, W, ky - 1, kx - 1)
+            ref = sum((Zm[:, j] @ Xm) @ (dYm.T @ Tk @ Zm[:, j]) for j in range(r)) / r
+            assert abs(est[0, 0, ky, kx] - ref) < 1e-11
+
+
+def test_p8_pointwise_kernel_is_a_plain_matmul():
+    """K = 1: dW = (1/r) L_flat Z_flat^T with L_flat [Cout, r*N], Z_flat [Cin, r*N]."""
+    g = _rng(10)
+    B, Cin, Cout, H, W, r = 3, 4, 5, 3, 3, 7
+    X = g.standard_normal((B, Cin, H, W)); dY = g.standard_normal((B, Cout, H, W))
+    Z = g.standard_normal((r, Cin, H, W))
+    S = Z.reshape(r, -1) @ X.reshape(B, -1).T
+    L = (S @ dY.reshape(B, -1)).reshape(r, Cout, H * W)
+    ref = L.transpose(1, 0, 2).reshape(Cout, -1) @ Z.reshape(r, Cin, -1).transpose(1, 0, 2).reshape(Cin, -1).T / r
+    est = O.wgrad_estimate(O.sketch(X, Z), dY, Z, KH=1, KW=1)
+    np.testing.assert_allclose(est[:, :, 0, 0], ref, rtol=0, atol=1e-11)
+
+
+def test_estimator_is_exact_wgrad_of_the_reconstructed_activation():
+    """Bilinearity: contracting L with Z equals the exact gradient with X replaced by (1/r) Z Z^T X."""
+    X, Wt, dY = _tiny(seed=12, B=3, Cin=2, Cout=2, H=4, W=4)
+    Z = _rng(13).standard_normal((6, 2, 4, 4))
+    S = O.sketch(X, Z)
+    Xrec = np.einsum("jb,jnyx->bnyx", S, Z) / 6
+    np.testing.assert_allclose(O.wgrad_estimate(S, dY, Z), _loops_dw(Xrec, dY, 3, 3, False), rtol=0, atol=1e-11)
+
+
+# ---------------------------------------------------------------- P3/P4: unbiasedness and closed-form variance
+
+def _C_blocks(X, dY, m, ky, kx):
+    """C_n'[p, q'] = sum_b X[b,n',p] dY[b,m,q'-k]; the estimate of dW[m,n,k] with one probe is
+    sum_n' z_n'^T C_n' z_n."""
+    B, Cin, H, W = X.shape
+    N = H * W
+    C = np.zeros((Cin, N, N))
+    for n in range(Cin):
+        for y in range(H):
+            for x in range(W):
+                yq, xq = y - (ky - 1), x - (kx - 1)     # q = q' - k
+                if 0 <= yq < H and 0 <= xq < W:
+                    for b in range(B):
+                        C[n, :, y * W + x] += X[b, n].ravel() * dY[b, m, yq, xq]
+    return C
+
+
+def _closed_form_variance(C, n, rademacher):
+    v = np.sum(C[n] ** 2) + np.trace(C[n] @ C[n])
+    if rademacher:
+        v -= 2.0 * np.sum(np.diag(C[n]) ** 2)
+    for k in range(C.shape[0]):
+        if k != n:
+            v += np.sum(C[k] ** 2)
+    return v
+
+
+@pytest.mark.parametrize("kind", ["gaussian", "rademacher"])
+def test_p3_p4_unbiased_with_hutchinson_variance(kind):
+    """Mean over independent probes tends to the exact gradient (Appendix, proof of Theorem 1, first part);
+    the per-probe variance is the textbook Hutchinson expression plus the cross-channel terms."""
+    X, Wt, dY = _tiny(seed=20, B=3, Cin=2, Cout=2, H=4, W=4)
+    exact = _loops_dw(X, dY, 3, 3, False)
+    T = 6000
+    g = _rng(21)
+    if kind == "gaussian":
+        Zall = g.standard_normal((T, 2, 4, 4))
+    else:
+        Zall = g.integers(0, 2, size=(T, 2, 4, 4)).astype(float) * 2 - 1
+    ests = np.stack([O.wgrad_estimate(O.sketch(X, Zall[t:t + 1]), dY, Zall[t:t + 1]) for t in range(T)])
+    mean, var = ests.mean(0), ests.var(0, ddof=1)
+    for m in range(2):
+        for ky in range(3):
+            for kx in range(3):
+                C = _C_blocks(X, dY, m, ky, kx)
+                for n in range(2):
+                    assert abs(np.trace(C[n]) - exact[m, n, ky, kx]) < 1e-10
+                    v = _closed_form_variance(C, n, kind == "rademacher")
+                    z = (mean[m, n, ky, kx] - exact[m, n, ky, kx]) / math.sqrt(v / T)
+                    assert abs(z) < 4.5, (m, n, ky, kx, z)
+                    assert 0.8 < var[m, n, ky, kx] / v < 1.25, (m, n, ky, kx, var[m, n, ky, kx], v)
+    # one r-probe estimate is the average of r one-probe estimates (scale 1/r)
+    r = 8
+    np.testing.assert_allclose(O.wgrad_estimate(O.sketch(X, Zall[:r]), dY, Zall[:r]), ests[:r].mean(0), atol=1e-11)
+
+
+def test_p3_block_sparse_probes_with_nnz_scale_are_unbiased():
+    """Eq. (7) probes (whole channel blocks zeroed with probability 1-p) with the 1/nnz(Z_n) scale of
+    Eq. (8) stay unbiased; with the plain 1/r scale they are biased by the factor nnz/r."""
+    X, Wt, dY = _tiny(seed=30, B=3, Cin=3, Cout=2, H=3, W=3)
+    exact = _loops_dw(X, dY, 3, 3, False)
+    g = _rng(31)
+    T, r, p = 1500, 6, 0.6
+    acc = np.zeros_like(exact); acc_plain = np.zeros_like(exact)
+    for _ in range(T):
+        Z = g.standard_normal((r, 3, 3, 3)) * (g.random((r, 3, 1, 1)) < p)
+        sc = O.channel_scale(Z)
+        S = O.sketch(X, Z)
+        acc += O.wgrad_estimate(S, dY, Z, scale=sc)
+        acc_plain += O.wgrad_estimate(S, dY, Z)
+    # channels with nnz = 0 give 0 (probability (1-p)^r = 0.4%): compare against (1-(1-p)^r) * exact
+    keep = 1 - (1 - p) ** r
+    assert O.rel_fro(acc / T, keep * exact) < 0.08
+    assert O.rel_fro(acc_plain / T, p * exact) < 0.08
+    assert O.rel_fro(acc_plain / T, exact) > 0.25
+
+
+def test_channel_scale_counts_nonzero_blocks():
+    Z = np.zeros((4, 3, 2, 2))
+    Z[0, 0] = 1; Z[2, 0, 1, 1] = -3; Z[1, 1, 0, 0] = 2
+    np.testing.assert_allclose(O.channel_scale(Z), [0.5, 1.0, 0.0])
+    np.testing.assert_allclose(O.channel_scale(np.ones((5, 2, 2, 2))), [0.2, 0.2])
+
+
+# ---------------------------------------------------------------- P5: Proposition 1
+
+def test_p5_proposition1_bound_holds_with_probability_1_minus_delta():
+    c2, cF = np.loadtxt(os.path.join(GOLD, "prop1_constants.txt"))
+    g = _rng(40)
+    H, W, B = 4, 4, 3
+    X = g.standard_normal((B, 1, H, W)); dY = g.standard_normal((B, 1, H, W))
+    exact = _loops_dw(X, dY, 3, 3, False)
+    T = 1500
+    for r in (1, 4, 32):
+        Zall = g.standard_normal((T, r, 1, H, W))
+        ests = np.stack([O.wgrad_estimate(O.sketch(X, Zall[t]), dY, Zall[t]) for t in range(T)])
+        for (ky, kx) in ((0, 0), (1, 1), (2, 1)):
+            A = _C_blocks(X, dY, 0, ky, kx)[0]
+            n2, nF = np.linalg.norm(A, 2), np.linalg.norm(A, "fro")
+            dev = np.abs(ests[:, 0, 0, ky, kx] - exact[0, 0, ky, kx])
+            for delta in (0.1, 0.01):
+                lg = math.log(2 / delta)
+                bound = c2 * n2 / r * lg + cF * nF / math.sqrt(r) * math.sqrt(lg)
+                frac = np.mean(dev > bound)
+                assert frac <= delta + 3 * math.sqrt(delta * (1 - delta) / T), (r, ky, kx, delta, frac)
+            # the bound is not vacuous for this estimator: a deviation of that size does occur at 1/50 of it
+            assert np.mean(dev > bound / 50) > 0
+
+
+# ---------------------------------------------------------------- P6: Theorem 1's shape
+
+def test_p6_error_decays_like_inverse_sqrt_r_and_respects_the_row_bound():
+    X, Wt, dY = _tiny(seed=50, B=4, Cin=3, Cout=2, H=4, W=4)
+    exact = _loops_dw(X, dY, 3, 3, False)
+    g = _rng(51)
+    rs, rms = (4, 16, 64, 256), []
+    for r in rs:
+        errs = []
+        for _ in range(60):
+            Z = g.standard_normal((r, 3, 4, 4))
+            errs.append(O.wgrad_estimate(O.sketch(X, Z), dY, Z) - exact)
+        rms.append(np.sqrt(np.mean(np.square(errs), axis=0)))
+    slope = np.polyfit(np.log(rs), np.log([np.sqrt(np.mean(e ** 2)) for e in rms]), 1)[0]
+    assert -0.6 < slope < -0.4, slope
+    # RMS error of entry (m,n) <= (sqrt(2)||C_n||_F + sum_{k != n} ||C_k||_F)/sqrt(r): own block plus
+    # the other blocks of the same output row (Theorem 1, large-r form, with the constant made explicit)
+    r = rs[-1]
+    for m in range(2):
+        C = _C_blocks(X, dY, m, 1, 2)
+        nf = [np.linalg.norm(C[n]) for n in range(3)]
+        for n in range(3):
+            bound = (math.sqrt(2) * nf[n] + sum(nf[k] for k in range(3) if k != n)) / math.sqrt(r)
+            assert rms[-1][m, n, 1, 2] <= 1.25 * bound
+
+
+# ---------------------------------------------------------------- P7: memory factor
+
+def test_p7_memory_factor_matches_printed_values():
+    rows = np.loadtxt(os.path.join(GOLD, "memory_factor.txt"))
+    for H, W, Cin, gamma, factor in rows:
+        assert O.memory_factor(int(Cin), int(H), int(W), 2 ** int(gamma)) == factor == 2 ** (14 - gamma)
+    assert 100 <= O.memory_factor(16, 32, 32, 2 ** 7) <= 130      # "roughly 100x"
