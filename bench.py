@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the XConv hot path: sketch (S = Z^T X) + weight-gradient estimate, layers per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--r R] [--impl xconv|reference]
+
+One step is one pass of the hot path over one synthetic layer batch: xconv_sketch, xconv_backprobe and
+xconv_contract (the last two are exactly xconv_wgrad) through the C ABI, inputs resident in HBM.  The
+line printed by rank 0 carries the whole-job throughput, the same metric end to end from pinned host
+buffers (`e2e`), the roofline of the dominant kernel (`roofline`), the float64 oracle timed on the
+host cores (`cpu_baseline`), per-phase times and, as context, torch's exact cuDNN weight gradient.
+With N > 1 every rank owns its own batch shard (same Z everywhere) and the dW estimates are summed
+with one NCCL all-reduce per step (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "sketch+wgrad layers/s"
+UNIT = "layers/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+def layer_work(c, r):
+    """Algorithmic bytes and flops per launch of each phase (what the method must move and compute)."""
+    s = 4 if c["dtype"] == "f32" else 2
+    N = c["H"] * c["W"]
+    B, Cin, Cout = c["B"], c["Cin"], c["Cout"]
+    T = 9
+    return {
+        "sketch": dict(bytes=s * (B + r) * Cin * N + 4 * r * B, flops=2.0 * r * B * Cin * N),
+        "backprobe": dict(bytes=s * (B + r) * Cout * N + 4 * r * B, flops=2.0 * r * B * Cout * N),
+        "contract": dict(bytes=s * r * (Cin + Cout) * N + 4 * T * Cin * Cout, flops=2.0 * T * r * Cout * Cin * N),
+    }
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for row in self.rows:
+            try:
+                sm.append(float(row[0])); mx.append(float(row[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, row[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------- oracle legs
+
+def oracle_sample_time(cfg, r, frac=8):
+    """The float64 oracle, as it stands, on a bounded sample of the workload: the sketch of B/frac
+    samples plus the estimator for Cout/frac output channels (all probes, input channels and pixels).
+    Both costs are linear in the sliced axis, so the layer time is frac x the sample time."""
+    from oracle import xconv_oracle as O
+    from paper_2106_06998_b200 import inputs
+    c = inputs.layer_shape(cfg)
+    if frac <= 0:       # about 0.3 s of oracle time per GFLOP-pair on a few cores: aim at 10-20 s
+        est = 2.0 * r * c["Cout"] * c["H"] * c["W"] * (c["B"] + 9 * c["Cin"]) / 4e9
+        frac = 1
+        while est / frac > 16 and frac < 64:
+            frac *= 2
+    Bs, Ms = max(1, c["B"] // frac), max(1, c["Cout"] // frac)
+    g = np.random.Generator(np.random.PCG64(1))
+    X = inputs.draw(c["x"], (Bs, c["Cin"], c["H"], c["W"]), 11, c["dtype"])
+    dY = inputs.draw("normal", (c["B"], Ms, c["H"], c["W"]), 12, c["dtype"], c["dy_var"] ** 0.5)
+    Z = inputs.draw(c["z"], (r, c["Cin"], c["H"], c["W"]), 13, c["dtype"])
+    S = g.standard_normal((r, c["B"]))
+    t0 = time.perf_counter()
+    O.sketch(X, Z)
+    t1 = time.perf_counter()
+    O.wgrad_estimate(S, dY, Z)
+    t2 = time.perf_counter()
+    sample = (f"sketch of B/{frac}={Bs} samples + estimator for Cout/{frac}={Ms} output channels "
+              f"(all r, Cin, pixels); layer time = {frac} x sample time")
+    return frac * (t2 - t0), frac * (t1 - t0), frac * (t2 - t1), sample
+
+
+def host_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([i.get("num_threads", 1) for i in threadpool_info()] or [1])
+    except Exception:
+        n = 1
+    return min(n, len(os.sched_getaffinity(0)))
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2106_06998_b200 import inputs
+    c = inputs.layer_shape(args.config)
+    times = []
+    sample = ""
+    for i in range(args.warmup + args.steps):
+        t, _, _, sample = oracle_sample_time(args.config, args.r, frac=args.oracle_frac)
+        if i >= args.warmup:
+            times.append(t)
+    t = float(np.mean(times))
+    val = 1.0 / t
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(args, c),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_config(args, c):
+    return {"workload": f"config {args.config}: 3x3 conv layer B={c['B']} Cin={c['Cin']} Cout={c['Cout']} "
+                        f"{c['H']}x{c['W']} {c['dtype']} storage, {c['z']} probes, r={args.r}",
+            "r": args.r, "layout": "channels_last", "l2": "inputs larger than L2 (X and dY 205 MB each)"
+            if args.config == 5 else "L2 flushed between steps by a 256 MB write"}
+
+
+# ----------------------------------------------------------------------------------- GPU arm
+
+def run_xconv(args):
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as entry
+    from paper_2106_06998_b200 import binding as xb
+    from paper_2106_06998_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    entry.build()
+
+    cfg, r = args.config, args.r
+    c = inputs.layer_shape(cfg)
+    tdt = torch.float32 if c["dtype"] == "f32" else torch.bfloat16
+    B, Cin, Cout, H, W = c["B"], c["Cin"], c["Cout"], c["H"], c["W"]
+    # seeded synthetic inputs of the workload's recipe, drawn on the host; each rank its own batch
+    # shard (X, dY differ per rank), the same probes Z on every rank
+    lay = inputs.make_layer(cfg, r, tensors=("Z",))
+    Z = xb.to_device(lay["Z"], c["dtype"], dev)
+    hX = inputs.draw(c["x"], (B, Cin, H, W), inputs.seed_for(cfg, r, "X") + 7919 * rank, c["dtype"])
+    hdY = inputs.draw("normal", (B, Cout, H, W), inputs.seed_for(cfg, r, "dY") + 7919 * rank, c["dtype"],
+                      c["dy_var"] ** 0.5)
+    X, dY = xb.to_device(hX, c["dtype"], dev), xb.to_device(hdY, c["dtype"], dev)
+    del lay
+
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, tdt)
+    S = torch.empty((r, B), dtype=torch.float32, device=dev)
+    dW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device=dev, memory_format=torch.channels_last)
+    L = torch.empty((r, Cout, H, W), dtype=tdt, device=dev, memory_format=torch.channels_last)
+    ws = torch.empty(max(xb.workspace_bytes(desc, xb.OP_SKETCH), xb.workspace_bytes(desc, xb.OP_WGRAD)),
+                     dtype=torch.uint8, device=dev)
+    flush = None if cfg == 5 else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    launches = [0]
+
+    def step(events=None):
+        if flush is not None:
+            flush.fill_(1)
+        if events:
+            events[0].record()
+        xb.sketch_into(desc, X, Z, S, ws)
+        launches[0] += xb.last_launch_count()
+        if events:
+            events[1].record()
+        xb.backprobe_into(desc, S, dY, L, ws)
+        launches[0] += xb.last_launch_count()
+        if events:
+            events[2].record()
+        xb.contract_into(desc, L, Z, dW, ws)
+        launches[0] += xb.last_launch_count()
+        if events:
+            events[3].record()
+        if world > 1:
+            dist.all_reduce(dW)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    if xb.workspace_status(ws) != 0:
+        raise SystemExit("a device-side wait ran out during warm-up")
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
+    if rank == 0:
+        sampler.start()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches[0] = 0
+    t_begin.record()
+    for i in range(args.steps):
+        step(ev[i])
+    t_end.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    if xb.workspace_status(ws) != 0:
+        raise SystemExit("a device-side wait ran out during the timed region")
+    ms_step = total_ms / args.steps
+    phase_ms = {n: float(np.mean([ev[i][k].elapsed_time(ev[i][k + 1]) for i in range(args.steps)]))
+                for k, n in enumerate(("sketch", "backprobe", "contract"))}
+
+    # ---- end to end from pinned host buffers through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        pX, pdY, pZ = X.cpu().pin_memory(), dY.cpu().pin_memory(), Z.cpu().pin_memory()
+        pS = torch.empty((r, B), dtype=torch.float32).pin_memory()
+        pdW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32).contiguous(memory_format=torch.channels_last).pin_memory()
+        arena = torch.empty(xb.host_arena_bytes(desc), dtype=torch.uint8, device=dev)
+        n_e2e = max(2, min(args.steps, 5))
+        for _ in range(2):
+            xb.xconv_sketch_wgrad_host(desc, pX, pdY, pZ, pS, pdW, arena)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            xb.xconv_sketch_wgrad_host(desc, pX, pdY, pZ, pS, pdW, arena)   # synchronises before returning
+        t_e2e = torch.tensor([(time.perf_counter() - t0) / n_e2e], device=dev)
+        if world > 1:
+            dist.all_reduce(t_e2e, op=dist.ReduceOp.MAX)
+        es = X.element_size()
+        e2e = {"value": world / float(t_e2e.item()), "unit": UNIT,
+               "h2d_bytes_per_step": (X.numel() + dY.numel() + Z.numel()) * es,
+               "d2h_bytes_per_step": (S.numel() + dW.numel()) * 4, "steps": n_e2e,
+               "note": "xconv_sketch_wgrad_host: pinned host buffers, copies and sync inside the call"}
+        del pX, pdY, pZ, arena
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (live CUDA-event times of the timed region)
+    peaks, peak_src = load_peaks()
+    work = layer_work(c, r)
+    dom = max(phase_ms, key=phase_ms.get)
+    engines = {"sketch": xb.engine_for(desc, xb.OP_SKETCH), "backprobe": xb.engine_for(desc, xb.OP_WGRAD),
+               "contract": xb.engine_for(desc, xb.OP_WGRAD)}
+    tensor_peak = peaks["bf16_tflops"] if total_ms < 2000 else peaks["bf16_tflops_sustained"]
+    phases = {}
+    for n, ms in phase_ms.items():
+        gbs = work[n]["bytes"] / (ms * 1e-3) / 1e9
+        tfs = work[n]["flops"] / (ms * 1e-3) / 1e12
+        comp_peak = tensor_peak if engines[n] == "tcgen05_bf16" else FP32_ALU_TFLOPS
+        t_mem, t_comp = work[n]["bytes"] / (peaks["hbm_gbs"] * 1e9), work[n]["flops"] / (comp_peak * 1e12)
+        bound = "hbm" if t_mem >= t_comp else ("tensor" if engines[n] == "tcgen05_bf16" else "alu")
+        phases[n] = {"ms": ms, "engine": engines[n], "GBps": gbs, "TFLOPps": tfs, "bound": bound,
+                     "frac": (gbs / peaks["hbm_gbs"]) if bound == "hbm" else tfs / comp_peak}
+    d = phases[dom]
+    roofline = {"kernel": dom, "bound": d["bound"],
+                "achieved": d["GBps"] if d["bound"] == "hbm" else d["TFLOPps"],
+                "peak": peaks["hbm_gbs"] if d["bound"] == "hbm" else (tensor_peak if d["engine"] == "tcgen05_bf16" else FP32_ALU_TFLOPS),
+                "unit": "GB/s" if d["bound"] == "hbm" else "TFLOP/s", "frac": d["frac"], "traffic": None,
+                "peak_source": f"of {peak_src}" + ("" if d["bound"] != "alu" else " (derived: 148 SMs x 128 FMA x 2 x 1.965 GHz)")}
+
+    cpu = None
+    if not args.no_cpu:
+        t, ts, tw, sample = oracle_sample_time(cfg, r, frac=args.oracle_frac)
+        cpu = {"value": 1.0 / t, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample,
+               "sketch_s": ts, "wgrad_s": tw}
+
+    context = {}
+    if not args.no_context:
+        try:
+            Wt = torch.empty((Cout, Cin, 3, 3), dtype=tdt, device=dev).contiguous(memory_format=torch.channels_last)
+            f = lambda: torch.ops.aten.convolution_backward(dY, X, Wt, None, [1, 1], [1, 1], [1, 1], False, [0, 0],
+                                                            1, [False, True, False])
+            for _ in range(3):
+                f()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(5):
+                f()
+            b.record(); torch.cuda.synchronize()
+            context["torch_cudnn_exact_wgrad_ms"] = a.elapsed_time(b) / 5
+        except Exception as e:      # context only
+            context["torch_cudnn_exact_wgrad_ms"] = f"unavailable: {type(e).__name__}"
+        context["paper"] = ("no timing table; text: up to 10x over im2col on a Xeon E3-1270 v6 for large images "
+                            "and batches at small r, competitive with cuDNN on an RTX 2000 Ada (Section 5.4)")
+    es = X.element_size()
+    line = {"metric": METRIC, "value": world * 1e3 / ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32" if c["dtype"] == "f32" else "bf16 (f32 accumulate)",
+            "data": "synthetic", "config": workload_config(args, c), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches[0], "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
+            "memory_ratio": {"elements": Cin * H * W / r, "stored_bytes": Cin * H * W * es / (4.0 * r)},
+            "context": context}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="xconv", choices=["xconv", "reference"])
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--r", type=int, default=64)
+    ap.add_argument("--oracle-frac", type=int, default=0, help="slice of the layer the oracle is timed on (0: pick for ~10-20 s)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-context", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_xconv(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,153 @@
+/*
+ * libxconv -- XConv layer kernels for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * XConv ("Low-memory stochastic backpropagation for convolutional layers") replaces the stored
+ * input activation X of a convolutional layer by its projection onto r random probing vectors,
+ * and estimates the weight gradient from that projection with a multi-channel randomized trace
+ * estimator (Section 3, Eq. 2-6; Section 4.1, Algorithm 1).  This library exposes the steps of
+ * Algorithm 1 for one layer:
+ *
+ *   forward :  Y = conv(X, w)            (Algorithm 1, forward step 1; Eq. 5)
+ *              S = Z^T X  in R^{r x B}   (forward step 3; the paper's X-bar, text after Eq. 4)
+ *   backward:  L = S dY^T                (backward step 3)
+ *              dw_i = (1/r) tr(L T_{-k(i)} Z)   for every kernel offset k(i)  (backward step 4; Eq. 6)
+ *              dX = conv^T(dY, w)        (standard back-propagation, which the method keeps exact)
+ *
+ * Index conventions (b batch, n input channel, m output channel, j probe, (y,x) pixel, (ky,kx) offset):
+ *   Y [b,m,y,x]      = sum_{n,ky,kx} W[m,n,ky,kx] * X[b,n,y+ky-pad_h,x+kx-pad_w]
+ *   S [j,b]          = sum_{n,y,x}   Z[j,n,y,x]   * X[b,n,y,x]
+ *   L [j,m,y,x]      = sum_b         S[j,b]       * dY[b,m,y,x]
+ *   dW[m,n,ky,kx]    = scale[n] * sum_{j,y,x} L[j,m,y,x] * Z[j,n,y+ky-pad_h,x+kx-pad_w]
+ *   dX[b,n,u,v]      = sum_{m,ky,kx} W[m,n,ky,kx] * dY[b,m,u-ky+pad_h,v-kx+pad_w]
+ * A pixel index outside [0,H)x[0,W) reads as zero (the truncating shift that matches a zero-padded
+ * convolution; the paper's circular shift T_k is not implemented).  scale[n] = 1/r (Eq. 6) unless
+ * chan_scale is given (Eq. 8: 1/nnz(Z_n) for block-sparse probes).
+ *
+ * MEMORY LAYOUT.  Every tensor is dense and channels-last: the channel index is the fastest one.
+ *   X, dY, Y, dX : element (b,c,y,x) at ((b*H + y)*W + x)*C + c
+ *   Z            : element (j,n,y,x) at ((j*H + y)*W + x)*Cin + n
+ *   W, dW        : element (m,n,ky,kx) at ((m*KH + ky)*KW + kx)*Cin + n
+ *   S            : element (j,b) at j*B + b, always float
+ * (This is torch's channels_last memory format of the logical NCHW / OIHW tensors.)
+ * X, W, dY, Z, Y, dX are stored in desc.dtype (float or bfloat16); S and dW are always float.
+ * With bfloat16 storage all sums are accumulated in float; L is kept in bfloat16 and S is rounded to
+ * bfloat16 where it feeds the tensor cores.
+ *
+ * OWNERSHIP AND EXECUTION.  All pointers are device pointers owned by the caller, 16-byte aligned,
+ * unless a parameter is documented as a host pointer.  The library allocates no device memory and
+ * keeps no state between calls; scratch memory is passed in as `ws` (size from
+ * xconv_workspace_bytes).  Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
+ * NULL = default stream) and the call returns without synchronising.  Outputs are overwritten, never
+ * accumulated into.  The same Z must be given to the forward and to the backward call of a layer.
+ * Results are bit-reproducible run to run (fixed reduction order, no atomics).
+ *
+ * ERRORS.  Every entry point returns an xconv_status.  A call that returns anything but XCONV_OK
+ * has launched nothing.  Shapes or options without a kernel return XCONV_ERR_UNSUPPORTED; there is
+ * no CPU or library fallback.  Pipelined kernels bound every device-side wait; a wait that runs
+ * out records a code in the first word of the workspace, which xconv_workspace_status() reads back.
+ */
+#ifndef XCONV_H_
+#define XCONV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { XCONV_F32 = 0, XCONV_BF16 = 1 } xconv_dtype;
+
+typedef enum {
+  XCONV_OK = 0,
+  XCONV_ERR_INVALID_ARG = 1, /* NULL descriptor/pointer, non-positive size */
+  XCONV_ERR_UNSUPPORTED = 2, /* valid request without a kernel (stride, even kernel size, circular shifts ...) */
+  XCONV_ERR_ALIGNMENT = 3,   /* a pointer is not 16-byte aligned */
+  XCONV_ERR_WORKSPACE = 4,   /* ws is NULL or smaller than xconv_workspace_bytes */
+  XCONV_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed; see xconv_last_cuda_error */
+  XCONV_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported by xconv_workspace_status) */
+} xconv_status;
+
+typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3 } xconv_op;
+
+/* Which arithmetic engine a call will use for its dominant kernel. */
+typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2 } xconv_engine;
+
+/* One convolutional layer: stride 1, dilation 1, one group, no bias, "same" output size
+ * (2*pad_h = KH-1, 2*pad_w = KW-1; KH = KW in {1, 3}). */
+typedef struct {
+  int32_t B, Cin, Cout, H, W;
+  int32_t KH, KW, pad_h, pad_w;
+  int32_t r;                /* number of probing vectors */
+  int32_t dtype;            /* xconv_dtype: storage of X, W, dY, Z, Y, dX */
+  int32_t circular;         /* must be 0 (truncating shifts) */
+  const float* chan_scale;  /* NULL: scale 1/r.  Else device pointer to Cin floats (Eq. 8). */
+} xconv_desc;
+
+/* Scratch bytes `op` needs for this layer (0 is possible).  Returns 0 for an invalid descriptor. */
+size_t xconv_workspace_bytes(const xconv_desc* desc, int op);
+
+/* Engine the dominant kernel of `op` runs on for this layer (XCONV_ENGINE_NONE if unsupported). */
+int xconv_engine_for(const xconv_desc* desc, int op);
+
+/* Algorithm 1, forward pass: Y = conv(X, W) (step 1, Eq. 5) and S = Z^T X (step 3).
+ * X [B,H,W,Cin], W [Cout,KH,KW,Cin], Z [r,H,W,Cin] in desc.dtype; Y [B,H,W,Cout] in desc.dtype;
+ * sketch [r,B] float.  After this call the caller may drop X and keep only `sketch` and Z (or the
+ * seed it drew Z from): a memory factor of N*Cin/r per sample (Section 3). */
+xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W, const void* Z,
+                           void* Y, float* sketch, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Forward step 3 alone, S = Z^T X (for callers whose convolution runs elsewhere). */
+xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
+                          void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Algorithm 1, backward steps 3-4: L = S dY^T, then dW[m,n,k] = scale[n] * tr(L^m T_{-k} Z_n) for
+ * every offset (Eq. 6; three-step procedure of Section 3).  sketch [r,B] float as written by
+ * xconv_forward; dY [B,H,W,Cout], Z [r,H,W,Cin] in desc.dtype; dW [Cout,KH,KW,Cin] float.
+ * L lives in the workspace only. */
+xconv_status xconv_wgrad(const xconv_desc* desc, const float* sketch, const void* dY, const void* Z,
+                         float* dW, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* The two halves of xconv_wgrad as calls of their own (for callers that overlap them with other work
+ * and for per-step timing).  xconv_backprobe: L = S dY^T (Algorithm 1 backward step 3), L [r,H,W,Cout]
+ * in desc.dtype (element (j,m,y,x) at ((j*H + y)*W + x)*Cout + m), xconv_backprobe_bytes(desc) bytes.
+ * xconv_contract: dW[m,n,k] = scale[n] * sum_{j,y,x} L[j,m,y,x] Z[j,n,(y,x)+k] (backward step 4; Eq. 6).
+ * xconv_wgrad(ws) is exactly xconv_backprobe + xconv_contract with L placed inside ws. */
+size_t xconv_backprobe_bytes(const xconv_desc* desc);
+xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const void* dY, void* L,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
+xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z, float* dW,
+                            void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Exact input gradient (the transposed convolution; the method leaves it as in standard
+ * back-propagation, Section 1).  dY [B,H,W,Cout], W [Cout,KH,KW,Cin]; dX [B,H,W,Cin] in desc.dtype. */
+xconv_status xconv_dgrad(const xconv_desc* desc, const void* dY, const void* W, void* dX,
+                         void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Sketch + weight-gradient estimate from HOST buffers (Algorithm 1 forward step 3 and backward
+ * steps 3-4 back to back).  hX, hdY, hZ are host pointers to desc.dtype data (pinned memory makes the
+ * copies asynchronous), hS [r,B] and hdW [Cout,KH,KW,Cin] host float outputs.  `arena` is caller-owned
+ * device memory of at least xconv_host_arena_bytes(desc) bytes that receives the inputs, the
+ * outputs and the workspace.  Copies in, runs xconv_sketch and xconv_wgrad, copies out and
+ * synchronises `cuda_stream` before returning. */
+size_t xconv_host_arena_bytes(const xconv_desc* desc);
+xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, const void* hdY, const void* hZ,
+                                     float* hS, float* hdW, void* arena, size_t arena_bytes,
+                                     void* cuda_stream);
+
+/* Reads the status word the kernels of the last call left in `ws` (synchronises `cuda_stream`).
+ * XCONV_OK, or XCONV_ERR_TIMEOUT if a bounded device-side wait ran out. */
+xconv_status xconv_workspace_status(const void* ws, void* cuda_stream);
+
+/* Number of kernels the last successful call on this host thread enqueued. */
+int xconv_last_launch_count(void);
+
+/* cudaError_t (as int) of the last failing CUDA call on this host thread, 0 if none. */
+int xconv_last_cuda_error(void);
+
+const char* xconv_status_string(xconv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XCONV_H_ */

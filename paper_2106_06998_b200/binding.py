@@ -1,0 +1,288 @@
+"""Python binding of libxconv: argument marshalling only -- every step runs in the CUDA library.
+
+Tensors are torch CUDA tensors of logical shape (batch, channel, H, W) / (Cout, Cin, KH, KW) /
+(r, Cin, H, W) held in ``torch.channels_last`` memory format (the library's layout), in float32 or
+bfloat16.  torch is used for device memory and streams only.  There is no fallback: if the shared
+library is missing or a layer has no kernel, a RuntimeError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_char_p, c_float, c_int, c_int32, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libxconv.so")
+
+XCONV_F32, XCONV_BF16 = 0, 1
+OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH = 0, 1, 2, 3
+ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16"}
+STATUS_OK = 0
+
+# every symbol include/xconv.h declares
+EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
+           "xconv_dgrad", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_workspace_status",
+           "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
+
+
+class XConvDesc(Structure):
+    _fields_ = [("B", c_int32), ("Cin", c_int32), ("Cout", c_int32), ("H", c_int32), ("W", c_int32),
+                ("KH", c_int32), ("KW", c_int32), ("pad_h", c_int32), ("pad_w", c_int32), ("r", c_int32),
+                ("dtype", c_int32), ("circular", c_int32), ("chan_scale", c_void_p)]
+
+
+class XConvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().xconv_status_string(status).decode()
+        extra = f" (cudaError {lib().xconv_last_cuda_error()})" if status == 5 else ""
+        super().__init__(f"{where}: {msg}{extra}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2106_06998_b200.build` "
+                           "(libxconv has no CPU or library fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    P = POINTER(XConvDesc)
+    L.xconv_workspace_bytes.argtypes = [P, c_int]; L.xconv_workspace_bytes.restype = c_size_t
+    L.xconv_engine_for.argtypes = [P, c_int]; L.xconv_engine_for.restype = c_int
+    L.xconv_forward.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_forward.restype = c_int
+    L.xconv_sketch.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_sketch.restype = c_int
+    L.xconv_wgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_wgrad.restype = c_int
+    L.xconv_backprobe_bytes.argtypes = [P]; L.xconv_backprobe_bytes.restype = c_size_t
+    L.xconv_backprobe.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_backprobe.restype = c_int
+    L.xconv_contract.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_contract.restype = c_int
+    L.xconv_dgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_dgrad.restype = c_int
+    L.xconv_host_arena_bytes.argtypes = [P]; L.xconv_host_arena_bytes.restype = c_size_t
+    L.xconv_sketch_wgrad_host.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
+                                          c_void_p]
+    L.xconv_sketch_wgrad_host.restype = c_int
+    L.xconv_workspace_status.argtypes = [c_void_p, c_void_p]; L.xconv_workspace_status.restype = c_int
+    L.xconv_last_launch_count.argtypes = []; L.xconv_last_launch_count.restype = c_int
+    L.xconv_last_cuda_error.argtypes = []; L.xconv_last_cuda_error.restype = c_int
+    L.xconv_status_string.argtypes = [c_int]; L.xconv_status_string.restype = c_char_p
+    _lib = L
+    return L
+
+
+def _dtype_code(t: torch.dtype) -> int:
+    if t == torch.float32:
+        return XCONV_F32
+    if t == torch.bfloat16:
+        return XCONV_BF16
+    raise TypeError(f"libxconv stores float32 or bfloat16, got {t}")
+
+
+def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None) -> XConvDesc:
+    code = dtype if isinstance(dtype, int) else _dtype_code(dtype)
+    cs = chan_scale.data_ptr() if chan_scale is not None else None
+    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs)
+
+
+def _cl(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dim() != 4 or not t.is_contiguous(memory_format=torch.channels_last):
+        raise ValueError(f"{name} must be a 4-d tensor in torch.channels_last memory format")
+    return t
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+_ws_cache: dict = {}
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    """A cached scratch buffer of at least ``nbytes`` on ``device`` (grown on demand)."""
+    key = str(device)
+    buf = _ws_cache.get(key)
+    if buf is None or buf.numel() < nbytes:
+        buf = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+        _ws_cache[key] = buf
+    return buf
+
+
+def workspace_bytes(desc: XConvDesc, op: int) -> int:
+    return lib().xconv_workspace_bytes(ctypes.byref(desc), op)
+
+
+def engine_for(desc: XConvDesc, op: int) -> str:
+    return ENGINE_NAMES[lib().xconv_engine_for(ctypes.byref(desc), op)]
+
+
+def _check(status: int, where: str):
+    if status != STATUS_OK:
+        raise XConvError(status, where)
+
+
+# ------------------------------------------------------------------ raw calls (preallocated outputs)
+
+def sketch_into(desc, X, Z, S, ws):
+    _check(lib().xconv_sketch(ctypes.byref(desc), X.data_ptr(), Z.data_ptr(), S.data_ptr(), ws.data_ptr(),
+                              ws.numel(), _stream()), "xconv_sketch")
+
+
+def forward_into(desc, X, W, Z, Y, S, ws):
+    _check(lib().xconv_forward(ctypes.byref(desc), X.data_ptr(), W.data_ptr(), Z.data_ptr(), Y.data_ptr(),
+                               S.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "xconv_forward")
+
+
+def wgrad_into(desc, S, dY, Z, dW, ws):
+    _check(lib().xconv_wgrad(ctypes.byref(desc), S.data_ptr(), dY.data_ptr(), Z.data_ptr(), dW.data_ptr(),
+                             ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad")
+
+
+def backprobe_into(desc, S, dY, L, ws):
+    _check(lib().xconv_backprobe(ctypes.byref(desc), S.data_ptr(), dY.data_ptr(), L.data_ptr(), ws.data_ptr(),
+                                 ws.numel(), _stream()), "xconv_backprobe")
+
+
+def contract_into(desc, L, Z, dW, ws):
+    _check(lib().xconv_contract(ctypes.byref(desc), L.data_ptr(), Z.data_ptr(), dW.data_ptr(), ws.data_ptr(),
+                                ws.numel(), _stream()), "xconv_contract")
+
+
+def dgrad_into(desc, dY, W, dX, ws):
+    _check(lib().xconv_dgrad(ctypes.byref(desc), dY.data_ptr(), W.data_ptr(), dX.data_ptr(), ws.data_ptr(),
+                             ws.numel(), _stream()), "xconv_dgrad")
+
+
+def workspace_status(ws) -> int:
+    return lib().xconv_workspace_status(ws.data_ptr(), _stream())
+
+
+def last_launch_count() -> int:
+    return lib().xconv_last_launch_count()
+
+
+# ------------------------------------------------------------------ same names as the C ABI
+
+def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
+    """S = Z^T X (Algorithm 1 forward step 3): float32 tensor [r, B]."""
+    _cl(X, "X"); _cl(Z, "Z")
+    B, Cin, H, W = X.shape
+    r = Z.shape[0]
+    if tuple(Z.shape[1:]) != (Cin, H, W) or Z.dtype != X.dtype:
+        raise ValueError("Z must be (r, Cin, H, W) in X's dtype")
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    S = torch.empty((r, B), dtype=torch.float32, device=X.device)
+    ws = workspace(workspace_bytes(desc, OP_SKETCH), X.device)
+    sketch_into(desc, X, Z, S, ws)
+    return S
+
+
+def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
+    """Y = conv(X, W) and the sketch S = Z^T X (Algorithm 1 forward steps 1 and 3)."""
+    _cl(X, "X"); _cl(W, "W"); _cl(Z, "Z")
+    B, Cin, H, Wd = X.shape
+    Cout, _, K, _ = W.shape
+    r = Z.shape[0]
+    if W.shape[1] != Cin or tuple(Z.shape[1:]) != (Cin, H, Wd) or W.dtype != X.dtype or Z.dtype != X.dtype:
+        raise ValueError("shape or dtype mismatch between X, W and Z")
+    desc = make_desc(B, Cin, Cout, H, Wd, r, X.dtype, K)
+    Y = torch.empty((B, Cout, H, Wd), dtype=X.dtype, device=X.device, memory_format=torch.channels_last)
+    S = torch.empty((r, B), dtype=torch.float32, device=X.device)
+    ws = workspace(workspace_bytes(desc, OP_FORWARD), X.device)
+    forward_into(desc, X, W, Z, Y, S, ws)
+    return Y, S
+
+
+def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
+                chan_scale: torch.Tensor | None = None) -> torch.Tensor:
+    """dW estimate (Algorithm 1 backward steps 3-4): float32 (Cout, Cin, K, K), channels_last."""
+    _cl(dY, "dY"); _cl(Z, "Z")
+    B, Cout, H, Wd = dY.shape
+    r, Cin = Z.shape[0], Z.shape[1]
+    if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
+        raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
+    if tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != dY.dtype:
+        raise ValueError("shape or dtype mismatch between dY and Z")
+    if chan_scale is not None and (chan_scale.dtype != torch.float32 or chan_scale.numel() != Cin):
+        raise ValueError("chan_scale must hold Cin float32 values")
+    K = kernel_size
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale)
+    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
+    wgrad_into(desc, sketch, dY, Z, dW, ws)
+    return dW
+
+
+def xconv_backprobe(sketch: torch.Tensor, dY: torch.Tensor) -> torch.Tensor:
+    """L = S dY^T (Algorithm 1 backward step 3): (r, Cout, H, W) in dY's dtype, channels_last."""
+    _cl(dY, "dY")
+    B, Cout, H, Wd = dY.shape
+    r = sketch.shape[0]
+    if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
+        raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
+    desc = make_desc(B, 1, Cout, H, Wd, r, dY.dtype)
+    L = torch.empty((r, Cout, H, Wd), dtype=dY.dtype, device=dY.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
+    backprobe_into(desc, sketch, dY, L, ws)
+    return L
+
+
+def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
+                   chan_scale: torch.Tensor | None = None) -> torch.Tensor:
+    """dW[m,n,k] = scale[n] * sum L[j,m,.] Z[j,n,.+k] (Algorithm 1 backward step 4)."""
+    _cl(L, "L"); _cl(Z, "Z")
+    r, Cout, H, Wd = L.shape
+    Cin = Z.shape[1]
+    if Z.shape[0] != r or tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != L.dtype:
+        raise ValueError("shape or dtype mismatch between L and Z")
+    K = kernel_size
+    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale)
+    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=L.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_WGRAD), L.device)
+    contract_into(desc, L, Z, dW, ws)
+    return dW
+
+
+def xconv_dgrad(dY: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+    """Exact dX (transposed convolution)."""
+    _cl(dY, "dY"); _cl(W, "W")
+    B, Cout, H, Wd = dY.shape
+    _, Cin, K, _ = W.shape
+    if W.shape[0] != Cout or W.dtype != dY.dtype:
+        raise ValueError("shape or dtype mismatch between dY and W")
+    desc = make_desc(B, Cin, Cout, H, Wd, 1, dY.dtype, K)
+    dX = torch.empty((B, Cin, H, Wd), dtype=dY.dtype, device=dY.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_DGRAD), dY.device)
+    dgrad_into(desc, dY, W, dX, ws)
+    return dX
+
+
+def host_arena_bytes(desc: XConvDesc) -> int:
+    return lib().xconv_host_arena_bytes(ctypes.byref(desc))
+
+
+def xconv_sketch_wgrad_host(desc: XConvDesc, hX, hdY, hZ, hS, hdW, arena: torch.Tensor):
+    """Sketch + dW estimate from host (ideally pinned) tensors; copies are inside the call."""
+    _check(lib().xconv_sketch_wgrad_host(ctypes.byref(desc), hX.data_ptr(), hdY.data_ptr(), hZ.data_ptr(),
+                                         hS.data_ptr(), hdW.data_ptr(), arena.data_ptr(), arena.numel(), _stream()),
+           "xconv_sketch_wgrad_host")
+
+
+def to_device(a, dtype: str, device="cuda") -> torch.Tensor:
+    """Host float32 array (logical NCHW, already rounded to ``dtype``) -> channels_last device tensor."""
+    t = torch.from_numpy(a).to(device)
+    if dtype == "bf16":
+        t = t.to(torch.bfloat16)
+    return t.contiguous(memory_format=torch.channels_last)

@@ -1,0 +1,440 @@
+// libxconv C ABI: argument checks, workspace planning and kernel dispatch.
+#include "../../include/xconv.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+#include "simt_kernels.cuh"
+#include "tc_api.h"
+
+namespace xconv {
+
+thread_local int g_last_cuda_error = 0;
+thread_local int g_launches = 0;
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline long cdiv(long a, long b) { return (a + b - 1) / b; }
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static xconv_status check_launch() {
+  ++g_launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return XCONV_OK;
+}
+
+static xconv_status clear_status(void* ws, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(ws, 0, 16, st);
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return XCONV_OK;
+}
+
+static xconv_status validate(const xconv_desc* d) {
+  if (!d) return XCONV_ERR_INVALID_ARG;
+  if (d->B <= 0 || d->Cin <= 0 || d->Cout <= 0 || d->H <= 0 || d->W <= 0 || d->r <= 0 || d->KH <= 0 || d->KW <= 0)
+    return XCONV_ERR_INVALID_ARG;
+  if (d->dtype != XCONV_F32 && d->dtype != XCONV_BF16) return XCONV_ERR_INVALID_ARG;
+  if (d->pad_h < 0 || d->pad_w < 0) return XCONV_ERR_INVALID_ARG;
+  if (d->circular != 0) return XCONV_ERR_UNSUPPORTED;
+  if (d->KH != d->KW || (d->KH != 1 && d->KH != 3)) return XCONV_ERR_UNSUPPORTED;
+  if (2 * d->pad_h != d->KH - 1 || 2 * d->pad_w != d->KW - 1) return XCONV_ERR_UNSUPPORTED;
+  // 32-bit grid and index limits of the kernels
+  const long Kdim = (long)d->H * d->W * d->Cin, Q = (long)d->H * d->W * d->Cout;
+  if (Kdim > (1L << 40) || Q > (1L << 40) || (long)d->B * d->H * cdiv(d->W, 32) > 2000000000L)
+    return XCONV_ERR_UNSUPPORTED;
+  return XCONV_OK;
+}
+
+// ----------------------------------------------------------------------------------- plans
+// A plan fixes every launch shape and workspace offset from the descriptor alone, so that
+// xconv_workspace_bytes and the entry points always agree.
+
+static const size_t WS_HEADER = 256;   // word 0: status left by pipelined kernels
+
+struct SketchPlan {
+  bool tc;
+  int splits; long k_per_split;        // simt
+  TcSketchPlan t;                      // tcgen05
+  size_t part_off, bytes;
+};
+
+static SketchPlan plan_sketch(const xconv_desc* d) {
+  SketchPlan p{};
+  const long K = (long)d->H * d->W * d->Cin;
+  p.part_off = WS_HEADER;
+  p.tc = tc_plan_sketch(d, &p.t);
+  if (p.tc) {
+    p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
+    return p;
+  }
+  const long tiles = cdiv(d->r, 64) * cdiv(d->B, 64);
+  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(K, 512)));
+  splits = std::min(splits, 2048L);
+  p.k_per_split = align_up((size_t)cdiv(K, splits), 16);
+  p.splits = (int)cdiv(K, p.k_per_split);
+  p.bytes = p.part_off + align_up((size_t)p.splits * d->r * d->B * sizeof(float), 256);
+  return p;
+}
+
+struct WgradPlan {
+  bool tc;
+  int splits; long items_per_split;    // simt contraction
+  TcWgradPlan t;                       // tcgen05
+  size_t l_off, sb_off, part_off, bytes;
+};
+
+static WgradPlan plan_wgrad(const xconv_desc* d) {
+  WgradPlan p{};
+  const long Q = (long)d->H * d->W * d->Cout;
+  const int T = d->KH * d->KW;
+  const size_t lsz = d->dtype == XCONV_F32 ? 4 : 2;
+  p.l_off = WS_HEADER;
+  p.sb_off = p.l_off + align_up((size_t)d->r * Q * lsz, 256);
+  p.part_off = p.sb_off + align_up((size_t)d->r * d->B * 2, 256);
+  p.tc = tc_plan_wgrad(d, &p.t);
+  if (p.tc) {
+    p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
+    return p;
+  }
+  const long items = (long)d->r * d->H * cdiv(d->W, 32);
+  const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32);
+  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(items, 8)));
+  splits = std::min(splits, 4096L);
+  p.items_per_split = cdiv(items, splits);
+  p.splits = (int)cdiv(items, p.items_per_split);
+  p.bytes = p.part_off + align_up((size_t)p.splits * d->Cout * T * d->Cin * sizeof(float), 256);
+  return p;
+}
+
+// ----------------------------------------------------------------------------------- launchers
+
+template <typename T>
+static xconv_status run_sketch_simt(const xconv_desc* d, const SketchPlan& p, const void* X, const void* Z,
+                                    float* S, char* ws, cudaStream_t st) {
+  const long K = (long)d->H * d->W * d->Cin;
+  float* part = reinterpret_cast<float*>(ws + p.part_off);
+  dim3 grid((unsigned)cdiv(d->B, 64), (unsigned)cdiv(d->r, 64), (unsigned)p.splits);
+  gemm_tn_simt<T><<<grid, 256, 0, st>>>(static_cast<const T*>(Z), static_cast<const T*>(X), part, d->r, d->B, K,
+                                        p.k_per_split, (K % 4 == 0) ? 1 : 0);
+  xconv_status s = check_launch();
+  if (s != XCONV_OK) return s;
+  const long count = (long)d->r * d->B;
+  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, S, count, p.splits, 1.0f, nullptr, 1);
+  return check_launch();
+}
+
+static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z, float* S, void* ws,
+                               size_t ws_bytes, cudaStream_t st) {
+  const SketchPlan p = plan_sketch(d);
+  if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
+  char* w = static_cast<char*>(ws);
+  if (clear_status(w, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st);
+  return d->dtype == XCONV_F32 ? run_sketch_simt<float>(d, p, X, Z, S, w, st)
+                               : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
+}
+
+template <typename T, typename TL>
+static xconv_status run_backprobe_simt(const xconv_desc* d, const float* S, const void* dY, void* Lv,
+                                       cudaStream_t st) {
+  const long Q = (long)d->H * d->W * d->Cout;
+  dim3 g1((unsigned)cdiv(Q, 1024), (unsigned)cdiv(d->r, 16));
+  backprobe_simt<T, TL><<<g1, 256, 0, st>>>(S, static_cast<const T*>(dY), static_cast<TL*>(Lv), d->r, d->B, Q,
+                                            (Q % 4 == 0) ? 1 : 0);
+  return check_launch();
+}
+
+template <typename T, typename TL>
+static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, const void* Lv, const void* Z,
+                                      float* dW, char* ws, cudaStream_t st) {
+  const int T9 = d->KH * d->KW;
+  const TL* L = static_cast<const TL*>(Lv);
+  float* part = reinterpret_cast<float*>(ws + p.part_off);
+  dim3 g2((unsigned)cdiv(d->Cin, 64), (unsigned)cdiv(d->Cout, 32), (unsigned)p.splits);
+  if (d->KH == 3)
+    contract_simt<TL, T, 3><<<g2, 256, 0, st>>>(L, static_cast<const T*>(Z), part, d->r, d->H, d->W, d->Cin, d->Cout,
+                                                p.items_per_split);
+  else
+    contract_simt<TL, T, 1><<<g2, 256, 0, st>>>(L, static_cast<const T*>(Z), part, d->r, d->H, d->W, d->Cin, d->Cout,
+                                                p.items_per_split);
+  xconv_status s = check_launch();
+  if (s != XCONV_OK) return s;
+  const long count = (long)d->Cout * T9 * d->Cin;
+  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, dW, count, p.splits, 1.0f / (float)d->r,
+                                                             d->chan_scale, d->Cin);
+  return check_launch();
+}
+
+template <typename T>
+static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* in, const void* Wt, void* out,
+                                  cudaStream_t st) {
+  const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
+  dim3 grid((unsigned)((long)d->B * d->H * cdiv(d->W, 32)), (unsigned)cdiv(Co, 64));
+  const T* i_ = static_cast<const T*>(in);
+  const T* w_ = static_cast<const T*>(Wt);
+  T* o_ = static_cast<T*>(out);
+  if (d->KH == 3) {
+    if (dgrad) conv_simt<T, 3, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+    else       conv_simt<T, 3, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+  } else {
+    if (dgrad) conv_simt<T, 1, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+    else       conv_simt<T, 1, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+  }
+  return check_launch();
+}
+
+static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, const void* Wt, void* out,
+                             cudaStream_t st) {
+  return d->dtype == XCONV_F32 ? run_conv_simt<float>(d, dgrad, in, Wt, out, st)
+                               : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
+}
+
+// L = S dY^T into `L`; `ws` supplies the bfloat16 copy of S for the tensor-core kernel.
+static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const float* S, const void* dY,
+                                  void* L, char* w, cudaStream_t st) {
+  if (p.tc) {
+    const long n = (long)d->r * d->B;
+    bf16* Sb = reinterpret_cast<bf16*>(w + p.sb_off);
+    cast_f32_to_bf16<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, Sb, n);
+    xconv_status s = check_launch();
+    if (s != XCONV_OK) return s;
+    return tc_run_backprobe(d, p.t, Sb, dY, L, w, st);
+  }
+  return d->dtype == XCONV_F32 ? run_backprobe_simt<float, float>(d, S, dY, L, st)
+                               : run_backprobe_simt<bf16, bf16>(d, S, dY, L, st);
+}
+
+static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const void* L, const void* Z,
+                                 float* dW, char* w, cudaStream_t st) {
+  if (p.tc) return tc_run_contract(d, p.t, L, Z, dW, w, w + p.part_off, st);
+  return d->dtype == XCONV_F32 ? run_contract_simt<float, float>(d, p, L, Z, dW, w, st)
+                               : run_contract_simt<bf16, bf16>(d, p, L, Z, dW, w, st);
+}
+
+static xconv_status check_ws(void* ws, size_t ws_bytes, size_t need) {
+  if (!ws || ws_bytes < need) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
+  return XCONV_OK;
+}
+
+static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* dY, const void* Z, float* dW,
+                              void* ws, size_t ws_bytes, cudaStream_t st) {
+  const WgradPlan p = plan_wgrad(d);
+  xconv_status s = check_ws(ws, ws_bytes, p.bytes);
+  if (s != XCONV_OK) return s;
+  char* w = static_cast<char*>(ws);
+  if (clear_status(w, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  s = run_backprobe(d, p, S, dY, w + p.l_off, w, st);
+  if (s != XCONV_OK) return s;
+  return run_contract(d, p, w + p.l_off, Z, dW, w, st);
+}
+
+int launches() { return g_launches; }
+void count_launch() { ++g_launches; }
+void set_cuda_error(int e) { g_last_cuda_error = e; }
+
+}  // namespace xconv
+
+using namespace xconv;
+
+extern "C" {
+
+size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
+  if (validate(desc) != XCONV_OK) return 0;
+  switch (op) {
+    case XCONV_OP_FORWARD:
+    case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
+    case XCONV_OP_WGRAD: return plan_wgrad(desc).bytes;
+    case XCONV_OP_DGRAD: return WS_HEADER;
+    default: return 0;
+  }
+}
+
+int xconv_engine_for(const xconv_desc* desc, int op) {
+  if (validate(desc) != XCONV_OK) return XCONV_ENGINE_NONE;
+  switch (op) {
+    case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_WGRAD: return plan_wgrad(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_FORWARD:
+    case XCONV_OP_DGRAD: return XCONV_ENGINE_SIMT_F32;
+    default: return XCONV_ENGINE_NONE;
+  }
+}
+
+xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, float* sketch, void* ws,
+                          size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!X || !Z || !sketch) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Z) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
+  g_launches = 0;
+  return run_sketch(desc, X, Z, sketch, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W, const void* Z, void* Y,
+                           float* sketch, void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!X || !W || !Z || !Y || !sketch) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Z) || !aligned16(Y) || !aligned16(sketch))
+    return XCONV_ERR_ALIGNMENT;
+  const SketchPlan p = plan_sketch(desc);
+  if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  g_launches = 0;
+  s = run_conv(desc, false, X, W, Y, st);
+  if (s != XCONV_OK) return s;
+  return run_sketch(desc, X, Z, sketch, ws, ws_bytes, st);
+}
+
+xconv_status xconv_wgrad(const xconv_desc* desc, const float* sketch, const void* dY, const void* Z, float* dW,
+                         void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!sketch || !dY || !Z || !dW) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(sketch) || !aligned16(dY) || !aligned16(Z) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
+  if (desc->chan_scale && (reinterpret_cast<uintptr_t>(desc->chan_scale) & 3u)) return XCONV_ERR_ALIGNMENT;
+  g_launches = 0;
+  return run_wgrad(desc, sketch, dY, Z, dW, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t xconv_backprobe_bytes(const xconv_desc* desc) {
+  if (validate(desc) != XCONV_OK) return 0;
+  return (size_t)desc->r * desc->H * desc->W * desc->Cout * (desc->dtype == XCONV_F32 ? 4 : 2);
+}
+
+xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const void* dY, void* L, void* ws,
+                             size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!sketch || !dY || !L) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(sketch) || !aligned16(dY) || !aligned16(L)) return XCONV_ERR_ALIGNMENT;
+  const WgradPlan p = plan_wgrad(desc);
+  s = check_ws(ws, ws_bytes, p.bytes);
+  if (s != XCONV_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  g_launches = 0;
+  if (clear_status(ws, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  return run_backprobe(desc, p, sketch, dY, L, static_cast<char*>(ws), st);
+}
+
+xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z, float* dW, void* ws,
+                            size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!L || !Z || !dW) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(L) || !aligned16(Z) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
+  if (desc->chan_scale && (reinterpret_cast<uintptr_t>(desc->chan_scale) & 3u)) return XCONV_ERR_ALIGNMENT;
+  const WgradPlan p = plan_wgrad(desc);
+  s = check_ws(ws, ws_bytes, p.bytes);
+  if (s != XCONV_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  g_launches = 0;
+  if (clear_status(ws, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  return run_contract(desc, p, L, Z, dW, static_cast<char*>(ws), st);
+}
+
+xconv_status xconv_dgrad(const xconv_desc* desc, const void* dY, const void* W, void* dX, void* ws,
+                         size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!dY || !W || !dX) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(W) || !aligned16(dX)) return XCONV_ERR_ALIGNMENT;
+  if (!ws || ws_bytes < WS_HEADER) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
+  g_launches = 0;
+  if (clear_status(ws, static_cast<cudaStream_t>(cuda_stream)) != XCONV_OK) return XCONV_ERR_CUDA;
+  return run_conv(desc, true, dY, W, dX, static_cast<cudaStream_t>(cuda_stream));
+}
+
+// Arena layout of the host-buffer entry point: X | dY | Z | S | dW | workspace, each 256-aligned.
+struct HostArena { size_t x, dy, z, s, dw, ws, ws_bytes, total, xb, dyb, zb, sb, dwb; };
+static HostArena host_arena(const xconv_desc* d) {
+  HostArena a{};
+  const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
+  const size_t px = (size_t)d->H * d->W;
+  a.xb = (size_t)d->B * px * d->Cin * es;
+  a.dyb = (size_t)d->B * px * d->Cout * es;
+  a.zb = (size_t)d->r * px * d->Cin * es;
+  a.sb = (size_t)d->r * d->B * 4;
+  a.dwb = (size_t)d->Cout * d->KH * d->KW * d->Cin * 4;
+  a.x = 0;
+  a.dy = a.x + align_up(a.xb, 256);
+  a.z = a.dy + align_up(a.dyb, 256);
+  a.s = a.z + align_up(a.zb, 256);
+  a.dw = a.s + align_up(a.sb, 256);
+  a.ws = a.dw + align_up(a.dwb, 256);
+  a.ws_bytes = std::max(plan_sketch(d).bytes, plan_wgrad(d).bytes);
+  a.total = a.ws + a.ws_bytes;
+  return a;
+}
+
+size_t xconv_host_arena_bytes(const xconv_desc* desc) {
+  if (validate(desc) != XCONV_OK) return 0;
+  return host_arena(desc).total;
+}
+
+xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, const void* hdY, const void* hZ,
+                                     float* hS, float* hdW, void* arena, size_t arena_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!hX || !hdY || !hZ || !hS || !hdW || !arena) return XCONV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(arena) & 255u) return XCONV_ERR_ALIGNMENT;
+  const HostArena a = host_arena(desc);
+  if (arena_bytes < a.total) return XCONV_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* base = static_cast<char*>(arena);
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(base + a.x, hX, a.xb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(base + a.z, hZ, a.zb, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(base + a.dy, hdY, a.dyb, cudaMemcpyHostToDevice, st)) != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return XCONV_ERR_CUDA;
+  }
+  g_launches = 0;
+  float* S = reinterpret_cast<float*>(base + a.s);
+  float* dW = reinterpret_cast<float*>(base + a.dw);
+  s = run_sketch(desc, base + a.x, base + a.z, S, base + a.ws, a.ws_bytes, st);
+  if (s != XCONV_OK) return s;
+  s = run_wgrad(desc, S, base + a.dy, base + a.z, dW, base + a.ws, a.ws_bytes, st);
+  if (s != XCONV_OK) return s;
+  if ((e = cudaMemcpyAsync(hS, S, a.sb, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(hdW, dW, a.dwb, cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+      (e = cudaStreamSynchronize(st)) != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return XCONV_ERR_CUDA;
+  }
+  return XCONV_OK;
+}
+
+xconv_status xconv_workspace_status(const void* ws, void* cuda_stream) {
+  if (!ws) return XCONV_ERR_INVALID_ARG;
+  unsigned int word = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return word == WS_OK ? XCONV_OK : XCONV_ERR_TIMEOUT;
+}
+
+int xconv_last_launch_count(void) { return g_launches; }
+int xconv_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* xconv_status_string(xconv_status s) {
+  switch (s) {
+    case XCONV_OK: return "ok";
+    case XCONV_ERR_INVALID_ARG: return "invalid argument";
+    case XCONV_ERR_UNSUPPORTED: return "unsupported layer or option (no kernel; there is no fallback)";
+    case XCONV_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case XCONV_ERR_WORKSPACE: return "workspace missing or too small";
+    case XCONV_ERR_CUDA: return "CUDA call failed";
+    case XCONV_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

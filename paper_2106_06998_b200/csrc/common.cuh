@@ -1,0 +1,62 @@
+// Shared device/host helpers for the libxconv kernels.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace xconv {
+
+typedef __nv_bfloat16 bf16;
+
+// Codes a kernel may leave in the first word of the workspace.
+enum : unsigned int { WS_OK = 0u, WS_TIMEOUT = 0x7157u };
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// Four consecutive elements as floats; the pointer must be aligned to 4 elements.
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 ld4(const bf16* p) {
+  const uint2 u = *reinterpret_cast<const uint2*>(p);
+  float4 f;
+  f.x = __uint_as_float(u.x << 16);
+  f.y = __uint_as_float(u.x & 0xffff0000u);
+  f.z = __uint_as_float(u.y << 16);
+  f.w = __uint_as_float(u.y & 0xffff0000u);
+  return f;
+}
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void st4(bf16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&a);
+  u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+// Elements idx..idx+3 of p, zero beyond `limit`; vector access when `vec` says rows are 4-aligned.
+template <typename T>
+__device__ __forceinline__ float4 ld4_guard(const T* p, long idx, long limit, bool vec) {
+  if (vec && idx + 3 < limit) return ld4(p + idx);
+  float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (idx + 0 < limit) f.x = to_f(p[idx + 0]);
+  if (idx + 1 < limit) f.y = to_f(p[idx + 1]);
+  if (idx + 2 < limit) f.z = to_f(p[idx + 2]);
+  if (idx + 3 < limit) f.w = to_f(p[idx + 3]);
+  return f;
+}
+template <typename T>
+__device__ __forceinline__ void st4_guard(T* p, long idx, long limit, bool vec, float4 v) {
+  if (vec && idx + 3 < limit) { st4(p + idx, v); return; }
+  if (idx + 0 < limit) p[idx + 0] = from_f<T>(v.x);
+  if (idx + 1 < limit) p[idx + 1] = from_f<T>(v.y);
+  if (idx + 2 < limit) p[idx + 2] = from_f<T>(v.z);
+  if (idx + 3 < limit) p[idx + 3] = from_f<T>(v.w);
+}
+
+}  // namespace xconv

@@ -1,0 +1,301 @@
+// FP32-FMA kernels for every step of the layer.  They serve float storage (where the 1e-5 parity
+// bar rules out TF32/BF16 tensor-core products) and any bfloat16 shape the tcgen05 kernels do not
+// cover.  All tensors are channels-last; all sums are accumulated in float.
+#pragma once
+
+#include "common.cuh"
+
+namespace xconv {
+
+// ---------------------------------------------------------------------------------------------
+// Sketch, S = Z^T X (Algorithm 1 forward step 3): D[m][n] = sum_k A[m,k] * Bm[n,k], both operands
+// contiguous along k (k runs over pixel-major, channel-minor positions of one sample / one probe).
+// Split over k: block z writes its partial tile to part[z][M][N]; reduce_partials sums them in order.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, const T* __restrict__ Bm,
+                                                    float* __restrict__ part, int M, int N, long K,
+                                                    long k_per_split, int vec) {
+  __shared__ __align__(16) float As[16][68];
+  __shared__ __align__(16) float Bs[16][68];
+  const int tid = threadIdx.x;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const long kb = (long)blockIdx.z * k_per_split;
+  const long ke = min(K, kb + k_per_split);
+  const int lr = tid >> 2, lk = (tid & 3) * 4;
+  const int tm = tid >> 4, tn = tid & 15;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (long k0 = kb; k0 < ke; k0 += 16) {
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (m0 + lr < M) a = ld4_guard(A + (long)(m0 + lr) * K, k0 + lk, ke, vec != 0);
+    if (n0 + lr < N) b = ld4_guard(Bm + (long)(n0 + lr) * K, k0 + lk, ke, vec != 0);
+    As[lk + 0][lr] = a.x; As[lk + 1][lr] = a.y; As[lk + 2][lr] = a.z; As[lk + 3][lr] = a.w;
+    Bs[lk + 0][lr] = b.x; Bs[lk + 1][lr] = b.y; Bs[lk + 2][lr] = b.z; Bs[lk + 3][lr] = b.w;
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[kk][tm * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tn * 4]);
+      const float ar[4] = {av.x, av.y, av.z, av.w};
+      const float br[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(ar[i], br[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* out = part + (long)blockIdx.z * M * N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + tm * 4 + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tn * 4 + j;
+      if (n < N) out[(long)m * N + n] = acc[i][j];
+    }
+  }
+}
+
+// out[i] = scale(i) * sum_s part[s][i], s ascending (fixed order: results are reproducible).
+// scale(i) = chan_scale[i % period] if chan_scale else alpha.
+__global__ void reduce_partials(const float* __restrict__ part, float* __restrict__ out, long count,
+                                int splits, float alpha, const float* __restrict__ chan_scale, int period) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= count) return;
+  float s = 0.f;
+  for (int k = 0; k < splits; ++k) s += part[(long)k * count + i];
+  out[i] = s * (chan_scale ? chan_scale[i % period] : alpha);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Back-probe, L = S dY^T (Algorithm 1 backward step 3): L[j][q] = sum_b S[j,b] * dY[b,q], q running
+// over the H*W*Cout positions of one sample.  A block owns 1024 q and 16 probes.
+// ---------------------------------------------------------------------------------------------
+template <typename T, typename TL>
+__global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ S, const T* __restrict__ dY,
+                                                      TL* __restrict__ L, int r, int B, long Q, int vec) {
+  __shared__ __align__(16) float Ss[128][16];
+  const int tid = threadIdx.x;
+  const long q = ((long)blockIdx.x * 256 + tid) * 4;
+  const int j0 = blockIdx.y * 16;
+  float4 acc[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  for (int b0 = 0; b0 < B; b0 += 128) {
+    for (int idx = tid; idx < 128 * 16; idx += 256) {
+      const int jj = idx >> 7, bb = idx & 127;   // consecutive threads read consecutive b
+      Ss[bb][jj] = (b0 + bb < B && j0 + jj < r) ? S[(long)(j0 + jj) * B + b0 + bb] : 0.f;
+    }
+    __syncthreads();
+    if (q < Q) {
+      const int nb = min(128, B - b0);
+      for (int bb = 0; bb < nb; ++bb) {
+        const float4 d = ld4_guard(dY + (long)(b0 + bb) * Q, q, Q, vec != 0);
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4) {
+          const float4 s = *reinterpret_cast<const float4*>(&Ss[bb][j4 * 4]);
+          const float sr[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            float4& a = acc[j4 * 4 + i];
+            a.x = fmaf(sr[i], d.x, a.x); a.y = fmaf(sr[i], d.y, a.y);
+            a.z = fmaf(sr[i], d.z, a.z); a.w = fmaf(sr[i], d.w, a.w);
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+  if (q < Q) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (j0 + j < r) st4_guard(L + (long)(j0 + j) * Q, q, Q, vec != 0, acc[j]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Offset contraction (Algorithm 1 backward step 4; Eq. 6 block by block):
+//   part[s][m][tap][n] = sum over the (j, y, x) of split s of L[j,y,x,m] * Z[j,y+ky-p,x+kx-p,n].
+// The shift of each kernel offset is an index offset into a haloed probe tile in shared memory, so
+// no shifted or im2col copy of Z exists.  A block owns 32 output x 64 input channels and all KS*KS
+// offsets; work items are (probe, row, 32-pixel chunk) triples dealt to grid.z splits in order.
+// ---------------------------------------------------------------------------------------------
+template <typename TL, typename TZ, int KS>
+__global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, const TZ* __restrict__ Z,
+                                                     float* __restrict__ part, int r, int H, int W, int Cin,
+                                                     int Cout, long items_per_split) {
+  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS;
+  __shared__ __align__(16) float Ls[XC][32];
+  __shared__ __align__(16) float Zs[KS][XC + KS - 1][64];
+  const int tid = threadIdx.x;
+  const int n0 = blockIdx.x * 64, m0 = blockIdx.y * 32;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int chunks = (W + XC - 1) / XC;
+  const long items = (long)r * H * chunks;
+  const long ib = (long)blockIdx.z * items_per_split;
+  const long ie = min(items, ib + items_per_split);
+
+  float acc[T][2][4];
+#pragma unroll
+  for (int t = 0; t < T; ++t)
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[t][i][k] = 0.f;
+
+  for (long it = ib; it < ie; ++it) {
+    const int xc = (int)(it % chunks);
+    const int y = (int)((it / chunks) % H);
+    const int j = (int)(it / ((long)chunks * H));
+    const int x0 = xc * XC;
+    for (int idx = tid; idx < XC * 32; idx += 256) {
+      const int mm = idx & 31, px = idx >> 5;
+      float v = 0.f;
+      if (x0 + px < W && m0 + mm < Cout) v = to_f(L[(((long)j * H + y) * W + x0 + px) * Cout + m0 + mm]);
+      Ls[px][mm] = v;
+    }
+    for (int idx = tid; idx < KS * (XC + KS - 1) * 64; idx += 256) {
+      const int nn = idx & 63;
+      const int px = (idx >> 6) % (XC + KS - 1);
+      const int dy = (idx >> 6) / (XC + KS - 1);
+      const int yy = y + dy - P, xx = x0 + px - P;
+      float v = 0.f;
+      if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
+        v = to_f(Z[(((long)j * H + yy) * W + xx) * Cin + n0 + nn]);
+      Zs[dy][px][nn] = v;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int px = 0; px < XC; ++px) {
+      const float2 l = *reinterpret_cast<const float2*>(&Ls[px][ty * 2]);
+#pragma unroll
+      for (int dy = 0; dy < KS; ++dy)
+#pragma unroll
+        for (int dx = 0; dx < KS; ++dx) {
+          const float4 z = *reinterpret_cast<const float4*>(&Zs[dy][px + dx][tx * 4]);
+          float* a0 = acc[dy * KS + dx][0];
+          float* a1 = acc[dy * KS + dx][1];
+          a0[0] = fmaf(l.x, z.x, a0[0]); a0[1] = fmaf(l.x, z.y, a0[1]);
+          a0[2] = fmaf(l.x, z.z, a0[2]); a0[3] = fmaf(l.x, z.w, a0[3]);
+          a1[0] = fmaf(l.y, z.x, a1[0]); a1[1] = fmaf(l.y, z.y, a1[1]);
+          a1[2] = fmaf(l.y, z.z, a1[2]); a1[3] = fmaf(l.y, z.w, a1[3]);
+        }
+    }
+    __syncthreads();
+  }
+  float* out = part + (long)blockIdx.z * Cout * T * Cin;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int m = m0 + ty * 2 + i;
+    if (m >= Cout) continue;
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int n = n0 + tx * 4 + k;
+        if (n < Cin) out[((long)m * T + t) * Cin + n] = acc[t][i][k];
+      }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Direct convolution, used for Y (Algorithm 1 forward step 1; Eq. 5) and, with the weights read
+// transposed and flipped, for the exact input gradient dX:
+//   out[b,y,x,co] = sum_{tap,ci} w(co,ci,tap) * in[b,y+dy-p,x+dx-p,ci]
+//   forward: w(co,ci,tap) = Wt[co][tap][ci]          (Wt is [Cout][T][Cin])
+//   dgrad  : w(co,ci,tap) = Wt[ci][T-1-tap][co]
+// A block owns 32 pixels of one image row and 64 output channels; input channels go by 16.
+// ---------------------------------------------------------------------------------------------
+template <typename T_, int KS, bool DGRAD>
+__global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, const T_* __restrict__ Wt,
+                                                 T_* __restrict__ out, int B, int H, int W, int Ci, int Co,
+                                                 int Cin_w) {
+  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS, CK = 16;
+  __shared__ __align__(16) float Xs[KS][XC + KS - 1][CK];
+  __shared__ __align__(16) float Ws[T][CK][64];
+  const int tid = threadIdx.x;
+  const int chunks = (W + XC - 1) / XC;
+  const int xc = blockIdx.x % chunks;
+  const int y = (blockIdx.x / chunks) % H;
+  const int b = blockIdx.x / (chunks * H);
+  const int x0 = xc * XC, co0 = blockIdx.y * 64;
+  const int cp = tid & 31, pg = tid >> 5;
+  float acc[4][2];
+#pragma unroll
+  for (int p = 0; p < 4; ++p) acc[p][0] = acc[p][1] = 0.f;
+
+  for (int ci0 = 0; ci0 < Ci; ci0 += CK) {
+    for (int idx = tid; idx < KS * (XC + KS - 1) * CK; idx += 256) {
+      const int cc = idx % CK;
+      const int px = (idx / CK) % (XC + KS - 1);
+      const int dy = idx / (CK * (XC + KS - 1));
+      const int yy = y + dy - P, xx = x0 + px - P;
+      float v = 0.f;
+      if (yy >= 0 && yy < H && xx >= 0 && xx < W && ci0 + cc < Ci)
+        v = to_f(in[(((long)b * H + yy) * W + xx) * Ci + ci0 + cc]);
+      Xs[dy][px][cc] = v;
+    }
+    for (int idx = tid; idx < T * CK * 64; idx += 256) {
+      int cc, tap, co;
+      if (DGRAD) { co = idx & 63; cc = (idx >> 6) % CK; tap = idx / (64 * CK); }
+      else       { cc = idx % CK; tap = (idx / CK) % T; co = idx / (CK * T); }
+      float v = 0.f;
+      if (co0 + co < Co && ci0 + cc < Ci) {
+        v = DGRAD ? to_f(Wt[((long)(ci0 + cc) * T + (T - 1 - tap)) * Cin_w + co0 + co])
+                  : to_f(Wt[((long)(co0 + co) * T + tap) * Cin_w + ci0 + cc]);
+      }
+      // pairs of output channels are XOR-swizzled by the input channel so that both the
+      // channel-fastest writes above and the pair reads below are free of bank conflicts
+      Ws[tap][cc][(((co >> 1) ^ cc) << 1) | (co & 1)] = v;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int cc = 0; cc < CK; ++cc) {
+#pragma unroll
+      for (int dy = 0; dy < KS; ++dy) {
+        float xv[4 + KS - 1];
+#pragma unroll
+        for (int p = 0; p < 4 + KS - 1; ++p) xv[p] = Xs[dy][pg * 4 + p][cc];
+#pragma unroll
+        for (int dx = 0; dx < KS; ++dx) {
+          const float2 w = *reinterpret_cast<const float2*>(&Ws[dy * KS + dx][cc][(cp ^ cc) << 1]);
+#pragma unroll
+          for (int p = 0; p < 4; ++p) {
+            acc[p][0] = fmaf(xv[p + dx], w.x, acc[p][0]);
+            acc[p][1] = fmaf(xv[p + dx], w.y, acc[p][1]);
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int p = 0; p < 4; ++p) {
+    const int x = x0 + pg * 4 + p;
+    if (x >= W) continue;
+    T_* o = out + (((long)b * H + y) * W + x) * Co;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int co = co0 + cp * 2 + i;
+      if (co < Co) o[co] = from_f<T_>(acc[p][i]);
+    }
+  }
+}
+
+// float -> bfloat16 copy (the sketch as tensor-core operand).
+__global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = __float2bfloat16_rn(in[i]);
+}
+
+__global__ void set_word(unsigned int* p, unsigned int v) { *p = v; }
+
+}  // namespace xconv

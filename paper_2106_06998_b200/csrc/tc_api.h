@@ -1,0 +1,45 @@
+// Interface between the C ABI layer and the tcgen05 (5th-generation tensor core) kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "../../include/xconv.h"
+
+namespace xconv {
+
+struct TcSketchPlan {
+  int swap;            // 0: MMA rows = probes, columns = samples; 1: rows = samples, columns = probes
+  int tile_m, tile_n;  // output tile of one CTA
+  int tiles_m, tiles_n, splits;
+  long kblocks, kblocks_per_split;
+  int stages;
+  size_t part_bytes;
+};
+
+struct TcWgradPlan {
+  // back-probe
+  int bp_tile_n, bp_tiles_q, bp_tiles_r, bp_stages;
+  // contraction
+  int ct_tile_n, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
+  int patch_h, patch_w, patches_y, patches_x;
+  long ct_items, ct_items_per_split;
+  size_t part_bytes;
+};
+
+// Fill the plan and return true when the tcgen05 kernels cover this layer.
+bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p);
+bool tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p);
+
+xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const void* X, const void* Z, float* S,
+                           char* ws_head, char* part, cudaStream_t st);
+xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const void* S_bf16, const void* dY,
+                              void* L, char* ws_head, cudaStream_t st);
+xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const void* L, const void* Z, float* dW,
+                             char* ws_head, char* part, cudaStream_t st);
+
+// bookkeeping shared with the ABI layer
+void count_launch();
+void set_cuda_error(int e);
+
+}  // namespace xconv

@@ -1,0 +1,192 @@
+"""GPU parity: libxconv (through the C ABI) against the float64 oracle, element by element on the
+same seeded inputs.  Tolerances: relative Frobenius error <= 1e-5 for float storage, <= 1e-2 for
+bfloat16 storage with float accumulation; the estimate is compared with the oracle's ESTIMATE for
+the same Z, never with the exact gradient."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import xconv_oracle as O
+from paper_2106_06998_b200 import binding as xb
+from paper_2106_06998_b200 import inputs
+from tests._util import TOL, check, dev, host, sketch_oracle_chunked
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    entry.build()
+    torch.cuda.set_device(0)
+
+
+def _full_layer_parity(lay, K=3):
+    tol = TOL[lay["dtype"]]
+    d = dev(lay)
+    Y, S = xb.xconv_forward(d["X"], d["W"], d["Z"])
+    S2 = xb.xconv_sketch(d["X"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"], kernel_size=K)
+    dX = xb.xconv_dgrad(d["dY"], d["W"])
+    torch.cuda.synchronize()
+    assert torch.equal(S, S2)
+    Yo, So, dWo, dXo = O.xconv_layer(lay["X"], lay["W"], lay["dY"], lay["Z"])
+    errs = dict(Y=check("Y", host(Y), Yo, tol), S=check("sketch", host(S), So, tol),
+                dX=check("dX", host(dX), dXo, tol))
+    # the estimator alone, from the oracle's own sketch (float), so that its error is not inherited
+    So32 = torch.from_numpy(So.astype(np.float32)).cuda()
+    dW_from_oracle_S = xb.xconv_wgrad(So32, d["dY"], d["Z"], kernel_size=K)
+    # the two halves on their own: L against Algorithm 1 backward step 3, the contraction against step 4
+    L = xb.xconv_backprobe(So32, d["dY"])
+    Lo = O.backprobe(So.astype(np.float32), lay["dY"])
+    errs["L"] = check("L", host(L), Lo, tol)
+    Lr = inputs.round_to_storage(Lo.astype(np.float32), lay["dtype"])
+    dWc = xb.xconv_contract(xb.to_device(Lr, lay["dtype"]), d["Z"], kernel_size=K)
+    check("dW (contraction alone)", host(dWc), O.wgrad_contract(Lr, lay["Z"], K, K), 1e-5 if lay["dtype"] == "f32" else 1e-4)
+    errs["dW"] = check("dW (end to end)", host(dW), dWo, tol)
+    check("dW (oracle sketch in)", host(dW_from_oracle_S), dWo, tol)
+    return errs
+
+
+# ------------------------------------------------------------------ small layers, every element
+
+EDGE_SHAPES = [
+    # B, Cin, Cout, H, W, r   -- odd sizes, ragged tiles, B = 1, r not a multiple of any tile
+    (1, 1, 1, 1, 1, 1),
+    (1, 3, 2, 5, 4, 3),
+    (3, 5, 7, 9, 11, 5),
+    (2, 16, 16, 8, 8, 8),
+    (5, 33, 65, 7, 35, 17),
+    (4, 64, 32, 12, 40, 70),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", EDGE_SHAPES)
+def test_edge_shapes_all_elements(shape, dtype):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape))
+    _full_layer_parity(lay)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_pointwise_kernel(dtype):
+    lay = inputs.make_custom(3, 12, 20, 6, 10, 9, dtype=dtype, seed=77, KH=1, KW=1)
+    _full_layer_parity(lay, K=1)
+
+
+@pytest.mark.parametrize("cfg,r,shrink", [
+    (1, 8, {}),                                   # the small configuration at full size
+    (2, 16, dict(B=32)), (2, 64, dict(B=32)),
+    (3, 32, dict(B=16, H=28, W=28)), (3, 128, dict(B=16, H=28, W=28)),
+    (4, 64, dict(B=16, H=48, W=40)),
+    (5, 16, dict(B=128, H=14, W=14)), (5, 64, dict(B=128, H=14, W=14)), (5, 256, dict(B=256, H=14, W=14)),
+])
+def test_config_recipes_reduced_all_elements(cfg, r, shrink):
+    """The five workload recipes (shapes shrunk where the oracle would take too long), all elements."""
+    _full_layer_parity(inputs.make_layer(cfg, r, **shrink))
+
+
+# ------------------------------------------------------------------ full sizes, sampled outputs
+
+FULL = [(2, 16), (2, 64), (3, 32), (3, 128), (4, 64), (5, 16), (5, 64), (5, 256), (5, 1024)]
+
+
+@pytest.mark.parametrize("cfg,r", FULL)
+def test_full_size_sampled(cfg, r):
+    """Full-size layers in the launch configuration the benchmark times.  The sketch is compared in
+    full (one float64 matrix product per slab of probes); dW, Y and dX on channel / sample subsets,
+    each of which the oracle computes as a smaller layer of its own."""
+    lay = inputs.make_layer(cfg, r)
+    tol = TOL[lay["dtype"]]
+    d = dev(lay)
+    Y, S = xb.xconv_forward(d["X"], d["W"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"])
+    dX = xb.xconv_dgrad(d["dY"], d["W"])
+    torch.cuda.synchronize()
+    assert xb.workspace_status(xb.workspace(256, S.device)) == 0
+    So = sketch_oracle_chunked(lay["X"], lay["Z"])
+    check("sketch", host(S), So, tol)
+    g = np.random.Generator(np.random.PCG64(cfg * 1000 + r))
+    ms = np.sort(g.choice(lay["Cout"], size=min(4, lay["Cout"]), replace=False))
+    ns = np.sort(g.choice(lay["Cin"], size=min(6, lay["Cin"]), replace=False))
+    dWo = O.wgrad_estimate(So, lay["dY"][:, ms], lay["Z"][:, ns])
+    check("dW block", host(dW)[np.ix_(ms, ns)], dWo, tol)
+    bs = np.sort(g.choice(lay["B"], size=min(2, lay["B"]), replace=False))
+    check("Y samples", host(Y[bs]), O.conv_forward(lay["X"][bs], lay["W"]), tol)
+    check("dX samples", host(dX[bs]), O.dx_exact(lay["dY"][bs], lay["W"]), tol)
+
+
+# ------------------------------------------------------------------ properties and options
+
+def test_results_are_bit_reproducible():
+    lay = inputs.make_layer(5, 64, B=128, H=14, W=14)
+    d = dev(lay)
+    S1 = xb.xconv_sketch(d["X"], d["Z"]).clone()
+    W1 = xb.xconv_wgrad(S1, d["dY"], d["Z"]).clone()
+    for _ in range(3):
+        S2 = xb.xconv_sketch(d["X"], d["Z"])
+        W2 = xb.xconv_wgrad(S2, d["dY"], d["Z"])
+        assert torch.equal(S1, S2) and torch.equal(W1, W2)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_block_sparse_probes_with_channel_scale(dtype):
+    """Eq. (7) probes with the 1/nnz(Z_n) scale of Eq. (8) passed as chan_scale."""
+    lay = inputs.make_custom(4, 16, 24, 10, 12, 12, dtype=dtype, seed=5)
+    g = np.random.Generator(np.random.PCG64(9))
+    mask = (g.random((12, 16, 1, 1)) < 0.5).astype(np.float32)
+    mask[:, 3] = 0                                     # one channel never probed: estimate must be 0
+    lay["Z"] = lay["Z"] * mask
+    sc = O.channel_scale(lay["Z"])
+    d = dev(lay)
+    S = xb.xconv_sketch(d["X"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"], chan_scale=torch.from_numpy(sc.astype(np.float32)).cuda())
+    want = O.wgrad_estimate(O.sketch(lay["X"], lay["Z"]), lay["dY"], lay["Z"], scale=sc)
+    check("dW nnz-scaled", host(dW), want, TOL[dtype])
+    assert float(dW[:, 3].abs().max()) == 0.0
+
+
+def test_orthogonal_probe_basis_recovers_exact_gradient_on_gpu():
+    """r = Cin*N with (1/r) Z Z^T = I: the float path reproduces the exact gradient."""
+    Cin, H, W = 2, 4, 4
+    lay = inputs.make_custom(3, Cin, 3, H, W, Cin * H * W, dtype="f32", seed=3)
+    from scipy.linalg import hadamard
+    lay["Z"] = hadamard(32).astype(np.float32).reshape(32, Cin, H, W)
+    d = dev(lay)
+    dW = xb.xconv_wgrad(xb.xconv_sketch(d["X"], d["Z"]), d["dY"], d["Z"])
+    check("exact recovery", host(dW), O.dw_exact(lay["X"], lay["dY"]), 1e-5)
+
+
+def test_host_buffer_entry_point_matches_device_entry_points():
+    lay = inputs.make_layer(5, 64, B=128, H=14, W=14)
+    d = dev(lay)
+    S = xb.xconv_sketch(d["X"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"])
+    desc = xb.make_desc(lay["B"], lay["Cin"], lay["Cout"], lay["H"], lay["W"], 64, torch.bfloat16)
+    hX, hdY, hZ = (d[k].cpu().pin_memory() for k in ("X", "dY", "Z"))
+    hS = torch.empty((64, lay["B"]), dtype=torch.float32).pin_memory()
+    hdW = torch.empty(dW.shape, dtype=torch.float32).contiguous(memory_format=torch.channels_last).pin_memory()
+    arena = torch.empty(xb.host_arena_bytes(desc), dtype=torch.uint8, device="cuda")
+    xb.xconv_sketch_wgrad_host(desc, hX, hdY, hZ, hS, hdW, arena)
+    assert torch.equal(hS, S.cpu()) and torch.equal(hdW, dW.cpu())
+
+
+def test_errors_launch_nothing_on_gpu():
+    lay = inputs.make_custom(2, 8, 8, 6, 6, 4, dtype="f32", seed=1)
+    d = dev(lay)
+    desc = xb.make_desc(2, 8, 8, 6, 6, 4, torch.float32)
+    S = torch.full((4, 2), 7.0, device="cuda")
+    ws = torch.empty(xb.workspace_bytes(desc, xb.OP_SKETCH), dtype=torch.uint8, device="cuda")
+    short = ws[: ws.numel() - 64]
+    st = xb.lib().xconv_sketch(ctypes.byref(desc), d["X"].data_ptr(), d["Z"].data_ptr(), S.data_ptr(),
+                               short.data_ptr(), short.numel(), None)
+    torch.cuda.synchronize()
+    assert st == 4 and float(S.min()) == 7.0 and float(S.max()) == 7.0
+
+
+def test_engines_reported():
+    d1 = xb.make_desc(8, 16, 16, 32, 32, 8, torch.float32)
+    assert xb.engine_for(d1, xb.OP_SKETCH) == "simt_f32" and xb.engine_for(d1, xb.OP_WGRAD) == "simt_f32"

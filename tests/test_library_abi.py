@@ -1,0 +1,82 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, sizes its workspace and rejects bad arguments before launching anything."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2106_06998_b200 import binding as xb
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return xb.lib()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    header = open(os.path.join(ROOT, "include", "xconv.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(xconv_[a-z0-9_]+)\s*\(", header))
+    assert declared == set(xb.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def _desc(**kw):
+    base = dict(B=8, Cin=16, Cout=16, H=32, W=32, r=8, dtype=xb.XCONV_F32, K=3)
+    base.update(kw)
+    return xb.make_desc(**base)
+
+
+def test_workspace_sizes_are_positive_and_monotone_in_r(lib):
+    a = xb.workspace_bytes(_desc(r=8), xb.OP_WGRAD)
+    b = xb.workspace_bytes(_desc(r=64), xb.OP_WGRAD)
+    assert 0 < a < b
+    assert xb.workspace_bytes(_desc(), xb.OP_SKETCH) > 0
+    assert xb.workspace_bytes(_desc(), xb.OP_DGRAD) > 0
+    assert xb.workspace_bytes(_desc(), 17) == 0
+
+
+def test_invalid_descriptors_are_rejected(lib):
+    assert xb.workspace_bytes(_desc(B=0), xb.OP_SKETCH) == 0
+    assert xb.engine_for(_desc(r=-1), xb.OP_SKETCH) == "none"
+    d = _desc()
+    d.circular = 1                       # the paper's circular shift has no kernel
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
+    d = _desc(K=5)                       # 5x5 kernels have no kernel yet
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
+    d = _desc()
+    d.pad_h = 0                          # not a "same" convolution
+    assert lib.xconv_wgrad(ctypes.byref(d), 16, 16, 16, 16, 16, 1 << 20, None) == 2
+    d = _desc()
+    d.dtype = 7
+    assert lib.xconv_dgrad(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 1
+
+
+def test_null_misaligned_and_short_workspace_return_codes_without_launching(lib):
+    d = _desc()
+    need = xb.workspace_bytes(d, xb.OP_SKETCH)
+    assert lib.xconv_sketch(None, 16, 16, 16, 16, need, None) == 1
+    assert lib.xconv_sketch(ctypes.byref(d), None, 16, 16, 16, need, None) == 1
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 24, 16, 16, need, None) == 3      # 24 is not 16-aligned
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, None, need, None) == 4
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, need - 1, None) == 4
+    needw = xb.workspace_bytes(d, xb.OP_WGRAD)
+    assert lib.xconv_wgrad(ctypes.byref(d), 16, 16, 16, 16, 16, needw - 1, None) == 4
+    assert lib.xconv_forward(ctypes.byref(d), 16, 16, 16, 16, 16, 16, 0, None) == 4
+    assert lib.xconv_sketch_wgrad_host(ctypes.byref(d), 16, 16, 16, 16, 16, 256, 10, None) == 4
+    assert xb.host_arena_bytes(d) > need
+    assert b"workspace" in lib.xconv_status_string(4)
+
+
+def test_binding_refuses_host_tensors_and_wrong_layout(lib):
+    import torch
+    X = torch.zeros(2, 4, 5, 5)
+    Z = torch.zeros(3, 4, 5, 5)
+    with pytest.raises(ValueError):
+        xb.xconv_sketch(X, Z)
