@@ -79,7 +79,7 @@ static SketchPlan plan_sketch(const xconv_desc* d) {
 }
 
 struct WgradPlan {
-  bool tc;
+  bool tc_bp, tc_ct;
   int splits; long items_per_split;    // simt contraction
   TcWgradPlan t;                       // tcgen05
   size_t l_off, sb_off, part_off, bytes;
@@ -93,8 +93,10 @@ static WgradPlan plan_wgrad(const xconv_desc* d) {
   p.l_off = WS_HEADER;
   p.sb_off = p.l_off + align_up((size_t)d->r * Q * lsz, 256);
   p.part_off = p.sb_off + align_up((size_t)d->r * d->B * 2, 256);
-  p.tc = tc_plan_wgrad(d, &p.t);
-  if (p.tc) {
+  const int mask = tc_plan_wgrad(d, &p.t);
+  p.tc_bp = (mask & 1) != 0;
+  p.tc_ct = (mask & 2) != 0;
+  if (p.tc_ct) {
     p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
     return p;
   }
@@ -195,7 +197,7 @@ static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, co
 // L = S dY^T into `L`; `ws` supplies the bfloat16 copy of S for the tensor-core kernel.
 static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const float* S, const void* dY,
                                   void* L, char* w, cudaStream_t st) {
-  if (p.tc) {
+  if (p.tc_bp) {
     const long n = (long)d->r * d->B;
     bf16* Sb = reinterpret_cast<bf16*>(w + p.sb_off);
     cast_f32_to_bf16<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, Sb, n);
@@ -209,7 +211,7 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
 
 static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const void* L, const void* Z,
                                  float* dW, char* w, cudaStream_t st) {
-  if (p.tc) return tc_run_contract(d, p.t, L, Z, dW, w, w + p.part_off, st);
+  if (p.tc_ct) return tc_run_contract(d, p.t, L, Z, dW, w, w + p.part_off, st);
   return d->dtype == XCONV_F32 ? run_contract_simt<float, float>(d, p, L, Z, dW, w, st)
                                : run_contract_simt<bf16, bf16>(d, p, L, Z, dW, w, st);
 }
@@ -257,7 +259,7 @@ int xconv_engine_for(const xconv_desc* desc, int op) {
   if (validate(desc) != XCONV_OK) return XCONV_ENGINE_NONE;
   switch (op) {
     case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
-    case XCONV_OP_WGRAD: return plan_wgrad(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_WGRAD: return plan_wgrad(desc).tc_ct ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_FORWARD:
     case XCONV_OP_DGRAD: return XCONV_ENGINE_SIMT_F32;
     default: return XCONV_ENGINE_NONE;

@@ -94,11 +94,11 @@ def layer_shape(config: int, **override) -> dict:
 
 def make_layer(config: int, r: int, *, tensors=("X", "W", "dY", "Z"), KH: int = 3, KW: int = 3,
                **override) -> dict:
-    """The tensors of one (config, r) workload.  ``override`` may shrink B, H, W, Cin, Cout
+    """The tensors of one (config, r) workload (key "W" holds the weights, "width" the image width).  ``override`` may shrink B, H, W, Cin, Cout
     (used by tests that want the same recipe at a size the oracle finishes quickly)."""
     c = layer_shape(config, **override)
     B, Cin, Cout, H, W, dt = c["B"], c["Cin"], c["Cout"], c["H"], c["W"], c["dtype"]
-    out = dict(config=config, r=r, B=B, Cin=Cin, Cout=Cout, H=H, W=W, KH=KH, KW=KW, dtype=dt)
+    out = dict(config=config, r=r, B=B, Cin=Cin, Cout=Cout, H=H, width=W, KH=KH, KW=KW, dtype=dt)
     if "X" in tensors:
         out["X"] = draw(c["x"], (B, Cin, H, W), seed_for(config, r, "X"), dt)
     if "W" in tensors:
@@ -114,7 +114,7 @@ def make_layer(config: int, r: int, *, tensors=("X", "W", "dY", "Z"), KH: int = 
 def make_custom(B, Cin, Cout, H, W, r, *, dtype="f32", z="gaussian", x="normal", seed=0,
                 KH=3, KW=3) -> dict:
     """A free-form layer for edge-case tests (odd sizes, ragged tails)."""
-    out = dict(config=0, r=r, B=B, Cin=Cin, Cout=Cout, H=H, W=W, KH=KH, KW=KW, dtype=dtype)
+    out = dict(config=0, r=r, B=B, Cin=Cin, Cout=Cout, H=H, width=W, KH=KH, KW=KW, dtype=dtype)
     out["X"] = draw(x, (B, Cin, H, W), seed * 10 + 0, dtype)
     out["W"] = draw("normal", (Cout, Cin, KH, KW), seed * 10 + 1, dtype, (2.0 / (Cin * KH * KW)) ** 0.5)
     out["dY"] = draw("normal", (B, Cout, H, W), seed * 10 + 2, dtype)

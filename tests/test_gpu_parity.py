@@ -165,7 +165,7 @@ def test_host_buffer_entry_point_matches_device_entry_points():
     d = dev(lay)
     S = xb.xconv_sketch(d["X"], d["Z"])
     dW = xb.xconv_wgrad(S, d["dY"], d["Z"])
-    desc = xb.make_desc(lay["B"], lay["Cin"], lay["Cout"], lay["H"], lay["W"], 64, torch.bfloat16)
+    desc = xb.make_desc(lay["B"], lay["Cin"], lay["Cout"], lay["H"], lay["width"], 64, torch.bfloat16)
     hX, hdY, hZ = (d[k].cpu().pin_memory() for k in ("X", "dY", "Z"))
     hS = torch.empty((64, lay["B"]), dtype=torch.float32).pin_memory()
     hdW = torch.empty(dW.shape, dtype=torch.float32).contiguous(memory_format=torch.channels_last).pin_memory()
