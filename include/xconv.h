@@ -135,6 +135,31 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
                                      float* hS, float* hdW, void* arena, size_t arena_bytes,
                                      void* cuda_stream);
 
+/* The sketch S = Z^T X without any workspace argument and without any allocation.  (The paper has no
+ * counterpart to this call; it computes exactly what xconv_sketch computes.)
+ *
+ * It is meant for callers that cannot allocate device memory when they need the sketch and have no
+ * spare buffer to lend as `ws`: code running inside a host application or framework that gave out
+ * all device memory at start-up and forbids cudaMalloc afterwards, or a latency-critical loop in
+ * which cudaMalloc's device-wide synchronisation is not acceptable.  The split-k partial sums go to
+ * a fixed array of XCONV_STATIC_SCRATCH_FLOATS floats (4 MiB) that is part of the library image:
+ * every GPU that loads the library holds it until the process exits.
+ *
+ *  - X [B,H,W,Cin] and Z [r,H,W,Cin] in desc.dtype and sketch [r,B] float are caller-owned device
+ *    pointers, 16-byte aligned, as for xconv_sketch.  desc.Cout, KH, KW and pad_* are ignored.
+ *  - Limit: r*B <= XCONV_STATIC_SCRATCH_FLOATS.  A larger layer returns XCONV_ERR_WORKSPACE ("too
+ *    small": the fixed array cannot hold even one [r,B] slab) and launches nothing.
+ *  - The call performs no cudaMalloc, cudaFree or other allocating call.  The first call on a device
+ *    resolves the device address of the array (cudaGetSymbolAddress, with that device current);
+ *    make that first call outside any stream capture.
+ *  - All calls on a device share the one array.  Nothing in it has to start at zero -- every call
+ *    overwrites the slabs it then sums -- so stale contents of an earlier call are harmless, but two
+ *    calls that overlap on the GPU (different streams, no dependency) race on it.  Serialise them.
+ *  - Always runs the FP32-FMA kernel; results agree with xconv_sketch to rounding (summation order). */
+#define XCONV_STATIC_SCRATCH_FLOATS (1 << 20)
+xconv_status xconv_sketch_static(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
+                                 void* cuda_stream);
+
 /* Reads the status word the kernels of the last call left in `ws` (synchronises `cuda_stream`).
  * XCONV_OK, or XCONV_ERR_TIMEOUT if a bounded device-side wait ran out. */
 xconv_status xconv_workspace_status(const void* ws, void* cuda_stream);

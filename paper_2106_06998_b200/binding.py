@@ -23,7 +23,8 @@ STATUS_OK = 0
 
 # every symbol include/xconv.h declares
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
-           "xconv_dgrad", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_workspace_status",
+           "xconv_dgrad", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
+           "xconv_workspace_status",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -73,6 +74,8 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_wgrad_host.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t,
                                           c_void_p]
     L.xconv_sketch_wgrad_host.restype = c_int
+    L.xconv_sketch_static.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
+    L.xconv_sketch_static.restype = c_int
     L.xconv_workspace_status.argtypes = [c_void_p, c_void_p]; L.xconv_workspace_status.restype = c_int
     L.xconv_last_launch_count.argtypes = []; L.xconv_last_launch_count.restype = c_int
     L.xconv_last_cuda_error.argtypes = []; L.xconv_last_cuda_error.restype = c_int
@@ -186,6 +189,26 @@ def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
     ws = workspace(workspace_bytes(desc, OP_SKETCH), X.device)
     sketch_into(desc, X, Z, S, ws)
+    return S
+
+
+STATIC_SCRATCH_FLOATS = 1 << 20
+
+
+def xconv_sketch_static(X: torch.Tensor, Z: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """S = Z^T X through the entry point that takes no workspace and allocates nothing in the library
+    (its partial sums live in a fixed 4 MiB array inside the library image).  For callers that may not
+    allocate device memory at this point; pass ``out`` to avoid even the output allocation here.
+    Raises XConvError (workspace too small) when r*B exceeds STATIC_SCRATCH_FLOATS."""
+    _cl(X, "X"); _cl(Z, "Z")
+    B, Cin, H, W = X.shape
+    r = Z.shape[0]
+    if tuple(Z.shape[1:]) != (Cin, H, W) or Z.dtype != X.dtype:
+        raise ValueError("Z must be (r, Cin, H, W) in X's dtype")
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    S = out if out is not None else torch.empty((r, B), dtype=torch.float32, device=X.device)
+    _check(lib().xconv_sketch_static(ctypes.byref(desc), X.data_ptr(), Z.data_ptr(), S.data_ptr(), _stream()),
+           "xconv_sketch_static")
     return S
 
 

@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, con
 
 // out[i] = scale(i) * sum_s part[s][i], s ascending (fixed order: results are reproducible).
 // scale(i) = chan_scale[i % period] if chan_scale else alpha.
-__global__ void reduce_partials(const float* __restrict__ part, float* __restrict__ out, long count,
+static __global__ void reduce_partials(const float* __restrict__ part, float* __restrict__ out, long count,
                                 int splits, float alpha, const float* __restrict__ chan_scale, int period) {
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= count) return;
@@ -291,11 +291,9 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
 }
 
 // float -> bfloat16 copy (the sketch as tensor-core operand).
-__global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
+static __global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = __float2bfloat16_rn(in[i]);
 }
-
-__global__ void set_word(unsigned int* p, unsigned int v) { *p = v; }
 
 }  // namespace xconv
