@@ -10,7 +10,7 @@ namespace xconv {
 
 struct TcSketchPlan {
   int swap;            // 0: MMA rows = probes, columns = samples; 1: rows = samples, columns = probes
-  int tile_m, tile_n;  // output tile of one CTA
+  int tile_m, tile_n, m_sub;  // output tile of one work unit; m_sub 128-row MMA tiles share the other operand
   int tiles_m, tiles_n, splits;
   long kblocks, kblocks_per_split;
   int stages;
@@ -21,7 +21,7 @@ struct TcWgradPlan {
   // back-probe
   int bp_tile_n, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps;
   // contraction
-  int ct_tile_n, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
+  int ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
   int patch_h, patch_w, patches_y, patches_x;
   long ct_items, ct_items_per_split;
   size_t part_bytes;

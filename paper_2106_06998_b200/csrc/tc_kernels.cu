@@ -23,6 +23,7 @@
 #include <cudaTypedefs.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -33,15 +34,19 @@ enum : int { MODE_SKETCH = 0, MODE_BACKPROBE = 1, MODE_CONTRACT = 2 };
 struct TcParams {
   int mode;
   int tile_n;              // MMA N (multiple of 16, <= 256)
-  int tmem_cols;           // power of two >= max(32, tile_n)
+  int m_sub;               // 128-row MMA tiles per work unit that share the B tile (1 or 2)
+  int acc_bufs;            // accumulator sets in tensor memory (2 = epilogue overlaps the next unit)
+  int tmem_cols;           // power of two >= max(32, tile_n * m_sub * acc_bufs)
   int stages;
+  int burst;               // k-blocks the producer issues back to back (<= stages)
   int ksteps;              // UMMA k-steps (of 16) per stage
   uint32_t a_stage_bytes, b_stage_bytes, tx_bytes;
-  int a_boxes, b_boxes;    // TMA boxes per stage and operand
-  uint32_t a_box_bytes, b_box_bytes;
+  int a_boxes, b_boxes;    // TMA boxes per stage: A per 128-row tile, B in all
+  uint32_t a_box_bytes, b_box_bytes, a_sub_bytes;
   int a_mn_major, b_mn_major;
   uint32_t a_lbo, b_lbo;   // leading byte offsets of the UMMA descriptors
-  int tiles_m, tiles_n;    // blockIdx.x = (tap * tiles_m + tm) * tiles_n + tn
+  int tiles_m, tiles_n, taps;
+  long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
   // contraction geometry
   int patch_w, patch_h, patches_x, patches_y, pad;
@@ -170,6 +175,33 @@ constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
 constexpr int TC_THREADS = 192;
 
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+struct Unit { int tm, tn, tap; long split, kb0; int nkb; };
+
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
+  Unit w;
+  if (p.mode == MODE_BACKPROBE) {           // probe tiles innermost: the dY tile is re-read while hot in L2
+    w.tm = (int)(u % p.tiles_m);
+    w.tn = (int)(u / p.tiles_m);
+    w.tap = 0;
+    w.split = 0;
+  } else {                                   // tiles of one k-split are adjacent: they share operands in L2
+    const long tiles = (long)p.taps * p.tiles_m * p.tiles_n;
+    long t = u % tiles;
+    w.split = u / tiles;
+    w.tn = (int)(t % p.tiles_n); t /= p.tiles_n;
+    w.tm = (int)(t % p.tiles_m); t /= p.tiles_m;
+    w.tap = (int)t;
+  }
+  w.kb0 = w.split * p.kblocks_per_split;
+  const long kb1 = min(p.kblocks, w.kb0 + p.kblocks_per_split);
+  w.nkb = (int)max(0L, kb1 - w.kb0);
+  return w;
+}
+
 // ------------------------------------------------------------------------------------ the kernel
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -178,7 +210,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
-  __shared__ __align__(8) uint64_t tmem_full_bar;
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int go;
 
@@ -190,19 +223,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-
-  // tile of this CTA
-  int t = blockIdx.x;
-  const int tn = t % p.tiles_n; t /= p.tiles_n;
-  const int tm = t % p.tiles_m; t /= p.tiles_m;
-  const int tap = t;
-  const long kb0 = (long)blockIdx.y * p.kblocks_per_split;
-  const long kb1 = min(p.kblocks, kb0 + p.kblocks_per_split);
-  const int nkb = (int)max(0L, kb1 - kb0);
+  const int acc_cols = p.tile_n * p.m_sub;                                    // columns of one accumulator set
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&tmem_full_bar, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     prefetch_tmap(&map_a);
@@ -217,43 +242,59 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued = 0;
+      long it = 0;                         // stages filled so far, across units
       bool ok = true;
-      for (int i = 0; i < nkb && ok; ++i) {
-        const int s = i % p.stages;
-        if (i >= p.stages) ok = mbar_wait(&empty_bar[s], (uint32_t)(((i / p.stages) - 1) & 1), p.status);
-        if (!ok) break;
-        const long kb = kb0 + i;
-        const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
-        const uint32_t b_dst = a_dst + p.a_stage_bytes;
-        mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
-        if (p.mode == MODE_SKETCH) {
-          tma_load_2d(a_dst, &map_a, (int)(kb * 64), tm * TILE_M, &full_bar[s]);
-          tma_load_2d(b_dst, &map_b, (int)(kb * 64), tn * p.tile_n, &full_bar[s]);
-        } else if (p.mode == MODE_BACKPROBE) {
-          const int brow = (int)kb * p.ksteps * 16;
-          for (int bx = 0; bx < p.a_boxes; ++bx)
-            tma_load_2d(a_dst + bx * p.a_box_bytes, &map_a, tm * TILE_M + bx * 64, brow, &full_bar[s]);
-          tma_load_2d(b_dst, &map_b, brow, tn * p.tile_n, &full_bar[s]);
-        } else {
-          long u = kb;
-          const int px = (int)(u % p.patches_x); u /= p.patches_x;
-          const int py = (int)(u % p.patches_y); u /= p.patches_y;
-          const int j = (int)u;
-          const int ks = 2 * p.pad + 1;
-          const int dy = tap / ks - p.pad, dx = tap % ks - p.pad;
-          const int x0 = px * p.patch_w, y0 = py * p.patch_h;
-          for (int bx = 0; bx < p.a_boxes; ++bx)
-            tma_load_4d(a_dst + bx * p.a_box_bytes, &map_a, tm * TILE_M + bx * 64, x0, y0, j, &full_bar[s]);
-          for (int bx = 0; bx < p.b_boxes; ++bx)
-            tma_load_4d(b_dst + bx * p.b_box_bytes, &map_b, tn * p.tile_n + bx * 64, x0 + dx, y0 + dy, j,
-                        &full_bar[s]);
+      for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        const int row0 = w.tm * p.m_sub * TILE_M;
+        for (int i = 0; i < w.nkb; ++i, ++it) {
+          const int s = (int)(it % p.stages);
+          if (p.burst > 1 && (i % p.burst) == 0) {
+            // issue `burst` consecutive k-blocks back to back: their rows are adjacent in memory, so
+            // the requests reach DRAM together and share open pages
+            const int n = min(p.burst, w.nkb - i);
+            for (int g = 1; g < n && ok; ++g) {
+              const long t = it + g;
+              if (t >= p.stages) ok = mbar_wait(&empty_bar[t % p.stages], (uint32_t)(((t / p.stages) - 1) & 1), p.status);
+            }
+            if (!ok) break;
+          }
+          if (it >= p.stages) ok = mbar_wait(&empty_bar[s], (uint32_t)(((it / p.stages) - 1) & 1), p.status);
+          if (!ok) break;
+          const long kb = w.kb0 + i;
+          const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
+          const uint32_t b_dst = a_dst + p.a_stage_bytes;
+          mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
+          if (p.mode == MODE_SKETCH) {
+            for (int mt = 0; mt < p.m_sub; ++mt)
+              tma_load_2d(a_dst + mt * p.a_sub_bytes, &map_a, (int)(kb * 64), row0 + mt * TILE_M, &full_bar[s]);
+            tma_load_2d(b_dst, &map_b, (int)(kb * 64), w.tn * p.tile_n, &full_bar[s]);
+          } else if (p.mode == MODE_BACKPROBE) {
+            const int brow = (int)kb * p.ksteps * 16;
+            tma_load_2d(a_dst, &map_a, brow, row0, &full_bar[s]);
+            for (int bx = 0; bx < p.b_boxes; ++bx)
+              tma_load_2d(b_dst + bx * p.b_box_bytes, &map_b, w.tn * p.tile_n + bx * 64, brow, &full_bar[s]);
+          } else {
+            long q = kb;
+            const int px = (int)(q % p.patches_x); q /= p.patches_x;
+            const int py = (int)(q % p.patches_y); q /= p.patches_y;
+            const int j = (int)q;
+            const int ks = 2 * p.pad + 1;
+            const int dy = w.tap / ks - p.pad, dx = w.tap % ks - p.pad;
+            const int x0 = px * p.patch_w, y0 = py * p.patch_h;
+            for (int mt = 0; mt < p.m_sub; ++mt)
+              for (int bx = 0; bx < p.a_boxes; ++bx)
+                tma_load_4d(a_dst + mt * p.a_sub_bytes + bx * p.a_box_bytes, &map_a, row0 + mt * TILE_M + bx * 64,
+                            x0, y0, j, &full_bar[s]);
+            for (int bx = 0; bx < p.b_boxes; ++bx)
+              tma_load_4d(b_dst + bx * p.b_box_bytes, &map_b, w.tn * p.tile_n + bx * 64, x0 + dx, y0 + dy, j,
+                          &full_bar[s]);
+          }
         }
-        issued = i + 1;
       }
       // drain: every copy issued must have landed in this CTA's shared memory before it exits
       // (immediate on the normal path, bounded on the failure path)
-      for (int i = max(0, issued - p.stages); i < issued; ++i)
+      for (long i = max(0L, it - p.stages); i < it; ++i)
         if (!mbar_wait(&full_bar[i % p.stages], (uint32_t)((i / p.stages) & 1), p.status)) break;
     }
   } else if (warp == 1) {
@@ -266,59 +307,94 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       // MN-major: 8-row (k) groups 1024 B apart, 64-column blocks `lbo` apart, k-step = 16 rows = 2048 B.
       const uint32_t a_step = p.a_mn_major ? 2048u : 32u, b_step = p.b_mn_major ? 2048u : 32u;
       const uint32_t a_lbo = p.a_mn_major ? p.a_lbo : 16u, b_lbo = p.b_mn_major ? p.b_lbo : 16u;
+      long it = 0, lu = 0;
       bool ok = true;
-      for (int i = 0; i < nkb; ++i) {
-        const int s = i % p.stages;
-        ok = mbar_wait(&full_bar[s], (uint32_t)((i / p.stages) & 1), p.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t a_src = tiles_base + (uint32_t)s * stage_bytes;
-        const uint32_t b_src = a_src + p.a_stage_bytes;
-        for (int k = 0; k < p.ksteps; ++k) {
-          const uint64_t da = make_desc(a_src + k * a_step, a_lbo, 1024u);
-          const uint64_t db = make_desc(b_src + k * b_step, b_lbo, 1024u);
-          umma_bf16(tmem_base, da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
+      for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
+        const Unit w = decode_unit(p, u);
+        if (w.nkb == 0) continue;
+        const int buf = (int)(lu % p.acc_bufs);
+        const long use = lu / p.acc_bufs;
+        if (use > 0) {                      // the epilogue must have emptied this accumulator set
+          ok = mbar_wait(&tmem_empty_bar[buf], (uint32_t)((use - 1) & 1), p.status);
+          if (!ok) break;
+          tc_fence_after();
         }
-        umma_commit(&empty_bar[s]);          // stage s may be refilled once these MMAs have read it
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
+        for (int i = 0; i < w.nkb; ++i, ++it) {
+          const int s = (int)(it % p.stages);
+          ok = mbar_wait(&full_bar[s], (uint32_t)((it / p.stages) & 1), p.status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a_src = tiles_base + (uint32_t)s * stage_bytes;
+          const uint32_t b_src = a_src + p.a_stage_bytes;
+          for (int k = 0; k < p.ksteps; ++k) {
+            const uint64_t db = make_desc(b_src + k * b_step, b_lbo, 1024u);
+            for (int mt = 0; mt < p.m_sub; ++mt) {
+              const uint64_t da = make_desc(a_src + mt * p.a_sub_bytes + k * a_step, a_lbo, 1024u);
+              umma_bf16(d_tmem + (uint32_t)(mt * p.tile_n), da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit(&empty_bar[s]);        // stage s may be refilled once these MMAs have read it
+        }
+        if (ok) umma_commit(&tmem_full_bar[buf]);
       }
-      if (ok && nkb > 0) umma_commit(&tmem_full_bar);
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
+    long lu = 0;
     bool ok = true;
-    if (nkb > 0) {
-      if (lane == 0) ok = mbar_wait(&tmem_full_bar, 0u, p.status);
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      tc_fence_after();
-    }
-    if (ok) {
-      const long row = (long)tm * TILE_M + quad * 32 + lane;
-      const long col0 = (long)tn * p.tile_n;
-      for (int c = 0; c < p.tile_n; c += 32) {
-        uint32_t v[32];
+    for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
+      const Unit w = decode_unit(p, u);
+      const int buf = (int)(lu % p.acc_bufs);
+      const long use = lu / p.acc_bufs;
+      if (w.nkb > 0) {
+        if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) break;
+        tc_fence_after();
+      }
+      const long col0 = (long)w.tn * p.tile_n;
+      for (int mt = 0; mt < p.m_sub; ++mt) {
+        const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;    // first row of this warp
+        if (row_w >= p.rows) continue;                                         // warp-uniform
+        const long row = row_w + lane;
+        for (int c = 0; c < p.tile_n; c += 32) {
+          if (col0 + c >= p.cols) break;
+          uint32_t v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = 0u;
-        if (nkb > 0) {
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c;
-          if (p.tile_n - c >= 32) tmem_ld32(taddr, v);
-          else { tmem_ld16(taddr, v); }
-        }
-        const int nc = min(32, p.tile_n - c);
-        if (p.mode == MODE_BACKPROBE) {
-          // D[q, j] -> L[j][q]: a warp writes 32 consecutive q of one probe per instruction
-          if (row < p.rows) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const long j = col0 + c + i;
-              if (i < nc && j < p.cols) p.L[j * p.Q + row] = __float2bfloat16_rn(__uint_as_float(v[i]));
-            }
+          for (int i = 0; i < 32; ++i) v[i] = 0u;
+          if (w.nkb > 0) {
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols + mt * p.tile_n + c);
+            if (p.tile_n - c >= 32) tmem_ld32(taddr, v);
+            else tmem_ld16(taddr, v);
           }
-        } else {
-          float* dst;
-          if (p.mode == MODE_SKETCH) dst = p.part + ((long)blockIdx.y * p.rows + row) * p.cols + col0 + c;
-          else dst = p.part + (((long)blockIdx.y * p.rows + row) * p.T + tap) * p.Cin + col0 + c;
-          if (row < p.rows) {
+          const int nc = min(32, p.tile_n - c);
+          if (row >= p.rows) continue;
+          if (p.mode == MODE_BACKPROBE) {
+            // D[j, q] -> L[j][q]: each thread owns 32 consecutive positions of one probe
+            bf16* dst = p.L + row * p.Q + col0 + c;
+            if (nc == 32 && col0 + c + 32 <= p.cols) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                uint4 o;
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+                *reinterpret_cast<uint4*>(dst + i) = o;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+            }
+          } else {
+            float* dst;
+            if (p.mode == MODE_SKETCH) dst = p.part + ((long)w.split * p.rows + row) * p.cols + col0 + c;
+            else dst = p.part + (((long)w.split * p.rows + row) * p.T + w.tap) * p.Cin + col0 + c;
             const bool vec = ((p.cols & 3) == 0);
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
@@ -335,6 +411,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
       }
+      // this accumulator set may be overwritten by the unit after next
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
     }
   }
 
@@ -346,26 +426,46 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
-// S[j][b] = sum_s part[s][row][col]; (row, col) = (b, j) when the samples were the MMA rows.
-__global__ void reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S, int r, int B,
-                                       int splits, int swapped) {
-  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+// S[j][b] = sum_s part[s][row][col] (s ascending within each of four interleaved groups, groups added in
+// order: a fixed tree, so results are reproducible); (row, col) = (b, j) when the samples were the MMA rows.
+__global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S,
+                                                              int r, int B, int splits, int swapped) {
+  __shared__ float acc[4][64];
+  const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
   const long count = (long)r * B;
-  if (i >= count) return;
-  const int j = (int)(i / B), b = (int)(i % B);
-  const long src = swapped ? (long)b * r + j : i;
+  const long i = (long)blockIdx.x * 64 + o;           // index in the layout of `part`
   float s = 0.f;
-  for (int k = 0; k < splits; ++k) s += part[(long)k * count + src];
-  S[i] = s;
+  if (i < count) {
+#pragma unroll 4
+    for (int k = g; k < splits; k += 4) s += part[(long)k * count + i];
+  }
+  acc[g][o] = s;
+  __syncthreads();
+  if (g == 0 && i < count) {
+    const float t = ((acc[0][o] + acc[1][o]) + acc[2][o]) + acc[3][o];
+    long dst = i;
+    if (swapped) { const long b = i / r, j = i % r; dst = j * B + b; }
+    S[dst] = t;
+  }
 }
 
-__global__ void reduce_contract_partials(const float* __restrict__ part, float* __restrict__ out, long count,
-                                         int splits, float alpha, const float* __restrict__ chan_scale, int period) {
-  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
-  float s = 0.f;
-  for (int k = 0; k < splits; ++k) s += part[(long)k * count + i];
-  out[i] = s * (chan_scale ? chan_scale[i % period] : alpha);
+__global__ void __launch_bounds__(256) reduce_contract_partials(const float* __restrict__ part, float* __restrict__ out,
+                                                                long count, int splits, float alpha,
+                                                                const float* __restrict__ chan_scale, int period) {
+  const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (i >= count) return;                              // count is a multiple of 4 (Cin % 8 == 0)
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+  for (int k = 0; k < splits; ++k) {
+    const float4 v = *reinterpret_cast<const float4*>(part + (long)k * count + i);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  float4 sc = make_float4(alpha, alpha, alpha, alpha);
+  if (chan_scale) {
+    const int n = (int)(i % period);
+    sc = make_float4(chan_scale[n], chan_scale[n + 1], chan_scale[n + 2], chan_scale[n + 3]);
+  }
+  *reinterpret_cast<float4*>(out + i) = make_float4(s.x * sc.x, s.y * sc.y, s.z * sc.z, s.w * sc.w);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -374,6 +474,7 @@ static inline long cdivl(long a, long b) { return (a + b - 1) / b; }
 static inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 static const int SMEM_LIMIT = 227 * 1024;
 static const int STATIC_SMEM_SLACK = 2048;     // barriers + alignment slack
+static const int NUM_SMS = 148;
 
 static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -403,6 +504,11 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
   return r == CUDA_SUCCESS;
 }
 
+static int env_int(const char* name, int dflt) {   // TUNING
+  const char* v = getenv(name);
+  return v ? atoi(v) : dflt;
+}
+
 static int pow2_cols(int n) { int c = 32; while (c < n) c *= 2; return c; }
 
 static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
@@ -411,15 +517,17 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
   return std::max(1, std::min(s, MAX_STAGES));
 }
 
-static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, dim3 grid,
+static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
                            cudaStream_t st) {
   const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
-  if (smem > (size_t)(SMEM_LIMIT - 1024)) return XCONV_ERR_UNSUPPORTED;
+  if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512) return XCONV_ERR_UNSUPPORTED;
   {
     cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
     if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   }
-  tc_gemm_kernel<<<grid, TC_THREADS, smem, st>>>(ma, mb, p);
+  TcParams q = p;
+  q.burst = std::min(env_int("XC_BURST", 1), q.stages);   // TUNING
+  tc_gemm_kernel<<<grid, TC_THREADS, smem, st>>>(ma, mb, q);
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -434,17 +542,19 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   if (K % 8 != 0 || K < 2048 || K > 2000000000L) return false;
   p->swap = d->B >= d->r ? 1 : 0;
   const int rows = p->swap ? d->B : d->r, cols = p->swap ? d->r : d->B;
-  p->tile_m = TILE_M;
   p->tile_n = std::min(256, round_up(cols, 16));
-  p->tiles_m = (int)cdivl(rows, TILE_M);
+  p->m_sub = rows > TILE_M ? 2 : 1;                      // two row tiles share each tile of the other operand
+  p->m_sub = env_int("XC_SK_MSUB", p->m_sub);
+  const int sk_ctas = env_int("XC_SK_CTAS", 1);
+  p->tile_m = TILE_M * p->m_sub;
+  p->tiles_m = (int)cdivl(rows, p->tile_m);
   p->tiles_n = (int)cdivl(cols, p->tile_n);
   p->kblocks = cdivl(K, 64);
-  const uint32_t stage = TILE_M * 128 + p->tile_n * 128;
-  const int ctas = (stage * 4 + STATIC_SMEM_SLACK <= SMEM_LIMIT / 2 && p->tile_n <= 128) ? 2 : 1;
-  p->stages = pick_stages(stage, ctas);
+  const uint32_t stage = (uint32_t)p->m_sub * TILE_M * 128 + p->tile_n * 128;
+  p->stages = std::min(pick_stages(stage, sk_ctas), env_int("XC_SK_STAGES", 8));
   const long tiles = (long)p->tiles_m * p->tiles_n;
-  long splits = std::max(1L, std::min((148L * ctas) / tiles, p->kblocks / 8));
-  if (tiles >= 148L * ctas) splits = 1;
+  long splits = std::max(1L, std::min((long)NUM_SMS * sk_ctas / tiles, p->kblocks / 8));
+  splits = env_int("XC_SK_SPLITS", (int)splits);
   splits = std::max(1L, std::min(splits, 512L));
   p->kblocks_per_split = cdivl(p->kblocks, splits);
   p->splits = (int)cdivl(p->kblocks, p->kblocks_per_split);
@@ -468,26 +578,31 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   TcParams p{};
   p.mode = MODE_SKETCH;
   p.tile_n = pl.tile_n;
-  p.tmem_cols = pow2_cols(pl.tile_n);
+  p.m_sub = pl.m_sub;
+  p.acc_bufs = 1;
+  p.tmem_cols = pow2_cols(pl.tile_n * pl.m_sub);
   p.stages = pl.stages;
   p.ksteps = 4;
-  p.a_stage_bytes = TILE_M * 128;
+  p.a_sub_bytes = TILE_M * 128;
+  p.a_stage_bytes = (uint32_t)pl.m_sub * p.a_sub_bytes;
   p.b_stage_bytes = (uint32_t)pl.tile_n * 128;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.a_boxes = p.b_boxes = 1;
   p.a_mn_major = p.b_mn_major = 0;
   p.tiles_m = pl.tiles_m;
   p.tiles_n = pl.tiles_n;
+  p.taps = 1;
   p.kblocks = pl.kblocks;
   p.kblocks_per_split = pl.kblocks_per_split;
+  p.units = (long)pl.tiles_m * pl.tiles_n * pl.splits;
   p.rows = rows;
   p.cols = cols;
   p.part = reinterpret_cast<float*>(part);
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  xconv_status s = launch(ma, mb, p, dim3((unsigned)(pl.tiles_m * pl.tiles_n), (unsigned)pl.splits), st);
+  xconv_status s = launch(ma, mb, p, (unsigned)p.units, st);
   if (s != XCONV_OK) return s;
   const long count = (long)d->r * d->B;
-  reduce_sketch_partials<<<(unsigned)cdivl(count, 256), 256, 0, st>>>(p.part, S, d->r, d->B, pl.splits, pl.swap);
+  reduce_sketch_partials<<<(unsigned)cdivl(count, 64), 256, 0, st>>>(p.part, S, d->r, d->B, pl.splits, pl.swap);
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -508,7 +623,7 @@ static void pick_patch(int H, int W, int* pw, int* ph) {
         best = waste; bw = w; bh = h; barea = w * h;
       }
     }
-  if (barea == 0) { bw = std::min(16, 128); bh = 1; }     // tiny images: one 16-pixel row box, mostly zero fill
+  if (barea == 0) { bw = 16; bh = 1; }     // tiny images: one 16-pixel row box, mostly zero fill
   *pw = bw; *ph = bh;
 }
 
@@ -516,15 +631,15 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   if (d->dtype != XCONV_BF16) return 0;
   int mask = 0;
   const long Q = (long)d->H * d->W * d->Cout;
-  // back-probe: D[q, j], rows = Q, cols = r, k = B
+  // back-probe: D[j, q], rows = r, cols = Q, k = B
   if (Q % 8 == 0 && d->B % 8 == 0 && Q >= 2048 && Q < 2000000000L) {
     mask |= 1;
-    p->bp_tile_n = std::min(256, round_up(d->r, 16));
-    p->bp_tiles_q = (int)cdivl(Q, TILE_M);
-    p->bp_tiles_r = (int)cdivl(d->r, p->bp_tile_n);
+    p->bp_tile_n = env_int("XC_BP_TILEN", 256);
+    p->bp_tiles_q = (int)cdivl(Q, p->bp_tile_n);
+    p->bp_tiles_r = (int)cdivl(d->r, TILE_M);
     p->bp_ksteps = std::min(4, (int)cdivl(d->B, 16));
-    const uint32_t stage = (uint32_t)p->bp_ksteps * 16 * 128 * 2 + (uint32_t)p->bp_tile_n * 128;
-    p->bp_stages = pick_stages(stage, p->bp_tile_n <= 128 ? 2 : 1);
+    const uint32_t stage = TILE_M * 128 + (uint32_t)p->bp_ksteps * 16 * 128 * (uint32_t)(p->bp_tile_n / 64);
+    p->bp_stages = std::min(pick_stages(stage, env_int("XC_BP_CTAS", 1)), env_int("XC_BP_STAGES", 8));
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
@@ -533,15 +648,18 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     pick_patch(d->H, d->W, &p->patch_w, &p->patch_h);
     p->patches_x = (int)cdivl(d->W, p->patch_w);
     p->patches_y = (int)cdivl(d->H, p->patch_h);
-    p->ct_tile_n = std::min(256, round_up(d->Cin, 16));
-    p->ct_tiles_m = (int)cdivl(d->Cout, TILE_M);
+    p->ct_tile_n = std::min(env_int("XC_CT_TILEN", 256), round_up(d->Cin, 16));
+    p->ct_m_sub = d->Cout > TILE_M ? 2 : 1;            // two output-channel tiles share each probe tile
+    p->ct_m_sub = env_int("XC_CT_MSUB", p->ct_m_sub);
+    p->ct_tiles_m = (int)cdivl(d->Cout, TILE_M * p->ct_m_sub);
     p->ct_tiles_n = (int)cdivl(d->Cin, p->ct_tile_n);
     const int bk = p->patch_w * p->patch_h;
-    const uint32_t stage = (uint32_t)bk * 128 * (2 + (uint32_t)cdivl(p->ct_tile_n, 64));
-    p->ct_stages = pick_stages(stage, 1);
+    const uint32_t stage = (uint32_t)bk * 128 * (2 * p->ct_m_sub + (uint32_t)cdivl(p->ct_tile_n, 64));
+    p->ct_stages = std::min(pick_stages(stage, env_int("XC_CT_CTAS", 1)), env_int("XC_CT_STAGES", 8));
     p->ct_items = (long)d->r * p->patches_x * p->patches_y;
     const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * T;
-    long splits = std::max(1L, std::min(148L / std::max(1L, tiles), p->ct_items / 4));
+    long splits = std::max(1L, std::min((long)NUM_SMS * env_int("XC_CT_CTAS", 1) / std::max(1L, tiles), p->ct_items / 4));
+    splits = env_int("XC_CT_SPLITS", (int)splits);
     splits = std::max(1L, std::min(splits, 512L));
     p->ct_items_per_split = cdivl(p->ct_items, splits);
     p->ct_splits = (int)cdivl(p->ct_items, p->ct_items_per_split);
@@ -555,37 +673,43 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const long Q = (long)d->H * d->W * d->Cout;
   const int bk = pl.bp_ksteps * 16;
   CUtensorMap ma, mb;
-  const uint64_t da[2] = {(uint64_t)Q, (uint64_t)d->B}, db[2] = {(uint64_t)d->B, (uint64_t)d->r};
-  const uint64_t sa[1] = {(uint64_t)Q * 2}, sb[1] = {(uint64_t)d->B * 2};
-  const uint32_t box_a[2] = {64, (uint32_t)bk};
-  const uint32_t box_b[2] = {64, (uint32_t)pl.bp_tile_n};     // 128-byte rows whatever bk is (zero fill past B)
-  if (!make_map(&ma, dY, 2, da, sa, box_a) || !make_map(&mb, S_bf16, 2, db, sb, box_b)) return XCONV_ERR_CUDA;
+  // A = S (bfloat16) [r][B], k = b contiguous; B operand = dY [B][Q], q contiguous (MN-major tile)
+  const uint64_t da[2] = {(uint64_t)d->B, (uint64_t)d->r}, db[2] = {(uint64_t)Q, (uint64_t)d->B};
+  const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[1] = {(uint64_t)Q * 2};
+  const uint32_t box_a[2] = {64, (uint32_t)TILE_M};    // 128-byte rows whatever bk is (zero fill past B)
+  const uint32_t box_b[2] = {64, (uint32_t)bk};
+  if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 2, db, sb, box_b)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_BACKPROBE;
   p.tile_n = pl.bp_tile_n;
-  p.tmem_cols = pow2_cols(pl.bp_tile_n);
+  p.m_sub = 1;
+  p.acc_bufs = 2;
+  p.tmem_cols = pow2_cols(2 * pl.bp_tile_n);
   p.stages = pl.bp_stages;
   p.ksteps = pl.bp_ksteps;
-  p.a_boxes = 2;
-  p.b_boxes = 1;
-  p.a_box_bytes = (uint32_t)bk * 128;
-  p.a_stage_bytes = 2 * p.a_box_bytes;
-  p.b_stage_bytes = (uint32_t)pl.bp_tile_n * 128;
-  p.b_box_bytes = p.b_stage_bytes;
+  p.a_boxes = 1;
+  p.b_boxes = pl.bp_tile_n / 64;
+  p.a_sub_bytes = TILE_M * 128;
+  p.a_stage_bytes = p.a_sub_bytes;
+  p.a_box_bytes = p.a_sub_bytes;
+  p.b_box_bytes = (uint32_t)bk * 128;
+  p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  p.a_mn_major = 1;
-  p.b_mn_major = 0;
-  p.a_lbo = p.a_box_bytes;
-  p.tiles_m = pl.bp_tiles_q;
-  p.tiles_n = pl.bp_tiles_r;
+  p.a_mn_major = 0;
+  p.b_mn_major = 1;
+  p.b_lbo = p.b_box_bytes;
+  p.tiles_m = pl.bp_tiles_r;
+  p.tiles_n = pl.bp_tiles_q;
+  p.taps = 1;
   p.kblocks = cdivl(d->B, bk);
   p.kblocks_per_split = p.kblocks;
-  p.rows = Q;
-  p.cols = d->r;
+  p.units = (long)pl.bp_tiles_q * pl.bp_tiles_r;
+  p.rows = d->r;
+  p.cols = Q;
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  return launch(ma, mb, p, dim3((unsigned)((long)pl.bp_tiles_q * pl.bp_tiles_r), 1), st);
+  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS * env_int("XC_BP_CTAS", 1)), st);
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
@@ -602,13 +726,16 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   TcParams p{};
   p.mode = MODE_CONTRACT;
   p.tile_n = pl.ct_tile_n;
-  p.tmem_cols = pow2_cols(pl.ct_tile_n);
+  p.m_sub = pl.ct_m_sub;
+  p.acc_bufs = 1;
+  p.tmem_cols = pow2_cols(pl.ct_tile_n * pl.ct_m_sub);
   p.stages = pl.ct_stages;
   p.ksteps = bk / 16;
   p.a_boxes = 2;
   p.b_boxes = (int)cdivl(pl.ct_tile_n, 64);
   p.a_box_bytes = p.b_box_bytes = (uint32_t)bk * 128;
-  p.a_stage_bytes = 2 * p.a_box_bytes;
+  p.a_sub_bytes = 2 * p.a_box_bytes;
+  p.a_stage_bytes = (uint32_t)pl.ct_m_sub * p.a_sub_bytes;
   p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.a_mn_major = p.b_mn_major = 1;
@@ -616,8 +743,10 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.b_lbo = p.b_box_bytes;
   p.tiles_m = pl.ct_tiles_m;
   p.tiles_n = pl.ct_tiles_n;
+  p.taps = T;
   p.kblocks = pl.ct_items;
   p.kblocks_per_split = pl.ct_items_per_split;
+  p.units = (long)pl.ct_tiles_m * pl.ct_tiles_n * T * pl.ct_splits;
   p.patch_w = pl.patch_w;
   p.patch_h = pl.patch_h;
   p.patches_x = pl.patches_x;
@@ -629,11 +758,11 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.Cin = d->Cin;
   p.part = reinterpret_cast<float*>(part);
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  xconv_status s = launch(ma, mb, p, dim3((unsigned)(pl.ct_tiles_m * pl.ct_tiles_n * T), (unsigned)pl.ct_splits), st);
+  xconv_status s = launch(ma, mb, p, (unsigned)std::min<long>(p.units, 4L * NUM_SMS), st);
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T * d->Cin;
-  reduce_contract_partials<<<(unsigned)cdivl(count, 256), 256, 0, st>>>(p.part, dW, count, pl.ct_splits,
-                                                                       1.0f / (float)d->r, d->chan_scale, d->Cin);
+  reduce_contract_partials<<<(unsigned)cdivl(count / 4, 256), 256, 0, st>>>(p.part, dW, count, pl.ct_splits,
+                                                                           1.0f / (float)d->r, d->chan_scale, d->Cin);
   count_launch();
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
