@@ -2,6 +2,7 @@
 #include "../../include/xconv.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -25,11 +26,14 @@ static xconv_status check_launch() {
   return XCONV_OK;
 }
 
-static xconv_status clear_status(void* ws, cudaStream_t st) {
-  cudaError_t e = cudaMemsetAsync(ws, 0, 16, st);
-  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
-  return XCONV_OK;
+// A fresh non-zero tag per API call (see the workspace header in common.cuh).
+static std::atomic<unsigned int> g_call_tag{0x51u};
+thread_local unsigned int g_tag = 1u;
+static void new_call() {
+  g_launches = 0;
+  g_tag = g_call_tag.fetch_add(2u) | 1u;
 }
+unsigned int call_tag() { return g_tag; }
 
 static xconv_status validate(const xconv_desc* d) {
   if (!d) return XCONV_ERR_INVALID_ARG;
@@ -133,7 +137,6 @@ static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z
   if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   char* w = static_cast<char*>(ws);
-  if (clear_status(w, st) != XCONV_OK) return XCONV_ERR_CUDA;
   if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st);
   return d->dtype == XCONV_F32 ? run_sketch_simt<float>(d, p, X, Z, S, w, st)
                                : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
@@ -200,9 +203,9 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
   if (p.tc_bp) {
     const long n = (long)d->r * d->B;
     bf16* Sb = reinterpret_cast<bf16*>(w + p.sb_off);
-    cast_f32_to_bf16<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, Sb, n);
-    xconv_status s = check_launch();
-    if (s != XCONV_OK) return s;
+    cudaError_t e = launch_pdl(cast_f32_to_bf16, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, Sb, n);
+    ++g_launches;
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
     return tc_run_backprobe(d, p.t, Sb, dY, L, w, st);
   }
   return d->dtype == XCONV_F32 ? run_backprobe_simt<float, float>(d, S, dY, L, st)
@@ -228,7 +231,6 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
   xconv_status s = check_ws(ws, ws_bytes, p.bytes);
   if (s != XCONV_OK) return s;
   char* w = static_cast<char*>(ws);
-  if (clear_status(w, st) != XCONV_OK) return XCONV_ERR_CUDA;
   s = run_backprobe(d, p, S, dY, w + p.l_off, w, st);
   if (s != XCONV_OK) return s;
   return run_contract(d, p, w + p.l_off, Z, dW, w, st);
@@ -272,7 +274,7 @@ xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, 
   if (s != XCONV_OK) return s;
   if (!X || !Z || !sketch) return XCONV_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(Z) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
-  g_launches = 0;
+  new_call();
   return run_sketch(desc, X, Z, sketch, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -287,7 +289,7 @@ xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W,
   if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  g_launches = 0;
+  new_call();
   s = run_conv(desc, false, X, W, Y, st);
   if (s != XCONV_OK) return s;
   return run_sketch(desc, X, Z, sketch, ws, ws_bytes, st);
@@ -300,7 +302,7 @@ xconv_status xconv_wgrad(const xconv_desc* desc, const float* sketch, const void
   if (!sketch || !dY || !Z || !dW) return XCONV_ERR_INVALID_ARG;
   if (!aligned16(sketch) || !aligned16(dY) || !aligned16(Z) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
   if (desc->chan_scale && (reinterpret_cast<uintptr_t>(desc->chan_scale) & 3u)) return XCONV_ERR_ALIGNMENT;
-  g_launches = 0;
+  new_call();
   return run_wgrad(desc, sketch, dY, Z, dW, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -319,8 +321,7 @@ xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const 
   s = check_ws(ws, ws_bytes, p.bytes);
   if (s != XCONV_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  g_launches = 0;
-  if (clear_status(ws, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  new_call();
   return run_backprobe(desc, p, sketch, dY, L, static_cast<char*>(ws), st);
 }
 
@@ -335,8 +336,7 @@ xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z
   s = check_ws(ws, ws_bytes, p.bytes);
   if (s != XCONV_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  g_launches = 0;
-  if (clear_status(ws, st) != XCONV_OK) return XCONV_ERR_CUDA;
+  new_call();
   return run_contract(desc, p, L, Z, dW, static_cast<char*>(ws), st);
 }
 
@@ -348,8 +348,7 @@ xconv_status xconv_dgrad(const xconv_desc* desc, const void* dY, const void* W, 
   if (!aligned16(dY) || !aligned16(W) || !aligned16(dX)) return XCONV_ERR_ALIGNMENT;
   if (!ws || ws_bytes < WS_HEADER) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
-  g_launches = 0;
-  if (clear_status(ws, static_cast<cudaStream_t>(cuda_stream)) != XCONV_OK) return XCONV_ERR_CUDA;
+  new_call();
   return run_conv(desc, true, dY, W, dX, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -397,7 +396,7 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
     g_last_cuda_error = (int)e;
     return XCONV_ERR_CUDA;
   }
-  g_launches = 0;
+  new_call();
   float* S = reinterpret_cast<float*>(base + a.s);
   float* dW = reinterpret_cast<float*>(base + a.dw);
   s = run_sketch(desc, base + a.x, base + a.z, S, base + a.ws, a.ws_bytes, st);
@@ -415,12 +414,12 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
 
 xconv_status xconv_workspace_status(const void* ws, void* cuda_stream) {
   if (!ws) return XCONV_ERR_INVALID_ARG;
-  unsigned int word = 0;
+  unsigned int word[2] = {0, 0};
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e = cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, st);
+  cudaError_t e = cudaMemcpyAsync(word, ws, sizeof(word), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
-  return word == WS_OK ? XCONV_OK : XCONV_ERR_TIMEOUT;
+  return (word[0] != WS_OK && word[0] == word[1]) ? XCONV_ERR_TIMEOUT : XCONV_OK;
 }
 
 int xconv_last_launch_count(void) { return g_launches; }

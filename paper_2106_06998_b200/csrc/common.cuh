@@ -9,8 +9,33 @@ namespace xconv {
 
 typedef __nv_bfloat16 bf16;
 
-// Codes a kernel may leave in the first word of the workspace.
-enum : unsigned int { WS_OK = 0u, WS_TIMEOUT = 0x7157u };
+// Workspace header (two 32-bit words).  Every API call draws a fresh non-zero tag; word 1 holds the
+// tag of the last call that ran a pipelined kernel, word 0 the tag of a call in which a bounded wait
+// ran out.  The last call timed out iff the two are equal and non-zero -- so the header never has to
+// be cleared, whatever the scratch memory held before.
+enum : unsigned int { WS_OK = 0u };
+
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while the kernel before
+// it in the stream is still draining; it must call pdl_wait() before it reads or overwrites anything
+// that kernel touches.  pdl_trigger() lets the kernel after this one start its own preamble early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 __device__ __forceinline__ float to_f(float v) { return v; }
 __device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }

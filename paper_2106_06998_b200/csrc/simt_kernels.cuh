@@ -292,6 +292,8 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
 
 // float -> bfloat16 copy (the sketch as tensor-core operand).
 static __global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
+  pdl_trigger();
+  pdl_wait();
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) out[i] = __float2bfloat16_rn(in[i]);
 }

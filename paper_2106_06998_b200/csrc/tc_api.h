@@ -42,5 +42,6 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const vo
 // bookkeeping shared with the ABI layer
 void count_launch();
 void set_cuda_error(int e);
+unsigned int call_tag();   // tag of the API call in progress on this host thread
 
 }  // namespace xconv

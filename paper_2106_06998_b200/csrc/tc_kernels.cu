@@ -15,7 +15,7 @@
 // Structure of a CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = epilogue (one TMEM lane quadrant each).  A ring of shared-memory stages is handed
 // from producer to issuer with mbarriers; tcgen05.commit returns stages and signals the epilogue.
-// Every wait is bounded: on expiry the CTA records WS_TIMEOUT in the workspace status word, drains
+// Every wait is bounded: on expiry the CTA records the call's tag in the workspace header, drains
 // its outstanding copies (bounded again), frees its tensor memory and returns.
 #include "tc_api.h"
 
@@ -38,7 +38,6 @@ struct TcParams {
   int acc_bufs;            // accumulator sets in tensor memory (2 = epilogue overlaps the next unit)
   int tmem_cols;           // power of two >= max(32, tile_n * m_sub * acc_bufs)
   int stages;
-  int burst;               // k-blocks the producer issues back to back (<= stages)
   int ksteps;              // UMMA k-steps (of 16) per stage
   uint32_t a_stage_bytes, b_stage_bytes, tx_bytes;
   int a_boxes, b_boxes;    // TMA boxes per stage: A per 128-row tile, B in all
@@ -57,7 +56,8 @@ struct TcParams {
   bf16* L;                 // BACKPROBE: [r][Q]
   long Q;
   int T, Cin;              // CONTRACT output indexing
-  unsigned int* status;
+  unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
+  unsigned int tag;        // tag of this call
 };
 
 // ------------------------------------------------------------------------------------ PTX wrappers
@@ -84,8 +84,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait: about one second after a short spin.  Returns false (and records the code) on expiry.
-__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* status) {
+// Bounded wait: about one second after a short spin.  Returns false (and records the tag) on expiry.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, unsigned int* status, unsigned int tag) {
   for (int i = 0; i < 4096; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
@@ -93,10 +93,14 @@ __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned 
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (global_ns() - t0 > 1000000000ull) {
-      atomicExch(status, (unsigned int)WS_TIMEOUT);
+      atomicExch(status, tag);
       return false;
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* status, unsigned int tag) {
+  if (mbar_try_wait(bar, parity)) return true;       // the common case costs one instruction
+  return mbar_wait_slow(bar, parity, status, tag);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
@@ -104,12 +108,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4,
                                             uint64_t* bar) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
-      : "memory");
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4),
+        "r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
@@ -126,14 +135,19 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem], bfloat16 inputs, float accumulate; issued by one thread.
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem], bfloat16 inputs, float accumulate; issued by one thread.  The two
+// shared-memory descriptors come as 32-bit halves: only the low half (start address) changes between
+// k-steps, so the issuing thread -- whose own instruction stream is the critical path of the CTA when
+// the tiles are small -- spends one 32-bit add per operand and k-step.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 // mbarrier arrive once every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -162,13 +176,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr) : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
-// Byte offsets are encoded without their 4 low bits.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
 }
 
 constexpr int TILE_M = 128;
@@ -215,16 +222,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ uint32_t tmem_slot;
   __shared__ int go;
 
-  // an earlier CTA gave up: leave at once (one thread reads the word so that the whole CTA agrees)
-  if (threadIdx.x == 0) go = (*reinterpret_cast<volatile unsigned int*>(p.status) == WS_OK) ? 1 : 0;
-  __syncthreads();
-  if (!go) return;
-
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   const int acc_cols = p.tile_n * p.m_sub;                                    // columns of one accumulator set
 
+  // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
@@ -234,80 +237,105 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     prefetch_tmap(&map_b);
   }
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
+  pdl_trigger();
+  pdl_wait();                              // from here on the previous kernel's results are visible
+  if (threadIdx.x == 0) {
+    // a CTA of this call gave up earlier: skip the work (one thread reads so that the whole CTA agrees)
+    go = (*reinterpret_cast<volatile unsigned int*>(p.status) != p.tag) ? 1 : 0;
+    if (blockIdx.x == 0) reinterpret_cast<volatile unsigned int*>(p.status)[1] = p.tag;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_slot);
 
-  if (warp == 0) {
+  if (!go) {
+    // fall through to the teardown
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
+    // One thread; its loop is kept free of divisions (coordinates advance incrementally).
     if (lane == 0) {
+      const int stages = p.stages;
+      int s = 0;                           // stage to fill next
+      long fill = 0;                       // how often the ring has wrapped
       long it = 0;                         // stages filled so far, across units
       bool ok = true;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
         const int row0 = w.tm * p.m_sub * TILE_M;
-        for (int i = 0; i < w.nkb; ++i, ++it) {
-          const int s = (int)(it % p.stages);
-          if (p.burst > 1 && (i % p.burst) == 0) {
-            // issue `burst` consecutive k-blocks back to back: their rows are adjacent in memory, so
-            // the requests reach DRAM together and share open pages
-            const int n = min(p.burst, w.nkb - i);
-            for (int g = 1; g < n && ok; ++g) {
-              const long t = it + g;
-              if (t >= p.stages) ok = mbar_wait(&empty_bar[t % p.stages], (uint32_t)(((t / p.stages) - 1) & 1), p.status);
-            }
+        const int col0 = w.tn * p.tile_n;
+        // running coordinates of the k-block
+        int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0;
+        if (p.mode == MODE_SKETCH) kc = (int)(w.kb0 * 64);
+        else if (p.mode == MODE_BACKPROBE) kc = (int)w.kb0 * p.ksteps * 16;
+        else {
+          long q = w.kb0;
+          px = (int)(q % p.patches_x); q /= p.patches_x;
+          py = (int)(q % p.patches_y); q /= p.patches_y;
+          pj = (int)q;
+          const int ks = 2 * p.pad + 1;
+          dy = w.tap / ks - p.pad;
+          dx = w.tap % ks - p.pad;
+        }
+        for (int i = 0; i < w.nkb; ++i) {
+          if (fill > 0) {
+            ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
             if (!ok) break;
           }
-          if (it >= p.stages) ok = mbar_wait(&empty_bar[s], (uint32_t)(((it / p.stages) - 1) & 1), p.status);
-          if (!ok) break;
-          const long kb = w.kb0 + i;
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
           const uint32_t b_dst = a_dst + p.a_stage_bytes;
           mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
           if (p.mode == MODE_SKETCH) {
-            for (int mt = 0; mt < p.m_sub; ++mt)
-              tma_load_2d(a_dst + mt * p.a_sub_bytes, &map_a, (int)(kb * 64), row0 + mt * TILE_M, &full_bar[s]);
-            tma_load_2d(b_dst, &map_b, (int)(kb * 64), w.tn * p.tile_n, &full_bar[s]);
+            // one box per operand: 128*m_sub rows of A, tile_n rows of B, 64 k each
+            tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
+            tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
+            kc += 64;
           } else if (p.mode == MODE_BACKPROBE) {
-            const int brow = (int)kb * p.ksteps * 16;
-            tma_load_2d(a_dst, &map_a, brow, row0, &full_bar[s]);
-            for (int bx = 0; bx < p.b_boxes; ++bx)
-              tma_load_2d(b_dst + bx * p.b_box_bytes, &map_b, w.tn * p.tile_n + bx * 64, brow, &full_bar[s]);
+            tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
+            // dY tile as one 3-d box (64 positions, k rows, tile_n/64 column groups)
+            tma_load_3d(b_dst, &map_b, 0, kc, col0 >> 6, &full_bar[s]);
+            kc += p.ksteps * 16;
           } else {
-            long q = kb;
-            const int px = (int)(q % p.patches_x); q /= p.patches_x;
-            const int py = (int)(q % p.patches_y); q /= p.patches_y;
-            const int j = (int)q;
-            const int ks = 2 * p.pad + 1;
-            const int dy = w.tap / ks - p.pad, dx = w.tap % ks - p.pad;
+            // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
-            for (int mt = 0; mt < p.m_sub; ++mt)
-              for (int bx = 0; bx < p.a_boxes; ++bx)
-                tma_load_4d(a_dst + mt * p.a_sub_bytes + bx * p.a_box_bytes, &map_a, row0 + mt * TILE_M + bx * 64,
-                            x0, y0, j, &full_bar[s]);
-            for (int bx = 0; bx < p.b_boxes; ++bx)
-              tma_load_4d(b_dst + bx * p.b_box_bytes, &map_b, w.tn * p.tile_n + bx * 64, x0 + dx, y0 + dy, j,
-                          &full_bar[s]);
+            tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> 6, pj, &full_bar[s]);
+            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> 6, pj, &full_bar[s]);
+            if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
           }
+          ++it;
+          if (++s == stages) { s = 0; ++fill; }
         }
       }
       // drain: every copy issued must have landed in this CTA's shared memory before it exits
       // (immediate on the normal path, bounded on the failure path)
-      for (long i = max(0L, it - p.stages); i < it; ++i)
-        if (!mbar_wait(&full_bar[i % p.stages], (uint32_t)((i / p.stages) & 1), p.status)) break;
+      for (long i = max(0L, it - stages); i < it; ++i)
+        if (!mbar_wait(&full_bar[i % stages], (uint32_t)((i / stages) & 1), p.status, p.tag)) break;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
+    // One thread.  With small tiles the time between two tcgen05.mma is set by this thread's own
+    // instruction stream, so the loop carries descriptors as 32-bit halves and does no division.
     if (lane == 0) {
       const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn_major << 15) |
                              ((uint32_t)p.b_mn_major << 16) | ((uint32_t)(p.tile_n >> 3) << 17) |
                              ((uint32_t)(TILE_M >> 4) << 24);
-      // K-major: 8-row groups 1024 B apart, k-step = 32 B inside the swizzled row.
+      // Shared-memory descriptor (128-byte swizzle): start address >> 4 | (lbo >> 4) << 16 in the low
+      // word; (sbo >> 4) | version 1 << 14 | layout SWIZZLE_128B << 29 in the high word.
+      // K-major: 8-row groups 1024 B apart (sbo), k-step = 32 B inside the swizzled row.
       // MN-major: 8-row (k) groups 1024 B apart, 64-column blocks `lbo` apart, k-step = 16 rows = 2048 B.
-      const uint32_t a_step = p.a_mn_major ? 2048u : 32u, b_step = p.b_mn_major ? 2048u : 32u;
-      const uint32_t a_lbo = p.a_mn_major ? p.a_lbo : 16u, b_lbo = p.b_mn_major ? p.b_lbo : 16u;
-      long it = 0, lu = 0;
+      const uint32_t a_step = (p.a_mn_major ? 2048u : 32u) >> 4, b_step = (p.b_mn_major ? 2048u : 32u) >> 4;
+      const uint32_t a_lo0 = ((p.a_mn_major ? p.a_lbo : 16u) >> 4) << 16;
+      const uint32_t b_lo0 = ((p.b_mn_major ? p.b_lbo : 16u) >> 4) << 16;
+      const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t a_sub = p.a_sub_bytes >> 4;
+      const uint32_t a_stage16 = p.a_stage_bytes >> 4, stage16 = stage_bytes >> 4;
+      const uint32_t base16 = (tiles_base & 0x3FFFFu) >> 4;
+      const int ksteps = p.ksteps, stages = p.stages;
+      const bool two = p.m_sub == 2;
+      const uint32_t tile_n = (uint32_t)p.tile_n;
+      int s = 0;
+      uint32_t full_parity = 0, s16 = base16;
+      long lu = 0;
       bool ok = true;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
         const Unit w = decode_unit(p, u);
@@ -315,26 +343,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int buf = (int)(lu % p.acc_bufs);
         const long use = lu / p.acc_bufs;
         if (use > 0) {                      // the epilogue must have emptied this accumulator set
-          ok = mbar_wait(&tmem_empty_bar[buf], (uint32_t)((use - 1) & 1), p.status);
+          ok = mbar_wait(&tmem_empty_bar[buf], (uint32_t)((use - 1) & 1), p.status, p.tag);
           if (!ok) break;
           tc_fence_after();
         }
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
-        for (int i = 0; i < w.nkb; ++i, ++it) {
-          const int s = (int)(it % p.stages);
-          ok = mbar_wait(&full_bar[s], (uint32_t)((it / p.stages) & 1), p.status);
+        uint32_t acc = 0;
+        for (int i = 0; i < w.nkb; ++i) {
+          ok = mbar_wait(&full_bar[s], full_parity, p.status, p.tag);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a_src = tiles_base + (uint32_t)s * stage_bytes;
-          const uint32_t b_src = a_src + p.a_stage_bytes;
-          for (int k = 0; k < p.ksteps; ++k) {
-            const uint64_t db = make_desc(b_src + k * b_step, b_lbo, 1024u);
-            for (int mt = 0; mt < p.m_sub; ++mt) {
-              const uint64_t da = make_desc(a_src + mt * p.a_sub_bytes + k * a_step, a_lbo, 1024u);
-              umma_bf16(d_tmem + (uint32_t)(mt * p.tile_n), da, db, idesc, (i > 0 || k > 0) ? 1u : 0u);
-            }
+          uint32_t a_lo = a_lo0 | s16;
+          uint32_t b_lo = b_lo0 | (s16 + a_stage16);
+          for (int k = 0; k < ksteps; ++k) {
+            umma_bf16(d_tmem, a_lo, desc_hi, b_lo, desc_hi, idesc, acc);
+            if (two) umma_bf16(d_tmem + tile_n, a_lo + a_sub, desc_hi, b_lo, desc_hi, idesc, acc);
+            acc = 1u;
+            a_lo += a_step;
+            b_lo += b_step;
           }
           umma_commit(&empty_bar[s]);        // stage s may be refilled once these MMAs have read it
+          s16 += stage16;
+          if (++s == stages) { s = 0; s16 = base16; full_parity ^= 1u; }
         }
         if (ok) umma_commit(&tmem_full_bar[buf]);
       }
@@ -349,7 +379,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int buf = (int)(lu % p.acc_bufs);
       const long use = lu / p.acc_bufs;
       if (w.nkb > 0) {
-        if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status);
+        if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status, p.tag);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         if (!ok) break;
         tc_fence_after();
@@ -431,6 +461,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 __global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S,
                                                               int r, int B, int splits, int swapped) {
   __shared__ float acc[4][64];
+  pdl_trigger();
+  pdl_wait();
   const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
   const long count = (long)r * B;
   const long i = (long)blockIdx.x * 64 + o;           // index in the layout of `part`
@@ -452,8 +484,10 @@ __global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __res
 __global__ void __launch_bounds__(256) reduce_contract_partials(const float* __restrict__ part, float* __restrict__ out,
                                                                 long count, int splits, float alpha,
                                                                 const float* __restrict__ chan_scale, int period) {
+  pdl_trigger();
+  pdl_wait();
   const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (i >= count) return;                              // count is a multiple of 4 (Cin % 8 == 0)
+  if (i >= count) return;                              // count is a multiple of 4 (Cin % 64 == 0)
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
   for (int k = 0; k < splits; ++k) {
@@ -520,16 +554,13 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
 static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
                            cudaStream_t st) {
   const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
-  if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512) return XCONV_ERR_UNSUPPORTED;
-  {
-    cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
-    if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
-  }
+  if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
+  cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
+  if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   TcParams q = p;
-  q.burst = std::min(env_int("XC_BURST", 1), q.stages);   // TUNING
-  tc_gemm_kernel<<<grid, TC_THREADS, smem, st>>>(ma, mb, q);
+  q.tag = call_tag();
+  e = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, q);
   count_launch();
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
 }
@@ -572,7 +603,7 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   const uint64_t da[2] = {(uint64_t)K, (uint64_t)rows}, db[2] = {(uint64_t)K, (uint64_t)cols};
   const uint64_t sa[1] = {(uint64_t)K * 2};
   // full boxes always: rows and k positions past the tensor are zero-filled by the TMA unit
-  const uint32_t box_a[2] = {64, (uint32_t)TILE_M};
+  const uint32_t box_a[2] = {64, (uint32_t)(TILE_M * pl.m_sub)};
   const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
   if (!make_map(&ma, A, 2, da, sa, box_a) || !make_map(&mb, Bm, 2, db, sa, box_b)) return XCONV_ERR_CUDA;
   TcParams p{};
@@ -602,9 +633,9 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   xconv_status s = launch(ma, mb, p, (unsigned)p.units, st);
   if (s != XCONV_OK) return s;
   const long count = (long)d->r * d->B;
-  reduce_sketch_partials<<<(unsigned)cdivl(count, 64), 256, 0, st>>>(p.part, S, d->r, d->B, pl.splits, pl.swap);
+  cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(count, 64)), dim3(256), 0, st, p.part, S,
+                             d->r, d->B, pl.splits, pl.swap);
   count_launch();
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
 }
@@ -632,7 +663,7 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   int mask = 0;
   const long Q = (long)d->H * d->W * d->Cout;
   // back-probe: D[j, q], rows = r, cols = Q, k = B
-  if (Q % 8 == 0 && d->B % 8 == 0 && Q >= 2048 && Q < 2000000000L) {
+  if (Q % 64 == 0 && d->B % 8 == 0 && Q >= 2048 && Q < 2000000000L) {
     mask |= 1;
     p->bp_tile_n = env_int("XC_BP_TILEN", 256);
     p->bp_tiles_q = (int)cdivl(Q, p->bp_tile_n);
@@ -643,7 +674,7 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
-  if (d->Cout % 8 == 0 && d->Cin % 8 == 0 && d->Cout >= 64 && d->Cin >= 64 && (long)d->H * d->W >= 16) {
+  if (d->Cout % 64 == 0 && d->Cin % 64 == 0 && (long)d->H * d->W >= 16) {
     mask |= 2;
     pick_patch(d->H, d->W, &p->patch_w, &p->patch_h);
     p->patches_x = (int)cdivl(d->W, p->patch_w);
@@ -674,11 +705,14 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const int bk = pl.bp_ksteps * 16;
   CUtensorMap ma, mb;
   // A = S (bfloat16) [r][B], k = b contiguous; B operand = dY [B][Q], q contiguous (MN-major tile)
-  const uint64_t da[2] = {(uint64_t)d->B, (uint64_t)d->r}, db[2] = {(uint64_t)Q, (uint64_t)d->B};
-  const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[1] = {(uint64_t)Q * 2};
+  // dY as (64 positions, B rows, Q/64 groups of 64 positions): one box fetches the whole [bk x tile_n] tile
+  // as tile_n/64 consecutive blocks of 128-byte rows
+  const uint64_t da[2] = {(uint64_t)d->B, (uint64_t)d->r};
+  const uint64_t db[3] = {64, (uint64_t)d->B, (uint64_t)(Q / 64)};
+  const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[2] = {(uint64_t)Q * 2, 128};
   const uint32_t box_a[2] = {64, (uint32_t)TILE_M};    // 128-byte rows whatever bk is (zero fill past B)
-  const uint32_t box_b[2] = {64, (uint32_t)bk};
-  if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 2, db, sb, box_b)) return XCONV_ERR_CUDA;
+  const uint32_t box_b[3] = {64, (uint32_t)bk, (uint32_t)(pl.bp_tile_n / 64)};
+  if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 3, db, sb, box_b)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_BACKPROBE;
   p.tile_n = pl.bp_tile_n;
@@ -717,12 +751,15 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   const int T = d->KH * d->KW;
   const int bk = pl.patch_w * pl.patch_h;
   CUtensorMap ma, mb;
-  const uint64_t da[4] = {(uint64_t)d->Cout, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)d->r};
-  const uint64_t sa[3] = {(uint64_t)d->Cout * 2, (uint64_t)d->W * d->Cout * 2, (uint64_t)d->H * d->W * d->Cout * 2};
-  const uint64_t db[4] = {(uint64_t)d->Cin, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)d->r};
-  const uint64_t sb[3] = {(uint64_t)d->Cin * 2, (uint64_t)d->W * d->Cin * 2, (uint64_t)d->H * d->W * d->Cin * 2};
-  const uint32_t box[4] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1};
-  if (!make_map(&ma, L, 4, da, sa, box) || !make_map(&mb, Z, 4, db, sb, box)) return XCONV_ERR_CUDA;
+  // (64 channels, x, y, groups of 64 channels, probe): one box = a whole [patch x channels] tile laid
+  // out as consecutive blocks of 128-byte rows, one block per channel group
+  const uint64_t da[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cout / 64), (uint64_t)d->r};
+  const uint64_t sa[4] = {(uint64_t)d->Cout * 2, (uint64_t)d->W * d->Cout * 2, 128, (uint64_t)d->H * d->W * d->Cout * 2};
+  const uint64_t db[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cin / 64), (uint64_t)d->r};
+  const uint64_t sb[4] = {(uint64_t)d->Cin * 2, (uint64_t)d->W * d->Cin * 2, 128, (uint64_t)d->H * d->W * d->Cin * 2};
+  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)(2 * pl.ct_m_sub), 1};
+  const uint32_t box_b[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)cdivl(pl.ct_tile_n, 64), 1};
+  if (!make_map(&ma, L, 5, da, sa, box_a) || !make_map(&mb, Z, 5, db, sb, box_b)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_CONTRACT;
   p.tile_n = pl.ct_tile_n;
@@ -761,10 +798,9 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   xconv_status s = launch(ma, mb, p, (unsigned)std::min<long>(p.units, 4L * NUM_SMS), st);
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T * d->Cin;
-  reduce_contract_partials<<<(unsigned)cdivl(count / 4, 256), 256, 0, st>>>(p.part, dW, count, pl.ct_splits,
-                                                                           1.0f / (float)d->r, d->chan_scale, d->Cin);
+  cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(count / 4, 256)), dim3(256), 0, st, p.part,
+                             dW, count, pl.ct_splits, 1.0f / (float)d->r, d->chan_scale, d->Cin);
   count_launch();
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
 }
