@@ -191,8 +191,17 @@ static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* i
   return check_launch();
 }
 
+// Scratch of the convolution calls: the header, and for the tensor-core dgrad the transposed weights.
+static size_t conv_ws_bytes(const xconv_desc* d, bool dgrad) {
+  TcConvPlan t;
+  if (tc_plan_conv(d, dgrad, &t)) return WS_HEADER + align_up(t.wt_bytes, 256);
+  return WS_HEADER;
+}
+
 static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, const void* Wt, void* out,
-                             cudaStream_t st) {
+                             char* ws, cudaStream_t st) {
+  TcConvPlan t;
+  if (tc_plan_conv(d, dgrad, &t)) return tc_run_conv(d, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
   return d->dtype == XCONV_F32 ? run_conv_simt<float>(d, dgrad, in, Wt, out, st)
                                : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
 }
@@ -252,7 +261,7 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
     case XCONV_OP_FORWARD:
     case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
     case XCONV_OP_WGRAD: return plan_wgrad(desc).bytes;
-    case XCONV_OP_DGRAD: return WS_HEADER;
+    case XCONV_OP_DGRAD: return conv_ws_bytes(desc, true);
     default: return 0;
   }
 }
@@ -263,7 +272,10 @@ int xconv_engine_for(const xconv_desc* desc, int op) {
     case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_WGRAD: return plan_wgrad(desc).tc_ct ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_FORWARD:
-    case XCONV_OP_DGRAD: return XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_DGRAD: {
+      TcConvPlan t;
+      return tc_plan_conv(desc, op == XCONV_OP_DGRAD, &t) ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    }
     default: return XCONV_ENGINE_NONE;
   }
 }
@@ -290,7 +302,7 @@ xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W,
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   new_call();
-  s = run_conv(desc, false, X, W, Y, st);
+  s = run_conv(desc, false, X, W, Y, static_cast<char*>(ws), st);
   if (s != XCONV_OK) return s;
   return run_sketch(desc, X, Z, sketch, ws, ws_bytes, st);
 }
@@ -346,10 +358,10 @@ xconv_status xconv_dgrad(const xconv_desc* desc, const void* dY, const void* W, 
   if (s != XCONV_OK) return s;
   if (!dY || !W || !dX) return XCONV_ERR_INVALID_ARG;
   if (!aligned16(dY) || !aligned16(W) || !aligned16(dX)) return XCONV_ERR_ALIGNMENT;
-  if (!ws || ws_bytes < WS_HEADER) return XCONV_ERR_WORKSPACE;
+  if (!ws || ws_bytes < conv_ws_bytes(desc, true)) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   new_call();
-  return run_conv(desc, true, dY, W, dX, static_cast<cudaStream_t>(cuda_stream));
+  return run_conv(desc, true, dY, W, dX, static_cast<char*>(ws), static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Arena layout of the host-buffer entry point: X | dY | Z | S | dW | workspace, each 256-aligned.

@@ -19,7 +19,7 @@ struct TcSketchPlan {
 
 struct TcWgradPlan {
   // back-probe
-  int bp_tile_n, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps;
+  int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps;
   // contraction
   int ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
   int patch_h, patch_w, patches_y, patches_x;
@@ -27,10 +27,19 @@ struct TcWgradPlan {
   size_t part_bytes;
 };
 
+struct TcConvPlan {
+  int tile_n, tiles_n, stages, patch_w, patch_h, patches_x, patches_y;
+  size_t wt_bytes;     // dgrad only: transposed, flipped copy of the weights
+};
+
 // Fill the plan and say whether the tcgen05 kernels cover this layer.  tc_plan_wgrad returns a mask:
 // bit 0 = back-probe covered, bit 1 = contraction covered.
 bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p);
 int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p);
+
+bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p);
+xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& p, bool dgrad, const void* in, const void* W,
+                         void* out, char* ws_head, char* wt, cudaStream_t st);
 
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const void* X, const void* Z, float* S,
                            char* ws_head, char* part, cudaStream_t st);

@@ -11,6 +11,10 @@
 //             reduction runs over image patches, and the offset is added to the patch coordinates of
 //             the TMA box of Z -- out-of-image rows are zero-filled by the TMA unit, which is exactly
 //             the zero padding of the convolution.  No shifted or im2col copy of Z is ever made.
+//   CONV      Y = conv(X, w)  (forward step 1, Eq. 5) and, with transposed and flipped weights, the exact
+//             dX: D[pixel, co] = sum_{offset, ci} In[pixel + offset, ci] W[co, offset, ci] for one image
+//             patch per work unit; both tiles K-major (channels contiguous), the reduction runs over
+//             (offset, 64-channel block), and the offset again moves the TMA box of the input.
 //
 // Structure of a CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
 // warps 2..5 = epilogue (one TMEM lane quadrant each).  A ring of shared-memory stages is handed
@@ -23,13 +27,12 @@
 #include <cudaTypedefs.h>
 
 #include <algorithm>
-#include <cstdlib>
 
 #include "common.cuh"
 
 namespace xconv {
 
-enum : int { MODE_SKETCH = 0, MODE_BACKPROBE = 1, MODE_CONTRACT = 2 };
+enum : int { MODE_SKETCH = 0, MODE_BACKPROBE = 1, MODE_CONTRACT = 2, MODE_CONV = 3 };
 
 struct TcParams {
   int mode;
@@ -53,9 +56,10 @@ struct TcParams {
   long rows, cols;         // valid MMA rows / columns of the whole problem
   // outputs
   float* part;             // SKETCH: [split][rows][cols]; CONTRACT: [split][Cout][T][Cin]
-  bf16* L;                 // BACKPROBE: [r][Q]
+  bf16* L;                 // BACKPROBE: [r][Q]; CONV: output [B][H][W][Co]
   long Q;
-  int T, Cin;              // CONTRACT output indexing
+  int T, Cin;              // CONTRACT output indexing; CONV: offsets and input channels
+  int H, W, cgroups;       // CONV: image size and input-channel blocks of 64
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
 };
@@ -186,11 +190,19 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-struct Unit { int tm, tn, tap; long split, kb0; int nkb; };
+struct Unit { int tm, tn, tap; long split, kb0; int nkb; int px, py, img; };
 
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
   Unit w;
-  if (p.mode == MODE_BACKPROBE) {           // probe tiles innermost: the dY tile is re-read while hot in L2
+  w.px = w.py = w.img = 0;
+  if (p.mode == MODE_CONV) {                 // channel tiles innermost, then patches of one image
+    long q = u;
+    w.tn = (int)(q % p.tiles_n); q /= p.tiles_n;
+    w.px = (int)(q % p.patches_x); q /= p.patches_x;
+    w.py = (int)(q % p.patches_y); q /= p.patches_y;
+    w.img = (int)q;
+    w.tm = 0; w.tap = 0; w.split = 0;
+  } else if (p.mode == MODE_BACKPROBE) {     // probe tiles innermost: the dY tile is re-read while hot in L2
     w.tm = (int)(u % p.tiles_m);
     w.tn = (int)(u / p.tiles_m);
     w.tap = 0;
@@ -268,6 +280,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0;
         if (p.mode == MODE_SKETCH) kc = (int)(w.kb0 * 64);
         else if (p.mode == MODE_BACKPROBE) kc = (int)w.kb0 * p.ksteps * 16;
+        else if (p.mode == MODE_CONV) { dx = dy = -p.pad; }     // pj counts channel blocks, kc = offset * Cin
         else {
           long q = w.kb0;
           px = (int)(q % p.patches_x); q /= p.patches_x;
@@ -295,6 +308,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // dY tile as one 3-d box (64 positions, k rows, tile_n/64 column groups)
             tma_load_3d(b_dst, &map_b, 0, kc, col0 >> 6, &full_bar[s]);
             kc += p.ksteps * 16;
+          } else if (p.mode == MODE_CONV) {
+            // input patch moved by the kernel offset (zero fill outside the image) and the matching
+            // [tile_n output channels x 64 input channels] block of the weights
+            tma_load_5d(a_dst, &map_a, 0, w.px * p.patch_w + dx, w.py * p.patch_h + dy, pj, w.img, &full_bar[s]);
+            tma_load_2d(b_dst, &map_b, kc + pj * 64, col0, &full_bar[s]);
+            if (++pj == p.cgroups) { pj = 0; kc += p.Cin; if (++dx > p.pad) { dx = -p.pad; ++dy; } }
           } else {
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
@@ -401,7 +420,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           const int nc = min(32, p.tile_n - c);
           if (row >= p.rows) continue;
-          if (p.mode == MODE_BACKPROBE) {
+          if (p.mode == MODE_CONV) {
+            // D[pixel of the patch, co] -> out[img][y][x][co]: 32 consecutive channels per thread
+            const int pr = (int)row / p.patch_w, pc = (int)row % p.patch_w;
+            const int y = w.py * p.patch_h + pr, x = w.px * p.patch_w + pc;
+            if (y < p.H && x < p.W) {
+              bf16* dst = p.L + (((long)w.img * p.H + y) * p.W + x) * p.cols + col0 + c;
+              if (nc == 32 && col0 + c + 32 <= p.cols) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 8) {
+                  uint4 o;
+                  __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
+                  __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                  __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                  __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+                  o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+                  o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+                  *reinterpret_cast<uint4*>(dst + i) = o;
+                }
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+              }
+            }
+          } else if (p.mode == MODE_BACKPROBE) {
             // D[j, q] -> L[j][q]: each thread owns 32 consecutive positions of one probe
             bf16* dst = p.L + row * p.Q + col0 + c;
             if (nc == 32 && col0 + c + 32 <= p.cols) {
@@ -538,11 +581,6 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
   return r == CUDA_SUCCESS;
 }
 
-static int env_int(const char* name, int dflt) {   // TUNING
-  const char* v = getenv(name);
-  return v ? atoi(v) : dflt;
-}
-
 static int pow2_cols(int n) { int c = 32; while (c < n) c *= 2; return c; }
 
 static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
@@ -575,17 +613,14 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   const int rows = p->swap ? d->B : d->r, cols = p->swap ? d->r : d->B;
   p->tile_n = std::min(256, round_up(cols, 16));
   p->m_sub = rows > TILE_M ? 2 : 1;                      // two row tiles share each tile of the other operand
-  p->m_sub = env_int("XC_SK_MSUB", p->m_sub);
-  const int sk_ctas = env_int("XC_SK_CTAS", 1);
   p->tile_m = TILE_M * p->m_sub;
   p->tiles_m = (int)cdivl(rows, p->tile_m);
   p->tiles_n = (int)cdivl(cols, p->tile_n);
   p->kblocks = cdivl(K, 64);
   const uint32_t stage = (uint32_t)p->m_sub * TILE_M * 128 + p->tile_n * 128;
-  p->stages = std::min(pick_stages(stage, sk_ctas), env_int("XC_SK_STAGES", 8));
+  p->stages = pick_stages(stage, 1);
   const long tiles = (long)p->tiles_m * p->tiles_n;
-  long splits = std::max(1L, std::min((long)NUM_SMS * sk_ctas / tiles, p->kblocks / 8));
-  splits = env_int("XC_SK_SPLITS", (int)splits);
+  long splits = std::max(1L, std::min((long)NUM_SMS / tiles, p->kblocks / 8));
   splits = std::max(1L, std::min(splits, 512L));
   p->kblocks_per_split = cdivl(p->kblocks, splits);
   p->splits = (int)cdivl(p->kblocks, p->kblocks_per_split);
@@ -665,12 +700,15 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   // back-probe: D[j, q], rows = r, cols = Q, k = B
   if (Q % 64 == 0 && d->B % 8 == 0 && Q >= 2048 && Q < 2000000000L) {
     mask |= 1;
-    p->bp_tile_n = env_int("XC_BP_TILEN", 256);
+    p->bp_tile_n = 256;
     p->bp_tiles_q = (int)cdivl(Q, p->bp_tile_n);
-    p->bp_tiles_r = (int)cdivl(d->r, TILE_M);
+    p->bp_m_sub = 1;
+    p->bp_acc_bufs = (2 * p->bp_m_sub * p->bp_tile_n <= 512) ? 2 : 1;
+    p->bp_tiles_r = (int)cdivl(d->r, TILE_M * p->bp_m_sub);
     p->bp_ksteps = std::min(4, (int)cdivl(d->B, 16));
-    const uint32_t stage = TILE_M * 128 + (uint32_t)p->bp_ksteps * 16 * 128 * (uint32_t)(p->bp_tile_n / 64);
-    p->bp_stages = std::min(pick_stages(stage, env_int("XC_BP_CTAS", 1)), env_int("XC_BP_STAGES", 8));
+    const uint32_t stage = (uint32_t)p->bp_m_sub * TILE_M * 128 +
+                           (uint32_t)p->bp_ksteps * 16 * 128 * (uint32_t)(p->bp_tile_n / 64);
+    p->bp_stages = pick_stages(stage, 1);
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
@@ -679,18 +717,18 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     pick_patch(d->H, d->W, &p->patch_w, &p->patch_h);
     p->patches_x = (int)cdivl(d->W, p->patch_w);
     p->patches_y = (int)cdivl(d->H, p->patch_h);
-    p->ct_tile_n = std::min(env_int("XC_CT_TILEN", 256), round_up(d->Cin, 16));
-    p->ct_m_sub = d->Cout > TILE_M ? 2 : 1;            // two output-channel tiles share each probe tile
-    p->ct_m_sub = env_int("XC_CT_MSUB", p->ct_m_sub);
+    p->ct_tile_n = std::min(256, round_up(d->Cin, 16));
+    // two output-channel tiles share each probe tile, unless the reduction is so short (few probes)
+    // that more, smaller work units finish sooner
+    p->ct_m_sub = (d->Cout > TILE_M && d->r >= 32) ? 2 : 1;
     p->ct_tiles_m = (int)cdivl(d->Cout, TILE_M * p->ct_m_sub);
     p->ct_tiles_n = (int)cdivl(d->Cin, p->ct_tile_n);
     const int bk = p->patch_w * p->patch_h;
     const uint32_t stage = (uint32_t)bk * 128 * (2 * p->ct_m_sub + (uint32_t)cdivl(p->ct_tile_n, 64));
-    p->ct_stages = std::min(pick_stages(stage, env_int("XC_CT_CTAS", 1)), env_int("XC_CT_STAGES", 8));
+    p->ct_stages = pick_stages(stage, 1);
     p->ct_items = (long)d->r * p->patches_x * p->patches_y;
     const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * T;
-    long splits = std::max(1L, std::min((long)NUM_SMS * env_int("XC_CT_CTAS", 1) / std::max(1L, tiles), p->ct_items / 4));
-    splits = env_int("XC_CT_SPLITS", (int)splits);
+    long splits = std::max(1L, std::min((long)NUM_SMS / std::max(1L, tiles), p->ct_items / 4));
     splits = std::max(1L, std::min(splits, 512L));
     p->ct_items_per_split = cdivl(p->ct_items, splits);
     p->ct_splits = (int)cdivl(p->ct_items, p->ct_items_per_split);
@@ -710,22 +748,22 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const uint64_t da[2] = {(uint64_t)d->B, (uint64_t)d->r};
   const uint64_t db[3] = {64, (uint64_t)d->B, (uint64_t)(Q / 64)};
   const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[2] = {(uint64_t)Q * 2, 128};
-  const uint32_t box_a[2] = {64, (uint32_t)TILE_M};    // 128-byte rows whatever bk is (zero fill past B)
+  const uint32_t box_a[2] = {64, (uint32_t)(TILE_M * pl.bp_m_sub)};   // 128-byte rows whatever bk is (zero fill past B)
   const uint32_t box_b[3] = {64, (uint32_t)bk, (uint32_t)(pl.bp_tile_n / 64)};
   if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 3, db, sb, box_b)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_BACKPROBE;
   p.tile_n = pl.bp_tile_n;
-  p.m_sub = 1;
-  p.acc_bufs = 2;
-  p.tmem_cols = pow2_cols(2 * pl.bp_tile_n);
+  p.m_sub = pl.bp_m_sub;
+  p.acc_bufs = pl.bp_acc_bufs;
+  p.tmem_cols = pow2_cols(pl.bp_acc_bufs * pl.bp_m_sub * pl.bp_tile_n);
   p.stages = pl.bp_stages;
   p.ksteps = pl.bp_ksteps;
   p.a_boxes = 1;
   p.b_boxes = pl.bp_tile_n / 64;
   p.a_sub_bytes = TILE_M * 128;
-  p.a_stage_bytes = p.a_sub_bytes;
-  p.a_box_bytes = p.a_sub_bytes;
+  p.a_stage_bytes = (uint32_t)pl.bp_m_sub * p.a_sub_bytes;
+  p.a_box_bytes = p.a_stage_bytes;
   p.b_box_bytes = (uint32_t)bk * 128;
   p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
@@ -743,7 +781,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS * env_int("XC_BP_CTAS", 1)), st);
+  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st);
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
@@ -803,6 +841,107 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
+}
+
+// ---- exact convolution and input gradient -----------------------------------------------------
+
+// Wd[n][T-1-t][m] = W[m][t][n]: the weights of the transposed convolution, laid out like W.
+__global__ void __launch_bounds__(256) flip_transpose_weights(const bf16* __restrict__ W, bf16* __restrict__ Wd,
+                                                              int Cout, int Cin, int T) {
+  pdl_trigger();
+  pdl_wait();
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long count = (long)Cout * T * Cin;
+  if (i >= count) return;
+  const int m = (int)(i % Cout);
+  const int t = (int)((i / Cout) % T);
+  const int n = (int)(i / ((long)Cout * T));
+  Wd[i] = W[((long)m * T + (T - 1 - t)) * Cin + n];
+}
+
+static void pick_patch_conv(int H, int W, int* pw, int* ph) {
+  // patch of at most 128 pixels (the MMA rows) covering the image with the least work per pixel:
+  // overhang and unused MMA rows both count
+  double best = 1e30; int bw = 1, bh = 1;
+  for (int w = 1; w <= std::min(W, 128); ++w)
+    for (int h = 1; h * w <= 128 && h <= H; ++h) {
+      const double cost = (double)cdivl(W, w) * (double)cdivl(H, h) * 128.0 / ((double)W * H);
+      if (cost < best - 1e-9 || (cost < best + 1e-9 && w > bw)) { best = cost; bw = w; bh = h; }
+    }
+  *pw = bw; *ph = bh;
+}
+
+bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
+  if (d->dtype != XCONV_BF16) return false;
+  const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
+  if (Ci % 64 != 0 || Co % 8 != 0 || Co < 16) return false;
+  p->tile_n = std::min(256, round_up(Co, 16));
+  p->tiles_n = (int)cdivl(Co, p->tile_n);
+  pick_patch_conv(d->H, d->W, &p->patch_w, &p->patch_h);
+  p->patches_x = (int)cdivl(d->W, p->patch_w);
+  p->patches_y = (int)cdivl(d->H, p->patch_h);
+  p->stages = pick_stages(TILE_M * 128 + (uint32_t)p->tile_n * 128, 1);
+  p->wt_bytes = dgrad ? (size_t)d->Cout * d->KH * d->KW * d->Cin * 2 : 0;
+  return true;
+}
+
+xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, const void* in, const void* W,
+                         void* out, char* ws_head, char* wt, cudaStream_t st) {
+  const int T = d->KH * d->KW;
+  const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
+  const void* Wk = W;
+  if (dgrad) {
+    const long count = (long)d->Cout * T * d->Cin;
+    cudaError_t e = launch_pdl(flip_transpose_weights, dim3((unsigned)cdivl(count, 256)), dim3(256), 0, st,
+                               static_cast<const bf16*>(W), reinterpret_cast<bf16*>(wt), d->Cout, d->Cin, T);
+    count_launch();
+    if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
+    Wk = wt;
+  }
+  CUtensorMap ma, mb;
+  // input as (64 channels, x, y, channel blocks of 64, image); weights as [Co][T*Ci]
+  const uint64_t da[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(Ci / 64), (uint64_t)d->B};
+  const uint64_t sa[4] = {(uint64_t)Ci * 2, (uint64_t)d->W * Ci * 2, 128, (uint64_t)d->H * d->W * Ci * 2};
+  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1, 1};
+  const uint64_t db[2] = {(uint64_t)T * Ci, (uint64_t)Co};
+  const uint64_t sb[1] = {(uint64_t)T * Ci * 2};
+  const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
+  if (!make_map(&ma, in, 5, da, sa, box_a) || !make_map(&mb, Wk, 2, db, sb, box_b)) return XCONV_ERR_CUDA;
+  TcParams p{};
+  p.mode = MODE_CONV;
+  p.tile_n = pl.tile_n;
+  p.m_sub = 1;
+  p.acc_bufs = 2;
+  p.tmem_cols = pow2_cols(2 * pl.tile_n);
+  p.stages = pl.stages;
+  p.ksteps = 4;
+  p.a_boxes = p.b_boxes = 1;
+  p.a_sub_bytes = TILE_M * 128;
+  p.a_stage_bytes = p.a_sub_bytes;                 // the patch fills its first patch_w*patch_h rows
+  p.b_stage_bytes = (uint32_t)pl.tile_n * 128;
+  p.tx_bytes = (uint32_t)(pl.patch_w * pl.patch_h) * 128 + p.b_stage_bytes;
+  p.a_mn_major = p.b_mn_major = 0;
+  p.tiles_m = 1;
+  p.tiles_n = pl.tiles_n;
+  p.taps = 1;
+  p.kblocks = (long)T * (Ci / 64);
+  p.kblocks_per_split = p.kblocks;
+  p.units = (long)d->B * pl.patches_y * pl.patches_x * pl.tiles_n;
+  p.patch_w = pl.patch_w;
+  p.patch_h = pl.patch_h;
+  p.patches_x = pl.patches_x;
+  p.patches_y = pl.patches_y;
+  p.pad = (d->KH - 1) / 2;
+  p.rows = (long)pl.patch_w * pl.patch_h;
+  p.cols = Co;
+  p.L = static_cast<bf16*>(out);
+  p.T = T;
+  p.Cin = Ci;
+  p.H = d->H;
+  p.W = d->W;
+  p.cgroups = Ci / 64;
+  p.status = reinterpret_cast<unsigned int*>(ws_head);
+  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, NUM_SMS), st);
 }
 
 }  // namespace xconv
