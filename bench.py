@@ -56,6 +56,15 @@ def layer_work(c, r):
     }
 
 
+# DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
+# profiles/ (None where the kernel has changed since, or was never captured).
+NCU_TRAFFIC = {}
+
+
+def ncu_traffic(cfg, r, phase):
+    return NCU_TRAFFIC.get((cfg, r, phase))
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -67,7 +76,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -206,71 +215,94 @@ def run_xconv(args):
     X, dY = xb.to_device(hX, c["dtype"], dev), xb.to_device(hdY, c["dtype"], dev)
     del lay
 
-    desc = xb.make_desc(B, Cin, Cout, H, W, r, tdt)
-    S = torch.empty((r, B), dtype=torch.float32, device=dev)
-    dW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device=dev, memory_format=torch.channels_last)
-    L = torch.empty((r, Cout, H, W), dtype=tdt, device=dev, memory_format=torch.channels_last)
-    ws = torch.empty(max(xb.workspace_bytes(desc, xb.OP_SKETCH), xb.workspace_bytes(desc, xb.OP_WGRAD)),
-                     dtype=torch.uint8, device=dev)
     flush = None if cfg == 5 else torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    launches = [0]
 
-    def step(events=None):
-        if flush is not None:
-            flush.fill_(1)
-        if events:
-            events[0].record()
-        xb.sketch_into(desc, X, Z, S, ws)
-        launches[0] += xb.last_launch_count()
-        if events:
-            events[1].record()
-        xb.backprobe_into(desc, S, dY, L, ws)
-        launches[0] += xb.last_launch_count()
-        if events:
-            events[2].record()
-        xb.contract_into(desc, L, Z, dW, ws)
-        launches[0] += xb.last_launch_count()
-        if events:
-            events[3].record()
-        dp.allreduce_dw(dW)
+    class Layer:
+        """Buffers and the timed step of one (config, r) workload."""
 
-    for _ in range(max(3, args.warmup)):
-        step()
-    torch.cuda.synchronize()
-    if xb.workspace_status(ws) != 0:
-        raise SystemExit("a device-side wait ran out during warm-up")
+        def __init__(self, r_, Z_):
+            self.r, self.Z = r_, Z_
+            self.desc = xb.make_desc(B, Cin, Cout, H, W, r_, tdt)
+            self.S = torch.empty((r_, B), dtype=torch.float32, device=dev)
+            self.dW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device=dev, memory_format=torch.channels_last)
+            self.L = torch.empty((r_, Cout, H, W), dtype=tdt, device=dev, memory_format=torch.channels_last)
+            self.ws = torch.empty(max(xb.workspace_bytes(self.desc, xb.OP_SKETCH),
+                                      xb.workspace_bytes(self.desc, xb.OP_WGRAD)), dtype=torch.uint8, device=dev)
+            self.launches = 0
 
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        def step(self, events=None):
+            if flush is not None:
+                flush.fill_(1)
+            if events:
+                events[0].record()
+            xb.sketch_into(self.desc, X, self.Z, self.S, self.ws)
+            self.launches += xb.last_launch_count()
+            if events:
+                events[1].record()
+            xb.backprobe_into(self.desc, self.S, dY, self.L, self.ws)
+            self.launches += xb.last_launch_count()
+            if events:
+                events[2].record()
+            xb.contract_into(self.desc, self.L, self.Z, self.dW, self.ws)
+            self.launches += xb.last_launch_count()
+            if events:
+                events[3].record()
+            dp.allreduce_dw(self.dW)
+
+        def measure(self, steps, warmup, sampler=None, phase_events=True):
+            """W warm-up steps, then exactly `steps` timed steps between barriers and synchronisations;
+            returns (total ms as the max over ranks, mean per-phase ms or None, clock record).
+            With phase_events an event is recorded between the three calls of every step: that gives
+            the per-phase times but costs about 15 us per step, because an event between two kernels
+            keeps the second from starting its preamble under the tail of the first."""
+            for _ in range(max(3, warmup)):
+                self.step()
+            torch.cuda.synchronize()
+            if xb.workspace_status(self.ws) != 0:
+                raise SystemExit("a device-side wait ran out during warm-up")
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+            t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if sampler is not None:
+                sampler.start()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            self.launches = 0
+            t_begin.record()
+            for i in range(steps):
+                self.step(ev[i] if phase_events else None)
+            t_end.record()
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            total = t_begin.elapsed_time(t_end)
+            clk = sampler.stop() if sampler is not None else None
+            if world > 1:
+                t = torch.tensor([total], device=dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                total = float(t.item())
+            if xb.workspace_status(self.ws) != 0:
+                raise SystemExit("a device-side wait ran out during the timed region")
+            ph = None
+            if phase_events:
+                ph = {n: float(np.mean([ev[i][k].elapsed_time(ev[i][k + 1]) for i in range(steps)]))
+                      for k, n in enumerate(("sketch", "backprobe", "contract"))}
+            return total, ph, clk
+
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
         gpu_id = str(local)
-    sampler = ClockSampler(gpu_id)
-    if rank == 0:
-        sampler.start()
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    launches[0] = 0
-    t_begin.record()
-    for i in range(args.steps):
-        step(ev[i])
-    t_end.record()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    total_ms = t_begin.elapsed_time(t_end)
-    clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    if xb.workspace_status(ws) != 0:
-        raise SystemExit("a device-side wait ran out during the timed region")
+    layer = Layer(r, Z)
+    # the timed region of the headline number: K steps, nothing but the three calls in the stream
+    total_ms, _, clocks = layer.measure(args.steps, args.warmup, ClockSampler(gpu_id) if rank == 0 else None,
+                                        phase_events=False)
     ms_step = total_ms / args.steps
-    phase_ms = {n: float(np.mean([ev[i][k].elapsed_time(ev[i][k + 1]) for i in range(args.steps)]))
-                for k, n in enumerate(("sketch", "backprobe", "contract"))}
+    n_launch = layer.launches
+    # the same K steps again with an event between the calls: per-phase times for the roofline
+    total_ev_ms, phase_ms, _ = layer.measure(args.steps, 3, None, phase_events=True)
+    desc, S, dW = layer.desc, layer.S, layer.dW
+    launches = [n_launch]
 
     # ---- end to end from pinned host buffers through the host-buffer entry point
     e2e = None
@@ -305,26 +337,74 @@ def run_xconv(args):
 
     # ---- roofline of the dominant kernel (live CUDA-event times of the timed region)
     peaks, peak_src = load_peaks()
-    work = layer_work(c, r)
-    dom = max(phase_ms, key=phase_ms.get)
-    engines = {"sketch": xb.engine_for(desc, xb.OP_SKETCH), "backprobe": xb.engine_for(desc, xb.OP_WGRAD),
-               "contract": xb.engine_for(desc, xb.OP_WGRAD)}
     tensor_peak = peaks["bf16_tflops"] if total_ms < 2000 else peaks["bf16_tflops_sustained"]
-    phases = {}
-    for n, ms in phase_ms.items():
-        gbs = work[n]["bytes"] / (ms * 1e-3) / 1e9
-        tfs = work[n]["flops"] / (ms * 1e-3) / 1e12
-        comp_peak = tensor_peak if engines[n] == "tcgen05_bf16" else FP32_ALU_TFLOPS
-        t_mem, t_comp = work[n]["bytes"] / (peaks["hbm_gbs"] * 1e9), work[n]["flops"] / (comp_peak * 1e12)
-        bound = "hbm" if t_mem >= t_comp else ("tensor" if engines[n] == "tcgen05_bf16" else "alu")
-        phases[n] = {"ms": ms, "engine": engines[n], "GBps": gbs, "TFLOPps": tfs, "bound": bound,
-                     "frac": (gbs / peaks["hbm_gbs"]) if bound == "hbm" else tfs / comp_peak}
+
+    def phase_table(r_, desc_, ph_ms):
+        work = layer_work(c, r_)
+        eng = {"sketch": xb.engine_for(desc_, xb.OP_SKETCH), "backprobe": xb.engine_for(desc_, xb.OP_WGRAD),
+               "contract": xb.engine_for(desc_, xb.OP_WGRAD)}
+        out = {}
+        for n, ms in ph_ms.items():
+            gbs = work[n]["bytes"] / (ms * 1e-3) / 1e9
+            tfs = work[n]["flops"] / (ms * 1e-3) / 1e12
+            comp_peak = tensor_peak if eng[n] == "tcgen05_bf16" else FP32_ALU_TFLOPS
+            t_mem, t_comp = work[n]["bytes"] / (peaks["hbm_gbs"] * 1e9), work[n]["flops"] / (comp_peak * 1e12)
+            bound = "hbm" if t_mem >= t_comp else ("tensor" if eng[n] == "tcgen05_bf16" else "alu")
+            out[n] = {"ms": ms, "engine": eng[n], "GBps": gbs, "TFLOPps": tfs, "bound": bound,
+                      "peak": peaks["hbm_gbs"] if bound == "hbm" else comp_peak,
+                      "frac": (gbs / peaks["hbm_gbs"]) if bound == "hbm" else tfs / comp_peak}
+        return out
+
+    phases = phase_table(r, desc, phase_ms)
+    dom = max(phase_ms, key=phase_ms.get)
     d = phases[dom]
-    roofline = {"kernel": dom, "bound": d["bound"],
-                "achieved": d["GBps"] if d["bound"] == "hbm" else d["TFLOPps"],
-                "peak": peaks["hbm_gbs"] if d["bound"] == "hbm" else (tensor_peak if d["engine"] == "tcgen05_bf16" else FP32_ALU_TFLOPS),
-                "unit": "GB/s" if d["bound"] == "hbm" else "TFLOP/s", "frac": d["frac"], "traffic": None,
+    roofline = {"kernel": dom + " (tc_gemm_kernel and its reduce/cast helper, timed together)", "bound": d["bound"],
+                "achieved": d["GBps"] if d["bound"] == "hbm" else d["TFLOPps"], "peak": d["peak"],
+                "unit": "GB/s" if d["bound"] == "hbm" else "TFLOP/s", "frac": d["frac"],
+                "traffic": ncu_traffic(cfg, r, dom),
                 "peak_source": f"of {peak_src}" + ("" if d["bound"] != "alu" else " (derived: 148 SMs x 128 FMA x 2 x 1.965 GHz)")}
+
+    # ---- the other probe counts of this workload's sweep (shorter runs), same step and timing
+    sweep = []
+    if not args.no_sweep and world == 1:
+        for r2 in c["r"]:
+            if r2 == r:
+                continue
+            Z2 = xb.to_device(inputs.make_layer(cfg, r2, tensors=("Z",))["Z"], c["dtype"], dev)
+            lay2 = Layer(r2, Z2)
+            n2 = max(5, min(args.steps, 30))
+            tot2, _, _ = lay2.measure(n2, 3, None, phase_events=False)
+            _, ph2, _ = lay2.measure(n2, 3, None, phase_events=True)
+            sweep.append({"r": r2, "ms_per_step": tot2 / n2, "value": 1e3 * n2 / tot2, "phases": phase_table(r2, lay2.desc, ph2)})
+            del lay2, Z2
+            torch.cuda.empty_cache()
+
+    # ---- the rest of the layer API on the same tensors: forward (conv + sketch) and exact dX
+    full = None
+    if not args.no_context:
+        Wt = xb.to_device(inputs.draw("normal", (Cout, Cin, 3, 3), inputs.seed_for(cfg, r, "W"), c["dtype"],
+                                      (2.0 / (Cin * 9)) ** 0.5), c["dtype"], dev)
+        Y = torch.empty((B, Cout, H, W), dtype=tdt, device=dev, memory_format=torch.channels_last)
+        dX = torch.empty((B, Cin, H, W), dtype=tdt, device=dev, memory_format=torch.channels_last)
+        wsf = torch.empty(max(xb.workspace_bytes(desc, xb.OP_FORWARD), xb.workspace_bytes(desc, xb.OP_DGRAD)),
+                          dtype=torch.uint8, device=dev)
+
+        def _time(f, n=5):
+            for _ in range(2):
+                f()
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record()
+            for _ in range(n):
+                f()
+            b_.record()
+            torch.cuda.synchronize()
+            return a_.elapsed_time(b_) / n
+
+        full = {"forward_ms": _time(lambda: xb.forward_into(desc, X, Wt, Z, Y, S, wsf)),
+                "dgrad_ms": _time(lambda: xb.dgrad_into(desc, dY, Wt, dX, wsf)),
+                "conv_engine": xb.engine_for(desc, xb.OP_FORWARD),
+                "note": "xconv_forward = conv + sketch; xconv_dgrad = exact dX; not part of the metric"}
+        del Y, dX, wsf
 
     cpu = None
     if not args.no_cpu:
@@ -356,6 +436,10 @@ def run_xconv(args):
             "vs_baseline": None, "dtype": "f32" if c["dtype"] == "f32" else "bf16 (f32 accumulate)",
             "data": "synthetic", "config": workload_config(args, c), "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches[0], "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
+            "phase_timing": {"ms_per_step_with_events": total_ev_ms / args.steps,
+                             "note": "phases and roofline come from a second timed region of the same K steps with a "
+                                     "CUDA event between the three calls; the events themselves add to that region"},
+            "sweep": sweep, "layer_api": full,
             "memory_ratio": {"elements": Cin * H * W / r, "stored_bytes": Cin * H * W * es / (4.0 * r)},
             "context": context}
     print(json.dumps(line))
@@ -366,7 +450,7 @@ def run_xconv(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="xconv", choices=["xconv", "reference"])
     ap.add_argument("--config", type=int, default=5)
@@ -375,6 +459,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-context", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
