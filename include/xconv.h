@@ -160,9 +160,19 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
 xconv_status xconv_sketch_static(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
                                  void* cuda_stream);
 
-/* Reads the status word the kernels of the last call left in `ws` (synchronises `cuda_stream`).
- * XCONV_OK, or XCONV_ERR_TIMEOUT if a bounded device-side wait ran out. */
+/* Reads the status the kernels of the last call left in the header of `ws` (synchronises
+ * `cuda_stream`).  XCONV_OK, or XCONV_ERR_TIMEOUT if a bounded device-side wait ran out in that call.
+ * The header never needs clearing: every call tags it afresh, so a later call on the same `ws`
+ * reports its own outcome.  (Only the tensor-core kernels wait on anything; calls served by the
+ * FP32-FMA kernels leave the header as it was.) */
 xconv_status xconv_workspace_status(const void* ws, void* cuda_stream);
+
+/* Self-test of the failure path: one warp waits, with the same bounded wait the pipelined kernels use,
+ * on a barrier that nothing completes; after `limit_ms` (1..2000) it gives up and records the
+ * time-out in the header of `ws` (at least 256 bytes), where xconv_workspace_status then reports
+ * XCONV_ERR_TIMEOUT.  Nothing faults or hangs; the context stays usable.  (No counterpart in the
+ * paper.) */
+xconv_status xconv_selftest_wait_limit(void* ws, size_t ws_bytes, unsigned int limit_ms, void* cuda_stream);
 
 /* Number of kernels the last successful call on this host thread enqueued. */
 int xconv_last_launch_count(void);

@@ -24,7 +24,7 @@ STATUS_OK = 0
 # every symbol include/xconv.h declares
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
            "xconv_dgrad", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
-           "xconv_workspace_status",
+           "xconv_workspace_status", "xconv_selftest_wait_limit",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -76,6 +76,8 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_wgrad_host.restype = c_int
     L.xconv_sketch_static.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
     L.xconv_sketch_static.restype = c_int
+    L.xconv_selftest_wait_limit.argtypes = [c_void_p, c_size_t, ctypes.c_uint, c_void_p]
+    L.xconv_selftest_wait_limit.restype = c_int
     L.xconv_workspace_status.argtypes = [c_void_p, c_void_p]; L.xconv_workspace_status.restype = c_int
     L.xconv_last_launch_count.argtypes = []; L.xconv_last_launch_count.restype = c_int
     L.xconv_last_cuda_error.argtypes = []; L.xconv_last_cuda_error.restype = c_int

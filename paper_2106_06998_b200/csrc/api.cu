@@ -424,6 +424,15 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
   return XCONV_OK;
 }
 
+xconv_status xconv_selftest_wait_limit(void* ws, size_t ws_bytes, unsigned int limit_ms, void* cuda_stream) {
+  if (!ws || ws_bytes < WS_HEADER) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
+  if (limit_ms == 0 || limit_ms > 2000) return XCONV_ERR_INVALID_ARG;
+  new_call();
+  return tc_run_wait_selftest(static_cast<char*>(ws), (unsigned long long)limit_ms * 1000000ull,
+                              static_cast<cudaStream_t>(cuda_stream));
+}
+
 xconv_status xconv_workspace_status(const void* ws, void* cuda_stream) {
   if (!ws) return XCONV_ERR_INVALID_ARG;
   unsigned int word[2] = {0, 0};

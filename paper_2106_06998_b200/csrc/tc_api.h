@@ -48,6 +48,8 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const v
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const void* L, const void* Z, float* dW,
                              char* ws_head, char* part, cudaStream_t st);
 
+xconv_status tc_run_wait_selftest(char* ws_head, unsigned long long limit_ns, cudaStream_t st);
+
 // bookkeeping shared with the ABI layer
 void count_launch();
 void set_cuda_error(int e);

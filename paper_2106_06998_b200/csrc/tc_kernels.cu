@@ -89,14 +89,15 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Bounded wait: about one second after a short spin.  Returns false (and records the tag) on expiry.
-__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, unsigned int* status, unsigned int tag) {
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, unsigned int* status, unsigned int tag,
+                                            unsigned long long limit_ns = 1000000000ull) {
   for (int i = 0; i < 4096; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (global_ns() - t0 > 1000000000ull) {
+    if (global_ns() - t0 > limit_ns) {
       atomicExch(status, tag);
       return false;
     }
@@ -839,6 +840,29 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(count / 4, 256)), dim3(256), 0, st, p.part,
                              dW, count, pl.ct_splits, 1.0f / (float)d->r, d->chan_scale, d->Cin);
   count_launch();
+  if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
+  return XCONV_OK;
+}
+
+// ---- self-test of the bounded wait ------------------------------------------------------------
+
+// One warp waits on an mbarrier that nothing will ever complete; the wait gives up after `limit_ns`,
+// records the call's tag in the workspace header exactly as a pipelined kernel would, and returns.
+__global__ void wait_limit_selftest_kernel(unsigned int* status, unsigned int tag, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  pdl_wait();
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    status[1] = tag;
+    mbar_wait_slow(&bar, 0u, status, tag, limit_ns);
+  }
+}
+
+xconv_status tc_run_wait_selftest(char* ws_head, unsigned long long limit_ns, cudaStream_t st) {
+  wait_limit_selftest_kernel<<<1, 32, 0, st>>>(reinterpret_cast<unsigned int*>(ws_head), call_tag(), limit_ns);
+  count_launch();
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
 }

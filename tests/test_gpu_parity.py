@@ -187,6 +187,27 @@ def test_errors_launch_nothing_on_gpu():
     assert st == 4 and float(S.min()) == 7.0 and float(S.max()) == 7.0
 
 
+def test_bounded_wait_reports_timeout_and_next_call_recovers():
+    """A wait that nothing satisfies gives up after its limit, the status says so, the context stays
+    usable and the next call on the same workspace reports its own (clean) outcome."""
+    lay = inputs.make_layer(5, 16, B=128, H=14, W=14)
+    d = dev(lay, ("X", "Z"))
+    desc = xb.make_desc(128, 256, 256, 14, 14, 16, torch.bfloat16)
+    ws = torch.empty(xb.workspace_bytes(desc, xb.OP_SKETCH), dtype=torch.uint8, device="cuda")
+    st = xb.lib().xconv_selftest_wait_limit(ws.data_ptr(), ws.numel(), 50, torch.cuda.current_stream().cuda_stream)
+    assert st == 0
+    assert xb.workspace_status(ws) == 6                      # XCONV_ERR_TIMEOUT
+    S = torch.empty((16, 128), dtype=torch.float32, device="cuda")
+    xb.sketch_into(desc, d["X"], d["Z"], S, ws)
+    assert xb.workspace_status(ws) == 0
+    check("sketch after a timed-out call", host(S), O.sketch(lay["X"], lay["Z"]), 1e-2)
+
+
 def test_engines_reported():
     d1 = xb.make_desc(8, 16, 16, 32, 32, 8, torch.float32)
     assert xb.engine_for(d1, xb.OP_SKETCH) == "simt_f32" and xb.engine_for(d1, xb.OP_WGRAD) == "simt_f32"
+    d5 = xb.make_desc(512, 256, 256, 28, 28, 64, torch.bfloat16)
+    for op in (xb.OP_SKETCH, xb.OP_WGRAD, xb.OP_FORWARD, xb.OP_DGRAD):
+        assert xb.engine_for(d5, op) == "tcgen05_bf16"
+    d4 = xb.make_desc(16, 32, 32, 256, 256, 64, torch.bfloat16)      # 32 channels: contraction on FP32 FMA
+    assert xb.engine_for(d4, xb.OP_SKETCH) == "tcgen05_bf16" and xb.engine_for(d4, xb.OP_WGRAD) == "simt_f32"
