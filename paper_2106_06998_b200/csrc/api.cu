@@ -89,7 +89,7 @@ struct WgradPlan {
   size_t l_off, sb_off, part_off, bytes;
 };
 
-static WgradPlan plan_wgrad(const xconv_desc* d) {
+static WgradPlan plan_wgrad_core(const xconv_desc* d) {
   WgradPlan p{};
   const long Q = (long)d->H * d->W * d->Cout;
   const int T = d->KH * d->KW;
@@ -111,6 +111,47 @@ static WgradPlan plan_wgrad(const xconv_desc* d) {
   p.items_per_split = cdiv(items, splits);
   p.splits = (int)cdiv(items, p.items_per_split);
   p.bytes = p.part_off + align_up((size_t)p.splits * d->Cout * T * d->Cin * sizeof(float), 256);
+  return p;
+}
+
+// Re-association for r > B.  The estimate is one bilinear form,
+//   dW[m,n,k] = scale_n * sum_{j,b,q} S[j,b] dY[b,m,q] Z[j,n,q+k],
+// and Algorithm 1 sums over b first (L = S dY^T, cost r*Cout*N*(B + 9*Cin)).  Summing over j first
+// gives Xr[b,n,p] = sum_j S[j,b] Z[j,n,p] -- the activation rebuilt from its sketch -- followed by the
+// same offset contraction over the batch, dW = scale * sum_{b,q} dY[b,m,q] Xr[b,n,q+k]
+// (cost B*Cin*N*(r + 9*Cout)): cheaper exactly when r > B.  Both steps are the kernels of the other
+// order with the roles of the tensors swapped, so xconv_wgrad picks the cheaper order; the explicit
+// halves xconv_backprobe / xconv_contract always follow the paper's order.
+struct SwappedWgrad {
+  bool on;
+  xconv_desc d1, d2;       // d1: "back-probe" producing Xr; d2: contraction over the batch
+  WgradPlan p1, p2;
+  size_t x_off, st_off, sb_off, part_off, bytes;
+};
+
+static SwappedWgrad plan_wgrad_swapped(const xconv_desc* d) {
+  SwappedWgrad w{};
+  w.on = d->r > d->B;
+  if (!w.on) return w;
+  w.d1 = *d; w.d1.B = d->r; w.d1.r = d->B; w.d1.Cout = d->Cin; w.d1.chan_scale = nullptr;
+  w.d2 = *d; w.d2.r = d->B;
+  w.p1 = plan_wgrad_core(&w.d1);
+  w.p2 = plan_wgrad_core(&w.d2);
+  const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
+  const int T = d->KH * d->KW;
+  w.x_off = WS_HEADER;
+  w.st_off = w.x_off + align_up((size_t)d->B * d->H * d->W * d->Cin * es, 256);
+  w.sb_off = w.st_off + align_up((size_t)d->r * d->B * 4, 256);
+  w.part_off = w.sb_off + align_up((size_t)d->r * d->B * 2, 256);
+  const size_t part = w.p2.tc_ct ? w.p2.t.part_bytes : (size_t)w.p2.splits * d->Cout * T * d->Cin * sizeof(float);
+  w.bytes = w.part_off + align_up(part, 256);
+  return w;
+}
+
+static WgradPlan plan_wgrad(const xconv_desc* d) {
+  WgradPlan p = plan_wgrad_core(d);
+  const SwappedWgrad w = plan_wgrad_swapped(d);
+  if (w.on) p.bytes = std::max(p.bytes, w.bytes);
   return p;
 }
 
@@ -154,10 +195,9 @@ static xconv_status run_backprobe_simt(const xconv_desc* d, const float* S, cons
 
 template <typename T, typename TL>
 static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, const void* Lv, const void* Z,
-                                      float* dW, char* ws, cudaStream_t st) {
+                                      float* dW, float alpha, float* part, cudaStream_t st) {
   const int T9 = d->KH * d->KW;
   const TL* L = static_cast<const TL*>(Lv);
-  float* part = reinterpret_cast<float*>(ws + p.part_off);
   dim3 g2((unsigned)cdiv(d->Cin, 64), (unsigned)cdiv(d->Cout, 32), (unsigned)p.splits);
   if (d->KH == 3)
     contract_simt<TL, T, 3><<<g2, 256, 0, st>>>(L, static_cast<const T*>(Z), part, d->r, d->H, d->W, d->Cin, d->Cout,
@@ -168,8 +208,7 @@ static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, c
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T9 * d->Cin;
-  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, dW, count, p.splits, 1.0f / (float)d->r,
-                                                             d->chan_scale, d->Cin);
+  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, dW, count, p.splits, alpha, d->chan_scale, d->Cin);
   return check_launch();
 }
 
@@ -206,12 +245,12 @@ static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, co
                                : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
 }
 
-// L = S dY^T into `L`; `ws` supplies the bfloat16 copy of S for the tensor-core kernel.
+// L = S dY^T into `L`; `Sb` receives the bfloat16 copy of S that the tensor-core kernel reads.
 static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const float* S, const void* dY,
-                                  void* L, char* w, cudaStream_t st) {
+                                  void* L, void* Sb_, char* w, cudaStream_t st) {
   if (p.tc_bp) {
     const long n = (long)d->r * d->B;
-    bf16* Sb = reinterpret_cast<bf16*>(w + p.sb_off);
+    bf16* Sb = static_cast<bf16*>(Sb_);
     cudaError_t e = launch_pdl(cast_f32_to_bf16, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, Sb, n);
     ++g_launches;
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
@@ -222,10 +261,11 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
 }
 
 static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const void* L, const void* Z,
-                                 float* dW, char* w, cudaStream_t st) {
-  if (p.tc_ct) return tc_run_contract(d, p.t, L, Z, dW, w, w + p.part_off, st);
-  return d->dtype == XCONV_F32 ? run_contract_simt<float, float>(d, p, L, Z, dW, w, st)
-                               : run_contract_simt<bf16, bf16>(d, p, L, Z, dW, w, st);
+                                 float* dW, float alpha, char* part, char* w, cudaStream_t st) {
+  if (p.tc_ct) return tc_run_contract(d, p.t, L, Z, dW, alpha, w, part, st);
+  return d->dtype == XCONV_F32
+             ? run_contract_simt<float, float>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st)
+             : run_contract_simt<bf16, bf16>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st);
 }
 
 static xconv_status check_ws(void* ws, size_t ws_bytes, size_t need) {
@@ -240,9 +280,22 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
   xconv_status s = check_ws(ws, ws_bytes, p.bytes);
   if (s != XCONV_OK) return s;
   char* w = static_cast<char*>(ws);
-  s = run_backprobe(d, p, S, dY, w + p.l_off, w, st);
+  const float alpha = 1.0f / (float)d->r;
+  const SwappedWgrad sw = plan_wgrad_swapped(d);
+  if (sw.on) {
+    // Xr = S^T Z, then the offset contraction over the batch (see plan_wgrad_swapped)
+    float* St = reinterpret_cast<float*>(w + sw.st_off);
+    const long n = (long)d->r * d->B;
+    transpose_f32<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, St, d->r, d->B);
+    s = check_launch();
+    if (s != XCONV_OK) return s;
+    s = run_backprobe(&sw.d1, sw.p1, St, Z, w + sw.x_off, w + sw.sb_off, w, st);
+    if (s != XCONV_OK) return s;
+    return run_contract(&sw.d2, sw.p2, dY, w + sw.x_off, dW, alpha, w + sw.part_off, w, st);
+  }
+  s = run_backprobe(d, p, S, dY, w + p.l_off, w + p.sb_off, w, st);
   if (s != XCONV_OK) return s;
-  return run_contract(d, p, w + p.l_off, Z, dW, w, st);
+  return run_contract(d, p, w + p.l_off, Z, dW, alpha, w + p.part_off, w, st);
 }
 
 int launches() { return g_launches; }
@@ -334,7 +387,7 @@ xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const 
   if (s != XCONV_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   new_call();
-  return run_backprobe(desc, p, sketch, dY, L, static_cast<char*>(ws), st);
+  return run_backprobe(desc, p, sketch, dY, L, static_cast<char*>(ws) + p.sb_off, static_cast<char*>(ws), st);
 }
 
 xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z, float* dW, void* ws,
@@ -349,7 +402,8 @@ xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z
   if (s != XCONV_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   new_call();
-  return run_contract(desc, p, L, Z, dW, static_cast<char*>(ws), st);
+  return run_contract(desc, p, L, Z, dW, 1.0f / (float)desc->r, static_cast<char*>(ws) + p.part_off,
+                      static_cast<char*>(ws), st);
 }
 
 xconv_status xconv_dgrad(const xconv_desc* desc, const void* dY, const void* W, void* dX, void* ws,

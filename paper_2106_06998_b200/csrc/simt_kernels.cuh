@@ -290,6 +290,14 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
   }
 }
 
+// out[b][j] = in[j][b] for a small [rows][cols] float matrix (the sketch, transposed).
+static __global__ void transpose_f32(const float* __restrict__ in, float* __restrict__ out, int rows, int cols) {
+  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long)rows * cols) return;
+  const int j = (int)(i / cols), b = (int)(i % cols);
+  out[(long)b * rows + j] = in[i];
+}
+
 // float -> bfloat16 copy (the sketch as tensor-core operand).
 static __global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
   pdl_trigger();

@@ -46,7 +46,7 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const voi
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const void* S_bf16, const void* dY,
                               void* L, char* ws_head, cudaStream_t st);
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const void* L, const void* Z, float* dW,
-                             char* ws_head, char* part, cudaStream_t st);
+                             float alpha, char* ws_head, char* part, cudaStream_t st);
 
 xconv_status tc_run_wait_selftest(char* ws_head, unsigned long long limit_ns, cudaStream_t st);
 

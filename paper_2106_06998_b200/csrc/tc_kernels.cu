@@ -786,7 +786,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
-                             char* ws_head, char* part, cudaStream_t st) {
+                             float alpha, char* ws_head, char* part, cudaStream_t st) {
   const int T = d->KH * d->KW;
   const int bk = pl.patch_w * pl.patch_h;
   CUtensorMap ma, mb;
@@ -838,7 +838,7 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T * d->Cin;
   cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(count / 4, 256)), dim3(256), 0, st, p.part,
-                             dW, count, pl.ct_splits, 1.0f / (float)d->r, d->chan_scale, d->Cin);
+                             dW, count, pl.ct_splits, alpha, d->chan_scale, d->Cin);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
