@@ -180,7 +180,7 @@ def workload_config(args, c):
     return {"workload": f"config {args.config}: 3x3 conv layer B={c['B']} Cin={c['Cin']} Cout={c['Cout']} "
                         f"{c['H']}x{c['W']} {c['dtype']} storage, {c['z']} probes, r={args.r}",
             "r": args.r, "layout": "channels_last", "l2": "inputs larger than L2 (X and dY 205 MB each)"
-            if args.config == 5 else "L2 flushed between steps by a 256 MB write"}
+            if args.config == 5 else "L2 flushed before every step by a 256 MB write (inside the step time, outside the phase times)"}
 
 
 # ----------------------------------------------------------------------------------- GPU arm
@@ -344,8 +344,8 @@ def run_xconv(args):
 
     def phase_table(r_, desc_, ph_ms):
         work = layer_work(c, r_)
-        eng = {"sketch": xb.engine_for(desc_, xb.OP_SKETCH), "backprobe": xb.engine_for(desc_, xb.OP_WGRAD),
-               "contract": xb.engine_for(desc_, xb.OP_WGRAD)}
+        eng = {"sketch": xb.engine_for(desc_, xb.OP_SKETCH), "backprobe": xb.engine_for(desc_, xb.OP_BACKPROBE),
+               "contract": xb.engine_for(desc_, xb.OP_CONTRACT)}
         out = {}
         for n, ms in ph_ms.items():
             gbs = work[n]["bytes"] / (ms * 1e-3) / 1e9

@@ -68,7 +68,8 @@ typedef enum {
   XCONV_ERR_TIMEOUT = 6      /* a bounded device-side wait ran out (reported by xconv_workspace_status) */
 } xconv_status;
 
-typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3 } xconv_op;
+typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3,
+               XCONV_OP_BACKPROBE = 4, XCONV_OP_CONTRACT = 5 } xconv_op;
 
 /* Which arithmetic engine a call will use for its dominant kernel. */
 typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2 } xconv_engine;

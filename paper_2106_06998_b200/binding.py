@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxconv.so")
 
 XCONV_F32, XCONV_BF16 = 0, 1
-OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH = 0, 1, 2, 3
+OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT = 0, 1, 2, 3, 4, 5
 ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16"}
 STATUS_OK = 0
 

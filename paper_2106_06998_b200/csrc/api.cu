@@ -313,7 +313,9 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
   switch (op) {
     case XCONV_OP_FORWARD:
     case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
-    case XCONV_OP_WGRAD: return plan_wgrad(desc).bytes;
+    case XCONV_OP_WGRAD:
+    case XCONV_OP_BACKPROBE:
+    case XCONV_OP_CONTRACT: return plan_wgrad(desc).bytes;
     case XCONV_OP_DGRAD: return conv_ws_bytes(desc, true);
     default: return 0;
   }
@@ -323,7 +325,9 @@ int xconv_engine_for(const xconv_desc* desc, int op) {
   if (validate(desc) != XCONV_OK) return XCONV_ENGINE_NONE;
   switch (op) {
     case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
-    case XCONV_OP_WGRAD: return plan_wgrad(desc).tc_ct ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_WGRAD:
+    case XCONV_OP_CONTRACT: return plan_wgrad(desc).tc_ct ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_BACKPROBE: return plan_wgrad(desc).tc_bp ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_FORWARD:
     case XCONV_OP_DGRAD: {
       TcConvPlan t;

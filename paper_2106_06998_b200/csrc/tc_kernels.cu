@@ -47,6 +47,10 @@ struct TcParams {
   uint32_t a_box_bytes, b_box_bytes, a_sub_bytes;
   int a_mn_major, b_mn_major;
   uint32_t a_lbo, b_lbo;   // leading byte offsets of the UMMA descriptors
+  // swizzle of the stage tiles: 128-byte rows (layout 2, 8-row groups 1024 B apart) everywhere except
+  // the contraction of layers with 32-channel multiples, which uses 64-byte rows (layout 4, 512 B)
+  uint32_t sbo, mn_step, layout;
+  int cw_shift;            // log2 of the channels per tile block (6 or 5)
   int tiles_m, tiles_n, taps;
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
@@ -183,6 +187,19 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Optional per-CTA cycle counters (build with -DXC_TIMELINE): time the producer and the MMA-issue thread
+// spend waiting on barriers and issuing work, read back through xconv_debug_waits.
+#ifdef XC_TIMELINE
+__device__ long long g_waits[1024 * 8];
+#define TW_BEGIN long long _tw0 = clock64()
+#define TW_END(acc) acc += clock64() - _tw0
+#define TW_STORE(slot, acc) do { if (blockIdx.x < 1024) g_waits[blockIdx.x * 8 + (slot)] = (acc); } while (0)
+#else
+#define TW_BEGIN do {} while (0)
+#define TW_END(acc) do {} while (0)
+#define TW_STORE(slot, acc) do {} while (0)
+#endif
+
 constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
 constexpr int TC_THREADS = 192;
@@ -273,6 +290,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       long fill = 0;                       // how often the ring has wrapped
       long it = 0;                         // stages filled so far, across units
       bool ok = true;
+      long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
         const int row0 = w.tm * p.m_sub * TILE_M;
@@ -293,9 +311,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int i = 0; i < w.nkb; ++i) {
           if (fill > 0) {
+            TW_BEGIN;
             ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
+            TW_END(tw_pw);
             if (!ok) break;
           }
+          TW_BEGIN;
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
           const uint32_t b_dst = a_dst + p.a_stage_bytes;
           mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
@@ -318,14 +339,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else {
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
-            tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> 6, pj, &full_bar[s]);
-            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> 6, pj, &full_bar[s]);
+            tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
+            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
             if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
           }
           ++it;
           if (++s == stages) { s = 0; ++fill; }
+          TW_END(tw_pi);
         }
       }
+      TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it);
       // drain: every copy issued must have landed in this CTA's shared memory before it exits
       // (immediate on the normal path, bounded on the failure path)
       for (long i = max(0L, it - stages); i < it; ++i)
@@ -340,13 +363,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                              ((uint32_t)p.b_mn_major << 16) | ((uint32_t)(p.tile_n >> 3) << 17) |
                              ((uint32_t)(TILE_M >> 4) << 24);
       // Shared-memory descriptor (128-byte swizzle): start address >> 4 | (lbo >> 4) << 16 in the low
-      // word; (sbo >> 4) | version 1 << 14 | layout SWIZZLE_128B << 29 in the high word.
-      // K-major: 8-row groups 1024 B apart (sbo), k-step = 32 B inside the swizzled row.
-      // MN-major: 8-row (k) groups 1024 B apart, 64-column blocks `lbo` apart, k-step = 16 rows = 2048 B.
-      const uint32_t a_step = (p.a_mn_major ? 2048u : 32u) >> 4, b_step = (p.b_mn_major ? 2048u : 32u) >> 4;
+      // word; (sbo >> 4) | version 1 << 14 | layout (2 = SWIZZLE_128B, 4 = SWIZZLE_64B) << 29 in the high word.
+      // K-major: 8-row groups `sbo` = 1024 B apart, k-step = 32 B inside the swizzled row.
+      // MN-major: 8-row (k) groups `sbo` apart, column blocks `lbo` apart, k-step = 16 rows = `mn_step` bytes.
+      const uint32_t a_step = (p.a_mn_major ? p.mn_step : 32u) >> 4, b_step = (p.b_mn_major ? p.mn_step : 32u) >> 4;
       const uint32_t a_lo0 = ((p.a_mn_major ? p.a_lbo : 16u) >> 4) << 16;
       const uint32_t b_lo0 = ((p.b_mn_major ? p.b_lbo : 16u) >> 4) << 16;
-      const uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t desc_hi = (p.sbo >> 4) | (1u << 14) | (p.layout << 29);
       const uint32_t a_sub = p.a_sub_bytes >> 4;
       const uint32_t a_stage16 = p.a_stage_bytes >> 4, stage16 = stage_bytes >> 4;
       const uint32_t base16 = (tiles_base & 0x3FFFFu) >> 4;
@@ -357,6 +380,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t full_parity = 0, s16 = base16;
       long lu = 0;
       bool ok = true;
+      long long tw_mw = 0, tw_mi = 0; (void)tw_mw; (void)tw_mi;
+      const long long t_start = clock64(); (void)t_start;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
         const Unit w = decode_unit(p, u);
         if (w.nkb == 0) continue;
@@ -370,8 +395,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
         uint32_t acc = 0;
         for (int i = 0; i < w.nkb; ++i) {
+          { TW_BEGIN;
           ok = mbar_wait(&full_bar[s], full_parity, p.status, p.tag);
+          TW_END(tw_mw); }
           if (!ok) break;
+          TW_BEGIN;
           tc_fence_after();
           uint32_t a_lo = a_lo0 | s16;
           uint32_t b_lo = b_lo0 | (s16 + a_stage16);
@@ -385,8 +413,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           umma_commit(&empty_bar[s]);        // stage s may be refilled once these MMAs have read it
           s16 += stage16;
           if (++s == stages) { s = 0; s16 = base16; full_parity ^= 1u; }
+          TW_END(tw_mi);
         }
         if (ok) umma_commit(&tmem_full_bar[buf]);
+        TW_STORE(2, tw_mw); TW_STORE(3, tw_mi); TW_STORE(4, clock64() - t_start);
       }
     }
   } else {
@@ -566,9 +596,9 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// bfloat16 tensor map with 128-byte swizzle; dims/strides innermost first, strides in bytes for dims 1..rank-1.
+// bfloat16 tensor map, 128-byte swizzle unless told otherwise; dims/strides innermost first, strides in bytes for dims 1..rank-1.
 static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
-                     const uint32_t* box) {
+                     const uint32_t* box, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (!fn) return false;
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -577,7 +607,7 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, bx, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -598,6 +628,7 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   TcParams q = p;
   q.tag = call_tag();
+  if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
   e = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, q);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -713,7 +744,8 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
-  if (d->Cout % 64 == 0 && d->Cin % 64 == 0 && (long)d->H * d->W >= 16) {
+  p->ct_cw = (d->Cout % 64 == 0 && d->Cin % 64 == 0) ? 64 : ((d->Cout % 32 == 0 && d->Cin % 32 == 0) ? 32 : 0);
+  if (p->ct_cw && (long)d->H * d->W >= 16) {
     mask |= 2;
     pick_patch(d->H, d->W, &p->patch_w, &p->patch_h);
     p->patches_x = (int)cdivl(d->W, p->patch_w);
@@ -725,7 +757,8 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     p->ct_tiles_m = (int)cdivl(d->Cout, TILE_M * p->ct_m_sub);
     p->ct_tiles_n = (int)cdivl(d->Cin, p->ct_tile_n);
     const int bk = p->patch_w * p->patch_h;
-    const uint32_t stage = (uint32_t)bk * 128 * (2 * p->ct_m_sub + (uint32_t)cdivl(p->ct_tile_n, 64));
+    const uint32_t a_groups = d->Cout == p->ct_cw ? 1u : (uint32_t)((TILE_M / p->ct_cw) * p->ct_m_sub);
+    const uint32_t stage = (uint32_t)bk * (uint32_t)p->ct_cw * 2 * (a_groups + (uint32_t)cdivl(p->ct_tile_n, p->ct_cw));
     p->ct_stages = pick_stages(stage, 1);
     p->ct_items = (long)d->r * p->patches_x * p->patches_y;
     const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * T;
@@ -790,15 +823,25 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   const int T = d->KH * d->KW;
   const int bk = pl.patch_w * pl.patch_h;
   CUtensorMap ma, mb;
-  // (64 channels, x, y, groups of 64 channels, probe): one box = a whole [patch x channels] tile laid
-  // out as consecutive blocks of 128-byte rows, one block per channel group
-  const uint64_t da[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cout / 64), (uint64_t)d->r};
-  const uint64_t sa[4] = {(uint64_t)d->Cout * 2, (uint64_t)d->W * d->Cout * 2, 128, (uint64_t)d->H * d->W * d->Cout * 2};
-  const uint64_t db[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cin / 64), (uint64_t)d->r};
-  const uint64_t sb[4] = {(uint64_t)d->Cin * 2, (uint64_t)d->W * d->Cin * 2, 128, (uint64_t)d->H * d->W * d->Cin * 2};
-  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)(2 * pl.ct_m_sub), 1};
-  const uint32_t box_b[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)cdivl(pl.ct_tile_n, 64), 1};
-  if (!make_map(&ma, L, 5, da, sa, box_a) || !make_map(&mb, Z, 5, db, sb, box_b)) return XCONV_ERR_CUDA;
+  // (cw channels, x, y, groups of cw channels, probe), cw = 64 or 32: one box = a whole
+  // [patch x channels] tile laid out as consecutive blocks of (2*cw)-byte rows, one block per channel
+  // group.  A layer with a single group of output channels loads just that block and gives the UMMA
+  // descriptor a zero leading-dimension offset: all 128/cw row blocks of the MMA then read the same
+  // block, and the accumulator rows past Cout hold copies that are never stored.
+  const int cw = pl.ct_cw;
+  const uint32_t row_bytes = (uint32_t)cw * 2;
+  const bool one_group = d->Cout == cw;
+  const int groups_a = one_group ? 1 : (TILE_M / cw) * pl.ct_m_sub, groups_b = (int)cdivl(pl.ct_tile_n, cw);
+  const CUtensorMapSwizzle swz = cw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  const uint64_t da[5] = {(uint64_t)cw, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cout / cw), (uint64_t)d->r};
+  const uint64_t sa[4] = {(uint64_t)d->Cout * 2, (uint64_t)d->W * d->Cout * 2, row_bytes,
+                          (uint64_t)d->H * d->W * d->Cout * 2};
+  const uint64_t db[5] = {(uint64_t)cw, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cin / cw), (uint64_t)d->r};
+  const uint64_t sb[4] = {(uint64_t)d->Cin * 2, (uint64_t)d->W * d->Cin * 2, row_bytes,
+                          (uint64_t)d->H * d->W * d->Cin * 2};
+  const uint32_t box_a[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)groups_a, 1};
+  const uint32_t box_b[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)groups_b, 1};
+  if (!make_map(&ma, L, 5, da, sa, box_a, swz) || !make_map(&mb, Z, 5, db, sb, box_b, swz)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_CONTRACT;
   p.tile_n = pl.ct_tile_n;
@@ -807,15 +850,19 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.tmem_cols = pow2_cols(pl.ct_tile_n * pl.ct_m_sub);
   p.stages = pl.ct_stages;
   p.ksteps = bk / 16;
-  p.a_boxes = 2;
-  p.b_boxes = (int)cdivl(pl.ct_tile_n, 64);
-  p.a_box_bytes = p.b_box_bytes = (uint32_t)bk * 128;
-  p.a_sub_bytes = 2 * p.a_box_bytes;
+  p.a_boxes = one_group ? 1 : TILE_M / cw;
+  p.b_boxes = groups_b;
+  p.a_box_bytes = p.b_box_bytes = (uint32_t)bk * row_bytes;
+  p.a_sub_bytes = (uint32_t)p.a_boxes * p.a_box_bytes;
   p.a_stage_bytes = (uint32_t)pl.ct_m_sub * p.a_sub_bytes;
+  p.sbo = 8 * row_bytes;
+  p.mn_step = 16 * row_bytes;
+  p.layout = cw == 64 ? 2u : 4u;
+  p.cw_shift = cw == 64 ? 6 : 5;
   p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.a_mn_major = p.b_mn_major = 1;
-  p.a_lbo = p.a_box_bytes;
+  p.a_lbo = one_group ? 0u : p.a_box_bytes;
   p.b_lbo = p.b_box_bytes;
   p.tiles_m = pl.ct_tiles_m;
   p.tiles_n = pl.ct_tiles_n;
@@ -969,3 +1016,9 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
 }
 
 }  // namespace xconv
+
+#ifdef XC_TIMELINE
+extern "C" int xconv_debug_waits(long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, xconv::g_waits, sizeof(long long) * 1024 * 8);
+}
+#endif

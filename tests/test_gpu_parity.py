@@ -209,5 +209,7 @@ def test_engines_reported():
     d5 = xb.make_desc(512, 256, 256, 28, 28, 64, torch.bfloat16)
     for op in (xb.OP_SKETCH, xb.OP_WGRAD, xb.OP_FORWARD, xb.OP_DGRAD):
         assert xb.engine_for(d5, op) == "tcgen05_bf16"
-    d4 = xb.make_desc(16, 32, 32, 256, 256, 64, torch.bfloat16)      # 32 channels: contraction on FP32 FMA
-    assert xb.engine_for(d4, xb.OP_SKETCH) == "tcgen05_bf16" and xb.engine_for(d4, xb.OP_WGRAD) == "simt_f32"
+    d4 = xb.make_desc(16, 32, 32, 256, 256, 64, torch.bfloat16)      # 32 channels: 64-byte-swizzle tiles
+    assert xb.engine_for(d4, xb.OP_SKETCH) == "tcgen05_bf16" and xb.engine_for(d4, xb.OP_WGRAD) == "tcgen05_bf16"
+    d6 = xb.make_desc(16, 24, 40, 30, 30, 8, torch.bfloat16)         # channels not multiples of 32: FP32 FMA
+    assert xb.engine_for(d6, xb.OP_WGRAD) == "simt_f32"
