@@ -112,6 +112,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsign
   return mbar_wait_slow(bar, parity, status, tag);
 }
 
+// The same operations on a 32-bit shared-memory address the caller keeps in a register.
+__device__ __forceinline__ bool mbar_try_wait_a(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void umma_commit_a(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -158,6 +172,22 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32
       "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
+// All MMAs of one stage, fully unrolled.  The issuing thread runs alone in its warp, so every instruction
+// it executes costs a full dependent-issue slot (~6 cycles): a 128x64x16 MMA occupies the tensor pipe for
+// 32 cycles, i.e. about five instructions.  KS k-steps, TWO = two 128-row tiles share the B tile.
+template <int KS, bool TWO>
+__device__ __forceinline__ void umma_stage(uint32_t d, uint32_t tile_n, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                           uint32_t idesc, uint32_t acc, uint32_t a_step, uint32_t b_step,
+                                           uint32_t a_sub) {
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    umma_bf16(d, a_lo, hi, b_lo, hi, idesc, k == 0 ? acc : 1u);
+    if (TWO) umma_bf16(d + tile_n, a_lo + a_sub, hi, b_lo, hi, idesc, k == 0 ? acc : 1u);
+    a_lo += a_step;
+    b_lo += b_step;
+  }
+}
+
 // mbarrier arrive once every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -378,6 +408,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t tile_n = (uint32_t)p.tile_n;
       int s = 0;
       uint32_t full_parity = 0, s16 = base16;
+      const uint32_t full_a0 = smem_u32(&full_bar[0]), empty_a0 = smem_u32(&empty_bar[0]);
+      uint32_t full_a = full_a0, empty_a = empty_a0;
       long lu = 0;
       bool ok = true;
       long long tw_mw = 0, tw_mi = 0; (void)tw_mw; (void)tw_mi;
@@ -396,23 +428,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t acc = 0;
         for (int i = 0; i < w.nkb; ++i) {
           { TW_BEGIN;
-          ok = mbar_wait(&full_bar[s], full_parity, p.status, p.tag);
+          if (!mbar_try_wait_a(full_a, full_parity)) ok = mbar_wait_slow(&full_bar[s], full_parity, p.status, p.tag);
           TW_END(tw_mw); }
           if (!ok) break;
           TW_BEGIN;
           tc_fence_after();
           uint32_t a_lo = a_lo0 | s16;
           uint32_t b_lo = b_lo0 | (s16 + a_stage16);
-          for (int k = 0; k < ksteps; ++k) {
-            umma_bf16(d_tmem, a_lo, desc_hi, b_lo, desc_hi, idesc, acc);
-            if (two) umma_bf16(d_tmem + tile_n, a_lo + a_sub, desc_hi, b_lo, desc_hi, idesc, acc);
-            acc = 1u;
-            a_lo += a_step;
-            b_lo += b_step;
+#define XC_STAGE(KS, TWO) umma_stage<KS, TWO>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, a_sub)
+          if (two) {
+            switch (ksteps) {
+              case 4: XC_STAGE(4, true); break;
+              case 7: XC_STAGE(7, true); break;
+              case 8: XC_STAGE(8, true); break;
+              default:
+                for (int k = 0; k < ksteps; ++k) {
+                  XC_STAGE(1, true);
+                  acc = 1u; a_lo += a_step; b_lo += b_step;
+                }
+            }
+          } else {
+            switch (ksteps) {
+              case 1: XC_STAGE(1, false); break;
+              case 4: XC_STAGE(4, false); break;
+              case 7: XC_STAGE(7, false); break;
+              case 8: XC_STAGE(8, false); break;
+              default:
+                for (int k = 0; k < ksteps; ++k) {
+                  XC_STAGE(1, false);
+                  acc = 1u; a_lo += a_step; b_lo += b_step;
+                }
+            }
           }
-          umma_commit(&empty_bar[s]);        // stage s may be refilled once these MMAs have read it
-          s16 += stage16;
-          if (++s == stages) { s = 0; s16 = base16; full_parity ^= 1u; }
+#undef XC_STAGE
+          acc = 1u;
+          umma_commit_a(empty_a);            // stage s may be refilled once these MMAs have read it
+          s16 += stage16; full_a += 8; empty_a += 8;
+          if (++s == stages) { s = 0; s16 = base16; full_a = full_a0; empty_a = empty_a0; full_parity ^= 1u; }
           TW_END(tw_mi);
         }
         if (ok) umma_commit(&tmem_full_bar[buf]);
