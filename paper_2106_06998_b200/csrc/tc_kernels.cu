@@ -811,10 +811,12 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     const int bk = p->patch_w * p->patch_h;
     const uint32_t a_groups = d->Cout == p->ct_cw ? 1u : (uint32_t)((TILE_M / p->ct_cw) * p->ct_m_sub);
     const uint32_t stage = (uint32_t)bk * (uint32_t)p->ct_cw * 2 * (a_groups + (uint32_t)cdivl(p->ct_tile_n, p->ct_cw));
-    p->ct_stages = pick_stages(stage, 1);
+    // narrow tiles are bound by the one MMA-issuing thread of a CTA: run two CTAs per SM then
+    const int ct_ctas = (p->ct_tile_n * p->ct_m_sub <= 128 && stage * 2 <= 100 * 1024) ? 2 : 1;
+    p->ct_stages = pick_stages(stage, ct_ctas);
     p->ct_items = (long)d->r * p->patches_x * p->patches_y;
     const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * T;
-    long splits = std::max(1L, std::min((long)NUM_SMS / std::max(1L, tiles), p->ct_items / 4));
+    long splits = std::max(1L, std::min((long)NUM_SMS * ct_ctas / std::max(1L, tiles), p->ct_items / 4));
     splits = std::max(1L, std::min(splits, 512L));
     p->ct_items_per_split = cdivl(p->ct_items, splits);
     p->ct_splits = (int)cdivl(p->ct_items, p->ct_items_per_split);
