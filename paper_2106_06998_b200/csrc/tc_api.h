@@ -19,7 +19,7 @@ struct TcSketchPlan {
 
 struct TcWgradPlan {
   // back-probe
-  int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps;
+  int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps, bp_staged;
   // contraction
   int ct_cw, ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
   int patch_h, patch_w, patches_y, patches_x;

@@ -51,6 +51,7 @@ struct TcParams {
   // the contraction of layers with 32-channel multiples, which uses 64-byte rows (layout 4, 512 B)
   uint32_t sbo, mn_step, layout;
   int cw_shift;            // log2 of the channels per tile block (6 or 5)
+  uint32_t epi_pitch;      // BACKPROBE: row pitch of the shared-memory staging of the output tile (0 = none)
   int tiles_m, tiles_n, taps;
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
@@ -474,6 +475,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
+    const uint32_t epi_base = tiles_base + (uint32_t)p.stages * stage_bytes;
     long lu = 0;
     bool ok = true;
     for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
@@ -527,6 +529,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
               }
             }
+          } else if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
+            // D[j, q] -> staging row of this probe; the warp writes whole rows out afterwards
+            const uint32_t sdst = epi_base + (uint32_t)(quad * 32 + lane) * p.epi_pitch + (uint32_t)c * 2u;
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
+              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sdst + (uint32_t)i * 2u),
+                           "r"(*reinterpret_cast<uint32_t*>(&h0)), "r"(*reinterpret_cast<uint32_t*>(&h1)),
+                           "r"(*reinterpret_cast<uint32_t*>(&h2)), "r"(*reinterpret_cast<uint32_t*>(&h3)) : "memory");
+            }
           } else if (p.mode == MODE_BACKPROBE) {
             // D[j, q] -> L[j][q]: each thread owns 32 consecutive positions of one probe
             bf16* dst = p.L + row * p.Q + col0 + c;
@@ -571,6 +586,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
+      if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
+        // Write the staged rows out: one 512-byte row (32 lanes x 16 B) per instruction.  Storing
+        // straight from the accumulator layout would send the 32 lanes of every store to 32 probe rows
+        // that lie H*W*Cout*2 bytes apart -- one page each for large images.
+        const long row_w = (long)w.tm * TILE_M + quad * 32;
+        const long col = col0 + lane * 8;
+        for (int rr = 0; rr < 32; ++rr) {
+          if (row_w + rr >= p.rows) break;
+          uint4 o;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o.x), "=r"(o.y), "=r"(o.z), "=r"(o.w)
+                       : "r"(epi_base + (uint32_t)(quad * 32 + rr) * p.epi_pitch + (uint32_t)lane * 16u) : "memory");
+          if (col + 8 <= p.cols) *reinterpret_cast<uint4*>(p.L + (row_w + rr) * p.Q + col) = o;
+        }
+        __syncwarp();
+      }
     }
   }
 
@@ -635,6 +665,7 @@ static inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 static const int SMEM_LIMIT = 227 * 1024;
 static const int STATIC_SMEM_SLACK = 2048;     // barriers + alignment slack
 static const int NUM_SMS = 148;
+static const int BP_EPI_PITCH = 512 + 16;   // staged back-probe output rows: 256 bf16 + padding against bank conflicts
 
 static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -674,7 +705,7 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
 
 static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
                            cudaStream_t st) {
-  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
+  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_pitch * TILE_M;
   if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -792,7 +823,11 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     p->bp_ksteps = std::min(4, (int)cdivl(d->B, 16));
     const uint32_t stage = (uint32_t)p->bp_m_sub * TILE_M * 128 +
                            (uint32_t)p->bp_ksteps * 16 * 128 * (uint32_t)(p->bp_tile_n / 64);
-    p->bp_stages = pick_stages(stage, 1);
+    // rows of L lie Q*2 bytes apart; once that reaches a 2 MB page the direct stores of the epilogue (32
+    // lanes = 32 rows per instruction) touch 32 pages each, and staging whole rows in shared memory pays
+    p->bp_staged = Q >= (1L << 20) ? 1 : 0;
+    p->bp_stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK -
+                                                     (p->bp_staged ? BP_EPI_PITCH * TILE_M : 0)) / (int)stage));
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
@@ -858,6 +893,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.a_mn_major = 0;
   p.b_mn_major = 1;
   p.b_lbo = p.b_box_bytes;
+  p.epi_pitch = pl.bp_staged ? BP_EPI_PITCH : 0;
   p.tiles_m = pl.bp_tiles_r;
   p.tiles_n = pl.bp_tiles_q;
   p.taps = 1;
