@@ -562,10 +562,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int i = 0; i < 32; ++i)
                 if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
             }
+          } else if (p.mode == MODE_CONTRACT) {
+            // Partial tile in the order the accumulator comes out of tensor memory:
+            // block(split, offset, tile) [128-row tile][32-column chunk][4-column group][row][4 floats],
+            // so that the 32 lanes of every store write 512 contiguous bytes.  The reduce kernel undoes it.
+            float* blk = p.part + ((((long)w.split * p.T + w.tap) * p.tiles_m + w.tm) * p.tiles_n + w.tn) *
+                                      ((long)p.m_sub * TILE_M * p.tile_n);
+            float* dst = blk + ((long)(mt * (p.tile_n >> 5) + (c >> 5)) * 8 * TILE_M + quad * 32 + lane) * 4;
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+              if (i >= nc) break;
+              *reinterpret_cast<float4*>(dst + (long)(i >> 2) * TILE_M * 4) =
+                  make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]), __uint_as_float(v[i + 2]),
+                              __uint_as_float(v[i + 3]));
+            }
           } else {
-            float* dst;
-            if (p.mode == MODE_SKETCH) dst = p.part + ((long)w.split * p.rows + row) * p.cols + col0 + c;
-            else dst = p.part + (((long)w.split * p.rows + row) * p.T + w.tap) * p.Cin + col0 + c;
+            float* dst = p.part + ((long)w.split * p.rows + row) * p.cols + col0 + c;
             const bool vec = ((p.cols & 3) == 0);
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
@@ -637,25 +649,38 @@ __global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __res
   }
 }
 
+// out[m][offset][n] = scale(n) * sum_s block_s[...]: walks one split's blocks in their stored order (see the
+// epilogue of MODE_CONTRACT), four consecutive input channels per thread, splits added in ascending order.
 __global__ void __launch_bounds__(256) reduce_contract_partials(const float* __restrict__ part, float* __restrict__ out,
-                                                                long count, int splits, float alpha,
-                                                                const float* __restrict__ chan_scale, int period) {
+                                                                long groups, long split_stride, int splits, int T,
+                                                                int tiles_m, int tiles_n, int m_sub, int tile_n,
+                                                                int Cout, int Cin, float alpha,
+                                                                const float* __restrict__ chan_scale) {
   pdl_trigger();
   pdl_wait();
-  const long i = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (i >= count) return;                              // count is a multiple of 4 (Cin % 64 == 0)
+  long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= groups) return;
+  const long idx = t;
+  const int row = (int)(t % TILE_M); t /= TILE_M;
+  const int q = (int)(t % 8); t /= 8;
+  const int chunks = tile_n >> 5;
+  const int chunk = (int)(t % chunks); t /= chunks;
+  const int mt = (int)(t % m_sub); t /= m_sub;
+  const int tn = (int)(t % tiles_n); t /= tiles_n;
+  const int tm = (int)(t % tiles_m); t /= tiles_m;
+  const int tap = (int)t;
+  const int m = (tm * m_sub + mt) * TILE_M + row;
+  const int n = tn * tile_n + chunk * 32 + q * 4;
+  if (m >= Cout || n >= Cin) return;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
   for (int k = 0; k < splits; ++k) {
-    const float4 v = *reinterpret_cast<const float4*>(part + (long)k * count + i);
+    const float4 v = *reinterpret_cast<const float4*>(part + (long)k * split_stride + idx * 4);
     s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
   }
   float4 sc = make_float4(alpha, alpha, alpha, alpha);
-  if (chan_scale) {
-    const int n = (int)(i % period);
-    sc = make_float4(chan_scale[n], chan_scale[n + 1], chan_scale[n + 2], chan_scale[n + 3]);
-  }
-  *reinterpret_cast<float4*>(out + i) = make_float4(s.x * sc.x, s.y * sc.y, s.z * sc.z, s.w * sc.w);
+  if (chan_scale) sc = make_float4(chan_scale[n], chan_scale[n + 1], chan_scale[n + 2], chan_scale[n + 3]);
+  *reinterpret_cast<float4*>(out + ((long)m * T + tap) * Cin + n) = make_float4(s.x * sc.x, s.y * sc.y, s.z * sc.z, s.w * sc.w);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -855,7 +880,8 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     splits = std::max(1L, std::min(splits, 512L));
     p->ct_items_per_split = cdivl(p->ct_items, splits);
     p->ct_splits = (int)cdivl(p->ct_items, p->ct_items_per_split);
-    p->part_bytes = (size_t)p->ct_splits * d->Cout * T * d->Cin * sizeof(float);
+    p->part_bytes = (size_t)p->ct_splits * T * p->ct_tiles_m * p->ct_tiles_n * p->ct_m_sub * TILE_M * p->ct_tile_n *
+                    sizeof(float);
   }
   return mask;
 }
@@ -973,9 +999,11 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.status = reinterpret_cast<unsigned int*>(ws_head);
   xconv_status s = launch(ma, mb, p, (unsigned)std::min<long>(p.units, 4L * NUM_SMS), st);
   if (s != XCONV_OK) return s;
-  const long count = (long)d->Cout * T * d->Cin;
-  cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(count / 4, 256)), dim3(256), 0, st, p.part,
-                             dW, count, pl.ct_splits, alpha, d->chan_scale, d->Cin);
+  const long split_stride = (long)T * pl.ct_tiles_m * pl.ct_tiles_n * pl.ct_m_sub * TILE_M * pl.ct_tile_n;
+  const long groups = split_stride / 4;
+  cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(groups, 256)), dim3(256), 0, st, p.part,
+                             dW, groups, split_stride, pl.ct_splits, T, pl.ct_tiles_m, pl.ct_tiles_n, pl.ct_m_sub,
+                             pl.ct_tile_n, d->Cout, d->Cin, alpha, d->chan_scale);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
