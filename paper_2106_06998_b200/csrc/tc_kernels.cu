@@ -562,34 +562,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int i = 0; i < 32; ++i)
                 if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
             }
-          } else if (p.mode == MODE_CONTRACT) {
-            // Partial tile in the order the accumulator comes out of tensor memory:
+          } else {
+            // SKETCH / CONTRACT: partial tile in the order the accumulator comes out of tensor memory:
             // block(split, offset, tile) [128-row tile][32-column chunk][4-column group][row][4 floats],
-            // so that the 32 lanes of every store write 512 contiguous bytes.  The reduce kernel undoes it.
-            float* blk = p.part + ((((long)w.split * p.T + w.tap) * p.tiles_m + w.tm) * p.tiles_n + w.tn) *
-                                      ((long)p.m_sub * TILE_M * p.tile_n);
-            float* dst = blk + ((long)(mt * (p.tile_n >> 5) + (c >> 5)) * 8 * TILE_M + quad * 32 + lane) * 4;
+            // so that the 32 lanes of every store write 512 contiguous bytes.  The reduce kernels undo it.
+            const int chunks = (p.tile_n + 31) >> 5, qn = p.tile_n < 32 ? p.tile_n >> 2 : 8;   // 4-column groups per chunk
+            float* blk = p.part + ((((long)w.split * p.taps + w.tap) * p.tiles_m + w.tm) * p.tiles_n + w.tn) *
+                                      ((long)p.m_sub * TILE_M * chunks * qn * 4);
+            float* dst = blk + ((long)(mt * chunks + (c >> 5)) * qn * TILE_M + quad * 32 + lane) * 4;
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
               if (i >= nc) break;
               *reinterpret_cast<float4*>(dst + (long)(i >> 2) * TILE_M * 4) =
                   make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]), __uint_as_float(v[i + 2]),
                               __uint_as_float(v[i + 3]));
-            }
-          } else {
-            float* dst = p.part + ((long)w.split * p.rows + row) * p.cols + col0 + c;
-            const bool vec = ((p.cols & 3) == 0);
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              if (i >= nc) break;
-              if (vec && col0 + c + i + 3 < p.cols) {
-                *reinterpret_cast<float4*>(dst + i) = make_float4(__uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                                                  __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-              } else {
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                  if (col0 + c + i + e < p.cols) dst[i + e] = __uint_as_float(v[i + e]);
-              }
             }
           }
         }
@@ -624,28 +610,53 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   }
 }
 
-// S[j][b] = sum_s part[s][row][col] (s ascending within each of four interleaved groups, groups added in
-// order: a fixed tree, so results are reproducible); (row, col) = (b, j) when the samples were the MMA rows.
+// S[j][b] = sum over splits of the partial tiles, which are stored in accumulator order (see the
+// epilogue).  Four threads share a group of four columns and take the splits in turn; the four sums are
+// added in a fixed order, so the result is reproducible.  (row, col) = (b, j) when the samples were
+// the MMA rows.
 __global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S,
-                                                              int r, int B, int splits, int swapped) {
-  __shared__ float acc[4][64];
+                                                              long groups, long split_stride, int splits, int tiles_n,
+                                                              int m_sub, int tile_n, int rows, int cols, int B,
+                                                              int swapped) {
+  __shared__ float4 acc[4][64];
   pdl_trigger();
   pdl_wait();
   const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
-  const long count = (long)r * B;
-  const long i = (long)blockIdx.x * 64 + o;           // index in the layout of `part`
-  float s = 0.f;
-  if (i < count) {
+  const long idx = (long)blockIdx.x * 64 + o;          // group of four columns, in stored order
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (idx < groups) {
 #pragma unroll 4
-    for (int k = g; k < splits; k += 4) s += part[(long)k * count + i];
+    for (int k = g; k < splits; k += 4) {
+      const float4 v = *reinterpret_cast<const float4*>(part + (long)k * split_stride + idx * 4);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
   }
   acc[g][o] = s;
   __syncthreads();
-  if (g == 0 && i < count) {
-    const float t = ((acc[0][o] + acc[1][o]) + acc[2][o]) + acc[3][o];
-    long dst = i;
-    if (swapped) { const long b = i / r, j = i % r; dst = j * B + b; }
-    S[dst] = t;
+  if (g != 0 || idx >= groups) return;
+  float t4[4];
+  t4[0] = ((acc[0][o].x + acc[1][o].x) + acc[2][o].x) + acc[3][o].x;
+  t4[1] = ((acc[0][o].y + acc[1][o].y) + acc[2][o].y) + acc[3][o].y;
+  t4[2] = ((acc[0][o].z + acc[1][o].z) + acc[2][o].z) + acc[3][o].z;
+  t4[3] = ((acc[0][o].w + acc[1][o].w) + acc[2][o].w) + acc[3][o].w;
+  long t = idx;
+  const int qn = tile_n < 32 ? tile_n >> 2 : 8;
+  const int row = (int)(t % TILE_M); t /= TILE_M;
+  const int q = (int)(t % qn); t /= qn;
+  const int chunks = (tile_n + 31) >> 5;
+  const int chunk = (int)(t % chunks); t /= chunks;
+  const int mt = (int)(t % m_sub); t /= m_sub;
+  const int tn = (int)(t % tiles_n); t /= tiles_n;
+  const int tm = (int)t;
+  const long rr = (long)(tm * m_sub + mt) * TILE_M + row;
+  const int cl = chunk * 32 + q * 4;
+  if (rr >= rows || cl >= tile_n) return;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const long cc = (long)tn * tile_n + cl + e;
+    if (cc >= cols) break;
+    if (swapped) S[cc * B + rr] = t4[e];      // rows are samples, columns probes
+    else S[rr * B + cc] = t4[e];              // rows are probes, columns samples
   }
 }
 
@@ -720,6 +731,9 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
   return r == CUDA_SUCCESS;
 }
 
+// Columns a partial tile occupies in its stored (accumulator-order) layout.
+static int tile_cols_stored(int tile_n) { return tile_n < 32 ? tile_n : (tile_n + 31) / 32 * 32; }
+
 static int pow2_cols(int n) { int c = 32; while (c < n) c *= 2; return c; }
 
 static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
@@ -764,7 +778,8 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   splits = std::max(1L, std::min(splits, 512L));
   p->kblocks_per_split = cdivl(p->kblocks, splits);
   p->splits = (int)cdivl(p->kblocks, p->kblocks_per_split);
-  p->part_bytes = (size_t)p->splits * rows * cols * sizeof(float);
+  p->part_bytes = (size_t)p->splits * p->tiles_m * p->tiles_n * p->m_sub * TILE_M * tile_cols_stored(p->tile_n) *
+                  sizeof(float);
   return true;
 }
 
@@ -807,9 +822,11 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   p.status = reinterpret_cast<unsigned int*>(ws_head);
   xconv_status s = launch(ma, mb, p, (unsigned)p.units, st);
   if (s != XCONV_OK) return s;
-  const long count = (long)d->r * d->B;
-  cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(count, 64)), dim3(256), 0, st, p.part, S,
-                             d->r, d->B, pl.splits, pl.swap);
+  const long split_stride = (long)pl.tiles_m * pl.tiles_n * pl.m_sub * TILE_M * tile_cols_stored(pl.tile_n);
+  const long groups = split_stride / 4;
+  cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(groups, 64)), dim3(256), 0, st, p.part, S,
+                             groups, split_stride, pl.splits, pl.tiles_n, pl.m_sub, pl.tile_n, rows, cols, d->B,
+                             pl.swap);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
