@@ -283,6 +283,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ uint32_t tmem_slot;
   __shared__ int go;
 
+#ifdef XC_TIMELINE
+  const long long t_kernel0 = clock64();
+  if (threadIdx.x == 64 && blockIdx.x < 1024) g_waits[blockIdx.x * 8 + 5] = 0;
+#endif
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
@@ -488,6 +492,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
       }
+#ifdef XC_TIMELINE
+      const long long t_epi0 = clock64();
+#endif
       const long col0 = (long)w.tn * p.tile_n;
       for (int mt = 0; mt < p.m_sub; ++mt) {
         const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;    // first row of this warp
@@ -584,6 +591,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
+#ifdef XC_TIMELINE
+      if (warp == 2 && lane == 0 && blockIdx.x < 1024) {
+        g_waits[blockIdx.x * 8 + 5] += clock64() - t_epi0;
+        g_waits[blockIdx.x * 8 + 7] = clock64() - t_kernel0;
+      }
+#endif
       if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
         // Write the staged rows out: one 512-byte row (32 lanes x 16 B) per instruction.  Storing
         // straight from the accumulator layout would send the 32 lanes of every store to 32 probe rows

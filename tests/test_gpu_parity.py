@@ -71,6 +71,37 @@ def test_edge_shapes_all_elements(shape, dtype):
     _full_layer_parity(lay)
 
 
+# Shapes that reach the tcgen05 kernels with ragged tiles: channel counts that are not powers of two
+# (several 64- or 32-channel groups, partial last tile), images that no patch tiles exactly, probe counts
+# and batches that are not multiples of the MMA tile, r > B (re-associated wgrad) and r < B.
+TENSOR_EDGE_SHAPES = [
+    # B, Cin, Cout, H, W, r
+    (24, 192, 320, 9, 13, 40),        # Cout 320 = 256 + 64: two row tiles, the second half empty
+    (40, 320, 64, 10, 6, 24),         # Cin 320: column tiles 256 + 64
+    (16, 96, 160, 12, 20, 48),        # multiples of 32 only: 64-byte-swizzle contraction, several groups
+    (8, 32, 32, 40, 24, 72),          # one 32-channel group, r > B
+    (72, 64, 128, 7, 9, 136),         # r just above a 128-row tile, B % 64 != 0
+    (136, 128, 64, 5, 5, 8),          # tiny image (25 pixels), B above a tile, few probes
+    (8, 64, 64, 3, 70, 16),           # wide flat image
+]
+
+
+@pytest.mark.parametrize("shape", TENSOR_EDGE_SHAPES)
+def test_tensor_path_edge_shapes_all_elements(shape):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="bf16", seed=sum(shape), z="rademacher", x="relu")
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, torch.bfloat16)
+    assert xb.engine_for(desc, xb.OP_CONTRACT) == "tcgen05_bf16"
+    _full_layer_parity(lay)
+
+
+def test_pointwise_kernel_on_the_tensor_path():
+    lay = inputs.make_custom(16, 64, 128, 8, 12, 32, dtype="bf16", seed=78, KH=1, KW=1)
+    desc = xb.make_desc(16, 64, 128, 8, 12, 32, torch.bfloat16, 1)
+    assert xb.engine_for(desc, xb.OP_CONTRACT) == "tcgen05_bf16" and xb.engine_for(desc, xb.OP_FORWARD) == "tcgen05_bf16"
+    _full_layer_parity(lay, K=1)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_pointwise_kernel(dtype):
     lay = inputs.make_custom(3, 12, 20, 6, 10, 9, dtype=dtype, seed=77, KH=1, KW=1)
