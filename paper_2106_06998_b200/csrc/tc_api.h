@@ -12,6 +12,7 @@ struct TcSketchPlan {
   int swap;            // 0: MMA rows = probes, columns = samples; 1: rows = samples, columns = probes
   int tile_m, tile_n, m_sub;  // output tile of one work unit; m_sub 128-row MMA tiles share the other operand
   int tiles_m, tiles_n, splits;
+  int kgroup, rows_box;      // 64-wide k-blocks per stage; rows of the A box
   long kblocks, kblocks_per_split;
   int stages;
   size_t part_bytes;

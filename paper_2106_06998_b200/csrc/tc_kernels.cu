@@ -42,6 +42,8 @@ struct TcParams {
   int tmem_cols;           // power of two >= max(32, tile_n * m_sub * acc_bufs)
   int stages;
   int ksteps;              // UMMA k-steps (of 16) per stage
+  int kgroup;              // SKETCH: 64-wide k-blocks per stage (each its own K-major tile), 1 elsewhere
+  uint32_t a_jump, b_jump; // kgroup > 1: descriptor start-address step (>>4) from the last k-step of a block to the next block
   uint32_t a_stage_bytes, b_stage_bytes, tx_bytes;
   int a_boxes, b_boxes;    // TMA boxes per stage: A per 128-row tile, B in all
   uint32_t a_box_bytes, b_box_bytes, a_sub_bytes;
@@ -52,6 +54,7 @@ struct TcParams {
   uint32_t sbo, mn_step, layout;
   int cw_shift;            // log2 of the channels per tile block (6 or 5)
   uint32_t epi_pitch;      // BACKPROBE: row pitch of the shared-memory staging of the output tile (0 = none)
+  uint32_t smem_pad;       // bytes kept free behind the last stage: a 128-row MMA reads that far past a shorter A tile
   int tiles_m, tiles_n, taps;
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
@@ -176,16 +179,18 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32
 // All MMAs of one stage, fully unrolled.  The issuing thread runs alone in its warp, so every instruction
 // it executes costs a full dependent-issue slot (~6 cycles): a 128x64x16 MMA occupies the tensor pipe for
 // 32 cycles, i.e. about five instructions.  KS k-steps, TWO = two 128-row tiles share the B tile.
-template <int KS, bool TWO>
+// GROUPED: the stage holds KS/4 K-major tiles of 64 k each; after every fourth k-step the start
+// addresses jump to the next tile.
+template <int KS, bool TWO, bool GROUPED = false>
 __device__ __forceinline__ void umma_stage(uint32_t d, uint32_t tile_n, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
                                            uint32_t idesc, uint32_t acc, uint32_t a_step, uint32_t b_step,
-                                           uint32_t a_sub) {
+                                           uint32_t a_sub, uint32_t a_jump = 0, uint32_t b_jump = 0) {
 #pragma unroll
   for (int k = 0; k < KS; ++k) {
     umma_bf16(d, a_lo, hi, b_lo, hi, idesc, k == 0 ? acc : 1u);
     if (TWO) umma_bf16(d + tile_n, a_lo + a_sub, hi, b_lo, hi, idesc, k == 0 ? acc : 1u);
-    a_lo += a_step;
-    b_lo += b_step;
+    if (GROUPED && (k & 3) == 3) { a_lo += a_jump; b_lo += b_jump; }
+    else { a_lo += a_step; b_lo += b_step; }
   }
 }
 
@@ -332,7 +337,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int col0 = w.tn * p.tile_n;
         // running coordinates of the k-block
         int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0;
-        if (p.mode == MODE_SKETCH) kc = (int)(w.kb0 * 64);
+        if (p.mode == MODE_SKETCH) kc = (int)(w.kb0 * 64 * p.kgroup);
         else if (p.mode == MODE_BACKPROBE) kc = (int)w.kb0 * p.ksteps * 16;
         else if (p.mode == MODE_CONV) { dx = dy = -p.pad; }     // pj counts channel blocks, kc = offset * Cin
         else {
@@ -357,9 +362,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
           if (p.mode == MODE_SKETCH) {
             // one box per operand: 128*m_sub rows of A, tile_n rows of B, 64 k each
-            tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
-            tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
-            kc += 64;
+            if (p.kgroup > 1) {
+              // kgroup consecutive k-blocks per operand in one 3-d box (64 k, rows, k-blocks)
+              tma_load_3d(a_dst, &map_a, 0, row0, kc >> 6, &full_bar[s]);
+              tma_load_3d(b_dst, &map_b, 0, col0, kc >> 6, &full_bar[s]);
+              kc += 64 * p.kgroup;
+            } else {
+              tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
+              tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
+              kc += 64;
+            }
           } else if (p.mode == MODE_BACKPROBE) {
             tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
             // dY tile as one 3-d box (64 positions, k rows, tile_n/64 column groups)
@@ -441,7 +453,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           uint32_t a_lo = a_lo0 | s16;
           uint32_t b_lo = b_lo0 | (s16 + a_stage16);
 #define XC_STAGE(KS, TWO) umma_stage<KS, TWO>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, a_sub)
-          if (two) {
+#define XC_GROUP(KS, TWO) umma_stage<KS, TWO, true>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, \
+                                                    a_sub, p.a_jump, p.b_jump)
+          if (p.kgroup > 1) {
+            if (two) { if (ksteps == 8) XC_GROUP(8, true); else XC_GROUP(16, true); }
+            else { if (ksteps == 8) XC_GROUP(8, false); else XC_GROUP(16, false); }
+          } else if (two) {
             switch (ksteps) {
               case 4: XC_STAGE(4, true); break;
               case 7: XC_STAGE(7, true); break;
@@ -466,6 +483,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
 #undef XC_STAGE
+#undef XC_GROUP
           acc = 1u;
           umma_commit_a(empty_a);            // stage s may be refilled once these MMAs have read it
           s16 += stage16; full_a += 8; empty_a += 8;
@@ -757,7 +775,7 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
 
 static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
                            cudaStream_t st) {
-  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_pitch * TILE_M;
+  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_pitch * TILE_M + p.smem_pad;
   if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -783,11 +801,16 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   p->tile_m = TILE_M * p->m_sub;
   p->tiles_m = (int)cdivl(rows, p->tile_m);
   p->tiles_n = (int)cdivl(cols, p->tile_n);
-  p->kblocks = cdivl(K, 64);
-  const uint32_t stage = (uint32_t)p->m_sub * TILE_M * 128 + p->tile_n * 128;
-  p->stages = pick_stages(stage, 1);
+  // Small tiles: the cost of a stage is set by the two single-thread roles (barrier waits, copy issue,
+  // commit), not by its bytes, so a stage takes up to four 64-wide k-blocks of each operand at once.
+  p->rows_box = p->m_sub == 1 ? std::min(TILE_M, round_up(rows, 8)) : TILE_M * 2;
+  const uint32_t block = (uint32_t)p->rows_box * 128 + p->tile_n * 128;
+  p->kgroup = 1;
+  if (K % 64 == 0) p->kgroup = block <= 24 * 1024 ? 4 : block <= 36 * 1024 ? 2 : 1;
+  p->kblocks = cdivl(K, 64L * p->kgroup);
+  p->stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - TILE_M * 128) / (int)(block * p->kgroup)));
   const long tiles = (long)p->tiles_m * p->tiles_n;
-  long splits = std::max(1L, std::min((long)NUM_SMS / tiles, p->kblocks / 8));
+  long splits = std::max(1L, std::min((long)NUM_SMS / tiles, cdivl(K, 64) / 8));
   splits = std::max(1L, std::min(splits, 512L));
   p->kblocks_per_split = cdivl(p->kblocks, splits);
   p->splits = (int)cdivl(p->kblocks, p->kblocks_per_split);
@@ -803,12 +826,24 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   const void* A = pl.swap ? X : Z;
   const void* Bm = pl.swap ? Z : X;
   CUtensorMap ma, mb;
-  const uint64_t da[2] = {(uint64_t)K, (uint64_t)rows}, db[2] = {(uint64_t)K, (uint64_t)cols};
-  const uint64_t sa[1] = {(uint64_t)K * 2};
-  // full boxes always: rows and k positions past the tensor are zero-filled by the TMA unit
-  const uint32_t box_a[2] = {64, (uint32_t)(TILE_M * pl.m_sub)};
-  const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
-  if (!make_map(&ma, A, 2, da, sa, box_a) || !make_map(&mb, Bm, 2, db, sa, box_b)) return XCONV_ERR_CUDA;
+  // Rows and k positions past the tensor are zero-filled by the TMA unit.  When the whole operand has
+  // fewer rows than a tile the box stops at the last row (rounded to the 8-row swizzle group): rows the
+  // box never writes only feed accumulator rows that are never stored.
+  const uint32_t rows_box = (uint32_t)pl.rows_box;
+  if (pl.kgroup > 1) {
+    // (64 k, rows, k-blocks): one box brings kgroup K-major tiles, one behind the other in shared memory
+    const uint64_t da[3] = {64, (uint64_t)rows, (uint64_t)(K / 64)}, db[3] = {64, (uint64_t)cols, (uint64_t)(K / 64)};
+    const uint64_t sa[2] = {(uint64_t)K * 2, 128};
+    const uint32_t box_a[3] = {64, rows_box, (uint32_t)pl.kgroup};
+    const uint32_t box_b[3] = {64, (uint32_t)pl.tile_n, (uint32_t)pl.kgroup};
+    if (!make_map(&ma, A, 3, da, sa, box_a) || !make_map(&mb, Bm, 3, db, sa, box_b)) return XCONV_ERR_CUDA;
+  } else {
+    const uint64_t da[2] = {(uint64_t)K, (uint64_t)rows}, db[2] = {(uint64_t)K, (uint64_t)cols};
+    const uint64_t sa[1] = {(uint64_t)K * 2};
+    const uint32_t box_a[2] = {64, rows_box};
+    const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
+    if (!make_map(&ma, A, 2, da, sa, box_a) || !make_map(&mb, Bm, 2, db, sa, box_b)) return XCONV_ERR_CUDA;
+  }
   TcParams p{};
   p.mode = MODE_SKETCH;
   p.tile_n = pl.tile_n;
@@ -816,11 +851,18 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   p.acc_bufs = 1;
   p.tmem_cols = pow2_cols(pl.tile_n * pl.m_sub);
   p.stages = pl.stages;
-  p.ksteps = 4;
+  p.kgroup = pl.kgroup;
+  p.ksteps = 4 * pl.kgroup;
   p.a_sub_bytes = TILE_M * 128;
-  p.a_stage_bytes = (uint32_t)pl.m_sub * p.a_sub_bytes;
-  p.b_stage_bytes = (uint32_t)pl.tile_n * 128;
+  const uint32_t a_tile = rows_box * 128, b_tile = (uint32_t)pl.tile_n * 128;
+  p.a_stage_bytes = a_tile * pl.kgroup;
+  p.b_stage_bytes = b_tile * pl.kgroup;
+  p.a_jump = (a_tile >> 4) - 6;
+  p.b_jump = (b_tile >> 4) - 6;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  // The MMA always reads 128 rows of A.  Behind a shorter tile it reads whatever follows (the rows it
+  // produces are never stored), which must still be this CTA's shared memory.
+  p.smem_pad = TILE_M * 128 - std::min<uint32_t>(a_tile, TILE_M * 128);
   p.a_boxes = p.b_boxes = 1;
   p.a_mn_major = p.b_mn_major = 0;
   p.tiles_m = pl.tiles_m;

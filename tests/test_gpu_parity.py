@@ -95,6 +95,24 @@ def test_tensor_path_edge_shapes_all_elements(shape):
     _full_layer_parity(lay)
 
 
+@pytest.mark.parametrize("shape", [
+    # B, Cin, H, W, r
+    (8, 24, 11, 13, 16),      # K = 3432: a multiple of 8 but not of 64 -> one k-block per stage, short A tile
+    (24, 8, 17, 19, 8),       # K = 2584, samples on the MMA rows
+    (8, 64, 6, 35, 8),        # K = 13440 = 64 * 210: four k-blocks per stage, the last stage half past K
+    (200, 64, 5, 10, 8),      # two 128-row tiles, the second ragged; two k-blocks per stage
+])
+def test_sketch_tensor_path_k_blocking(shape):
+    B, Cin, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, 8, H, W, r, dtype="bf16", seed=sum(shape), z="gaussian", x="normal")
+    desc = xb.make_desc(B, Cin, 8, H, W, r, torch.bfloat16)
+    assert xb.engine_for(desc, xb.OP_SKETCH) == "tcgen05_bf16"
+    d = dev(lay)
+    S = xb.xconv_sketch(d["X"], d["Z"])
+    torch.cuda.synchronize()
+    check("sketch", host(S), O.sketch(lay["X"], lay["Z"]), TOL["bf16"])
+
+
 def test_pointwise_kernel_on_the_tensor_path():
     lay = inputs.make_custom(16, 64, 128, 8, 12, 32, dtype="bf16", seed=78, KH=1, KW=1)
     desc = xb.make_desc(16, 64, 128, 8, 12, 32, torch.bfloat16, 1)
