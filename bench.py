@@ -59,8 +59,8 @@ def layer_work(c, r):
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
 # profiles/ (None where the kernel has changed since, or was never captured).
 NCU_TRAFFIC = {   # (config, r, phase): bytes; profiles/tc_gemm_kernel_config5_r64_r256.md
-    (5, 64, "sketch"): 238.4e6, (5, 64, "backprobe"): 220.0e6, (5, 64, "contract"): 54.9e6,
-    (5, 256, "sketch"): 316.0e6, (5, 256, "backprobe"): 271.5e6, (5, 256, "contract"): 209.4e6,
+    (5, 64, "sketch"): 238.1e6, (5, 64, "backprobe"): 220.5e6, (5, 64, "contract"): 55.1e6,
+    (5, 256, "sketch"): 316.4e6, (5, 256, "backprobe"): 271.8e6, (5, 256, "contract"): 210.0e6,
 }
 
 
