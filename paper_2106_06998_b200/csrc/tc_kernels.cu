@@ -227,6 +227,9 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
 // spend waiting on barriers and issuing work, read back through xconv_debug_waits.
 #ifdef XC_TIMELINE
 __device__ long long g_waits[1024 * 8];
+__device__ long long g_times[1024 * 8];      // globaltimer (ns) at fixed points of the kernel, per CTA
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TT(slot) do { if (blockIdx.x < 1024) g_times[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
 #define TW_BEGIN long long _tw0 = clock64()
 #define TW_END(acc) acc += clock64() - _tw0
 #define TW_STORE(slot, acc) do { if (blockIdx.x < 1024) g_waits[blockIdx.x * 8 + (slot)] = (acc); } while (0)
@@ -234,6 +237,7 @@ __device__ long long g_waits[1024 * 8];
 #define TW_BEGIN do {} while (0)
 #define TW_END(acc) do {} while (0)
 #define TW_STORE(slot, acc) do {} while (0)
+#define TT(slot) do {} while (0)
 #endif
 
 constexpr int TILE_M = 128;
@@ -292,6 +296,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const long long t_kernel0 = clock64();
   if (threadIdx.x == 64 && blockIdx.x < 1024) g_waits[blockIdx.x * 8 + 5] = 0;
 #endif
+  if (threadIdx.x == 0) TT(0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
@@ -309,6 +314,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
   pdl_trigger();
   pdl_wait();                              // from here on the previous kernel's results are visible
+  if (threadIdx.x == 0) TT(1);
   if (threadIdx.x == 0) {
     // a CTA of this call gave up earlier: skip the work (one thread reads so that the whole CTA agrees)
     go = (*reinterpret_cast<volatile unsigned int*>(p.status) != p.tag) ? 1 : 0;
@@ -448,6 +454,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!mbar_try_wait_a(full_a, full_parity)) ok = mbar_wait_slow(&full_bar[s], full_parity, p.status, p.tag);
           TW_END(tw_mw); }
           if (!ok) break;
+#ifdef XC_TIMELINE
+          if (lu == 0 && i == 0) TT(2);
+#endif
           TW_BEGIN;
           tc_fence_after();
           uint32_t a_lo = a_lo0 | s16;
@@ -491,6 +500,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           TW_END(tw_mi);
         }
         if (ok) umma_commit(&tmem_full_bar[buf]);
+        TT(3);
         TW_STORE(2, tw_mw); TW_STORE(3, tw_mi); TW_STORE(4, clock64() - t_start);
       }
     }
@@ -512,6 +522,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
 #ifdef XC_TIMELINE
       const long long t_epi0 = clock64();
+      if (warp == 2 && lane == 0) TT(4);
 #endif
       const long col0 = (long)w.tn * p.tile_n;
       for (int mt = 0; mt < p.m_sub; ++mt) {
@@ -613,6 +624,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (warp == 2 && lane == 0 && blockIdx.x < 1024) {
         g_waits[blockIdx.x * 8 + 5] += clock64() - t_epi0;
         g_waits[blockIdx.x * 8 + 7] = clock64() - t_kernel0;
+        TT(5);
       }
 #endif
       if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
@@ -639,6 +651,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
+  if (threadIdx.x == 0) TT(6);
 }
 
 // S[j][b] = sum over splits of the partial tiles, which are stored in accumulator order (see the
@@ -1210,5 +1223,8 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
 #ifdef XC_TIMELINE
 extern "C" int xconv_debug_waits(long long* out) {
   return (int)cudaMemcpyFromSymbol(out, xconv::g_waits, sizeof(long long) * 1024 * 8);
+}
+extern "C" int xconv_debug_times(long long* out) {
+  return (int)cudaMemcpyFromSymbol(out, xconv::g_times, sizeof(long long) * 1024 * 8);
 }
 #endif
