@@ -810,7 +810,10 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   p->swap = d->B >= d->r ? 1 : 0;
   const int rows = p->swap ? d->B : d->r, cols = p->swap ? d->r : d->B;
   p->tile_n = std::min(256, round_up(cols, 16));
-  p->m_sub = rows > TILE_M ? 2 : 1;                      // two row tiles share each tile of the other operand
+  // Two row tiles that share each tile of the other operand halve the traffic into the SM per MMA, which
+  // pays once the sketch is bound by the tensor pipe (r*B/(r+B) flops per byte against the machine's
+  // ~250); below that it only doubles the split-k partial sums each CTA writes and the reduce re-reads.
+  p->m_sub = (rows > TILE_M && (long)d->r * d->B > 250L * (d->r + d->B)) ? 2 : 1;
   p->tile_m = TILE_M * p->m_sub;
   p->tiles_m = (int)cdivl(rows, p->tile_m);
   p->tiles_n = (int)cdivl(cols, p->tile_n);

@@ -100,7 +100,8 @@ def test_tensor_path_edge_shapes_all_elements(shape):
     (8, 24, 11, 13, 16),      # K = 3432: a multiple of 8 but not of 64 -> one k-block per stage, short A tile
     (24, 8, 17, 19, 8),       # K = 2584, samples on the MMA rows
     (8, 64, 6, 35, 8),        # K = 13440 = 64 * 210: four k-blocks per stage, the last stage half past K
-    (200, 64, 5, 10, 8),      # two 128-row tiles, the second ragged; two k-blocks per stage
+    (200, 64, 5, 10, 8),      # two 128-row tiles, the second ragged
+    (520, 8, 16, 16, 504),    # r*B/(r+B) > 250: pairs of row tiles share the column tile; both axes ragged
 ])
 def test_sketch_tensor_path_k_blocking(shape):
     B, Cin, H, W, r = shape
