@@ -68,6 +68,7 @@ struct TcParams {
   long Q;
   int T, Cin;              // CONTRACT output indexing; CONV: offsets and input channels
   int H, W, cgroups;       // CONV: image size and input-channel blocks of 64
+  int nimg;                // CONV: images; with m_sub = 2 a unit covers the same patch of images img and img + 1
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
 };
@@ -258,7 +259,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
     w.tn = (int)(q % p.tiles_n); q /= p.tiles_n;
     w.px = (int)(q % p.patches_x); q /= p.patches_x;
     w.py = (int)(q % p.patches_y); q /= p.patches_y;
-    w.img = (int)q;
+    w.img = (int)q * p.m_sub;
     w.tm = 0; w.tap = 0; w.split = 0;
   } else if (p.mode == MODE_BACKPROBE) {     // probe tiles innermost: the dY tile is re-read while hot in L2
     w.tm = (int)(u % p.tiles_m);
@@ -526,8 +527,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #endif
       const long col0 = (long)w.tn * p.tile_n;
       for (int mt = 0; mt < p.m_sub; ++mt) {
-        const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;    // first row of this warp
+        // first row of this warp; CONV: rows are the pixels of the patch, the row tile picks the image
+        const long row_w = (p.mode == MODE_CONV ? 0L : ((long)w.tm * p.m_sub + mt) * TILE_M) + quad * 32;
         if (row_w >= p.rows) continue;                                         // warp-uniform
+        if (p.mode == MODE_CONV && w.img + mt >= p.nimg) continue;
         const long row = row_w + lane;
         for (int c = 0; c < p.tile_n; c += 32) {
           if (col0 + c >= p.cols) break;
@@ -546,7 +549,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int pr = (int)row / p.patch_w, pc = (int)row % p.patch_w;
             const int y = w.py * p.patch_h + pr, x = w.px * p.patch_w + pc;
             if (y < p.H && x < p.W) {
-              bf16* dst = p.L + (((long)w.img * p.H + y) * p.W + x) * p.cols + col0 + c;
+              bf16* dst = p.L + (((long)(w.img + mt) * p.H + y) * p.W + x) * p.cols + col0 + c;
               if (nc == 32 && col0 + c + 32 <= p.cols) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
@@ -1157,7 +1160,12 @@ bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
   pick_patch_conv(d->H, d->W, &p->patch_w, &p->patch_h);
   p->patches_x = (int)cdivl(d->W, p->patch_w);
   p->patches_y = (int)cdivl(d->H, p->patch_h);
-  p->stages = pick_stages(TILE_M * 128 + (uint32_t)p->tile_n * 128, 1);
+  // Two images share each weight tile when the patch is a whole number of 8-row swizzle groups (the
+  // second image's rows then start on a group boundary): the traffic into the SM per MMA cycle falls
+  // from 94 to 62.5 bytes, which is what bounded the convolution.
+  const int px = p->patch_w * p->patch_h;
+  p->m_sub = (px % 8 == 0 && d->B >= 2) ? 2 : 1;
+  p->stages = pick_stages((uint32_t)(p->m_sub == 2 ? px + TILE_M : TILE_M) * 128 + (uint32_t)p->tile_n * 128, 1);
   p->wt_bytes = dgrad ? (size_t)d->Cout * d->KH * d->KW * d->Cin * 2 : 0;
   return true;
 }
@@ -1179,7 +1187,7 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   // input as (64 channels, x, y, channel blocks of 64, image); weights as [Co][T*Ci]
   const uint64_t da[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(Ci / 64), (uint64_t)d->B};
   const uint64_t sa[4] = {(uint64_t)Ci * 2, (uint64_t)d->W * Ci * 2, 128, (uint64_t)d->H * d->W * Ci * 2};
-  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1, 1};
+  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1, (uint32_t)pl.m_sub};
   const uint64_t db[2] = {(uint64_t)T * Ci, (uint64_t)Co};
   const uint64_t sb[1] = {(uint64_t)T * Ci * 2};
   const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
@@ -1187,23 +1195,27 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   TcParams p{};
   p.mode = MODE_CONV;
   p.tile_n = pl.tile_n;
-  p.m_sub = 1;
-  p.acc_bufs = 2;
-  p.tmem_cols = pow2_cols(2 * pl.tile_n);
+  const uint32_t px = (uint32_t)(pl.patch_w * pl.patch_h);
+  p.m_sub = pl.m_sub;
+  p.acc_bufs = (2 * pl.m_sub * pl.tile_n <= 512) ? 2 : 1;
+  p.tmem_cols = pow2_cols(p.acc_bufs * pl.m_sub * pl.tile_n);
   p.stages = pl.stages;
   p.ksteps = 4;
   p.a_boxes = p.b_boxes = 1;
-  p.a_sub_bytes = TILE_M * 128;
-  p.a_stage_bytes = p.a_sub_bytes;                 // the patch fills its first patch_w*patch_h rows
+  // one image: the patch fills the first px rows of a 128-row tile.  Two images: the second image's px
+  // rows follow the first's directly and its MMA tile starts there; 128 rows behind that start belong to the stage.
+  p.a_sub_bytes = (pl.m_sub == 2 ? px : (uint32_t)TILE_M) * 128;
+  p.a_stage_bytes = (pl.m_sub == 2 ? px + TILE_M : (uint32_t)TILE_M) * 128;
   p.b_stage_bytes = (uint32_t)pl.tile_n * 128;
-  p.tx_bytes = (uint32_t)(pl.patch_w * pl.patch_h) * 128 + p.b_stage_bytes;
+  p.tx_bytes = (uint32_t)pl.m_sub * px * 128 + p.b_stage_bytes;
   p.a_mn_major = p.b_mn_major = 0;
   p.tiles_m = 1;
   p.tiles_n = pl.tiles_n;
   p.taps = 1;
   p.kblocks = (long)T * (Ci / 64);
   p.kblocks_per_split = p.kblocks;
-  p.units = (long)d->B * pl.patches_y * pl.patches_x * pl.tiles_n;
+  p.units = cdivl(d->B, pl.m_sub) * pl.patches_y * pl.patches_x * pl.tiles_n;
+  p.nimg = d->B;
   p.patch_w = pl.patch_w;
   p.patch_h = pl.patch_h;
   p.patches_x = pl.patches_x;

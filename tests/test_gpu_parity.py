@@ -83,6 +83,7 @@ TENSOR_EDGE_SHAPES = [
     (72, 64, 128, 7, 9, 136),         # r just above a 128-row tile, B % 64 != 0
     (136, 128, 64, 5, 5, 8),          # tiny image (25 pixels), B above a tile, few probes
     (8, 64, 64, 3, 70, 16),           # wide flat image
+    (9, 64, 64, 6, 12, 16),           # odd batch: the last image pair of the convolution is half empty
 ]
 
 
