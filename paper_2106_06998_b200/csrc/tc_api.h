@@ -23,6 +23,7 @@ struct TcWgradPlan {
   int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps, bp_staged;
   // contraction
   int ct_cw, ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
+  int ct_tpu;                // kernel offsets per work unit (they share the L tile of every stage)
   int patch_h, patch_w, patches_y, patches_x;
   long ct_items, ct_items_per_split;
   size_t part_bytes;

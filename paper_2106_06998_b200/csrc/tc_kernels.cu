@@ -56,6 +56,12 @@ struct TcParams {
   uint32_t epi_pitch;      // BACKPROBE: row pitch of the shared-memory staging of the output tile (0 = none)
   uint32_t smem_pad;       // bytes kept free behind the last stage: a 128-row MMA reads that far past a shorter A tile
   int tiles_m, tiles_n, taps;
+  // CONTRACT: kernel offsets per work unit (1, 3 or 9).  The offsets of a unit share the L tile of every
+  // stage; their Z tiles lie one behind the other in the stage as consecutive column blocks, so one MMA
+  // spans several offsets: columns [0, tpu * tile_n) of the accumulator, in `pieces` MMAs of whole blocks.
+  int tpu, pieces;
+  uint32_t b_tap_bytes;    // bytes of one offset's Z tile
+  int piece_cols[2];       // N of each MMA
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
   // contraction geometry
@@ -267,12 +273,13 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
     w.tap = 0;
     w.split = 0;
   } else {                                   // tiles of one k-split are adjacent: they share operands in L2
-    const long tiles = (long)p.taps * p.tiles_m * p.tiles_n;
+    const int tpu = p.mode == MODE_CONTRACT ? p.tpu : 1;
+    const long tiles = (long)(p.taps / tpu) * p.tiles_m * p.tiles_n;
     long t = u % tiles;
     w.split = u / tiles;
     w.tn = (int)(t % p.tiles_n); t /= p.tiles_n;
     w.tm = (int)(t % p.tiles_m); t /= p.tiles_m;
-    w.tap = (int)t;
+    w.tap = (int)t * tpu;                      // first offset of the unit
   }
   w.kb0 = w.split * p.kblocks_per_split;
   const long kb1 = min(p.kblocks, w.kb0 + p.kblocks_per_split);
@@ -301,7 +308,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  const int acc_cols = p.tile_n * p.m_sub;                                    // columns of one accumulator set
+  const int unit_cols = p.mode == MODE_CONTRACT ? p.tile_n * p.tpu : p.tile_n;  // columns of one row tile's accumulator
+  const int acc_cols = unit_cols * p.m_sub;                                   // columns of one accumulator set
 
   // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
@@ -394,7 +402,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
             tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
-            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
+            if (p.tpu == 1) tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
+            else {
+              // the unit's offsets in row-major order from (dy, dx): one Z tile each, one behind the other
+              int ex = dx, ey = dy;
+              for (int t = 0; t < p.tpu; ++t) {
+                tma_load_5d(b_dst + (uint32_t)t * p.b_tap_bytes, &map_b, 0, x0 + ex, y0 + ey, col0 >> p.cw_shift, pj,
+                            &full_bar[s]);
+                if (++ex > p.pad) { ex = -p.pad; ++ey; }
+              }
+            }
             if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
           }
           ++it;
@@ -465,7 +482,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #define XC_STAGE(KS, TWO) umma_stage<KS, TWO>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, a_sub)
 #define XC_GROUP(KS, TWO) umma_stage<KS, TWO, true>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, \
                                                     a_sub, p.a_jump, p.b_jump)
-          if (p.kgroup > 1) {
+          if (p.mode == MODE_CONTRACT && p.tpu > 1) {
+            // several offsets per unit: per k-step one MMA per piece (and row tile), each spanning whole
+            // column blocks of consecutive offsets
+            const uint32_t b_piece = (uint32_t)(p.piece_cols[0] >> p.cw_shift) * (p.b_lbo >> 4);
+            const uint32_t id0 = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(p.piece_cols[0] >> 3) << 17);
+            const uint32_t id1 = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(p.piece_cols[1] >> 3) << 17);
+            for (int k = 0; k < ksteps; ++k) {
+              umma_bf16(d_tmem, a_lo, desc_hi, b_lo, desc_hi, id0, acc);
+              if (p.pieces > 1) umma_bf16(d_tmem + (uint32_t)p.piece_cols[0], a_lo, desc_hi, b_lo + b_piece, desc_hi, id1, acc);
+              if (two) {
+                umma_bf16(d_tmem + (uint32_t)unit_cols, a_lo + a_sub, desc_hi, b_lo, desc_hi, id0, acc);
+                if (p.pieces > 1)
+                  umma_bf16(d_tmem + (uint32_t)(unit_cols + p.piece_cols[0]), a_lo + a_sub, desc_hi, b_lo + b_piece, desc_hi, id1, acc);
+              }
+              acc = 1u; a_lo += a_step; b_lo += b_step;
+            }
+          } else if (p.kgroup > 1) {
             if (two) { if (ksteps == 8) XC_GROUP(8, true); else XC_GROUP(16, true); }
             else { if (ksteps == 8) XC_GROUP(8, false); else XC_GROUP(16, false); }
           } else if (two) {
@@ -532,13 +565,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (row_w >= p.rows) continue;                                         // warp-uniform
         if (p.mode == MODE_CONV && w.img + mt >= p.nimg) continue;
         const long row = row_w + lane;
-        for (int c = 0; c < p.tile_n; c += 32) {
+        for (int cu = 0; cu < unit_cols; cu += 32) {
+          // several offsets per unit (CONTRACT): tile_n is then a multiple of 32 and a chunk lies in one offset
+          const int tap_l = unit_cols > p.tile_n ? cu / p.tile_n : 0;
+          const int c = cu - tap_l * p.tile_n;
           if (col0 + c >= p.cols) break;
           uint32_t v[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = 0u;
           if (w.nkb > 0) {
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols + mt * p.tile_n + c);
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * acc_cols + mt * unit_cols + cu);
             if (p.tile_n - c >= 32) tmem_ld32(taddr, v);
             else tmem_ld16(taddr, v);
           }
@@ -606,7 +642,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // block(split, offset, tile) [128-row tile][32-column chunk][4-column group][row][4 floats],
             // so that the 32 lanes of every store write 512 contiguous bytes.  The reduce kernels undo it.
             const int chunks = (p.tile_n + 31) >> 5, qn = p.tile_n < 32 ? p.tile_n >> 2 : 8;   // 4-column groups per chunk
-            float* blk = p.part + ((((long)w.split * p.taps + w.tap) * p.tiles_m + w.tm) * p.tiles_n + w.tn) *
+            float* blk = p.part + ((((long)w.split * p.taps + w.tap + tap_l) * p.tiles_m + w.tm) * p.tiles_n + w.tn) *
                                       ((long)p.m_sub * TILE_M * chunks * qn * 4);
             float* dst = blk + ((long)(mt * chunks + (c >> 5)) * qn * TILE_M + quad * 32 + lane) * 4;
 #pragma unroll
@@ -961,12 +997,25 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     p->ct_tiles_n = (int)cdivl(d->Cin, p->ct_tile_n);
     const int bk = p->patch_w * p->patch_h;
     const uint32_t a_groups = d->Cout == p->ct_cw ? 1u : (uint32_t)((TILE_M / p->ct_cw) * p->ct_m_sub);
-    const uint32_t stage = (uint32_t)bk * (uint32_t)p->ct_cw * 2 * (a_groups + (uint32_t)cdivl(p->ct_tile_n, p->ct_cw));
+    const uint32_t b_groups = (uint32_t)cdivl(p->ct_tile_n, p->ct_cw);
+    const uint32_t block = (uint32_t)bk * (uint32_t)p->ct_cw * 2;
+    // Several kernel offsets per work unit while the accumulators fit tensor memory and two stages fit
+    // shared memory: the L tile of a stage is fetched once for all of them, and with few input channels
+    // one MMA spans the Z tiles of several offsets instead of issuing a narrow MMA for each.
+    p->ct_tpu = 1;
+    if (T == 9 && p->ct_tiles_n == 1 && p->ct_tile_n % 32 == 0 && p->ct_tile_n % p->ct_cw == 0)
+      for (int t = 9; t > 1; t /= 3)
+        if (t * p->ct_tile_n * p->ct_m_sub <= 512 && t * p->ct_tile_n <= 512 &&
+            2 * block * (a_groups + t * b_groups) <= (uint32_t)(SMEM_LIMIT - STATIC_SMEM_SLACK)) {
+          p->ct_tpu = t;
+          break;
+        }
+    const uint32_t stage = block * (a_groups + (uint32_t)p->ct_tpu * b_groups);
     // narrow tiles are bound by the one MMA-issuing thread of a CTA: run two CTAs per SM then
-    const int ct_ctas = (p->ct_tile_n * p->ct_m_sub <= 128 && stage * 2 <= 100 * 1024) ? 2 : 1;
+    const int ct_ctas = (p->ct_tpu * p->ct_tile_n * p->ct_m_sub <= 128 && stage * 2 <= 100 * 1024) ? 2 : 1;
     p->ct_stages = pick_stages(stage, ct_ctas);
     p->ct_items = (long)d->r * p->patches_x * p->patches_y;
-    const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * T;
+    const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * (T / p->ct_tpu);
     long splits = std::max(1L, std::min((long)NUM_SMS * ct_ctas / std::max(1L, tiles), p->ct_items / 4));
     splits = std::max(1L, std::min(splits, 512L));
     p->ct_items_per_split = cdivl(p->ct_items, splits);
@@ -1054,7 +1103,12 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.tile_n = pl.ct_tile_n;
   p.m_sub = pl.ct_m_sub;
   p.acc_bufs = 1;
-  p.tmem_cols = pow2_cols(pl.ct_tile_n * pl.ct_m_sub);
+  p.tpu = pl.ct_tpu;
+  const int n_total = pl.ct_tpu * pl.ct_tile_n, blocks = n_total / cw;
+  p.pieces = n_total > 256 ? 2 : 1;
+  p.piece_cols[0] = p.pieces == 2 ? (blocks + 1) / 2 * cw : n_total;
+  p.piece_cols[1] = n_total - p.piece_cols[0];
+  p.tmem_cols = pow2_cols(n_total * pl.ct_m_sub);
   p.stages = pl.ct_stages;
   p.ksteps = bk / 16;
   p.a_boxes = one_group ? 1 : TILE_M / cw;
@@ -1066,7 +1120,8 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.mn_step = 16 * row_bytes;
   p.layout = cw == 64 ? 2u : 4u;
   p.cw_shift = cw == 64 ? 6 : 5;
-  p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
+  p.b_tap_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
+  p.b_stage_bytes = (uint32_t)pl.ct_tpu * p.b_tap_bytes;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
   p.a_mn_major = p.b_mn_major = 1;
   p.a_lbo = one_group ? 0u : p.a_box_bytes;
@@ -1076,7 +1131,7 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.taps = T;
   p.kblocks = pl.ct_items;
   p.kblocks_per_split = pl.ct_items_per_split;
-  p.units = (long)pl.ct_tiles_m * pl.ct_tiles_n * T * pl.ct_splits;
+  p.units = (long)pl.ct_tiles_m * pl.ct_tiles_n * (T / pl.ct_tpu) * pl.ct_splits;
   p.patch_w = pl.patch_w;
   p.patch_h = pl.patch_h;
   p.patches_x = pl.patches_x;
