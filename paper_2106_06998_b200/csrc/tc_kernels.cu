@@ -201,6 +201,26 @@ __device__ __forceinline__ void umma_stage(uint32_t d, uint32_t tile_n, uint32_t
   }
 }
 
+// The same for a CONTRACT unit with several kernel offsets: per k-step one MMA per piece of the unit's
+// columns (`b_piece` = start-address step to the second piece's Z blocks) and per row tile.
+template <int KS, bool TWO, bool PIECES2>
+__device__ __forceinline__ void umma_stage_taps(uint32_t d, uint32_t unit_cols, uint32_t piece0_cols, uint32_t a_lo,
+                                                uint32_t b_lo, uint32_t b_piece, uint32_t hi, uint32_t id0, uint32_t id1,
+                                                uint32_t acc, uint32_t a_step, uint32_t b_step, uint32_t a_sub) {
+#pragma unroll
+  for (int k = 0; k < KS; ++k) {
+    const uint32_t ac = k == 0 ? acc : 1u;
+    umma_bf16(d, a_lo, hi, b_lo, hi, id0, ac);
+    if (PIECES2) umma_bf16(d + piece0_cols, a_lo, hi, b_lo + b_piece, hi, id1, ac);
+    if (TWO) {
+      umma_bf16(d + unit_cols, a_lo + a_sub, hi, b_lo, hi, id0, ac);
+      if (PIECES2) umma_bf16(d + unit_cols + piece0_cols, a_lo + a_sub, hi, b_lo + b_piece, hi, id1, ac);
+    }
+    a_lo += a_step;
+    b_lo += b_step;
+  }
+}
+
 // mbarrier arrive once every MMA issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
@@ -336,6 +356,58 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (!go) {
     // fall through to the teardown
+  } else if (warp == 0 && p.mode == MODE_CONTRACT && p.tpu > 1) {
+    // ------------------------------------------------------------------ TMA producer, several offsets per unit
+    // A 5-d tensor copy costs its issuing thread some 150-200 cycles, and a stage takes one per offset
+    // plus one: lane 0 waits for the stage, arms its barrier and fetches the L tile, lanes 1..tpu
+    // fetch the Z tile of one offset each, all at once.  Every lane walks the same loop.
+    const int stages = p.stages;
+    const int ks = 2 * p.pad + 1;
+    int s = 0;
+    long fill = 0, it = 0;
+    bool ok = true;
+    long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
+    for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+      const Unit w = decode_unit(p, u);
+      const int row0 = w.tm * p.m_sub * TILE_M;
+      const int col0 = w.tn * p.tile_n;
+      long q = w.kb0;
+      int px = (int)(q % p.patches_x); q /= p.patches_x;
+      int py = (int)(q % p.patches_y); q /= p.patches_y;
+      int pj = (int)q;
+      const int tap = w.tap + max(0, min(lane - 1, p.tpu - 1));          // this lane's offset
+      const int dy = tap / ks - p.pad, dx = tap % ks - p.pad;
+      for (int i = 0; i < w.nkb; ++i) {
+        if (fill > 0) {
+          TW_BEGIN;
+          if (lane == 0) ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+          TW_END(tw_pw);
+          if (!ok) break;
+        }
+        TW_BEGIN;
+        const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
+        const uint32_t b_dst = a_dst + p.a_stage_bytes;
+        const int x0 = px * p.patch_w, y0 = py * p.patch_h;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
+          tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
+        }
+        __syncwarp();                                 // the barrier is armed before any Z tile can land
+        if (lane >= 1 && lane <= p.tpu)
+          tma_load_5d(b_dst + (uint32_t)(lane - 1) * p.b_tap_bytes, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj,
+                      &full_bar[s]);
+        if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
+        ++it;
+        if (++s == stages) { s = 0; ++fill; }
+        TW_END(tw_pi);
+      }
+    }
+    if (lane == 0) { TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it); }
+    // drain: every copy issued must have landed in this CTA's shared memory before it exits
+    if (lane == 0)
+      for (long i = max(0L, it - stages); i < it; ++i)
+        if (!mbar_wait(&full_bar[i % stages], (uint32_t)((i / stages) & 1), p.status, p.tag)) break;
   } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     // One thread; its loop is kept free of divisions (coordinates advance incrementally).
@@ -402,16 +474,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
             tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
-            if (p.tpu == 1) tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
-            else {
-              // the unit's offsets in row-major order from (dy, dx): one Z tile each, one behind the other
-              int ex = dx, ey = dy;
-              for (int t = 0; t < p.tpu; ++t) {
-                tma_load_5d(b_dst + (uint32_t)t * p.b_tap_bytes, &map_b, 0, x0 + ex, y0 + ey, col0 >> p.cw_shift, pj,
-                            &full_bar[s]);
-                if (++ex > p.pad) { ex = -p.pad; ++ey; }
-              }
-            }
+            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
             if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
           }
           ++it;
@@ -488,16 +551,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t b_piece = (uint32_t)(p.piece_cols[0] >> p.cw_shift) * (p.b_lbo >> 4);
             const uint32_t id0 = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(p.piece_cols[0] >> 3) << 17);
             const uint32_t id1 = (idesc & ~(0x3Fu << 17)) | ((uint32_t)(p.piece_cols[1] >> 3) << 17);
-            for (int k = 0; k < ksteps; ++k) {
-              umma_bf16(d_tmem, a_lo, desc_hi, b_lo, desc_hi, id0, acc);
-              if (p.pieces > 1) umma_bf16(d_tmem + (uint32_t)p.piece_cols[0], a_lo, desc_hi, b_lo + b_piece, desc_hi, id1, acc);
-              if (two) {
-                umma_bf16(d_tmem + (uint32_t)unit_cols, a_lo + a_sub, desc_hi, b_lo, desc_hi, id0, acc);
-                if (p.pieces > 1)
-                  umma_bf16(d_tmem + (uint32_t)(unit_cols + p.piece_cols[0]), a_lo + a_sub, desc_hi, b_lo + b_piece, desc_hi, id1, acc);
+#define XC_TAPS(KS, TWO, P2) umma_stage_taps<KS, TWO, P2>(d_tmem, (uint32_t)unit_cols, (uint32_t)p.piece_cols[0], a_lo, \
+                                                         b_lo, b_piece, desc_hi, id0, id1, acc, a_step, b_step, a_sub)
+            const int shape = (two ? 2 : 0) | (p.pieces > 1 ? 1 : 0);
+            if (ksteps == 7 && shape == 0) XC_TAPS(7, false, false);
+            else if (ksteps == 7 && shape == 1) XC_TAPS(7, false, true);
+            else if (ksteps == 7 && shape == 2) XC_TAPS(7, true, false);
+            else if (ksteps == 7 && shape == 3) XC_TAPS(7, true, true);
+            else if (ksteps == 8 && shape == 0) XC_TAPS(8, false, false);
+            else if (ksteps == 8 && shape == 1) XC_TAPS(8, false, true);
+            else if (ksteps == 8 && shape == 2) XC_TAPS(8, true, false);
+            else if (ksteps == 8 && shape == 3) XC_TAPS(8, true, true);
+            else
+              for (int k = 0; k < ksteps; ++k) {
+                if (shape == 0) XC_TAPS(1, false, false);
+                else if (shape == 1) XC_TAPS(1, false, true);
+                else if (shape == 2) XC_TAPS(1, true, false);
+                else XC_TAPS(1, true, true);
+                acc = 1u; a_lo += a_step; b_lo += b_step;
               }
-              acc = 1u; a_lo += a_step; b_lo += b_step;
-            }
+#undef XC_TAPS
           } else if (p.kgroup > 1) {
             if (two) { if (ksteps == 8) XC_GROUP(8, true); else XC_GROUP(16, true); }
             else { if (ksteps == 8) XC_GROUP(8, false); else XC_GROUP(16, false); }
