@@ -13,19 +13,20 @@ struct TcSketchPlan {
   int tile_m, tile_n, m_sub;  // output tile of one work unit; m_sub 128-row MMA tiles share the other operand
   int tiles_m, tiles_n, splits;
   int kgroup, rows_box;      // 64-wide k-blocks per stage; rows of the A box
-  long kblocks, kblocks_per_split;
+  long kblocks, kblocks_per_split, kb_rem;   // the first kb_rem splits take one k-block more
   int stages;
   size_t part_bytes;
 };
 
 struct TcWgradPlan {
   // back-probe
-  int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps, bp_staged;
+  int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps, bp_rows_box, bp_slots;
+  long bp_base, bp_rem;      // column tiles: bp_base blocks of 64 positions each, the first bp_rem one more
   // contraction
   int ct_cw, ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
   int ct_tpu;                // kernel offsets per work unit (they share the L tile of every stage)
   int patch_h, patch_w, patches_y, patches_x;
-  long ct_items, ct_items_per_split;
+  long ct_items, ct_items_per_split, ct_items_rem;   // the first ct_items_rem splits take one item more
   size_t part_bytes;
 };
 

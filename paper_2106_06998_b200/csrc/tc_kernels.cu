@@ -53,7 +53,12 @@ struct TcParams {
   // the contraction of layers with 32-channel multiples, which uses 64-byte rows (layout 4, 512 B)
   uint32_t sbo, mn_step, layout;
   int cw_shift;            // log2 of the channels per tile block (6 or 5)
-  uint32_t epi_pitch;      // BACKPROBE: row pitch of the shared-memory staging of the output tile (0 = none)
+  // BACKPROBE: behind the stages every epilogue warp owns a ring of epi_slots staging slots of 4 KB (32 rows x
+  // 64 positions) from which it stores L with tensor stores; epi_bytes = 4 warps x epi_slots x 4 KB (0 elsewhere).
+  // Column tiles have bp_base blocks of 64 positions, the first bp_rem tiles one more (at most 4).
+  uint32_t epi_bytes;
+  int epi_slots;
+  long bp_base, bp_rem;
   uint32_t smem_pad;       // bytes kept free behind the last stage: a 128-row MMA reads that far past a shorter A tile
   int tiles_m, tiles_n, taps;
   // CONTRACT: kernel offsets per work unit (1, 3 or 9).  The offsets of a unit share the L tile of every
@@ -64,6 +69,7 @@ struct TcParams {
   int piece_cols[2];       // N of each MMA
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
+  long kb_rem;             // the first kb_rem k-splits take one k-block more than kblocks_per_split
   // contraction geometry
   int patch_w, patch_h, patches_x, patches_y, pad;
   // extents for the epilogue guards
@@ -154,6 +160,25 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4),
         "r"(smem_u32(bar)) : "memory");
 }
+// Tensor store shared -> global (bulk async-group completion) and its bookkeeping.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all earlier bulk stores of this thread have finished READING shared memory / have completed
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// at most `pending` (1, 3 or 7) of this thread's bulk stores may still be reading shared memory
+__device__ __forceinline__ void bulk_wait_read_upto(int pending) {
+  if (pending >= 7) bulk_wait_read<7>();
+  else if (pending >= 3) bulk_wait_read<3>();
+  else if (pending >= 1) bulk_wait_read<1>();
+  else bulk_wait_read<0>();
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -254,9 +279,9 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
 // spend waiting on barriers and issuing work, read back through xconv_debug_waits.
 #ifdef XC_TIMELINE
 __device__ long long g_waits[1024 * 8];
-__device__ long long g_times[1024 * 8];      // globaltimer (ns) at fixed points of the kernel, per CTA
+__device__ long long g_times[4 * 1024 * 8];  // globaltimer (ns) at fixed points of the kernel, per mode and CTA
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TT(slot) do { if (blockIdx.x < 1024) g_times[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
+#define TT(slot) do { if (blockIdx.x < 1024) g_times[((p.mode & 3) * 1024 + blockIdx.x) * 8 + (slot)] = gtime(); } while (0)
 #define TW_BEGIN long long _tw0 = clock64()
 #define TW_END(acc) acc += clock64() - _tw0
 #define TW_STORE(slot, acc) do { if (blockIdx.x < 1024) g_waits[blockIdx.x * 8 + (slot)] = (acc); } while (0)
@@ -275,11 +300,12 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-struct Unit { int tm, tn, tap; long split, kb0; int nkb; int px, py, img; };
+struct Unit { int tm, tn, tap; long split, kb0; int nkb; int px, py, img; int blk0, nblk; };
 
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
   Unit w;
   w.px = w.py = w.img = 0;
+  w.blk0 = w.nblk = 0;
   if (p.mode == MODE_CONV) {                 // channel tiles innermost, then patches of one image
     long q = u;
     w.tn = (int)(q % p.tiles_n); q /= p.tiles_n;
@@ -292,6 +318,9 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
     w.tn = (int)(u / p.tiles_m);
     w.tap = 0;
     w.split = 0;
+    // column tile tn covers blocks [blk0, blk0 + nblk) of 64 positions
+    w.blk0 = (int)(w.tn * p.bp_base + min((long)w.tn, p.bp_rem));
+    w.nblk = (int)p.bp_base + (w.tn < p.bp_rem ? 1 : 0);
   } else {                                   // tiles of one k-split are adjacent: they share operands in L2
     const int tpu = p.mode == MODE_CONTRACT ? p.tpu : 1;
     const long tiles = (long)(p.taps / tpu) * p.tiles_m * p.tiles_n;
@@ -301,8 +330,8 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
     w.tm = (int)(t % p.tiles_m); t /= p.tiles_m;
     w.tap = (int)t * tpu;                      // first offset of the unit
   }
-  w.kb0 = w.split * p.kblocks_per_split;
-  const long kb1 = min(p.kblocks, w.kb0 + p.kblocks_per_split);
+  w.kb0 = w.split * p.kblocks_per_split + min(w.split, p.kb_rem);
+  const long kb1 = min(p.kblocks, w.kb0 + p.kblocks_per_split + (w.split < p.kb_rem ? 1 : 0));
   w.nkb = (int)max(0L, kb1 - w.kb0);
   return w;
 }
@@ -311,7 +340,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
 
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const TcParams p) {
+               const __grid_constant__ CUtensorMap map_c, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[MAX_STAGES];
   __shared__ __align__(8) uint64_t empty_bar[MAX_STAGES];
@@ -339,6 +368,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     prefetch_tmap(&map_a);
     prefetch_tmap(&map_b);
+    if (p.mode == MODE_BACKPROBE) prefetch_tmap(&map_c);
   }
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
   pdl_trigger();
@@ -446,7 +476,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           TW_BEGIN;
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
           const uint32_t b_dst = a_dst + p.a_stage_bytes;
-          mbar_arrive_expect_tx(&full_bar[s], p.tx_bytes);
+          mbar_arrive_expect_tx(&full_bar[s], p.mode == MODE_BACKPROBE
+                                                  ? p.a_stage_bytes + (uint32_t)w.nblk * p.b_box_bytes : p.tx_bytes);
           if (p.mode == MODE_SKETCH) {
             // one box per operand: 128*m_sub rows of A, tile_n rows of B, 64 k each
             if (p.kgroup > 1) {
@@ -461,8 +492,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           } else if (p.mode == MODE_BACKPROBE) {
             tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
-            // dY tile as one 3-d box (64 positions, k rows, tile_n/64 column groups)
-            tma_load_3d(b_dst, &map_b, 0, kc, col0 >> 6, &full_bar[s]);
+            // dY tile: one box (64 positions x k rows) per block of the column tile, one behind the other
+            for (int b = 0; b < w.nblk; ++b)
+              tma_load_3d(b_dst + (uint32_t)b * p.b_box_bytes, &map_b, 0, kc, w.blk0 + b, &full_bar[s]);
             kc += p.ksteps * 16;
           } else if (p.mode == MODE_CONV) {
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
@@ -530,6 +562,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
         uint32_t acc = 0;
+        // BACKPROBE: the MMA spans the blocks this column tile has
+        const uint32_t idesc_u = p.mode == MODE_BACKPROBE
+                                     ? (idesc & ~(0x3Fu << 17)) | ((uint32_t)(w.nblk * 8) << 17) : idesc;
         for (int i = 0; i < w.nkb; ++i) {
           { TW_BEGIN;
           if (!mbar_try_wait_a(full_a, full_parity)) ok = mbar_wait_slow(&full_bar[s], full_parity, p.status, p.tag);
@@ -542,7 +577,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_fence_after();
           uint32_t a_lo = a_lo0 | s16;
           uint32_t b_lo = b_lo0 | (s16 + a_stage16);
-#define XC_STAGE(KS, TWO) umma_stage<KS, TWO>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, a_sub)
+#define XC_STAGE(KS, TWO) umma_stage<KS, TWO>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc_u, acc, a_step, b_step, a_sub)
 #define XC_GROUP(KS, TWO) umma_stage<KS, TWO, true>(d_tmem, tile_n, a_lo, b_lo, desc_hi, idesc, acc, a_step, b_step, \
                                                     a_sub, p.a_jump, p.b_jump)
           if (p.mode == MODE_CONTRACT && p.tpu > 1) {
@@ -615,6 +650,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------------------------------------------ epilogue (warps 2..5)
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
     const uint32_t epi_base = tiles_base + (uint32_t)p.stages * stage_bytes;
+    uint32_t epi_slot = 0;                    // BACKPROBE: next staging slot of this warp's ring
     long lu = 0;
     bool ok = true;
     for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
@@ -632,6 +668,47 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       if (warp == 2 && lane == 0) TT(4);
 #endif
       const long col0 = (long)w.tn * p.tile_n;
+      if (p.mode == MODE_BACKPROBE) {
+        // D[j, q] -> L[j][q].  Each warp stages 32 rows x 64 positions at a time in the layout the tensor store
+        // wants (128-byte rows, 16-byte pieces swizzled by the row; lane = row) and stores the block with one
+        // instruction; rows past the last probe are clipped by the TMA unit.  Storing straight from the
+        // accumulator layout would send the 32 lanes of every store instruction to 32 different rows of L.
+        for (int mt = 0; mt < p.m_sub; ++mt) {
+          const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;
+          if (row_w >= p.rows) continue;                                       // warp-uniform
+          for (int b = 0; b < w.nblk; ++b) {
+            // the store that used this slot epi_slots blocks ago must have read it
+            if (lane == 0) bulk_wait_read_upto(p.epi_slots - 1);
+            __syncwarp();
+            const uint32_t slot_base = epi_base + ((uint32_t)quad * p.epi_slots + epi_slot) * 4096u;
+            const uint32_t rowbase = slot_base + (uint32_t)lane * 128u;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+              uint32_t v[32];
+              tmem_ld32(tmem_base + ((uint32_t)(quad * 32) << 16) +
+                            (uint32_t)(buf * acc_cols + mt * unit_cols + b * 64 + half * 32), v);
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
+                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
+                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
+                const uint32_t sdst = rowbase + ((((uint32_t)half * 4u + (uint32_t)(i >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sdst),
+                             "r"(*reinterpret_cast<uint32_t*>(&h0)), "r"(*reinterpret_cast<uint32_t*>(&h1)),
+                             "r"(*reinterpret_cast<uint32_t*>(&h2)), "r"(*reinterpret_cast<uint32_t*>(&h3)) : "memory");
+              }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_3d(&map_c, slot_base, 0, (int)row_w, w.blk0 + b);
+              bulk_commit();
+            }
+            if (++epi_slot == (uint32_t)p.epi_slots) epi_slot = 0;
+          }
+        }
+      } else
       for (int mt = 0; mt < p.m_sub; ++mt) {
         // first row of this warp; CONV: rows are the pixels of the patch, the row tile picks the image
         const long row_w = (p.mode == MODE_CONV ? 0L : ((long)w.tm * p.m_sub + mt) * TILE_M) + quad * 32;
@@ -677,39 +754,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                   if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
               }
             }
-          } else if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
-            // D[j, q] -> staging row of this probe; the warp writes whole rows out afterwards
-            const uint32_t sdst = epi_base + (uint32_t)(quad * 32 + lane) * p.epi_pitch + (uint32_t)c * 2u;
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
-              __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-              __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sdst + (uint32_t)i * 2u),
-                           "r"(*reinterpret_cast<uint32_t*>(&h0)), "r"(*reinterpret_cast<uint32_t*>(&h1)),
-                           "r"(*reinterpret_cast<uint32_t*>(&h2)), "r"(*reinterpret_cast<uint32_t*>(&h3)) : "memory");
-            }
-          } else if (p.mode == MODE_BACKPROBE) {
-            // D[j, q] -> L[j][q]: each thread owns 32 consecutive positions of one probe
-            bf16* dst = p.L + row * p.Q + col0 + c;
-            if (nc == 32 && col0 + c + 32 <= p.cols) {
-#pragma unroll
-              for (int i = 0; i < 32; i += 8) {
-                uint4 o;
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
-                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-                o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
-                o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
-                *reinterpret_cast<uint4*>(dst + i) = o;
-              }
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
-            }
           } else {
             // SKETCH / CONTRACT: partial tile in the order the accumulator comes out of tensor memory:
             // block(split, offset, tile) [128-row tile][32-column chunk][4-column group][row][4 floats],
@@ -739,22 +783,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         TT(5);
       }
 #endif
-      if (p.mode == MODE_BACKPROBE && p.epi_pitch) {
-        // Write the staged rows out: one 512-byte row (32 lanes x 16 B) per instruction.  Storing
-        // straight from the accumulator layout would send the 32 lanes of every store to 32 probe rows
-        // that lie H*W*Cout*2 bytes apart -- one page each for large images.
-        const long row_w = (long)w.tm * TILE_M + quad * 32;
-        const long col = col0 + lane * 8;
-        for (int rr = 0; rr < 32; ++rr) {
-          if (row_w + rr >= p.rows) break;
-          uint4 o;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o.x), "=r"(o.y), "=r"(o.z), "=r"(o.w)
-                       : "r"(epi_base + (uint32_t)(quad * 32 + rr) * p.epi_pitch + (uint32_t)lane * 16u) : "memory");
-          if (col + 8 <= p.cols) *reinterpret_cast<uint4*>(p.L + (row_w + rr) * p.Q + col) = o;
-        }
-        __syncwarp();
-      }
     }
+    // the tensor stores read this CTA's shared memory: they must be done before it exits
+    if (p.mode == MODE_BACKPROBE && lane == 0) bulk_wait_all();
   }
 
   tc_fence_before();
@@ -767,22 +798,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 }
 
 // S[j][b] = sum over splits of the partial tiles, which are stored in accumulator order (see the
-// epilogue).  Four threads share a group of four columns and take the splits in turn; the four sums are
-// added in a fixed order, so the result is reproducible.  (row, col) = (b, j) when the samples were
-// the MMA rows.
-__global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S,
-                                                              long groups, long split_stride, int splits, int tiles_n,
-                                                              int m_sub, int tile_n, int rows, int cols, int B,
-                                                              int swapped) {
-  __shared__ float4 acc[4][64];
+// epilogue).  Sixteen threads share a group of four columns and take the splits in turn (with some 150
+// splits of a small tile the kernel is a chain of dependent loads otherwise); their sums are added in a
+// fixed order, so the result is reproducible.  (row, col) = (b, j) when the samples were the MMA rows.
+constexpr int RS_LANES = 16, RS_GROUPS = 16;
+__global__ void __launch_bounds__(RS_LANES * RS_GROUPS)
+reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S, long groups, long split_stride,
+                       int splits, int tiles_n, int m_sub, int tile_n, int rows, int cols, int B, int swapped) {
+  __shared__ float4 acc[RS_LANES][RS_GROUPS];
   pdl_trigger();
   pdl_wait();
-  const int o = threadIdx.x & 63, g = threadIdx.x >> 6;
-  const long idx = (long)blockIdx.x * 64 + o;          // group of four columns, in stored order
+  const int o = threadIdx.x % RS_GROUPS, g = threadIdx.x / RS_GROUPS;
+  const long idx = (long)blockIdx.x * RS_GROUPS + o;   // group of four columns, in stored order
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
   if (idx < groups) {
 #pragma unroll 4
-    for (int k = g; k < splits; k += 4) {
+    for (int k = g; k < splits; k += RS_LANES) {
       const float4 v = *reinterpret_cast<const float4*>(part + (long)k * split_stride + idx * 4);
       s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
     }
@@ -790,11 +821,11 @@ __global__ void __launch_bounds__(256) reduce_sketch_partials(const float* __res
   acc[g][o] = s;
   __syncthreads();
   if (g != 0 || idx >= groups) return;
-  float t4[4];
-  t4[0] = ((acc[0][o].x + acc[1][o].x) + acc[2][o].x) + acc[3][o].x;
-  t4[1] = ((acc[0][o].y + acc[1][o].y) + acc[2][o].y) + acc[3][o].y;
-  t4[2] = ((acc[0][o].z + acc[1][o].z) + acc[2][o].z) + acc[3][o].z;
-  t4[3] = ((acc[0][o].w + acc[1][o].w) + acc[2][o].w) + acc[3][o].w;
+  float t4[4] = {acc[0][o].x, acc[0][o].y, acc[0][o].z, acc[0][o].w};
+#pragma unroll
+  for (int l = 1; l < RS_LANES; ++l) {
+    t4[0] += acc[l][o].x; t4[1] += acc[l][o].y; t4[2] += acc[l][o].z; t4[3] += acc[l][o].w;
+  }
   long t = idx;
   const int qn = tile_n < 32 ? tile_n >> 2 : 8;
   const int row = (int)(t % TILE_M); t /= TILE_M;
@@ -857,7 +888,7 @@ static inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 static const int SMEM_LIMIT = 227 * 1024;
 static const int STATIC_SMEM_SLACK = 2048;     // barriers + alignment slack
 static const int NUM_SMS = 148;
-static const int BP_EPI_PITCH = 512 + 16;   // staged back-probe output rows: 256 bf16 + padding against bank conflicts
+static const int BP_SLOT_BYTES = 4 * 32 * 128;      // back-probe output staging: per slot, 4 warps x 32 rows x 64 positions
 
 static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -899,15 +930,15 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
 }
 
 static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
-                           cudaStream_t st) {
-  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_pitch * TILE_M + p.smem_pad;
+                           cudaStream_t st, const CUtensorMap* mc = nullptr) {
+  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_bytes + p.smem_pad;
   if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
   cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   TcParams q = p;
   q.tag = call_tag();
   if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
-  e = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, q);
+  e = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, mc ? *mc : ma, q);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
@@ -934,14 +965,17 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   p->rows_box = p->m_sub == 1 ? std::min(TILE_M, round_up(rows, 8)) : TILE_M * 2;
   const uint32_t block = (uint32_t)p->rows_box * 128 + p->tile_n * 128;
   p->kgroup = 1;
-  if (K % 64 == 0) p->kgroup = block <= 24 * 1024 ? 4 : block <= 36 * 1024 ? 2 : 1;
+  if (K % 64 == 0) p->kgroup = block <= 12 * 1024 ? 4 : block <= 36 * 1024 ? 2 : 1;
   p->kblocks = cdivl(K, 64L * p->kgroup);
   p->stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - TILE_M * 128) / (int)(block * p->kgroup)));
   const long tiles = (long)p->tiles_m * p->tiles_n;
   long splits = std::max(1L, std::min((long)NUM_SMS / tiles, cdivl(K, 64) / 8));
   splits = std::max(1L, std::min(splits, 512L));
-  p->kblocks_per_split = cdivl(p->kblocks, splits);
-  p->splits = (int)cdivl(p->kblocks, p->kblocks_per_split);
+  // k-blocks dealt as evenly as they go: every split takes kblocks_per_split, the first kb_rem one more
+  splits = std::min(splits, p->kblocks);
+  p->splits = (int)splits;
+  p->kblocks_per_split = p->kblocks / splits;
+  p->kb_rem = p->kblocks % splits;
   p->part_bytes = (size_t)p->splits * p->tiles_m * p->tiles_n * p->m_sub * TILE_M * tile_cols_stored(p->tile_n) *
                   sizeof(float);
   return true;
@@ -998,6 +1032,7 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   p.taps = 1;
   p.kblocks = pl.kblocks;
   p.kblocks_per_split = pl.kblocks_per_split;
+  p.kb_rem = pl.kb_rem;
   p.units = (long)pl.tiles_m * pl.tiles_n * pl.splits;
   p.rows = rows;
   p.cols = cols;
@@ -1007,7 +1042,8 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   if (s != XCONV_OK) return s;
   const long split_stride = (long)pl.tiles_m * pl.tiles_n * pl.m_sub * TILE_M * tile_cols_stored(pl.tile_n);
   const long groups = split_stride / 4;
-  cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(groups, 64)), dim3(256), 0, st, p.part, S,
+  cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(groups, RS_GROUPS)),
+                             dim3(RS_LANES * RS_GROUPS), 0, st, p.part, S,
                              groups, split_stride, pl.splits, pl.tiles_n, pl.m_sub, pl.tile_n, rows, cols, d->B,
                              pl.swap);
   count_launch();
@@ -1041,18 +1077,33 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   if (Q % 64 == 0 && d->B % 8 == 0 && Q >= 2048 && Q < 2000000000L) {
     mask |= 1;
     p->bp_tile_n = 256;
-    p->bp_tiles_q = (int)cdivl(Q, p->bp_tile_n);
     p->bp_m_sub = 1;
     p->bp_acc_bufs = (2 * p->bp_m_sub * p->bp_tile_n <= 512) ? 2 : 1;
     p->bp_tiles_r = (int)cdivl(d->r, TILE_M * p->bp_m_sub);
+    // Column tiles of up to four 64-position blocks, sized so that every CTA of the persistent grid gets
+    // the same number of units and (to within one block) the same number of blocks: with tiles of a fixed
+    // width the CTAs that run one tile more than the rest finish alone, at a fraction of the bandwidth.
+    const long NB = Q / 64, TM = p->bp_tiles_r;
+    const long rounds = cdivl(NB * TM, 4L * NUM_SMS), units = rounds * NUM_SMS;
+    long NT = cdivl(NB, 4);
+    if (units % TM == 0 && units / TM <= NB && units / TM >= NT) NT = units / TM;
+    p->bp_tiles_q = (int)NT;
+    p->bp_base = NB / NT;
+    p->bp_rem = NB % NT;
     p->bp_ksteps = std::min(4, (int)cdivl(d->B, 16));
-    const uint32_t stage = (uint32_t)p->bp_m_sub * TILE_M * 128 +
-                           (uint32_t)p->bp_ksteps * 16 * 128 * (uint32_t)(p->bp_tile_n / 64);
-    // rows of L lie Q*2 bytes apart; once that reaches a 2 MB page the direct stores of the epilogue (32
-    // lanes = 32 rows per instruction) touch 32 pages each, and staging whole rows in shared memory pays
-    p->bp_staged = Q >= (1L << 20) ? 1 : 0;
-    p->bp_stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK -
-                                                     (p->bp_staged ? BP_EPI_PITCH * TILE_M : 0)) / (int)stage));
+    // the S tile of a stage holds only the probes there are (in 8-row swizzle groups): the 128-row MMA then
+    // reads on into the dY tile and whatever lies behind it in this CTA's shared memory, and the rows it
+    // makes of that are never stored
+    p->bp_rows_box = p->bp_m_sub == 1 ? std::min(TILE_M, round_up(d->r, 8)) : TILE_M * p->bp_m_sub;
+    const int stage = p->bp_rows_box * 128 + p->bp_ksteps * 16 * 128 * (p->bp_tile_n / 64);
+    // Behind the stages: the epilogue warps' rings of staging slots.  Deeper rings let more tensor stores
+    // be in flight, but a unit's k-blocks should all fit the stage ring (at least four stages otherwise).
+    const int budget = SMEM_LIMIT - STATIC_SMEM_SLACK;
+    const int want = std::min(4, (int)cdivl(d->B, p->bp_ksteps * 16) + 1);
+    p->bp_slots = 2;
+    for (int slots = 8; slots >= 2; slots /= 2)
+      if ((budget - slots * BP_SLOT_BYTES) / stage >= want) { p->bp_slots = slots; break; }
+    p->bp_stages = std::max(1, std::min(MAX_STAGES, (budget - p->bp_slots * BP_SLOT_BYTES) / stage));
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
   const int T = d->KH * d->KW;
@@ -1091,8 +1142,10 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     const long tiles = (long)p->ct_tiles_m * p->ct_tiles_n * (T / p->ct_tpu);
     long splits = std::max(1L, std::min((long)NUM_SMS * ct_ctas / std::max(1L, tiles), p->ct_items / 4));
     splits = std::max(1L, std::min(splits, 512L));
-    p->ct_items_per_split = cdivl(p->ct_items, splits);
-    p->ct_splits = (int)cdivl(p->ct_items, p->ct_items_per_split);
+    splits = std::min(splits, p->ct_items);
+    p->ct_splits = (int)splits;
+    p->ct_items_per_split = p->ct_items / splits;
+    p->ct_items_rem = p->ct_items % splits;
     p->part_bytes = (size_t)p->ct_splits * T * p->ct_tiles_m * p->ct_tiles_n * p->ct_m_sub * TILE_M * p->ct_tile_n *
                     sizeof(float);
   }
@@ -1105,14 +1158,20 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const int bk = pl.bp_ksteps * 16;
   CUtensorMap ma, mb;
   // A = S (bfloat16) [r][B], k = b contiguous; B operand = dY [B][Q], q contiguous (MN-major tile)
-  // dY as (64 positions, B rows, Q/64 groups of 64 positions): one box fetches the whole [bk x tile_n] tile
-  // as tile_n/64 consecutive blocks of 128-byte rows
+  // dY as (64 positions, B rows, Q/64 blocks of 64 positions): one box fetches the [bk x 64] piece of one
+  // block as 128-byte rows; the blocks of a column tile lie one behind the other in the stage
   const uint64_t da[2] = {(uint64_t)d->B, (uint64_t)d->r};
   const uint64_t db[3] = {64, (uint64_t)d->B, (uint64_t)(Q / 64)};
   const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[2] = {(uint64_t)Q * 2, 128};
-  const uint32_t box_a[2] = {64, (uint32_t)(TILE_M * pl.bp_m_sub)};   // 128-byte rows whatever bk is (zero fill past B)
-  const uint32_t box_b[3] = {64, (uint32_t)bk, (uint32_t)(pl.bp_tile_n / 64)};
+  const uint32_t box_a[2] = {64, (uint32_t)pl.bp_rows_box};           // 128-byte rows whatever bk is (zero fill past B)
+  const uint32_t box_b[3] = {64, (uint32_t)bk, 1};
   if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 3, db, sb, box_b)) return XCONV_ERR_CUDA;
+  // L [r][Q] for the epilogue's stores, as (64 positions, r rows, Q/64 groups): one box = the 32 rows of one
+  // epilogue warp x one block of positions
+  CUtensorMap mc;
+  const uint64_t dc[3] = {64, (uint64_t)d->r, (uint64_t)(Q / 64)};
+  const uint32_t box_c[3] = {64, 32, 1};
+  if (!make_map(&mc, L, 3, dc, sb, box_c)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_BACKPROBE;
   p.tile_n = pl.bp_tile_n;
@@ -1124,7 +1183,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.a_boxes = 1;
   p.b_boxes = pl.bp_tile_n / 64;
   p.a_sub_bytes = TILE_M * 128;
-  p.a_stage_bytes = (uint32_t)pl.bp_m_sub * p.a_sub_bytes;
+  p.a_stage_bytes = (uint32_t)pl.bp_rows_box * 128;
   p.a_box_bytes = p.a_stage_bytes;
   p.b_box_bytes = (uint32_t)bk * 128;
   p.b_stage_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
@@ -1132,7 +1191,10 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.a_mn_major = 0;
   p.b_mn_major = 1;
   p.b_lbo = p.b_box_bytes;
-  p.epi_pitch = pl.bp_staged ? BP_EPI_PITCH : 0;
+  p.epi_bytes = (uint32_t)pl.bp_slots * BP_SLOT_BYTES;
+  p.epi_slots = pl.bp_slots;
+  p.bp_base = pl.bp_base;
+  p.bp_rem = pl.bp_rem;
   p.tiles_m = pl.bp_tiles_r;
   p.tiles_n = pl.bp_tiles_q;
   p.taps = 1;
@@ -1144,7 +1206,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st);
+  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st, &mc);
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
@@ -1204,6 +1266,7 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.taps = T;
   p.kblocks = pl.ct_items;
   p.kblocks_per_split = pl.ct_items_per_split;
+  p.kb_rem = pl.ct_items_rem;
   p.units = (long)pl.ct_tiles_m * pl.ct_tiles_n * (T / pl.ct_tpu) * pl.ct_splits;
   p.patch_w = pl.patch_w;
   p.patch_h = pl.patch_h;
@@ -1368,6 +1431,6 @@ extern "C" int xconv_debug_waits(long long* out) {
   return (int)cudaMemcpyFromSymbol(out, xconv::g_waits, sizeof(long long) * 1024 * 8);
 }
 extern "C" int xconv_debug_times(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, xconv::g_times, sizeof(long long) * 1024 * 8);
+  return (int)cudaMemcpyFromSymbol(out, xconv::g_times, sizeof(long long) * 4 * 1024 * 8);
 }
 #endif

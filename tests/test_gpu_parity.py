@@ -115,6 +115,23 @@ def test_sketch_tensor_path_k_blocking(shape):
     check("sketch", host(S), O.sketch(lay["X"], lay["Z"]), TOL["bf16"])
 
 
+@pytest.mark.parametrize("shape", [
+    # B, Cout, H, W, r -- the persistent grid runs several rounds of column tiles of unequal width
+    (16, 64, 24, 40, 136),    # 960 blocks of 64 positions, two probe tiles (the second has 8 rows)
+    (24, 64, 30, 33, 40),     # 990 blocks: tiles of four and of three blocks, r not a multiple of 32
+    (8, 128, 31, 29, 200),    # 1798 blocks, B below one 64-wide k-block
+])
+def test_backprobe_tensor_path_column_tiles(shape):
+    B, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, 8, Cout, H, W, r, dtype="bf16", seed=sum(shape), z="gaussian", x="normal")
+    desc = xb.make_desc(B, 8, Cout, H, W, r, torch.bfloat16)
+    assert xb.engine_for(desc, xb.OP_BACKPROBE) == "tcgen05_bf16"
+    S = np.random.Generator(np.random.PCG64(sum(shape))).standard_normal((r, B)).astype(np.float32)
+    L = xb.xconv_backprobe(torch.from_numpy(S).cuda(), dev(lay)["dY"])
+    torch.cuda.synchronize()
+    check("L", host(L), O.backprobe(S, lay["dY"]), TOL["bf16"])
+
+
 def test_pointwise_kernel_on_the_tensor_path():
     lay = inputs.make_custom(16, 64, 128, 8, 12, 32, dtype="bf16", seed=78, KH=1, KW=1)
     desc = xb.make_desc(16, 64, 128, 8, 12, 32, torch.bfloat16, 1)
