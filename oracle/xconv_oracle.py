@@ -33,6 +33,9 @@ Pinned by tests/test_oracle_pins.py: brute-force loops and finite differences
 (conv_forward, dw_exact, dx_exact), exact recovery with an orthogonal probe basis,
 unbiasedness, the closed-form Hutchinson variance, Proposition 1's bound and the
 literal block-matrix estimator of Eq. (6) (sketch, backprobe, wgrad_estimate).
+philox4x32_10 and rademacher_probes (probing vectors redrawn from a stored seed, Algorithm 1) are pinned
+by the generator's published known-answer vectors (tests/golden/philox4x32_10_kat.txt), by the
+balance and independence of the signs, and by the unbiasedness of the estimator run on them.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -228,6 +231,49 @@ def wgrad_estimate_literal(X, dY, Z, KH=3, KW=3, pad=None, circular=False):
                         acc += Zc[n * N:(n + 1) * N, j] @ AZ[m * N:(m + 1) * N, j]   # (iii)
                     dW[m, n, ky, kx] = acc / r
     return dW
+
+
+def philox4x32_10(counter, key):
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2,
+    3", SC'11, Section 3.3 and Table 2): a counter-based generator, 128-bit counter -> 128 random bits.
+
+    ``counter``: four arrays of 32-bit words (c0 least significant), ``key``: two 32-bit words.
+    One round: (hi0, lo0) = M0 * c0, (hi1, lo1) = M1 * c2 (32 x 32 -> 64-bit products),
+    c <- (hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0); after every round the key is bumped by the Weyl
+    constants (k0 += W0, k1 += W1).  Returns the four output words as uint64 arrays below 2^32.
+    """
+    M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+    u = np.uint64
+    mask = u(0xFFFFFFFF)
+    c = [np.asarray(x, dtype=np.uint64) & mask for x in counter]
+    k0, k1 = u(int(key[0]) & 0xFFFFFFFF), u(int(key[1]) & 0xFFFFFFFF)
+    for _ in range(10):
+        p0, p1 = u(M0) * c[0], u(M1) * c[2]
+        hi0, lo0, hi1, lo1 = p0 >> u(32), p0 & mask, p1 >> u(32), p1 & mask
+        c = [hi1 ^ c[1] ^ k0, lo1, hi0 ^ c[3] ^ k1, lo0]
+        k0, k1 = (k0 + u(W0)) & mask, (k1 + u(W1)) & mask
+    return c
+
+
+def rademacher_probes(seed: int, r: int, Cin: int, H: int, W: int) -> np.ndarray:
+    """The probing vectors Z[s] redrawn from the stored seed s (Algorithm 1: forward step 2 draws the seed,
+    backward step 2 redraws "Z = randn(N, r)" from it), with Rademacher entries.
+
+    Definition (fixed by this library, the paper leaves the generator open): number the entries of Z by
+    e = ((j*H + y)*W + x)*Cin + n (probe j, pixel (y, x), input channel n).  Entry e is +1 if bit (e mod
+    128) of philox4x32_10(counter = e div 128 as a 128-bit number, key = the two 32-bit halves of the seed)
+    is 0 and -1 if it is 1; bit b is bit (b mod 32) of output word (b div 32).
+    Returns Z [r, Cin, H, W] float64.
+    """
+    total = r * Cin * H * W
+    blocks = np.arange((total + 127) // 128, dtype=np.uint64)
+    zero = np.zeros_like(blocks)
+    words = philox4x32_10((blocks & np.uint64(0xFFFFFFFF), blocks >> np.uint64(32), zero, zero),
+                          (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    shifts = np.arange(32, dtype=np.uint64)
+    bits = np.stack([(w[:, None] >> shifts[None, :]) & np.uint64(1) for w in words], axis=1)   # [block, word, bit]
+    signs = 1.0 - 2.0 * bits.reshape(-1)[:total].astype(F64)
+    return np.ascontiguousarray(signs.reshape(r, H, W, Cin).transpose(0, 3, 1, 2))
 
 
 def memory_factor(Cin, H, W, r):

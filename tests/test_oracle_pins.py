@@ -372,3 +372,57 @@ def test_p7_memory_factor_matches_printed_values():
     for H, W, Cin, gamma, factor in rows:
         assert O.memory_factor(int(Cin), int(H), int(W), 2 ** int(gamma)) == factor == 2 ** (14 - gamma)
     assert 100 <= O.memory_factor(16, 32, 32, 2 ** 7) <= 130      # "roughly 100x"
+
+
+# ------------------------------------------------------------------ probes redrawn from a seed (Algorithm 1)
+
+def test_philox_known_answer_vectors():
+    rows = [l.split() for l in open(os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 3
+    for row in rows:
+        v = [int(x, 16) for x in row]
+        out = O.philox4x32_10([np.array([c]) for c in v[0:4]], v[4:6])
+        assert [int(o[0]) for o in out] == v[6:10]
+
+
+def test_rademacher_probes_follow_the_stated_bit_order():
+    # entry e = ((j*H + y)*W + x)*Cin + n takes bit (e mod 128) of block (e div 128): re-derive a few entries
+    # one by one, straight from the definition
+    r, Cin, H, W, seed = 3, 5, 4, 7, 0x1234567890ABCDEF
+    Z = O.rademacher_probes(seed, r, Cin, H, W)
+    assert Z.shape == (r, Cin, H, W) and set(np.unique(Z)) == {-1.0, 1.0}
+    for (j, n, y, x) in [(0, 0, 0, 0), (0, 4, 0, 0), (1, 2, 3, 6), (2, 4, 3, 6), (2, 0, 1, 5)]:
+        e = ((j * H + y) * W + x) * Cin + n
+        blk, bit = divmod(e, 128)
+        words = O.philox4x32_10([np.array([blk & 0xFFFFFFFF]), np.array([blk >> 32]), np.array([0]), np.array([0])],
+                                (seed & 0xFFFFFFFF, seed >> 32))
+        b = (int(words[bit // 32][0]) >> (bit % 32)) & 1
+        assert Z[j, n, y, x] == (1.0 - 2.0 * b)
+
+
+def test_rademacher_probes_are_balanced_independent_and_seed_dependent():
+    r, Cin, H, W = 4096, 2, 3, 3          # 4096 probes of dimension 18
+    Z = O.rademacher_probes(7, r, Cin, H, W).reshape(r, -1)
+    assert abs(Z.mean()) < 4.0 / np.sqrt(Z.size)
+    C = Z.T @ Z / r                       # E[z z^T] = I, the only property the estimator needs (Section 3)
+    assert np.allclose(np.diag(C), 1.0)
+    off = C - np.eye(C.shape[0])
+    assert np.abs(off).max() < 5.0 / np.sqrt(r)
+    Z2 = O.rademacher_probes(8, r, Cin, H, W).reshape(r, -1)
+    assert 0.4 < (Z != Z2).mean() < 0.6
+
+
+def test_estimator_on_redrawn_probes_is_unbiased():
+    # mean of the estimate over many seeds -> exact gradient (Section 3: E[z z^T] = I)
+    g = np.random.Generator(np.random.PCG64(5))
+    B, Cin, Cout, H, W, r, T = 3, 2, 2, 4, 4, 8, 3000
+    X, dY = g.standard_normal((B, Cin, H, W)), g.standard_normal((B, Cout, H, W))
+    exact = O.dw_exact(X, dY)
+    acc = np.zeros_like(exact)
+    for t in range(T):
+        Z = O.rademacher_probes(1000 + t, r, Cin, H, W)
+        acc += O.wgrad_estimate(O.sketch(X, Z), dY, Z)
+    err = np.abs(acc / T - exact).max()
+    single = np.std([O.wgrad_estimate(O.sketch(X, Z), dY, Z) for Z in (O.rademacher_probes(s, r, Cin, H, W) for s in range(50))], axis=0).max()
+    assert err < 5.0 * single / np.sqrt(T)
