@@ -415,11 +415,19 @@ def run_xconv(args):
             torch.cuda.synchronize()
             return a_.elapsed_time(b_) / n
 
+        # Algorithm 1 with only the seed kept: Z redrawn inside the sketch kernel / into the workspace
+        wss = torch.empty(max(xb.workspace_bytes(desc, xb.OP_SKETCH_SEEDED), xb.workspace_bytes(desc, xb.OP_WGRAD_SEEDED)),
+                          dtype=torch.uint8, device=dev)
+        S2 = torch.empty_like(S)
         full = {"forward_ms": _time(lambda: xb.forward_into(desc, X, Wt, Z, Y, S, wsf)),
                 "dgrad_ms": _time(lambda: xb.dgrad_into(desc, dY, Wt, dX, wsf)),
+                "wgrad_ms": _time(lambda: xb.wgrad_into(desc, S, dY, Z, dW, layer.ws)),
+                "sketch_seeded_ms": _time(lambda: xb.sketch_seeded_into(desc, X, 12345, S2, wss)),
+                "wgrad_seeded_ms": _time(lambda: xb.wgrad_seeded_into(desc, S, dY, 12345, dW, wss)),
                 "conv_engine": xb.engine_for(desc, xb.OP_FORWARD),
-                "note": "xconv_forward = conv + sketch; xconv_dgrad = exact dX; not part of the metric"}
-        del Y, dX, wsf
+                "note": "xconv_forward = conv + sketch; xconv_dgrad = exact dX; xconv_wgrad = back-probe + contraction "
+                        "in one call; *_seeded: probes redrawn from a seed instead of read from memory; not part of the metric"}
+        del Y, dX, wsf, wss
 
     cpu = None
     if not args.no_cpu:

@@ -69,7 +69,8 @@ typedef enum {
 } xconv_status;
 
 typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3,
-               XCONV_OP_BACKPROBE = 4, XCONV_OP_CONTRACT = 5 } xconv_op;
+               XCONV_OP_BACKPROBE = 4, XCONV_OP_CONTRACT = 5, XCONV_OP_SKETCH_SEEDED = 6,
+               XCONV_OP_WGRAD_SEEDED = 7 } xconv_op;
 
 /* Which arithmetic engine a call will use for its dominant kernel. */
 typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2 } xconv_engine;
@@ -101,6 +102,31 @@ xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W,
 /* Forward step 3 alone, S = Z^T X (for callers whose convolution runs elsewhere). */
 xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
                           void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Probing vectors redrawn from a seed.  Algorithm 1 stores the random seed s in the forward pass (step 2)
+ * and redraws Z[s] in the backward pass (step 2) instead of keeping Z; the paper leaves the generator
+ * open.  This library fixes it as follows (Rademacher entries, for which E[z z^T] = I holds as Section 3
+ * requires): number the entries of Z in memory order, e = ((j*H + y)*W + x)*Cin + n.  Entry e is +1 if bit
+ * (e mod 128) of the Philox-4x32-10 block with counter (e div 128) and key (seed & 0xffffffff, seed >> 32)
+ * is 0, and -1 if it is 1; bit b of a block is bit (b mod 32) of its output word (b div 32).  (Philox:
+ * Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11.)
+ *
+ * xconv_probes_from_seed writes Z [r,H,W,Cin] in desc.dtype (desc.B, Cout, KH.. are ignored beyond validity).
+ * xconv_sketch_seeded computes S = Z[seed]^T X (Algorithm 1 forward step 3) without reading Z from memory:
+ * where the tensor-core kernel covers the layer and H*W*Cin is a multiple of 64 the tiles of Z are redrawn
+ * inside the kernel, so that only X leaves HBM; otherwise Z is first written into `ws` and the regular
+ * kernels run on it (xconv_workspace_bytes(desc, XCONV_OP_SKETCH_SEEDED) covers both cases).  The result
+ * equals xconv_sketch on xconv_probes_from_seed's Z up to the order of summation.
+ * xconv_wgrad_seeded is Algorithm 1's backward pass from the stored seed: step 2 redraws Z[seed] into `ws`
+ * (xconv_workspace_bytes(desc, XCONV_OP_WGRAD_SEEDED) = the scratch of xconv_wgrad plus one Z), steps 3-4
+ * are xconv_wgrad on it; the estimate equals xconv_wgrad(sketch, dY, xconv_probes_from_seed(seed)) bit for
+ * bit.  With these two calls a layer keeps S (r*B floats) and the 8-byte seed between its forward and its
+ * backward pass, the memory factor the paper quotes. */
+xconv_status xconv_probes_from_seed(const xconv_desc* desc, unsigned long long seed, void* Z, void* cuda_stream);
+xconv_status xconv_sketch_seeded(const xconv_desc* desc, const void* X, unsigned long long seed, float* sketch,
+                                 void* ws, size_t ws_bytes, void* cuda_stream);
+xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, const void* dY, unsigned long long seed,
+                                float* dW, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Algorithm 1, backward steps 3-4: L = S dY^T, then dW[m,n,k] = scale[n] * tr(L^m T_{-k} Z_n) for
  * every offset (Eq. 6; three-step procedure of Section 3).  sketch [r,B] float as written by

@@ -17,13 +17,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxconv.so")
 
 XCONV_F32, XCONV_BF16 = 0, 1
-OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT = 0, 1, 2, 3, 4, 5
+OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT, OP_SKETCH_SEEDED, OP_WGRAD_SEEDED = 0, 1, 2, 3, 4, 5, 6, 7
 ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16"}
 STATUS_OK = 0
 
 # every symbol include/xconv.h declares
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
-           "xconv_dgrad", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
+           "xconv_dgrad", "xconv_probes_from_seed", "xconv_sketch_seeded", "xconv_wgrad_seeded", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
            "xconv_workspace_status", "xconv_selftest_wait_limit",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
@@ -61,6 +61,12 @@ def lib() -> ctypes.CDLL:
     L.xconv_forward.restype = c_int
     L.xconv_sketch.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_sketch.restype = c_int
+    L.xconv_probes_from_seed.argtypes = [P, ctypes.c_ulonglong, c_void_p, c_void_p]
+    L.xconv_probes_from_seed.restype = c_int
+    L.xconv_sketch_seeded.argtypes = [P, c_void_p, ctypes.c_ulonglong, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_sketch_seeded.restype = c_int
+    L.xconv_wgrad_seeded.argtypes = [P, c_void_p, c_void_p, ctypes.c_ulonglong, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_wgrad_seeded.restype = c_int
     L.xconv_wgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad.restype = c_int
     L.xconv_backprobe_bytes.argtypes = [P]; L.xconv_backprobe_bytes.restype = c_size_t
@@ -145,6 +151,16 @@ def sketch_into(desc, X, Z, S, ws):
                               ws.numel(), _stream()), "xconv_sketch")
 
 
+def sketch_seeded_into(desc, X, seed, S, ws):
+    _check(lib().xconv_sketch_seeded(ctypes.byref(desc), X.data_ptr(), seed, S.data_ptr(), ws.data_ptr(),
+                                     ws.numel(), _stream()), "xconv_sketch_seeded")
+
+
+def wgrad_seeded_into(desc, S, dY, seed, dW, ws):
+    _check(lib().xconv_wgrad_seeded(ctypes.byref(desc), S.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
+                                    ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_seeded")
+
+
 def forward_into(desc, X, W, Z, Y, S, ws):
     _check(lib().xconv_forward(ctypes.byref(desc), X.data_ptr(), W.data_ptr(), Z.data_ptr(), Y.data_ptr(),
                                S.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "xconv_forward")
@@ -192,6 +208,42 @@ def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
     ws = workspace(workspace_bytes(desc, OP_SKETCH), X.device)
     sketch_into(desc, X, Z, S, ws)
     return S
+
+
+def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=torch.bfloat16, device="cuda") -> torch.Tensor:
+    """Z[seed]: Rademacher probing vectors (r, Cin, H, W), channels_last, from the library's Philox stream."""
+    desc = make_desc(1, Cin, 1, H, W, r, dtype)
+    Z = torch.empty((r, Cin, H, W), dtype=dtype, device=device, memory_format=torch.channels_last)
+    _check(lib().xconv_probes_from_seed(ctypes.byref(desc), seed, Z.data_ptr(), _stream()), "xconv_probes_from_seed")
+    return Z
+
+
+def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int) -> torch.Tensor:
+    """S = Z[seed]^T X without a stored Z (Algorithm 1 keeps the seed): float32 tensor [r, B]."""
+    _cl(X, "X")
+    B, Cin, H, W = X.shape
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    S = torch.empty((r, B), dtype=torch.float32, device=X.device)
+    ws = workspace(workspace_bytes(desc, OP_SKETCH_SEEDED), X.device)
+    sketch_seeded_into(desc, X, seed, S, ws)
+    return S
+
+
+def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: int, kernel_size: int = 3) -> torch.Tensor:
+    """dW estimate from the sketch and the seed (Algorithm 1 backward steps 2-4): Z[seed] is redrawn into the
+    workspace, never passed in.  float32 (Cout, Cin, K, K), channels_last."""
+    _cl(dY, "dY")
+    B, Cout, H, Wd = dY.shape
+    r = sketch.shape[0]
+    if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
+        raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
+    K = kernel_size
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K)
+    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_WGRAD_SEEDED), dY.device)
+    _check(lib().xconv_wgrad_seeded(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
+                                    ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_seeded")
+    return dW
 
 
 STATIC_SCRATCH_FLOATS = 1 << 20

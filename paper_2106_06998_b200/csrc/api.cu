@@ -64,11 +64,11 @@ struct SketchPlan {
   size_t part_off, bytes;
 };
 
-static SketchPlan plan_sketch(const xconv_desc* d) {
+static SketchPlan plan_sketch(const xconv_desc* d, bool seeded = false) {
   SketchPlan p{};
   const long K = (long)d->H * d->W * d->Cin;
   p.part_off = WS_HEADER;
-  p.tc = tc_plan_sketch(d, &p.t);
+  p.tc = tc_plan_sketch(d, &p.t, seeded && tc_sketch_can_redraw(d));
   if (p.tc) {
     p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
     return p;
@@ -155,6 +155,50 @@ static WgradPlan plan_wgrad(const xconv_desc* d) {
   return p;
 }
 
+// ----------------------------------------------------------------------------------- probes from a seed
+
+// Z redrawn from a seed: entry e (in memory order) is +1 if bit (e mod 128) of Philox block (e div 128) is 0,
+// -1 if it is 1; bit b is bit (b mod 32) of output word (b div 32).  One thread writes eight entries.
+template <typename T>
+__global__ void __launch_bounds__(256) probes_from_seed_kernel(T* __restrict__ Z, long total, uint32_t k0, uint32_t k1) {
+  pdl_trigger();
+  pdl_wait();
+  const long e0 = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (e0 >= total) return;
+  const unsigned long long blk = (unsigned long long)e0 >> 7;
+  const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), k0, k1);
+  const int word = (int)((e0 & 127) >> 5);
+  const uint32_t wv = word == 0 ? w.x : word == 1 ? w.y : word == 2 ? w.z : w.w;
+  const uint32_t bits = (wv >> (e0 & 31)) & 0xFFu;
+  if (e0 + 8 <= total) {                     // Z is 16-byte aligned and e0 a multiple of 8: vector stores
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = ((bits >> i) & 1u) ? -1.0f : 1.0f;
+    st4(Z + e0, make_float4(v[0], v[1], v[2], v[3]));
+    st4(Z + e0 + 4, make_float4(v[4], v[5], v[6], v[7]));
+    return;
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
+    if (e0 + i < total) Z[e0 + i] = from_f<T>(((bits >> i) & 1u) ? -1.0f : 1.0f);
+}
+
+static xconv_status run_probes_from_seed(const xconv_desc* d, unsigned long long seed, void* Z, cudaStream_t st) {
+  const long total = (long)d->r * d->H * d->W * d->Cin;
+  const unsigned grid = (unsigned)cdiv(cdiv(total, 8), 256);
+  const uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFull), k1 = (uint32_t)(seed >> 32);
+  cudaError_t e = d->dtype == XCONV_F32
+      ? launch_pdl(probes_from_seed_kernel<float>, dim3(grid), dim3(256), 0, st, static_cast<float*>(Z), total, k0, k1)
+      : launch_pdl(probes_from_seed_kernel<bf16>, dim3(grid), dim3(256), 0, st, static_cast<bf16*>(Z), total, k0, k1);
+  ++g_launches;
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return XCONV_OK;
+}
+
+static size_t probes_bytes(const xconv_desc* d) {
+  return align_up((size_t)d->r * d->H * d->W * d->Cin * (d->dtype == XCONV_F32 ? 4 : 2), 256);
+}
+
 // ----------------------------------------------------------------------------------- launchers
 
 template <typename T>
@@ -172,13 +216,24 @@ static xconv_status run_sketch_simt(const xconv_desc* d, const SketchPlan& p, co
   return check_launch();
 }
 
+// Whether the sketch kernel of this layer redraws Z itself; otherwise the seeded call first writes Z
+// into the workspace (behind the regular scratch) and runs the regular kernels on it.
+static bool sketch_redraws(const xconv_desc* d, const SketchPlan& p) { return p.tc && tc_sketch_can_redraw(d); }
+
 static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z, float* S, void* ws,
-                               size_t ws_bytes, cudaStream_t st) {
-  const SketchPlan p = plan_sketch(d);
-  if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
+                               size_t ws_bytes, cudaStream_t st, const unsigned long long* seed = nullptr) {
+  const SketchPlan p = plan_sketch(d, seed != nullptr);
+  const bool redraw = seed && sketch_redraws(d, p);
+  const size_t need = p.bytes + (seed && !redraw ? probes_bytes(d) : 0);
+  if (!ws || ws_bytes < need) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   char* w = static_cast<char*>(ws);
-  if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st);
+  if (seed && !redraw) {
+    xconv_status s = run_probes_from_seed(d, *seed, w + p.bytes, st);
+    if (s != XCONV_OK) return s;
+    Z = w + p.bytes;
+  }
+  if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st, redraw ? seed : nullptr);
   return d->dtype == XCONV_F32 ? run_sketch_simt<float>(d, p, X, Z, S, w, st)
                                : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
 }
@@ -313,6 +368,11 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
   switch (op) {
     case XCONV_OP_FORWARD:
     case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
+    case XCONV_OP_WGRAD_SEEDED: return plan_wgrad(desc).bytes + probes_bytes(desc);
+    case XCONV_OP_SKETCH_SEEDED: {
+      const SketchPlan p = plan_sketch(desc, true);
+      return p.bytes + (sketch_redraws(desc, p) ? 0 : probes_bytes(desc));
+    }
     case XCONV_OP_WGRAD:
     case XCONV_OP_BACKPROBE:
     case XCONV_OP_CONTRACT: return plan_wgrad(desc).bytes;
@@ -345,6 +405,43 @@ xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, 
   if (!aligned16(X) || !aligned16(Z) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
   new_call();
   return run_sketch(desc, X, Z, sketch, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+xconv_status xconv_probes_from_seed(const xconv_desc* desc, unsigned long long seed, void* Z, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!Z) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(Z)) return XCONV_ERR_ALIGNMENT;
+  new_call();
+  return run_probes_from_seed(desc, seed, Z, static_cast<cudaStream_t>(cuda_stream));
+}
+
+xconv_status xconv_sketch_seeded(const xconv_desc* desc, const void* X, unsigned long long seed, float* sketch,
+                                 void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!X || !sketch) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
+  new_call();
+  return run_sketch(desc, X, nullptr, sketch, ws, ws_bytes, static_cast<cudaStream_t>(cuda_stream), &seed);
+}
+
+xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, const void* dY, unsigned long long seed,
+                                float* dW, void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!sketch || !dY || !dW) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(sketch) || !aligned16(dY) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
+  const size_t base = plan_wgrad(desc).bytes;
+  s = check_ws(ws, ws_bytes, base + probes_bytes(desc));
+  if (s != XCONV_OK) return s;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // Algorithm 1 backward step 2: redraw Z from the seed (behind the regular scratch), then steps 3-4
+  char* Z = static_cast<char*>(ws) + base;
+  s = run_probes_from_seed(desc, seed, Z, st);
+  if (s != XCONV_OK) return s;
+  return run_wgrad(desc, sketch, dY, Z, dW, ws, base, st);
 }
 
 xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W, const void* Z, void* Y,

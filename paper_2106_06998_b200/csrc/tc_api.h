@@ -38,15 +38,18 @@ struct TcConvPlan {
 
 // Fill the plan and say whether the tcgen05 kernels cover this layer.  tc_plan_wgrad returns a mask:
 // bit 0 = back-probe covered, bit 1 = contraction covered.
-bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p);
+bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p, bool redraw = false);   // redraw: plan for a seeded call
 int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p);
 
 bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p);
 xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& p, bool dgrad, const void* in, const void* W,
                          void* out, char* ws_head, char* wt, cudaStream_t st);
 
+// `seed` != nullptr: Z is not read; its tiles are redrawn inside the kernel from the Philox stream of *seed
+// (Rademacher entries; see xconv_probes_from_seed).  Only for layers tc_sketch_can_redraw accepts.
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const void* X, const void* Z, float* S,
-                           char* ws_head, char* part, cudaStream_t st);
+                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed = nullptr);
+bool tc_sketch_can_redraw(const xconv_desc* d);
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const void* S_bf16, const void* dY,
                               void* L, char* ws_head, cudaStream_t st);
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const void* L, const void* Z, float* dW,

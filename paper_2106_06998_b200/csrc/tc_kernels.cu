@@ -81,6 +81,13 @@ struct TcParams {
   int T, Cin;              // CONTRACT output indexing; CONV: offsets and input channels
   int H, W, cgroups;       // CONV: image size and input-channel blocks of 64
   int nimg;                // CONV: images; with m_sub = 2 a unit covers the same patch of images img and img + 1
+  // Probing vectors redrawn inside the kernel (Algorithm 1 keeps the seed, not Z): the tile of Z is not copied
+  // from global memory; the epilogue warps write it into the stage from the Philox stream of the seed.
+  int seeded;              // 0: Z is read from memory
+  uint32_t seed_lo, seed_hi;
+  int z_is_a;              // SKETCH: Z is the A operand (probes on the MMA rows) instead of the B operand
+  long z_row_len;          // entries of one probing vector, H*W*Cin
+  long rows_z;             // probing vectors (rows of Z)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
 };
@@ -275,6 +282,40 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// The 64 sign bits of entries e0 .. e0+63 of Z (e0 a multiple of 64): entry e takes bit (e mod 128) of the
+// Philox block (e div 128); bit b is bit (b mod 32) of output word (b div 32).
+__device__ __forceinline__ uint2 z_sign_bits64(long e0, uint32_t k0, uint32_t k1) {
+  const unsigned long long blk = (unsigned long long)e0 >> 7;
+  const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), k0, k1);
+  return (e0 & 64) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y);
+}
+// Eight consecutive entries as bfloat16 (+1 = 0x3F80, -1 = 0xBF80) from bits 0..7 of `t` (higher bits are
+// ignored).  Two sign bits b0, b1 at positions 2i, 2i+1 go to bits 15 and 31 of a word: the product of
+// (t & (3 << 2i)) with (0x40008000 >> 2i) holds b0 at bits 15 and 30 and b1 at bits 16 and 31.
+__device__ __forceinline__ uint4 z_pack8(uint32_t t) {
+  uint4 o;
+  o.x = (((t & 0x03u) * 0x40008000u) & 0x80008000u) | 0x3F803F80u;
+  o.y = (((t & 0x0Cu) * 0x10002000u) & 0x80008000u) | 0x3F803F80u;
+  o.z = (((t & 0x30u) * 0x04000800u) & 0x80008000u) | 0x3F803F80u;
+  o.w = (((t & 0xC0u) * 0x01000200u) & 0x80008000u) | 0x3F803F80u;
+  return o;
+}
+
+// 64 entries of one row of a K-major, 128-byte-swizzled tile (row base `rbase`): eight 16-byte pieces.
+__device__ __forceinline__ void z_store64(uint32_t rbase, int row, uint2 bits) {
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint4 o = z_pack8((c < 4 ? bits.x : bits.y) >> ((c & 3) * 8));
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (((uint32_t)c ^ ((uint32_t)row & 7u)) << 4)),
+                 "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+  }
+}
+// 128 entries: the same row of two consecutive k-block tiles, `tile_bytes` apart.
+__device__ __forceinline__ void z_store128(uint32_t rbase, uint32_t tile_bytes, int row, uint4 w) {
+  z_store64(rbase, row, make_uint2(w.x, w.y));
+  z_store64(rbase + tile_bytes, row, make_uint2(w.z, w.w));
+}
+
 // Optional per-CTA cycle counters (build with -DXC_TIMELINE): time the producer and the MMA-issue thread
 // spend waiting on barriers and issuing work, read back through xconv_debug_waits.
 #ifdef XC_TIMELINE
@@ -362,7 +403,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 5 : 1); mbar_init(&empty_bar[s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -480,14 +521,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                                   ? p.a_stage_bytes + (uint32_t)w.nblk * p.b_box_bytes : p.tx_bytes);
           if (p.mode == MODE_SKETCH) {
             // one box per operand: 128*m_sub rows of A, tile_n rows of B, 64 k each
+            const bool get_a = !(p.seeded && p.z_is_a), get_b = !(p.seeded && !p.z_is_a);
             if (p.kgroup > 1) {
               // kgroup consecutive k-blocks per operand in one 3-d box (64 k, rows, k-blocks)
-              tma_load_3d(a_dst, &map_a, 0, row0, kc >> 6, &full_bar[s]);
-              tma_load_3d(b_dst, &map_b, 0, col0, kc >> 6, &full_bar[s]);
+              if (get_a) tma_load_3d(a_dst, &map_a, 0, row0, kc >> 6, &full_bar[s]);
+              if (get_b) tma_load_3d(b_dst, &map_b, 0, col0, kc >> 6, &full_bar[s]);
               kc += 64 * p.kgroup;
             } else {
-              tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
-              tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
+              if (get_a) tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
+              if (get_b) tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
               kc += 64;
             }
           } else if (p.mode == MODE_BACKPROBE) {
@@ -651,12 +693,62 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
     const uint32_t epi_base = tiles_base + (uint32_t)p.stages * stage_bytes;
     uint32_t epi_slot = 0;                    // BACKPROBE: next staging slot of this warp's ring
+    int gen_s = 0;                            // seeded: stage the generator fills next, and how often the ring wrapped
+    long gen_fill = 0;
     long lu = 0;
     bool ok = true;
     for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
       const Unit w = decode_unit(p, u);
       const int buf = (int)(lu % p.acc_bufs);
       const long use = lu / p.acc_bufs;
+      if (p.seeded && p.mode == MODE_SKETCH) {
+        // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
+        // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
+        // copy would have produced, hand the stage over with one arrival per warp.
+        const int gtid = (int)threadIdx.x - 64;                       // 0..127
+        const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
+        const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
+        const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
+        const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
+        long kc = w.kb0 * 64 * p.kgroup;
+        for (int i = 0; i < w.nkb && ok; ++i) {
+          if (gen_fill > 0) {
+            if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+          }
+          const uint32_t zbase = tiles_base + (uint32_t)gen_s * stage_bytes + z_off;
+          const uint32_t tile_bytes = (uint32_t)tile_rows * 128u;
+          if ((p.kgroup & 1) == 0 && (p.z_row_len & 127) == 0) {
+            // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
+            // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
+            const int nitems = nrows * (p.kgroup >> 1);
+            for (int it0 = gtid; it0 < nitems; it0 += 256) {
+              const int it1 = it0 + 128;
+              const bool two = it1 < nitems;
+              const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
+              const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
+              const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
+              const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
+              const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
+              z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0);
+              if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1);
+            }
+          } else {
+            for (int item = gtid; item < nrows * p.kgroup; item += 128) {
+              const int row = item % nrows, g = item / nrows;
+              const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
+              z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits);
+            }
+          }
+          fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full_bar[gen_s]);
+          kc += 64 * p.kgroup;
+          if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
+        }
+        if (!ok) break;
+      }
       if (w.nkb > 0) {
         if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status, p.tag);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -946,7 +1038,7 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
 
 // ---- sketch --------------------------------------------------------------------------------
 
-bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
+bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p, bool redraw) {
   if (d->dtype != XCONV_BF16) return false;
   const long K = (long)d->H * d->W * d->Cin;
   if (K % 8 != 0 || K < 2048 || K > 2000000000L) return false;
@@ -966,6 +1058,9 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   const uint32_t block = (uint32_t)p->rows_box * 128 + p->tile_n * 128;
   p->kgroup = 1;
   if (K % 64 == 0) p->kgroup = block <= 12 * 1024 ? 4 : block <= 36 * 1024 ? 2 : 1;
+  // Z redrawn in the kernel: a Philox block covers 128 consecutive entries of a row, i.e. two k-blocks
+  if (redraw && K % 128 == 0 && p->kgroup == 1 && 2 * 2 * block + TILE_M * 128 <= (uint32_t)(SMEM_LIMIT - STATIC_SMEM_SLACK))
+    p->kgroup = 2;
   p->kblocks = cdivl(K, 64L * p->kgroup);
   p->stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - TILE_M * 128) / (int)(block * p->kgroup)));
   const long tiles = (long)p->tiles_m * p->tiles_n;
@@ -981,10 +1076,15 @@ bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p) {
   return true;
 }
 
+bool tc_sketch_can_redraw(const xconv_desc* d) {
+  return ((long)d->H * d->W * d->Cin) % 64 == 0;     // a row of Z starts on a 64-entry boundary of the stream
+}
+
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const void* X, const void* Z, float* S,
-                           char* ws_head, char* part, cudaStream_t st) {
+                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed) {
   const long K = (long)d->H * d->W * d->Cin;
   const int rows = pl.swap ? d->B : d->r, cols = pl.swap ? d->r : d->B;
+  if (seed) Z = X;                                   // the map of Z is built but never used: any valid base
   const void* A = pl.swap ? X : Z;
   const void* Bm = pl.swap ? Z : X;
   CUtensorMap ma, mb;
@@ -1022,6 +1122,15 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   p.a_jump = (a_tile >> 4) - 6;
   p.b_jump = (b_tile >> 4) - 6;
   p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  if (seed) {                                        // Z is written by the generator warps, only X is copied
+    p.seeded = 1;
+    p.seed_lo = (uint32_t)(*seed & 0xFFFFFFFFull);
+    p.seed_hi = (uint32_t)(*seed >> 32);
+    p.z_is_a = pl.swap ? 0 : 1;
+    p.z_row_len = K;
+    p.rows_z = d->r;
+    p.tx_bytes = p.z_is_a ? p.b_stage_bytes : p.a_stage_bytes;
+  }
   // The MMA always reads 128 rows of A.  Behind a shorter tile it reads whatever follows (the rows it
   // produces are never stored), which must still be this CTA's shared memory.
   p.smem_pad = TILE_M * 128 - std::min<uint32_t>(a_tile, TILE_M * 128);

@@ -1,0 +1,87 @@
+"""GPU parity of the seeded calls: probing vectors redrawn from a seed (Algorithm 1 stores the seed, not
+Z).  The generator is compared bit for bit with the oracle's own implementation of the same published
+definition; the seeded sketch with the oracle's sketch on the oracle's Z, and bit for bit with the
+library's sketch on the library's Z."""
+import numpy as np
+import pytest
+import torch
+
+import __graft_entry__ as entry
+from oracle import xconv_oracle as O
+from paper_2106_06998_b200 import binding as xb
+from paper_2106_06998_b200 import inputs
+from tests._util import TOL, check, host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    entry.build()
+    torch.cuda.set_device(0)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("shape", [(1, 1, 1, 1), (3, 5, 4, 7), (8, 16, 9, 9), (5, 64, 6, 12), (130, 8, 5, 13)])
+def test_probes_from_seed_match_the_oracle_generator_bit_for_bit(shape, dtype):
+    r, Cin, H, W = shape
+    for seed in (0, 0x1234567890ABCDEF, 2**64 - 1):
+        Z = xb.xconv_probes_from_seed(seed, r, Cin, H, W, dtype)
+        torch.cuda.synchronize()
+        assert np.array_equal(host(Z), O.rademacher_probes(seed, r, Cin, H, W))
+
+
+SEEDED_SKETCH_SHAPES = [
+    # B, Cin, H, W, r
+    (24, 8, 16, 16, 8),       # samples on the MMA rows, K = 2048: four k-blocks per stage
+    (8, 64, 6, 35, 40),       # probes on the MMA rows (r > B): Z is the A operand; last stage half past K
+    (200, 64, 5, 10, 72),     # two 128-row tiles of samples, 72 probes
+    (520, 8, 16, 16, 504),    # pairs of row tiles share the redrawn tile; both axes ragged
+    (16, 32, 24, 24, 300),    # r > B with three probe tiles, the last one ragged
+    (8, 24, 11, 13, 16),      # K = 3432 is not a multiple of 64: Z is written to the workspace first
+    (3, 5, 7, 9, 5),          # no tensor-core kernel at all
+]
+
+
+@pytest.mark.parametrize("shape", SEEDED_SKETCH_SHAPES)
+def test_seeded_sketch_matches_oracle_and_the_stored_probe_path(shape):
+    B, Cin, H, W, r = shape
+    seed = 1000003 * sum(shape) + 17
+    lay = inputs.make_custom(B, Cin, 8, H, W, r, dtype="bf16", seed=sum(shape), z="rademacher", x="normal")
+    X = xb.to_device(lay["X"], "bf16")
+    S = xb.xconv_sketch_seeded(X, seed, r)
+    Zg = xb.xconv_probes_from_seed(seed, r, Cin, H, W, torch.bfloat16)
+    S_stored = xb.xconv_sketch(X, Zg)
+    torch.cuda.synchronize()
+    # the same sum in a possibly different order (the seeded plan may take more k-blocks per stage)
+    check("seeded sketch against the stored-probe sketch", host(S), host(S_stored), 1e-5)
+    check("seeded sketch", host(S), O.sketch(lay["X"], O.rademacher_probes(seed, r, Cin, H, W)), TOL["bf16"])
+
+
+def test_seeded_sketch_float_storage():
+    B, Cin, H, W, r, seed = 6, 16, 8, 8, 12, 99
+    lay = inputs.make_custom(B, Cin, 8, H, W, r, dtype="f32", seed=5, z="rademacher", x="normal")
+    X = xb.to_device(lay["X"], "f32")
+    S = xb.xconv_sketch_seeded(X, seed, r)
+    torch.cuda.synchronize()
+    check("seeded sketch", host(S), O.sketch(lay["X"], O.rademacher_probes(seed, r, Cin, H, W)), TOL["f32"])
+
+
+@pytest.mark.parametrize("shape,dtype", [((16, 64, 64, 12, 20, 24), "bf16"), ((8, 32, 32, 40, 24, 72), "bf16"),
+                                         ((3, 5, 7, 9, 11, 5), "f32"), ((2, 16, 16, 8, 8, 8), "f32")])
+def test_seeded_layer_matches_the_oracle_with_redrawn_probes(shape, dtype):
+    """Algorithm 1 end to end with nothing but S and the seed kept between the passes."""
+    B, Cin, Cout, H, W, r = shape
+    seed = 7919 * sum(shape) + 3
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape), z="rademacher", x="relu")
+    X, dY = xb.to_device(lay["X"], dtype), xb.to_device(lay["dY"], dtype)
+    S = xb.xconv_sketch_seeded(X, seed, r)
+    dW = xb.xconv_wgrad_seeded(S, dY, seed, Cin)
+    Zg = xb.xconv_probes_from_seed(seed, r, Cin, H, W, X.dtype)
+    dW_stored = xb.xconv_wgrad(S, dY, Zg)
+    torch.cuda.synchronize()
+    assert torch.equal(dW, dW_stored)
+    Zo = O.rademacher_probes(seed, r, Cin, H, W)
+    So = O.sketch(lay["X"], Zo)
+    check("sketch", host(S), So, TOL[dtype])
+    check("dW", host(dW), O.wgrad_estimate(So, lay["dY"], Zo), TOL[dtype])
