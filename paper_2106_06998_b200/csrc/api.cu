@@ -74,9 +74,11 @@ static SketchPlan plan_sketch(const xconv_desc* d, bool seeded = false) {
     return p;
   }
   const long tiles = cdiv(d->r, 64) * cdiv(d->B, 64);
-  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(K, 512)));
+  // short chains: a block walks its k-range step by step with one step of loads in flight, so the time of a
+  // sketch is (steps per block) x (load latency) unless the range is dealt to many blocks
+  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(K, 128)));
   splits = std::min(splits, 2048L);
-  p.k_per_split = align_up((size_t)cdiv(K, splits), 16);
+  p.k_per_split = align_up((size_t)cdiv(K, splits), 32);
   p.splits = (int)cdiv(K, p.k_per_split);
   p.bytes = p.part_off + align_up((size_t)p.splits * d->r * d->B * sizeof(float), 256);
   return p;
@@ -106,7 +108,8 @@ static WgradPlan plan_wgrad_core(const xconv_desc* d) {
   }
   const long items = (long)d->r * d->H * cdiv(d->W, 32);
   const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32);
-  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(items, 8)));
+  // one wave of the grid: two blocks of this kernel fit an SM (its 72 accumulators per thread)
+  long splits = std::max(1L, std::min(std::max(1L, 2L * 148 / tiles), cdiv(items, 2)));
   splits = std::min(splits, 4096L);
   p.items_per_split = cdiv(items, splits);
   p.splits = (int)cdiv(items, p.items_per_split);
@@ -212,7 +215,7 @@ static xconv_status run_sketch_simt(const xconv_desc* d, const SketchPlan& p, co
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
   const long count = (long)d->r * d->B;
-  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, S, count, p.splits, 1.0f, nullptr, 1);
+  reduce_partials<<<(unsigned)cdiv(count, RP_OUT), RP_OUT * RP_LANES, 0, st>>>(part, S, count, p.splits, 1.0f, nullptr, 1);
   return check_launch();
 }
 
@@ -254,16 +257,19 @@ static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, c
   const int T9 = d->KH * d->KW;
   const TL* L = static_cast<const TL*>(Lv);
   dim3 g2((unsigned)cdiv(d->Cin, 64), (unsigned)cdiv(d->Cout, 32), (unsigned)p.splits);
-  if (d->KH == 3)
-    contract_simt<TL, T, 3><<<g2, 256, 0, st>>>(L, static_cast<const T*>(Z), part, d->r, d->H, d->W, d->Cin, d->Cout,
-                                                p.items_per_split);
-  else
-    contract_simt<TL, T, 1><<<g2, 256, 0, st>>>(L, static_cast<const T*>(Z), part, d->r, d->H, d->W, d->Cin, d->Cout,
-                                                p.items_per_split);
+  const T* Zt = static_cast<const T*>(Z);
+  const bool vec = d->Cin % 4 == 0 && d->Cout % 4 == 0;      // rows of L and Z then start on 4-element boundaries
+  if (d->KH == 3) {
+    if (vec) contract_simt<TL, T, 3, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
+    else contract_simt<TL, T, 3, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
+  } else {
+    if (vec) contract_simt<TL, T, 1, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
+    else contract_simt<TL, T, 1, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
+  }
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T9 * d->Cin;
-  reduce_partials<<<(unsigned)cdiv(count, 256), 256, 0, st>>>(part, dW, count, p.splits, alpha, d->chan_scale, d->Cin);
+  reduce_partials<<<(unsigned)cdiv(count, RP_OUT), RP_OUT * RP_LANES, 0, st>>>(part, dW, count, p.splits, alpha, d->chan_scale, d->Cin);
   return check_launch();
 }
 

@@ -16,13 +16,20 @@ template <typename T>
 __global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, const T* __restrict__ Bm,
                                                     float* __restrict__ part, int M, int N, long K,
                                                     long k_per_split, int vec) {
-  __shared__ __align__(16) float As[16][68];
-  __shared__ __align__(16) float Bs[16][68];
+  // 64 x 64 outputs per block, 32 k per step (128 consecutive bytes of a row; rows lie K elements apart);
+  // the loads of the next step are issued before the arithmetic of this one.
+  constexpr int KS = 32;
+  __shared__ __align__(16) float As[KS][68];
+  __shared__ __align__(16) float Bs[KS][68];
   const int tid = threadIdx.x;
   const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
   const long kb = (long)blockIdx.z * k_per_split;
   const long ke = min(K, kb + k_per_split);
-  const int lr = tid >> 2, lk = (tid & 3) * 4;
+  // A warp reads 32 bytes (two threads) of 16 rows at a time, and warps 0..3 / 4..7 cover the eight 16-byte
+  // pieces of a step for rows 0..15 / 16..31: the transposing stores below then hit 32 different banks
+  // ((lk + c) * 68 + row = 16 * (lane & 1) + (lane >> 1) + const, modulo 32).
+  const int lane_ = tid & 31, warp_ = tid >> 5;
+  const int lr = (warp_ >> 2) * 16 + (lane_ >> 1), lk = ((warp_ & 3) * 2 + (lane_ & 1)) * 4;   // rows lr and lr + 32
   const int tm = tid >> 4, tn = tid & 15;
   float acc[4][4];
 #pragma unroll
@@ -30,15 +37,28 @@ __global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, con
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  for (long k0 = kb; k0 < ke; k0 += 16) {
-    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-    if (m0 + lr < M) a = ld4_guard(A + (long)(m0 + lr) * K, k0 + lk, ke, vec != 0);
-    if (n0 + lr < N) b = ld4_guard(Bm + (long)(n0 + lr) * K, k0 + lk, ke, vec != 0);
-    As[lk + 0][lr] = a.x; As[lk + 1][lr] = a.y; As[lk + 2][lr] = a.z; As[lk + 3][lr] = a.w;
-    Bs[lk + 0][lr] = b.x; Bs[lk + 1][lr] = b.y; Bs[lk + 2][lr] = b.z; Bs[lk + 3][lr] = b.w;
-    __syncthreads();
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 a[2], b[2];
+  auto fetch = [&](long k0) {
 #pragma unroll
-    for (int kk = 0; kk < 16; ++kk) {
+    for (int h = 0; h < 2; ++h) {
+      const int row = lr + 32 * h;
+      a[h] = (m0 + row < M) ? ld4_guard(A + (long)(m0 + row) * K, k0 + lk, ke, vec != 0) : zero;
+      b[h] = (n0 + row < N) ? ld4_guard(Bm + (long)(n0 + row) * K, k0 + lk, ke, vec != 0) : zero;
+    }
+  };
+  if (kb < ke) fetch(kb);
+  for (long k0 = kb; k0 < ke; k0 += KS) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int row = lr + 32 * h;
+      As[lk + 0][row] = a[h].x; As[lk + 1][row] = a[h].y; As[lk + 2][row] = a[h].z; As[lk + 3][row] = a[h].w;
+      Bs[lk + 0][row] = b[h].x; Bs[lk + 1][row] = b[h].y; Bs[lk + 2][row] = b[h].z; Bs[lk + 3][row] = b[h].w;
+    }
+    __syncthreads();
+    if (k0 + KS < ke) fetch(k0 + KS);
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
       const float4 av = *reinterpret_cast<const float4*>(&As[kk][tm * 4]);
       const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tn * 4]);
       const float ar[4] = {av.x, av.y, av.z, av.w};
@@ -63,15 +83,29 @@ __global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, con
   }
 }
 
-// out[i] = scale(i) * sum_s part[s][i], s ascending (fixed order: results are reproducible).
-// scale(i) = chan_scale[i % period] if chan_scale else alpha.
-static __global__ void reduce_partials(const float* __restrict__ part, float* __restrict__ out, long count,
-                                int splits, float alpha, const float* __restrict__ chan_scale, int period) {
-  const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= count) return;
+// out[i] = scale(i) * sum_s part[s][i].  Eight threads share an output and take the splits in turn (one
+// thread per output would walk a chain of `splits` dependent loads); their eight sums are added in a
+// fixed order, so results are reproducible.  scale(i) = chan_scale[i % period] if chan_scale else alpha.
+// Launch with 256 threads: 32 outputs per block.
+constexpr int RP_OUT = 32, RP_LANES = 8;
+static __global__ void __launch_bounds__(RP_OUT * RP_LANES)
+reduce_partials(const float* __restrict__ part, float* __restrict__ out, long count, int splits, float alpha,
+                const float* __restrict__ chan_scale, int period) {
+  __shared__ float acc[RP_LANES][RP_OUT];
+  const int o = threadIdx.x % RP_OUT, g = threadIdx.x / RP_OUT;
+  const long i = (long)blockIdx.x * RP_OUT + o;
   float s = 0.f;
-  for (int k = 0; k < splits; ++k) s += part[(long)k * count + i];
-  out[i] = s * (chan_scale ? chan_scale[i % period] : alpha);
+  if (i < count) {
+#pragma unroll 4
+    for (int k = g; k < splits; k += RP_LANES) s += part[(long)k * count + i];
+  }
+  acc[g][o] = s;
+  __syncthreads();
+  if (g != 0 || i >= count) return;
+  float t = acc[0][o];
+#pragma unroll
+  for (int l = 1; l < RP_LANES; ++l) t += acc[l][o];
+  out[i] = t * (chan_scale ? chan_scale[i % period] : alpha);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -97,17 +131,27 @@ __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ 
     __syncthreads();
     if (q < Q) {
       const int nb = min(128, B - b0);
-      for (int bb = 0; bb < nb; ++bb) {
-        const float4 d = ld4_guard(dY + (long)(b0 + bb) * Q, q, Q, vec != 0);
+      // eight samples at a time: their loads are issued together (one load in flight per thread keeps
+      // only a few KB per SM on the way from HBM), then consumed in order
+      for (int bb0 = 0; bb0 < nb; bb0 += 8) {
+        float4 d8[8];
 #pragma unroll
-        for (int j4 = 0; j4 < 4; ++j4) {
-          const float4 s = *reinterpret_cast<const float4*>(&Ss[bb][j4 * 4]);
-          const float sr[4] = {s.x, s.y, s.z, s.w};
+        for (int u = 0; u < 8; ++u)
+          d8[u] = bb0 + u < nb ? ld4_guard(dY + (long)(b0 + bb0 + u) * Q, q, Q, vec != 0) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            float4& a = acc[j4 * 4 + i];
-            a.x = fmaf(sr[i], d.x, a.x); a.y = fmaf(sr[i], d.y, a.y);
-            a.z = fmaf(sr[i], d.z, a.z); a.w = fmaf(sr[i], d.w, a.w);
+        for (int u = 0; u < 8; ++u) {
+          const float4 d = d8[u];
+          const int bb = min(bb0 + u, 127);          // rows past nb hold zeros in d8; any valid row of Ss will do
+#pragma unroll
+          for (int j4 = 0; j4 < 4; ++j4) {
+            const float4 s = *reinterpret_cast<const float4*>(&Ss[bb][j4 * 4]);
+            const float sr[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float4& a = acc[j4 * 4 + i];
+              a.x = fmaf(sr[i], d.x, a.x); a.y = fmaf(sr[i], d.y, a.y);
+              a.z = fmaf(sr[i], d.z, a.z); a.w = fmaf(sr[i], d.w, a.w);
+            }
           }
         }
       }
@@ -128,7 +172,7 @@ __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ 
 // no shifted or im2col copy of Z exists.  A block owns 32 output x 64 input channels and all KS*KS
 // offsets; work items are (probe, row, 32-pixel chunk) triples dealt to grid.z splits in order.
 // ---------------------------------------------------------------------------------------------
-template <typename TL, typename TZ, int KS>
+template <typename TL, typename TZ, int KS, bool VEC>
 __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, const TZ* __restrict__ Z,
                                                      float* __restrict__ part, int r, int H, int W, int Cin,
                                                      int Cout, long items_per_split) {
@@ -156,6 +200,26 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
     const int y = (int)((it / chunks) % H);
     const int j = (int)(it / ((long)chunks * H));
     const int x0 = xc * XC;
+    if (VEC) {
+      // channel counts are multiples of 4: four consecutive channels per load (the tiles fill in a quarter
+      // of the instructions; the fill costs about as much as the arithmetic otherwise)
+      {
+        const int mm = (tid & 7) * 4, px = tid >> 3;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (x0 + px < W && m0 + mm < Cout) v = ld4(L + (((long)j * H + y) * W + x0 + px) * Cout + m0 + mm);
+        *reinterpret_cast<float4*>(&Ls[px][mm]) = v;
+      }
+      for (int idx = tid; idx < KS * (XC + KS - 1) * 16; idx += 256) {
+        const int nn = (idx & 15) * 4;
+        const int px = (idx >> 4) % (XC + KS - 1);
+        const int dy = (idx >> 4) / (XC + KS - 1);
+        const int yy = y + dy - P, xx = x0 + px - P;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
+          v = ld4(Z + (((long)j * H + yy) * W + xx) * Cin + n0 + nn);
+        *reinterpret_cast<float4*>(&Zs[dy][px][nn]) = v;
+      }
+    } else {
     for (int idx = tid; idx < XC * 32; idx += 256) {
       const int mm = idx & 31, px = idx >> 5;
       float v = 0.f;
@@ -171,6 +235,7 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
       if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
         v = to_f(Z[(((long)j * H + yy) * W + xx) * Cin + n0 + nn]);
       Zs[dy][px][nn] = v;
+    }
     }
     __syncthreads();
 #pragma unroll 4

@@ -67,7 +67,7 @@ static xconv_status sketch_static_run(const xconv_desc* d, const void* X, const 
                                         k_per_split, (K % 4 == 0) ? 1 : 0);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
-  reduce_partials<<<(unsigned)((out_elems + 255) / 256), 256, 0, st>>>(scratch, S, out_elems, (int)splits, 1.0f,
+  reduce_partials<<<(unsigned)((out_elems + RP_OUT - 1) / RP_OUT), RP_OUT * RP_LANES, 0, st>>>(scratch, S, out_elems, (int)splits, 1.0f,
                                                                        nullptr, 1);
   e = cudaGetLastError();
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
