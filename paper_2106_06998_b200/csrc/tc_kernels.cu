@@ -64,6 +64,14 @@ struct TcParams {
   // CONTRACT: kernel offsets per work unit (1, 3 or 9).  The offsets of a unit share the L tile of every
   // stage; their Z tiles lie one behind the other in the stage as consecutive column blocks, so one MMA
   // spans several offsets: columns [0, tpu * tile_n) of the accumulator, in `pieces` MMAs of whole blocks.
+  // CONTRACT, one offset per unit: a k-block's tiles arrive as two halves (the upper and the lower image rows of
+  // the patch), each with barriers of its own, in a ring of `stages` half-slots.  A half is released as soon
+  // as the last MMA that reads it is done, so four halves cover the load latency where two whole stages
+  // cannot.  `ks_h0` k-steps lie wholly in the first half, then (if the half has an odd number of 8-row
+  // groups) one k-step takes its first 8 rows from the end of the first half and its last 8 from the start
+  // of the second -- the descriptor's stride between 8-row groups, `sbo_x`, spans the gap -- then `ks_h1`.
+  int halves, ks_h0, ks_x, ks_h1;
+  uint32_t a_half_bytes, sbo_x;
   int tpu, pieces;
   uint32_t b_tap_bytes;    // bytes of one offset's Z tile
   int piece_cols[2];       // N of each MMA
@@ -479,6 +487,112 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0)
       for (long i = max(0L, it - stages); i < it; ++i)
         if (!mbar_wait(&full_bar[i % stages], (uint32_t)((i / stages) & 1), p.status, p.tag)) break;
+  } else if (warp == 0 && p.mode == MODE_CONTRACT && p.halves) {
+    // ------------------------------------------------------------------ TMA producer, k-blocks in two halves
+    if (lane == 0) {
+      const int slots = p.stages;          // half-slots
+      int s = 0;
+      long fill = 0, it = 0;
+      bool ok = true;
+      long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
+      const int hrows = p.patch_h >> 1;    // image rows per half
+      for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        const int row0 = w.tm * p.m_sub * TILE_M, col0 = w.tn * p.tile_n;
+        long q = w.kb0;
+        int px = (int)(q % p.patches_x); q /= p.patches_x;
+        int py = (int)(q % p.patches_y); q /= p.patches_y;
+        int pj = (int)q;
+        const int ks = 2 * p.pad + 1, dy = w.tap / ks - p.pad, dx = w.tap % ks - p.pad;
+        for (int i = 0; i < 2 * w.nkb; ++i) {
+          if (fill > 0) {
+            TW_BEGIN;
+            ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
+            TW_END(tw_pw);
+            if (!ok) break;
+          }
+          TW_BEGIN;
+          const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes, b_dst = a_dst + p.a_half_bytes;
+          const int x0 = px * p.patch_w, y0 = py * p.patch_h + (i & 1) * hrows;
+          mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
+          tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
+          tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
+          if ((i & 1) && ++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
+          ++it;
+          if (++s == slots) { s = 0; ++fill; }
+          TW_END(tw_pi);
+        }
+      }
+      TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it);
+      for (long i = max(0L, it - slots); i < it; ++i)
+        if (!mbar_wait(&full_bar[i % slots], (uint32_t)((i / slots) & 1), p.status, p.tag)) break;
+    }
+  } else if (warp == 1 && p.mode == MODE_CONTRACT && p.halves) {
+    // ------------------------------------------------------------------ MMA issuer, k-blocks in two halves
+    if (lane == 0) {
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+                             ((uint32_t)(p.tile_n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
+      const uint32_t step = p.mn_step >> 4;                                   // 16 rows
+      const uint32_t a_lo0 = (p.a_lbo >> 4) << 16, b_lo0 = (p.b_lbo >> 4) << 16;
+      const uint32_t hi = (p.sbo >> 4) | (1u << 14) | (p.layout << 29);
+      const uint32_t hi_x = (p.sbo_x >> 4) | (1u << 14) | (p.layout << 29);    // the k-step across the two halves
+      const uint32_t a_sub = p.a_sub_bytes >> 4, a_half16 = p.a_half_bytes >> 4, slot16 = stage_bytes >> 4;
+      const uint32_t base16 = (tiles_base & 0x3FFFFu) >> 4;
+      const bool two = p.m_sub == 2;
+      const uint32_t tile_n = (uint32_t)p.tile_n;
+      int s = 0;                           // half-slot of the next first half (always even)
+      uint32_t parity = 0;
+      bool ok = true;
+      long long tw_mw = 0, tw_mi = 0; (void)tw_mw; (void)tw_mi;
+      const long long t_start = clock64(); (void)t_start;
+      for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        if (w.nkb == 0) continue;
+        const uint32_t d = tmem_base;      // one unit per CTA and accumulator set (acc_bufs = 1)
+        uint32_t acc = 0;
+        for (int i = 0; i < w.nkb; ++i) {
+          const uint32_t h0 = base16 + (uint32_t)s * slot16, h1 = h0 + slot16;
+          { TW_BEGIN; ok = mbar_wait(&full_bar[s], parity, p.status, p.tag); TW_END(tw_mw); }
+          if (!ok) break;
+#ifdef XC_TIMELINE
+          if (i == 0) TT(2);
+#endif
+          TW_BEGIN;
+          tc_fence_after();
+          uint32_t a = a_lo0 | h0, b = b_lo0 | (h0 + a_half16);
+          for (int k = 0; k < p.ks_h0; ++k) {
+            umma_bf16(d, a, hi, b, hi, idesc, acc);
+            if (two) umma_bf16(d + tile_n, a + a_sub, hi, b, hi, idesc, acc);
+            acc = 1u; a += step; b += step;
+          }
+          TW_END(tw_mi);
+          { TW_BEGIN; ok = mbar_wait(&full_bar[s + 1], parity, p.status, p.tag); TW_END(tw_mw); }
+          if (!ok) break;
+          { TW_BEGIN;
+          tc_fence_after();
+          if (p.ks_x) {                     // rows [16 ks_h0, +8) of the first half and [0, 8) of the second
+            umma_bf16(d, a, hi_x, b, hi_x, idesc, acc);
+            if (two) umma_bf16(d + tile_n, a + a_sub, hi_x, b, hi_x, idesc, acc);
+            acc = 1u;
+          }
+          umma_commit(&empty_bar[s]);       // the first half may be refilled
+          a = (a_lo0 | h1) + (p.ks_x ? (p.sbo >> 4) : 0u);
+          b = (b_lo0 | (h1 + a_half16)) + (p.ks_x ? (p.sbo >> 4) : 0u);
+          for (int k = 0; k < p.ks_h1; ++k) {
+            umma_bf16(d, a, hi, b, hi, idesc, acc);
+            if (two) umma_bf16(d + tile_n, a + a_sub, hi, b, hi, idesc, acc);
+            acc = 1u; a += step; b += step;
+          }
+          umma_commit(&empty_bar[s + 1]);
+          s += 2;
+          if (s == p.stages) { s = 0; parity ^= 1u; }
+          TW_END(tw_mi); }
+        }
+        if (ok) umma_commit(&tmem_full_bar[0]);
+        TT(3);
+        TW_STORE(2, tw_mw); TW_STORE(3, tw_mi); TW_STORE(4, clock64() - t_start);
+      }
+    }
   } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     // One thread; its loop is kept free of divisions (coordinates advance incrementally).
@@ -1257,6 +1371,16 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     p->ct_items_rem = p->ct_items % splits;
     p->part_bytes = (size_t)p->ct_splits * T * p->ct_tiles_m * p->ct_tiles_n * p->ct_m_sub * TILE_M * p->ct_tile_n *
                     sizeof(float);
+    // k-blocks in two halves (upper and lower image rows of the patch): four half-slots cover the load
+    // latency that two whole stages cannot.  Needs halves of whole 8-row swizzle groups and one unit per CTA.
+    const int hrows = (p->patch_h / 2) * p->patch_w;
+    p->ct_halves = (p->ct_tpu == 1 && p->ct_cw == 64 && p->patch_h % 2 == 0 && hrows % 8 == 0 && hrows >= 16 &&
+                    tiles * p->ct_splits <= NUM_SMS && ct_ctas == 1 && block * (a_groups + b_groups) >= 64 * 1024) ? 1 : 0;
+    if (p->ct_halves) {
+      const int half = (int)(block / 2 * (a_groups + b_groups));
+      p->ct_stages = std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK) / half) & ~1;      // half-slots, an even number
+      if (p->ct_stages < 4) p->ct_halves = 0, p->ct_stages = pick_stages(stage, ct_ctas);
+    }
   }
   return mask;
 }
@@ -1339,8 +1463,9 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   const uint64_t db[5] = {(uint64_t)cw, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(d->Cin / cw), (uint64_t)d->r};
   const uint64_t sb[4] = {(uint64_t)d->Cin * 2, (uint64_t)d->W * d->Cin * 2, row_bytes,
                           (uint64_t)d->H * d->W * d->Cin * 2};
-  const uint32_t box_a[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)groups_a, 1};
-  const uint32_t box_b[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, (uint32_t)groups_b, 1};
+  const uint32_t box_h = (uint32_t)(pl.ct_halves ? pl.patch_h / 2 : pl.patch_h);   // image rows per copy
+  const uint32_t box_a[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, box_h, (uint32_t)groups_a, 1};
+  const uint32_t box_b[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, box_h, (uint32_t)groups_b, 1};
   if (!make_map(&ma, L, 5, da, sa, box_a, swz) || !make_map(&mb, Z, 5, db, sb, box_b, swz)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_CONTRACT;
@@ -1373,6 +1498,24 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.tiles_m = pl.ct_tiles_m;
   p.tiles_n = pl.ct_tiles_n;
   p.taps = T;
+  if (pl.ct_halves) {
+    // every tile shrinks to half its rows; a "stage" of the ring is a half-slot
+    const int hrows = bk / 2;
+    p.halves = 1;
+    p.a_box_bytes = p.b_box_bytes = (uint32_t)hrows * row_bytes;
+    p.a_sub_bytes = (uint32_t)p.a_boxes * p.a_box_bytes;
+    p.a_stage_bytes = p.a_half_bytes = (uint32_t)pl.ct_m_sub * p.a_sub_bytes;
+    p.b_tap_bytes = (uint32_t)p.b_boxes * p.b_box_bytes;
+    p.b_stage_bytes = p.b_tap_bytes;
+    p.tx_bytes = p.a_stage_bytes + p.b_stage_bytes;
+    p.a_lbo = one_group ? 0u : p.a_box_bytes;
+    p.b_lbo = p.b_box_bytes;
+    p.ks_h0 = hrows / 16;
+    p.ks_x = (hrows % 16) ? 1 : 0;
+    p.ks_h1 = p.ks_x ? (hrows - 8) / 16 : hrows / 16;
+    // from the last 8-row group of a first half to the first group of the second half (same block, same operand)
+    p.sbo_x = (p.a_stage_bytes + p.b_stage_bytes) - (uint32_t)(p.ks_h0 * 16) * row_bytes;
+  }
   p.kblocks = pl.ct_items;
   p.kblocks_per_split = pl.ct_items_per_split;
   p.kb_rem = pl.ct_items_rem;

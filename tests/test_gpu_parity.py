@@ -132,6 +132,26 @@ def test_backprobe_tensor_path_column_tiles(shape):
     check("L", host(L), O.backprobe(S, lay["dY"]), TOL["bf16"])
 
 
+@pytest.mark.parametrize("shape", [
+    # B, Cin, Cout, H, W, r -- wide layers whose contraction copies every k-block in two halves
+    (16, 256, 256, 8, 28, 40),    # 28 x 4 patches: halves of 56 pixels, one MMA step spans the two halves
+    (16, 256, 256, 16, 16, 36),   # 16 x 8 patches: halves of 64 pixels, no step across the halves
+    (16, 256, 128, 8, 28, 24),    # one 128-row tile of output channels
+    (8, 256, 192, 12, 28, 33),    # 192 output channels: the second row tile half empty; odd probe count
+])
+def test_contraction_in_half_stages(shape):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="bf16", seed=sum(shape), z="rademacher", x="relu")
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, torch.bfloat16)
+    assert xb.engine_for(desc, xb.OP_CONTRACT) == "tcgen05_bf16"
+    d = dev(lay)
+    g = np.random.Generator(np.random.PCG64(sum(shape)))
+    Lr = inputs.round_to_storage(g.standard_normal((r, Cout, H, W)).astype(np.float32), "bf16")
+    dW = xb.xconv_contract(xb.to_device(Lr, "bf16"), d["Z"])
+    torch.cuda.synchronize()
+    check("dW (contraction alone)", host(dW), O.wgrad_contract(Lr, lay["Z"], 3, 3), 1e-4)
+
+
 def test_pointwise_kernel_on_the_tensor_path():
     lay = inputs.make_custom(16, 64, 128, 8, 12, 32, dtype="bf16", seed=78, KH=1, KW=1)
     desc = xb.make_desc(16, 64, 128, 8, 12, 32, torch.bfloat16, 1)
