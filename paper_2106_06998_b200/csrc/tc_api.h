@@ -34,6 +34,7 @@ struct TcWgradPlan {
 struct TcConvPlan {
   int tile_n, tiles_n, stages, patch_w, patch_h, patches_x, patches_y;
   int m_sub;           // 2 = a work unit covers the same patch of two images, which share the weight tile
+  int cw;              // input channels per stage: 64 (128-byte tile rows) or 32 (64-byte rows, more stages)
   size_t wt_bytes;     // dgrad only: transposed, flipped copy of the weights
 };
 

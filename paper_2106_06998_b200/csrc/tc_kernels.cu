@@ -656,7 +656,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
             // [tile_n output channels x 64 input channels] block of the weights
             tma_load_5d(a_dst, &map_a, 0, w.px * p.patch_w + dx, w.py * p.patch_h + dy, pj, w.img, &full_bar[s]);
-            tma_load_2d(b_dst, &map_b, kc + pj * 64, col0, &full_bar[s]);
+            tma_load_2d(b_dst, &map_b, kc + (pj << p.cw_shift), col0, &full_bar[s]);
             if (++pj == p.cgroups) { pj = 0; kc += p.Cin; if (++dx > p.pad) { dx = -p.pad; ++dy; } }
           } else {
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
@@ -1597,7 +1597,7 @@ static void pick_patch_conv(int H, int W, int* pw, int* ph) {
 bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
   if (d->dtype != XCONV_BF16) return false;
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
-  if (Ci % 64 != 0 || Co % 8 != 0 || Co < 16) return false;
+  if (Ci % 32 != 0 || Co % 8 != 0 || Co < 16) return false;
   p->tile_n = std::min(256, round_up(Co, 16));
   p->tiles_n = (int)cdivl(Co, p->tile_n);
   pick_patch_conv(d->H, d->W, &p->patch_w, &p->patch_h);
@@ -1608,7 +1608,12 @@ bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
   // from 94 to 62.5 bytes, which is what bounded the convolution.
   const int px = p->patch_w * p->patch_h;
   p->m_sub = (px % 8 == 0 && d->B >= 2) ? 2 : 1;
-  p->stages = pick_stages((uint32_t)(p->m_sub == 2 ? px + TILE_M : TILE_M) * 128 + (uint32_t)p->tile_n * 128, 1);
+  // Input channels go by 64 per stage (128-byte tile rows); layers whose channel count is a multiple of 32
+  // only take 32 per stage (64-byte rows, 64-byte swizzle).  (32 per stage everywhere, for more and smaller
+  // stages, was slower: 557 against 485 us on the 256-channel layer.)
+  const uint32_t rows = (uint32_t)(p->m_sub == 2 ? px + TILE_M : TILE_M) + (uint32_t)p->tile_n;
+  p->cw = Ci % 64 == 0 ? 64 : 32;
+  p->stages = pick_stages(rows * 2 * (uint32_t)p->cw, 1);
   p->wt_bytes = dgrad ? (size_t)d->Cout * d->KH * d->KW * d->Cin * 2 : 0;
   return true;
 }
@@ -1627,14 +1632,16 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
     Wk = wt;
   }
   CUtensorMap ma, mb;
-  // input as (64 channels, x, y, channel blocks of 64, image); weights as [Co][T*Ci]
-  const uint64_t da[5] = {64, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(Ci / 64), (uint64_t)d->B};
-  const uint64_t sa[4] = {(uint64_t)Ci * 2, (uint64_t)d->W * Ci * 2, 128, (uint64_t)d->H * d->W * Ci * 2};
-  const uint32_t box_a[5] = {64, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1, (uint32_t)pl.m_sub};
+  // input as (cw channels, x, y, channel blocks of cw, image); weights as [Co][T*Ci]; cw = 64 or 32
+  const uint32_t cw = (uint32_t)pl.cw, rb = 2 * cw;                      // channels and bytes per tile row
+  const CUtensorMapSwizzle swz = cw == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  const uint64_t da[5] = {cw, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)(Ci / cw), (uint64_t)d->B};
+  const uint64_t sa[4] = {(uint64_t)Ci * 2, (uint64_t)d->W * Ci * 2, rb, (uint64_t)d->H * d->W * Ci * 2};
+  const uint32_t box_a[5] = {cw, (uint32_t)pl.patch_w, (uint32_t)pl.patch_h, 1, (uint32_t)pl.m_sub};
   const uint64_t db[2] = {(uint64_t)T * Ci, (uint64_t)Co};
   const uint64_t sb[1] = {(uint64_t)T * Ci * 2};
-  const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
-  if (!make_map(&ma, in, 5, da, sa, box_a) || !make_map(&mb, Wk, 2, db, sb, box_b)) return XCONV_ERR_CUDA;
+  const uint32_t box_b[2] = {cw, (uint32_t)pl.tile_n};
+  if (!make_map(&ma, in, 5, da, sa, box_a, swz) || !make_map(&mb, Wk, 2, db, sb, box_b, swz)) return XCONV_ERR_CUDA;
   TcParams p{};
   p.mode = MODE_CONV;
   p.tile_n = pl.tile_n;
@@ -1643,19 +1650,20 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   p.acc_bufs = (2 * pl.m_sub * pl.tile_n <= 512) ? 2 : 1;
   p.tmem_cols = pow2_cols(p.acc_bufs * pl.m_sub * pl.tile_n);
   p.stages = pl.stages;
-  p.ksteps = 4;
+  p.ksteps = (int)cw / 16;
   p.a_boxes = p.b_boxes = 1;
   // one image: the patch fills the first px rows of a 128-row tile.  Two images: the second image's px
   // rows follow the first's directly and its MMA tile starts there; 128 rows behind that start belong to the stage.
-  p.a_sub_bytes = (pl.m_sub == 2 ? px : (uint32_t)TILE_M) * 128;
-  p.a_stage_bytes = (pl.m_sub == 2 ? px + TILE_M : (uint32_t)TILE_M) * 128;
-  p.b_stage_bytes = (uint32_t)pl.tile_n * 128;
-  p.tx_bytes = (uint32_t)pl.m_sub * px * 128 + p.b_stage_bytes;
+  p.a_sub_bytes = (pl.m_sub == 2 ? px : (uint32_t)TILE_M) * rb;
+  p.a_stage_bytes = (pl.m_sub == 2 ? px + TILE_M : (uint32_t)TILE_M) * rb;
+  p.b_stage_bytes = (uint32_t)pl.tile_n * rb;
+  p.tx_bytes = (uint32_t)pl.m_sub * px * rb + p.b_stage_bytes;
+  if (cw == 32) { p.layout = 4; p.sbo = 8 * rb; p.mn_step = 16 * rb; p.cw_shift = 5; }   // 64-byte swizzle
   p.a_mn_major = p.b_mn_major = 0;
   p.tiles_m = 1;
   p.tiles_n = pl.tiles_n;
   p.taps = 1;
-  p.kblocks = (long)T * (Ci / 64);
+  p.kblocks = (long)T * (Ci / cw);
   p.kblocks_per_split = p.kblocks;
   p.units = cdivl(d->B, pl.m_sub) * pl.patches_y * pl.patches_x * pl.tiles_n;
   p.nimg = d->B;
@@ -1671,7 +1679,7 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   p.Cin = Ci;
   p.H = d->H;
   p.W = d->W;
-  p.cgroups = Ci / 64;
+  p.cgroups = Ci / cw;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
   return launch(ma, mb, p, (unsigned)std::min<long>(p.units, NUM_SMS), st);
 }
