@@ -117,6 +117,9 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------------- oracle legs
 
+_ORACLE_INPUTS = {}
+
+
 def oracle_sample_time(cfg, r, frac=8):
     """The float64 oracle, as it stands, on a bounded sample of the workload: the sketch of B/frac
     samples plus the estimator for Cout/frac output channels (all probes, input channels and pixels).
@@ -130,11 +133,15 @@ def oracle_sample_time(cfg, r, frac=8):
         while est / frac > 16 and frac < 64:
             frac *= 2
     Bs, Ms = max(1, c["B"] // frac), max(1, c["Cout"] // frac)
-    g = np.random.Generator(np.random.PCG64(1))
-    X = inputs.draw(c["x"], (Bs, c["Cin"], c["H"], c["W"]), 11, c["dtype"])
-    dY = inputs.draw("normal", (c["B"], Ms, c["H"], c["W"]), 12, c["dtype"], c["dy_var"] ** 0.5)
-    Z = inputs.draw(c["z"], (r, c["Cin"], c["H"], c["W"]), 13, c["dtype"])
-    S = g.standard_normal((r, c["B"]))
+    key = (cfg, r, frac)
+    if key not in _ORACLE_INPUTS:            # drawn once per run, outside the timed calls
+        g = np.random.Generator(np.random.PCG64(1))
+        _ORACLE_INPUTS.clear()
+        _ORACLE_INPUTS[key] = (inputs.draw(c["x"], (Bs, c["Cin"], c["H"], c["W"]), 11, c["dtype"]),
+                               inputs.draw("normal", (c["B"], Ms, c["H"], c["W"]), 12, c["dtype"], c["dy_var"] ** 0.5),
+                               inputs.draw(c["z"], (r, c["Cin"], c["H"], c["W"]), 13, c["dtype"]),
+                               g.standard_normal((r, c["B"])))
+    X, dY, Z, S = _ORACLE_INPUTS[key]
     t0 = time.perf_counter()
     O.sketch(X, Z)
     t1 = time.perf_counter()
@@ -162,8 +169,19 @@ def run_reference(args):
     c = inputs.layer_shape(args.config)
     times = []
     sample = ""
+    frac = args.oracle_frac
+    if frac <= 0:
+        # every step times the oracle on a slice of the layer; the slice shrinks with the number of steps
+        # asked for, so that the whole run stays within a few minutes (about 0.3 s of oracle time per
+        # GFLOP-pair on a few cores; at most a 16th of the layer: on smaller slices the oracle's fixed costs take
+        # over and the layer time extrapolated from the slice comes out too long)
+        est = 2.0 * args.r * c["Cout"] * c["H"] * c["W"] * (c["B"] + 9 * c["Cin"]) / 4e9
+        per_step = min(16.0, 150.0 / max(1, args.warmup + args.steps))
+        frac = 1
+        while est / frac > per_step and frac < 16:
+            frac *= 2
     for i in range(args.warmup + args.steps):
-        t, _, _, sample = oracle_sample_time(args.config, args.r, frac=args.oracle_frac)
+        t, _, _, sample = oracle_sample_time(args.config, args.r, frac=frac)
         if i >= args.warmup:
             times.append(t)
     t = float(np.mean(times))
