@@ -204,7 +204,7 @@ def workload_config(args, c, copies=1):
           f"addresses, {copies * step_mb:.0f} MB in all, so that no step finds its inputs in the 126 MB L2")
     return {"workload": f"config {args.config}: 3x3 conv layer B={c['B']} Cin={c['Cin']} Cout={c['Cout']} "
                         f"{c['H']}x{c['W']} {c['dtype']} storage, {c['z']} probes, r={args.r}",
-            "r": args.r, "layout": "channels_last", "l2": l2}
+            "r": args.r, "layout": "channels_last", "accumulate": "f32", "l2": l2}
 
 
 # ----------------------------------------------------------------------------------- GPU arm
@@ -474,7 +474,7 @@ def run_xconv(args):
     es = X.element_size()
     line = {"metric": METRIC, "value": world * 1e3 / ms_step, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32" if c["dtype"] == "f32" else "bf16 (f32 accumulate)",
+            "vs_baseline": None, "dtype": "f32" if c["dtype"] == "f32" else "bf16",
             "data": "synthetic", "config": workload_config(args, c, layer.copies), "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches[0], "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
             "phase_timing": {"ms_per_step_with_events": total_ev_ms / args.steps,
