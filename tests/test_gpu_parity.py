@@ -202,6 +202,12 @@ def test_full_size_sampled(cfg, r):
     ns = np.sort(g.choice(lay["Cin"], size=min(6, lay["Cin"]), replace=False))
     dWo = O.wgrad_estimate(So, lay["dY"][:, ms], lay["Z"][:, ns])
     check("dW block", host(dW)[np.ix_(ms, ns)], dWo, tol)
+    # the two halves as the benchmark calls them (Algorithm 1's order, which xconv_wgrad leaves when r > B)
+    L = xb.xconv_backprobe(S, d["dY"])
+    dW2 = xb.xconv_contract(L, d["Z"])
+    torch.cuda.synchronize()
+    check("dW block (back-probe + contraction)", host(dW2)[np.ix_(ms, ns)], dWo, tol)
+    del L, dW2
     bs = np.sort(g.choice(lay["B"], size=min(2, lay["B"]), replace=False))
     check("Y samples", host(Y[bs]), O.conv_forward(lay["X"][bs], lay["W"]), tol)
     check("dX samples", host(dX[bs]), O.dx_exact(lay["dY"][bs], lay["W"]), tol)
