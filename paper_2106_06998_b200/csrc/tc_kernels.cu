@@ -78,6 +78,10 @@ struct TcParams {
   long units;              // work units = tiles x k-splits, dealt round-robin to the CTAs
   long kblocks, kblocks_per_split;
   long kb_rem;             // the first kb_rem k-splits take one k-block more than kblocks_per_split
+  // SKETCH: k-split s takes the k-blocks s, s + k_weave, s + 2 k_weave, ... (k_weave = number of splits) instead
+  // of a run of consecutive ones, so that the CTAs of a row tile read neighbouring pieces of the same rows at
+  // the same time.  0: consecutive k-blocks.
+  int k_weave;
   // contraction geometry
   int patch_w, patch_h, patches_x, patches_y, pad;
   // extents for the epilogue guards
@@ -609,7 +613,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int col0 = w.tn * p.tile_n;
         // running coordinates of the k-block
         int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0;
-        if (p.mode == MODE_SKETCH) kc = (int)(w.kb0 * 64 * p.kgroup);
+        if (p.mode == MODE_SKETCH) kc = (int)((p.k_weave ? w.split : w.kb0) * 64 * p.kgroup);
         else if (p.mode == MODE_BACKPROBE) kc = (int)w.kb0 * p.ksteps * 16;
         else if (p.mode == MODE_CONV) { dx = dy = -p.pad; }     // pj counts channel blocks, kc = offset * Cin
         else {
@@ -640,11 +644,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               // kgroup consecutive k-blocks per operand in one 3-d box (64 k, rows, k-blocks)
               if (get_a) tma_load_3d(a_dst, &map_a, 0, row0, kc >> 6, &full_bar[s]);
               if (get_b) tma_load_3d(b_dst, &map_b, 0, col0, kc >> 6, &full_bar[s]);
-              kc += 64 * p.kgroup;
+              kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
             } else {
               if (get_a) tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
               if (get_b) tma_load_2d(b_dst, &map_b, kc, col0, &full_bar[s]);
-              kc += 64;
+              kc += 64 * (p.k_weave ? p.k_weave : 1);
             }
           } else if (p.mode == MODE_BACKPROBE) {
             tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
@@ -824,7 +828,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
         const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
         const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
-        long kc = w.kb0 * 64 * p.kgroup;
+        long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
         for (int i = 0; i < w.nkb && ok; ++i) {
           if (gen_fill > 0) {
             if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
@@ -858,7 +862,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
           __syncwarp();
           if (lane == 0) mbar_arrive(&full_bar[gen_s]);
-          kc += 64 * p.kgroup;
+          kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
           if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
         }
         if (!ok) break;
@@ -1256,6 +1260,7 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   p.kblocks = pl.kblocks;
   p.kblocks_per_split = pl.kblocks_per_split;
   p.kb_rem = pl.kb_rem;
+  p.k_weave = pl.splits;
   p.units = (long)pl.tiles_m * pl.tiles_n * pl.splits;
   p.rows = rows;
   p.cols = cols;
