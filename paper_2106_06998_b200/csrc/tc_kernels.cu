@@ -345,6 +345,49 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 #define TT(slot) do {} while (0)
 #endif
 
+// The MMAs of `nkb` k-blocks that arrive in two halves (see TcParams::halves), with the numbers of k-steps known at
+// compile time so that the issuing thread runs straight-line code: it executes about one instruction per six
+// clocks, and every instruction between two tcgen05.mma counts.  Returns false if a wait ran out.
+template <int K0, int KX, int K1, bool TWO>
+__device__ __forceinline__ bool umma_halves_items(int nkb, int& s, uint32_t& parity, uint32_t& acc, int slots,
+                                                  uint64_t* full_bar, uint64_t* empty_bar, uint32_t base16, uint32_t slot16,
+                                                  uint32_t a_lo0, uint32_t b_lo0, uint32_t a_half16, uint32_t a_sub,
+                                                  uint32_t step, uint32_t sbo16, uint32_t hi, uint32_t hi_x, uint32_t idesc,
+                                                  uint32_t d, uint32_t tile_n, unsigned int* status, unsigned int tag) {
+  for (int i = 0; i < nkb; ++i) {
+    const uint32_t h0 = base16 + (uint32_t)s * slot16, h1 = h0 + slot16;
+    if (!mbar_wait(&full_bar[s], parity, status, tag)) return false;
+    tc_fence_after();
+    uint32_t a = a_lo0 | h0, b = b_lo0 | (h0 + a_half16);
+#pragma unroll
+    for (int k = 0; k < K0; ++k) {
+      umma_bf16(d, a, hi, b, hi, idesc, acc);
+      if (TWO) umma_bf16(d + tile_n, a + a_sub, hi, b, hi, idesc, acc);
+      acc = 1u; a += step; b += step;
+    }
+    if (!mbar_wait(&full_bar[s + 1], parity, status, tag)) return false;
+    tc_fence_after();
+    if (KX) {
+      umma_bf16(d, a, hi_x, b, hi_x, idesc, acc);
+      if (TWO) umma_bf16(d + tile_n, a + a_sub, hi_x, b, hi_x, idesc, acc);
+      acc = 1u;
+    }
+    umma_commit(&empty_bar[s]);
+    a = (a_lo0 | h1) + (KX ? sbo16 : 0u);
+    b = (b_lo0 | (h1 + a_half16)) + (KX ? sbo16 : 0u);
+#pragma unroll
+    for (int k = 0; k < K1; ++k) {
+      umma_bf16(d, a, hi, b, hi, idesc, acc);
+      if (TWO) umma_bf16(d + tile_n, a + a_sub, hi, b, hi, idesc, acc);
+      acc = 1u; a += step; b += step;
+    }
+    umma_commit(&empty_bar[s + 1]);
+    s += 2;
+    if (s == slots) { s = 0; parity ^= 1u; }
+  }
+  return true;
+}
+
 constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
 constexpr int TC_THREADS = 192;
@@ -554,6 +597,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (w.nkb == 0) continue;
         const uint32_t d = tmem_base;      // one unit per CTA and accumulator set (acc_bufs = 1)
         uint32_t acc = 0;
+#ifndef XC_TIMELINE
+        if (p.ks_h0 == 3 && p.ks_x == 1 && p.ks_h1 == 3) {      // halves of 56 pixels (28-wide images): unrolled
+          ok = two ? umma_halves_items<3, 1, 3, true>(w.nkb, s, parity, acc, p.stages, full_bar, empty_bar, base16, slot16,
+                                                       a_lo0, b_lo0, a_half16, a_sub, step, p.sbo >> 4, hi, hi_x, idesc, d,
+                                                       tile_n, p.status, p.tag)
+                   : umma_halves_items<3, 1, 3, false>(w.nkb, s, parity, acc, p.stages, full_bar, empty_bar, base16, slot16,
+                                                        a_lo0, b_lo0, a_half16, a_sub, step, p.sbo >> 4, hi, hi_x, idesc, d,
+                                                        tile_n, p.status, p.tag);
+          if (ok) umma_commit(&tmem_full_bar[0]);
+          continue;
+        }
+#endif
         for (int i = 0; i < w.nkb; ++i) {
           const uint32_t h0 = base16 + (uint32_t)s * slot16, h1 = h0 + slot16;
           { TW_BEGIN; ok = mbar_wait(&full_bar[s], parity, p.status, p.tag); TW_END(tw_mw); }
