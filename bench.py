@@ -7,9 +7,11 @@ One step is one pass of the hot path over one synthetic layer batch: xconv_sketc
 xconv_contract (the last two are exactly xconv_wgrad) through the C ABI, inputs resident in HBM.  The
 line printed by rank 0 carries the whole-job throughput, the same metric end to end from pinned host
 buffers (`e2e`), the roofline of the dominant kernel (`roofline`), the float64 oracle timed on the
-host cores (`cpu_baseline`), per-phase times and, as context, torch's exact cuDNN weight gradient.
+host cores (`cpu_baseline`), the time of every phase launched alone (`phases`: sketch, back-probe,
+contraction, and `wgrad` = the estimator as one call with L not counted in its algorithmic bytes)
+and, as context, torch's exact cuDNN weight gradient.
 With N > 1 every rank owns its own batch shard (same Z everywhere) and the dW estimates are summed
-with one NCCL all-reduce per step (weak scaling).
+with one NCCL all-reduce per step (weak scaling); `--gpus N` without a launcher starts the N ranks itself.
 """
 from __future__ import annotations
 
@@ -30,7 +32,8 @@ import numpy as np
 METRIC = "sketch+wgrad layers/s"
 UNIT = "layers/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12       # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+FP32_ALU_TFLOPS_DERIVED = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock (context)
+PHASE_STREAM_BYTES = 200 << 20                         # a phase that streams this much per launch evicts its own inputs
 L2_ROTATE_BYTES = 300 << 20                            # tensors of a step below this: rotate through copies
 
 
@@ -52,8 +55,13 @@ def layer_work(c, r):
     T = 9
     return {
         "sketch": dict(bytes=s * (B + r) * Cin * N + 4 * r * B, flops=2.0 * r * B * Cin * N),
+        # the two launches of the estimator, each charged the L it writes or reads ("L charged": diagnostics)
         "backprobe": dict(bytes=s * (B + r) * Cout * N + 4 * r * B, flops=2.0 * r * B * Cout * N),
         "contract": dict(bytes=s * r * (Cin + Cout) * N + 4 * T * Cin * Cout, flops=2.0 * T * r * Cout * Cin * N),
+        # the estimator as one unit of work: reads dY, Z and S, writes dW; L is not counted (what a kernel that
+        # never wrote L would move), so any round trip of L is overhead charged to the implementation
+        "wgrad": dict(bytes=s * (B * Cout * N + r * Cin * N) + 4 * r * B + 4 * T * Cout * Cin,
+                      flops=2.0 * r * Cout * N * (B + T * Cin)),
     }
 
 
@@ -184,13 +192,16 @@ def run_reference(args):
         t, _, _, sample = oracle_sample_time(args.config, args.r, frac=frac)
         if i >= args.warmup:
             times.append(t)
-    t = float(np.mean(times))
+    t = float(np.mean(times))              # layer time: frac x the time of one step's sample
     val = 1.0 / t
+    cfg_line = workload_config(args, c, 0)
+    cfg_line["layers_per_step"] = 1.0 / frac
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t, "higher_is_better": True,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / frac, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(args, c),
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample},
+            "config": cfg_line,
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": host_threads(), "kind": "oracle",
+                             "sample": sample + f"; a step is one sample = 1/{frac} layer, value = layers_per_step / step time"},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -199,7 +210,8 @@ def run_reference(args):
 def workload_config(args, c, copies=1):
     es = 4 if c["dtype"] == "f32" else 2
     step_mb = es * c["H"] * c["W"] * (c["B"] * (c["Cin"] + c["Cout"]) + args.r * (c["Cin"] + c["Cout"])) / 1e6
-    l2 = (f"the tensors of one step ({step_mb:.0f} MB) exceed the 126 MB L2" if copies == 1 else
+    l2 = ("not applicable: the oracle runs on the host" if copies == 0 else
+          f"the tensors of one step ({step_mb:.0f} MB) exceed the 126 MB L2" if copies == 1 else
           f"steps rotate through {copies} copies of the tensors of one step ({step_mb:.0f} MB each) at different "
           f"addresses, {copies * step_mb:.0f} MB in all, so that no step finds its inputs in the 126 MB L2")
     return {"workload": f"config {args.config}: 3x3 conv layer B={c['B']} Cin={c['Cin']} Cout={c['Cout']} "
@@ -221,7 +233,7 @@ def run_xconv(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world != args.gpus:
-        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -322,6 +334,58 @@ def run_xconv(args):
                       for k, n in enumerate(("sketch", "backprobe", "contract"))}
             return total, ph, clk
 
+        def phase_call(self, name, i):
+            """One launch of one phase on the i-th tensor set (through the C ABI, as in the step)."""
+            X_, dY_, Z_, L_ = self.sets[i % len(self.sets)]
+            if name == "sketch":
+                xb.sketch_into(self.desc, X_, Z_, self.S, self.ws)
+            elif name == "backprobe":
+                xb.backprobe_into(self.desc, self.S, dY_, L_, self.ws)
+            elif name == "contract":
+                xb.contract_into(self.desc, L_, Z_, self.dW, self.ws)
+            else:
+                xb.wgrad_into(self.desc, self.S, dY_, Z_, self.dW, self.ws)
+
+        def measure_phase(self, name, steps):
+            """Average duration of one phase (its main kernel and its helper kernels): `steps` launches of
+            that call back to back between two CUDA events on the launching stream, after warm-up.  No event
+            sits between two launches, so consecutive launches overlap preamble and tail exactly as the calls
+            of a step do.  A phase that moves less than PHASE_STREAM_BYTES per launch rotates through enough
+            tensor sets at different addresses that no launch finds its inputs in the 126 MB L2."""
+            es = X.element_size()
+            per = {"sketch": es * (X.numel() + self.sets[0][2].numel()),
+                   "backprobe": es * (dY.numel() + self.sets[0][3].numel()),
+                   "contract": es * (self.sets[0][2].numel() + self.sets[0][3].numel()),
+                   "wgrad": es * (dY.numel() + self.sets[0][2].numel())}[name]
+            need = 1 if per >= PHASE_STREAM_BYTES else min(64, -(-L2_ROTATE_BYTES // per) + 1)
+            while len(self.sets) < need:      # more copies of the tensors, made outside the timed region
+                X0, dY0, Z0, L0 = self.sets[0]
+                self.sets.append((X0, dY0, Z0.clone(), torch.empty_like(L0)) if name == "contract"
+                                 else (X0.clone(), dY0.clone(), Z0.clone(), torch.empty_like(L0)))
+            if name == "contract":            # every L the region reads holds this layer's back-probe
+                for i in range(need):
+                    xb.backprobe_into(self.desc, self.S, self.sets[i][1], self.sets[i][3], self.ws)
+            for i in range(max(3, need)):
+                self.phase_call(name, i)
+            torch.cuda.synchronize()
+            a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_.record()
+            for i in range(steps):
+                self.phase_call(name, i % need)
+            b_.record()
+            torch.cuda.synchronize()
+            if xb.workspace_status(self.ws) != 0:
+                raise SystemExit(f"a device-side wait ran out while timing {name}")
+            return a_.elapsed_time(b_) / steps, need
+
+        def measure_phases(self, steps):
+            out, sets = {}, {}
+            for n in ("sketch", "backprobe", "contract", "wgrad"):
+                out[n], sets[n] = self.measure_phase(n, steps)
+            del self.sets[max(1, self.copies):]
+            torch.cuda.empty_cache()
+            return out, sets
+
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
@@ -332,8 +396,11 @@ def run_xconv(args):
                                         phase_events=False)
     ms_step = total_ms / args.steps
     n_launch = layer.launches
-    # the same K steps again with an event between the calls: per-phase times for the roofline
-    total_ev_ms, phase_ms, _ = layer.measure(args.steps, 3, None, phase_events=True)
+    # every phase on its own: K launches back to back between two events (the roofline numbers), and the K
+    # steps once more with an event between the calls (diagnostic: the events keep the kernels from overlapping)
+    n_phase = max(5, min(args.steps, 100))
+    phase_ms, phase_sets = layer.measure_phases(n_phase)
+    total_ev_ms, phase_ev_ms, _ = layer.measure(n_phase, 3, None, phase_events=True)
     desc, S, dW = layer.desc, layer.S, layer.dW
     launches = [n_launch]
 
@@ -368,34 +435,46 @@ def run_xconv(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (live CUDA-event times of the timed region)
+    # ---- roofline of every phase (live CUDA-event times: K launches of the phase back to back)
     peaks, peak_src = load_peaks()
     tensor_peak = peaks["bf16_tflops"] if total_ms < 2000 else peaks["bf16_tflops_sustained"]
+    fma_tflops = xb.measure_fma_rate(dev)              # measured FP32 FMA rate: the ceiling of the FP32-FMA kernels
 
     def phase_table(r_, desc_, ph_ms):
         work = layer_work(c, r_)
         eng = {"sketch": xb.engine_for(desc_, xb.OP_SKETCH), "backprobe": xb.engine_for(desc_, xb.OP_BACKPROBE),
-               "contract": xb.engine_for(desc_, xb.OP_CONTRACT)}
+               "contract": xb.engine_for(desc_, xb.OP_CONTRACT), "wgrad": xb.engine_for(desc_, xb.OP_WGRAD)}
         out = {}
         for n, ms in ph_ms.items():
             gbs = work[n]["bytes"] / (ms * 1e-3) / 1e9
             tfs = work[n]["flops"] / (ms * 1e-3) / 1e12
-            comp_peak = tensor_peak if eng[n] == "tcgen05_bf16" else FP32_ALU_TFLOPS
+            comp_peak = tensor_peak if eng[n] == "tcgen05_bf16" else fma_tflops
             t_mem, t_comp = work[n]["bytes"] / (peaks["hbm_gbs"] * 1e9), work[n]["flops"] / (comp_peak * 1e12)
             bound = "hbm" if t_mem >= t_comp else ("tensor" if eng[n] == "tcgen05_bf16" else "alu")
             out[n] = {"ms": ms, "engine": eng[n], "GBps": gbs, "TFLOPps": tfs, "bound": bound,
                       "peak": peaks["hbm_gbs"] if bound == "hbm" else comp_peak,
+                      "roofline_ms": 1e3 * max(t_mem, t_comp),
                       "frac": (gbs / peaks["hbm_gbs"]) if bound == "hbm" else tfs / comp_peak}
+            if n in ("backprobe", "contract"):
+                out[n]["note"] = "L charged to this launch (diagnostic); the estimator as a whole is `wgrad`"
         return out
 
     phases = phase_table(r, desc, phase_ms)
-    dom = max(phase_ms, key=phase_ms.get)
+    kernels = {n: phase_ms[n] for n in ("sketch", "backprobe", "contract")}
+    dom = max(kernels, key=kernels.get)
     d = phases[dom]
+    low = min(("sketch", "wgrad"), key=lambda n: phases[n]["frac"])
     roofline = {"kernel": dom + " (tc_gemm_kernel and its reduce/cast helper, timed together)", "bound": d["bound"],
                 "achieved": d["GBps"] if d["bound"] == "hbm" else d["TFLOPps"], "peak": d["peak"],
                 "unit": "GB/s" if d["bound"] == "hbm" else "TFLOP/s", "frac": d["frac"],
                 "traffic": ncu_traffic(cfg, r, dom),
-                "peak_source": f"of {peak_src}" + ("" if d["bound"] != "alu" else " (derived: 148 SMs x 128 FMA x 2 x 1.965 GHz)")}
+                "peak_source": f"of {peak_src}" + ("" if d["bound"] != "alu" else
+                                                   " (FP32 FMA rate measured by xconv_measure_fma_rate; derived "
+                                                   f"148 SMs x 128 FMA x 2 x 1.965 GHz = {FP32_ALU_TFLOPS_DERIVED:.1f})"),
+                "timing": f"{n_phase} launches of the phase back to back between two CUDA events",
+                "furthest_below": {"phase": low, "bound": phases[low]["bound"], "frac": phases[low]["frac"],
+                                   "note": "of the two units of the method (sketch; estimator = back-probe + "
+                                           "contraction with L not counted), the one furthest below its roofline"}}
 
     # ---- the other probe counts of this workload's sweep (shorter runs), same step and timing
     sweep = []
@@ -407,7 +486,7 @@ def run_xconv(args):
             lay2 = Layer(r2, Z2)
             n2 = max(5, min(args.steps, 30))
             tot2, _, _ = lay2.measure(n2, 3, None, phase_events=False)
-            _, ph2, _ = lay2.measure(n2, 3, None, phase_events=True)
+            ph2, _ = lay2.measure_phases(n2)
             sweep.append({"r": r2, "ms_per_step": tot2 / n2, "value": 1e3 * n2 / tot2, "phases": phase_table(r2, lay2.desc, ph2)})
             del lay2, Z2
             torch.cuda.empty_cache()
@@ -477,15 +556,31 @@ def run_xconv(args):
             "vs_baseline": None, "dtype": "f32" if c["dtype"] == "f32" else "bf16",
             "data": "synthetic", "config": workload_config(args, c, layer.copies), "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches[0], "roofline": roofline, "cpu_baseline": cpu, "phases": phases,
-            "phase_timing": {"ms_per_step_with_events": total_ev_ms / args.steps,
-                             "note": "phases and roofline come from a second timed region of the same K steps with a "
-                                     "CUDA event between the three calls; the events themselves add to that region"},
+            "phase_timing": {"launches_per_phase": n_phase, "tensor_sets_per_phase": phase_sets,
+                             "fp32_fma_tflops_measured": fma_tflops,
+                             "with_events_between_calls_ms": dict(phase_ev_ms, step=total_ev_ms / n_phase),
+                             "note": "phases and roofline: each call timed alone, K launches back to back between two "
+                                     "CUDA events; with_events_between_calls_ms: the step with an event between its "
+                                     "three calls, which keeps a kernel's preamble from overlapping the previous "
+                                     "kernel's tail (diagnostic)"},
             "sweep": sweep, "layer_api": full,
             "memory_ratio": {"elements": Cin * H * W / r, "stored_bytes": Cin * H * W * es / (4.0 * r)},
             "context": context}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` started without a launcher: run the same command line as N ranks of one node
+    under torch.distributed.run (rendezvous on 127.0.0.1) and hand back its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), "--", os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -502,6 +597,8 @@ def main():
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -36,14 +36,20 @@
  * OWNERSHIP AND EXECUTION.  All pointers are device pointers owned by the caller, 16-byte aligned,
  * unless a parameter is documented as a host pointer.  The library allocates no device memory and
  * keeps no state between calls; scratch memory is passed in as `ws` (size from
- * xconv_workspace_bytes).  Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
+ * xconv_workspace_bytes).  (One documented exception: xconv_sketch_static, whose scratch is a fixed
+ * array inside the library image and whose first call per device resolves that array's address.)
+ * Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*,
  * NULL = default stream) and the call returns without synchronising.  Outputs are overwritten, never
  * accumulated into.  The same Z must be given to the forward and to the backward call of a layer.
  * Results are bit-reproducible run to run (fixed reduction order, no atomics).
  *
- * ERRORS.  Every entry point returns an xconv_status.  A call that returns anything but XCONV_OK
- * has launched nothing.  Shapes or options without a kernel return XCONV_ERR_UNSUPPORTED; there is
- * no CPU or library fallback.  Pipelined kernels bound every device-side wait; a wait that runs
+ * ERRORS.  Every entry point returns an xconv_status.  Every check of the arguments is made before the
+ * first launch: a call that returns XCONV_ERR_INVALID_ARG, XCONV_ERR_UNSUPPORTED, XCONV_ERR_ALIGNMENT
+ * or XCONV_ERR_WORKSPACE has launched nothing and touched no buffer.  XCONV_ERR_CUDA reports a CUDA
+ * runtime or driver call that failed in the middle of a call (a launch, a tensor-map encoding, a copy);
+ * kernels the call enqueued before that point still run, and the outputs are then undefined.
+ * Shapes or options without a kernel return XCONV_ERR_UNSUPPORTED; there is no CPU or library
+ * fallback.  Pipelined kernels bound every device-side wait; a wait that runs
  * out records a code in the first word of the workspace, which xconv_workspace_status() reads back.
  */
 #ifndef XCONV_H_
@@ -177,8 +183,12 @@ xconv_status xconv_sketch_wgrad_host(const xconv_desc* desc, const void* hX, con
  *  - Limit: r*B <= XCONV_STATIC_SCRATCH_FLOATS.  A larger layer returns XCONV_ERR_WORKSPACE ("too
  *    small": the fixed array cannot hold even one [r,B] slab) and launches nothing.
  *  - The call performs no cudaMalloc, cudaFree or other allocating call.  The first call on a device
- *    resolves the device address of the array (cudaGetSymbolAddress, with that device current);
- *    make that first call outside any stream capture.
+ *    resolves the device address of the array (cudaGetSymbolAddress, with that device current).  With
+ *    CUDA's lazy module loading that first call is also the moment at which the driver loads the
+ *    library's device code, fixed array included, onto that device: it can take the 4 MiB then,
+ *    synchronise, or fail if no device memory is left.  So make one warm-up call per device at
+ *    start-up -- before the memory budget is handed out, outside any stream capture and outside the
+ *    latency-critical loop; later calls on that device only launch kernels.
  *  - All calls on a device share the one array.  Nothing in it has to start at zero -- every call
  *    overwrites the slabs it then sums -- so stale contents of an earlier call are harmless, but two
  *    calls that overlap on the GPU (different streams, no dependency) race on it.  Serialise them.
@@ -200,6 +210,13 @@ xconv_status xconv_workspace_status(const void* ws, void* cuda_stream);
  * XCONV_ERR_TIMEOUT.  Nothing faults or hangs; the context stays usable.  (No counterpart in the
  * paper.) */
 xconv_status xconv_selftest_wait_limit(void* ws, size_t ws_bytes, unsigned int limit_ms, void* cuda_stream);
+
+/* Measurement aid (no counterpart in the paper): the FP32 fused-multiply-add rate this GPU sustains,
+ * which is the arithmetic ceiling of the FP32-FMA kernels that serve float storage.  Runs a kernel of
+ * register-only FMA chains a few times on `cuda_stream`, times it with CUDA events, synchronises, and
+ * writes the best rate in TFLOP/s (2 flops per FMA) to the HOST double `tflops`.  `scratch` is device
+ * memory of at least 148*16*256*4 bytes that the kernel writes its (meaningless) sums to. */
+xconv_status xconv_measure_fma_rate(void* scratch, size_t scratch_bytes, double* tflops, void* cuda_stream);
 
 /* Number of kernels the last successful call on this host thread enqueued. */
 int xconv_last_launch_count(void);

@@ -36,6 +36,7 @@ literal block-matrix estimator of Eq. (6) (sketch, backprobe, wgrad_estimate).
 philox4x32_10 and rademacher_probes (probing vectors redrawn from a stored seed, Algorithm 1) are pinned
 by the generator's published known-answer vectors (tests/golden/philox4x32_10_kat.txt), by the
 balance and independence of the signs, and by the unbiasedness of the estimator run on them.
+rel_fro, the metric every parity verdict passes through, is pinned on a hand-computed pair.
 No function here is "parity unpinned".
 """
 from __future__ import annotations

@@ -24,7 +24,7 @@ STATUS_OK = 0
 # every symbol include/xconv.h declares
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
            "xconv_dgrad", "xconv_probes_from_seed", "xconv_sketch_seeded", "xconv_wgrad_seeded", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
-           "xconv_workspace_status", "xconv_selftest_wait_limit",
+           "xconv_workspace_status", "xconv_selftest_wait_limit", "xconv_measure_fma_rate",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_static.restype = c_int
     L.xconv_selftest_wait_limit.argtypes = [c_void_p, c_size_t, ctypes.c_uint, c_void_p]
     L.xconv_selftest_wait_limit.restype = c_int
+    L.xconv_measure_fma_rate.argtypes = [c_void_p, c_size_t, POINTER(ctypes.c_double), c_void_p]
+    L.xconv_measure_fma_rate.restype = c_int
     L.xconv_workspace_status.argtypes = [c_void_p, c_void_p]; L.xconv_workspace_status.restype = c_int
     L.xconv_last_launch_count.argtypes = []; L.xconv_last_launch_count.restype = c_int
     L.xconv_last_cuda_error.argtypes = []; L.xconv_last_cuda_error.restype = c_int
@@ -188,6 +190,15 @@ def dgrad_into(desc, dY, W, dX, ws):
 
 def workspace_status(ws) -> int:
     return lib().xconv_workspace_status(ws.data_ptr(), _stream())
+
+
+def measure_fma_rate(device="cuda") -> float:
+    """FP32 FMA rate of the device in TFLOP/s, measured by the library's register-only FMA kernel."""
+    scratch = torch.empty(148 * 16 * 256, dtype=torch.float32, device=device)
+    out = ctypes.c_double(0.0)
+    _check(lib().xconv_measure_fma_rate(scratch.data_ptr(), scratch.numel() * 4, ctypes.byref(out), _stream()),
+           "xconv_measure_fma_rate")
+    return float(out.value)
 
 
 def last_launch_count() -> int:

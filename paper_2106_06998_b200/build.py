@@ -30,7 +30,7 @@ def _stale() -> bool:
 
 def build(force: bool = False, verbose: bool = False, extra_flags=()) -> str:
     """Compile every CUDA source into one shared library; returns its path.
-    ``extra_flags`` go to nvcc (e.g. ``-DXC_TIMELINE`` for the per-CTA wait counters)."""
+    ``extra_flags`` go to nvcc."""
     if not force and not _stale():
         return LIB
     objs = []

@@ -44,9 +44,15 @@ static xconv_status validate(const xconv_desc* d) {
   if (d->circular != 0) return XCONV_ERR_UNSUPPORTED;
   if (d->KH != d->KW || (d->KH != 1 && d->KH != 3)) return XCONV_ERR_UNSUPPORTED;
   if (2 * d->pad_h != d->KH - 1 || 2 * d->pad_w != d->KW - 1) return XCONV_ERR_UNSUPPORTED;
-  // 32-bit grid and index limits of the kernels
+  // 32-bit grid and index limits of the kernels.  r, B and the channel counts land on the y axis of a
+  // grid (at most 65535 blocks of 16 or more) in the FP32-FMA kernels, and r and B trade places when
+  // xconv_wgrad sums over the probes first.
   const long Kdim = (long)d->H * d->W * d->Cin, Q = (long)d->H * d->W * d->Cout;
   if (Kdim > (1L << 40) || Q > (1L << 40) || (long)d->B * d->H * cdiv(d->W, 32) > 2000000000L)
+    return XCONV_ERR_UNSUPPORTED;
+  const long axis_limit = 65535L * 16;
+  if (d->r > axis_limit || d->B > axis_limit || d->Cin > axis_limit || d->Cout > axis_limit ||
+      (long)d->r * d->B > (1L << 40))
     return XCONV_ERR_UNSUPPORTED;
   return XCONV_OK;
 }
@@ -345,6 +351,7 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
   const SwappedWgrad sw = plan_wgrad_swapped(d);
   if (sw.on) {
     // Xr = S^T Z, then the offset contraction over the batch (see plan_wgrad_swapped)
+    if ((s = validate(&sw.d1)) != XCONV_OK || (s = validate(&sw.d2)) != XCONV_OK) return s;
     float* St = reinterpret_cast<float*>(w + sw.st_off);
     const long n = (long)d->r * d->B;
     transpose_f32<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, St, d->r, d->B);
@@ -357,6 +364,23 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
   s = run_backprobe(d, p, S, dY, w + p.l_off, w + p.sb_off, w, st);
   if (s != XCONV_OK) return s;
   return run_contract(d, p, w + p.l_off, Z, dW, alpha, w + p.part_off, w, st);
+}
+
+// FP32 FMA throughput probe: every thread runs 16 independent chains of dependent FMAs on registers (no
+// memory traffic), 4 blocks of 256 threads per SM's worth of grid; the result is stored so that the
+// compiler keeps the arithmetic.
+__global__ void __launch_bounds__(256) fma_rate_kernel(float* __restrict__ sink, int iters, float a, float b) {
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = (float)(threadIdx.x + i);
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = fmaf(v[i], a, b);
+  }
+  float t = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) t += v[i];
+  sink[(long)blockIdx.x * blockDim.x + threadIdx.x] = t;
 }
 
 int launches() { return g_launches; }
@@ -602,6 +626,34 @@ xconv_status xconv_workspace_status(const void* ws, void* cuda_stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
   return (word[0] != WS_OK && word[0] == word[1]) ? XCONV_ERR_TIMEOUT : XCONV_OK;
+}
+
+xconv_status xconv_measure_fma_rate(void* scratch, size_t scratch_bytes, double* tflops, void* cuda_stream) {
+  const int blocks = 148 * 16, threads = 256, iters = 4096;
+  if (!scratch || !tflops) return XCONV_ERR_INVALID_ARG;
+  if (scratch_bytes < (size_t)blocks * threads * sizeof(float)) return XCONV_ERR_WORKSPACE;
+  if (!aligned16(scratch)) return XCONV_ERR_ALIGNMENT;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  cudaError_t e = cudaEventCreate(&e0);
+  if (e == cudaSuccess) e = cudaEventCreate(&e1);
+  float best_ms = 0.f;
+  new_call();
+  for (int rep = 0; rep < 6 && e == cudaSuccess; ++rep) {      // the first repetition warms up
+    cudaEventRecord(e0, st);
+    fma_rate_kernel<<<blocks, threads, 0, st>>>(static_cast<float*>(scratch), iters, 0.999f, 0.001f);
+    ++g_launches;
+    cudaEventRecord(e1, st);
+    e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && (best_ms == 0.f || ms < best_ms)) best_ms = ms;
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (e != cudaSuccess || best_ms <= 0.f) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  *tflops = 2.0 * 16.0 * iters * (double)blocks * threads / (best_ms * 1e-3) / 1e12;
+  return XCONV_OK;
 }
 
 int xconv_last_launch_count(void) { return g_launches; }

@@ -328,23 +328,6 @@ __device__ __forceinline__ void z_store128(uint32_t rbase, uint32_t tile_bytes, 
   z_store64(rbase + tile_bytes, row, make_uint2(w.z, w.w));
 }
 
-// Optional per-CTA cycle counters (build with -DXC_TIMELINE): time the producer and the MMA-issue thread
-// spend waiting on barriers and issuing work, read back through xconv_debug_waits.
-#ifdef XC_TIMELINE
-__device__ long long g_waits[1024 * 8];
-__device__ long long g_times[4 * 1024 * 8];  // globaltimer (ns) at fixed points of the kernel, per mode and CTA
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TT(slot) do { if (blockIdx.x < 1024) g_times[((p.mode & 3) * 1024 + blockIdx.x) * 8 + (slot)] = gtime(); } while (0)
-#define TW_BEGIN long long _tw0 = clock64()
-#define TW_END(acc) acc += clock64() - _tw0
-#define TW_STORE(slot, acc) do { if (blockIdx.x < 1024) g_waits[blockIdx.x * 8 + (slot)] = (acc); } while (0)
-#else
-#define TW_BEGIN do {} while (0)
-#define TW_END(acc) do {} while (0)
-#define TW_STORE(slot, acc) do {} while (0)
-#define TT(slot) do {} while (0)
-#endif
-
 // The MMAs of `nkb` k-blocks that arrive in two halves (see TcParams::halves), with the numbers of k-steps known at
 // compile time so that the issuing thread runs straight-line code: it executes about one instruction per six
 // clocks, and every instruction between two tcgen05.mma counts.  Returns false if a wait ran out.
@@ -445,11 +428,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ uint32_t tmem_slot;
   __shared__ int go;
 
-#ifdef XC_TIMELINE
-  const long long t_kernel0 = clock64();
-  if (threadIdx.x == 64 && blockIdx.x < 1024) g_waits[blockIdx.x * 8 + 5] = 0;
-#endif
-  if (threadIdx.x == 0) TT(0);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
   const uint32_t stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
@@ -469,7 +447,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
   pdl_trigger();
   pdl_wait();                              // from here on the previous kernel's results are visible
-  if (threadIdx.x == 0) TT(1);
   if (threadIdx.x == 0) {
     // a CTA of this call gave up earlier: skip the work (one thread reads so that the whole CTA agrees)
     go = (*reinterpret_cast<volatile unsigned int*>(p.status) != p.tag) ? 1 : 0;
@@ -492,7 +469,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     int s = 0;
     long fill = 0, it = 0;
     bool ok = true;
-    long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
     for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
       const Unit w = decode_unit(p, u);
       const int row0 = w.tm * p.m_sub * TILE_M;
@@ -505,13 +481,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int dy = tap / ks - p.pad, dx = tap % ks - p.pad;
       for (int i = 0; i < w.nkb; ++i) {
         if (fill > 0) {
-          TW_BEGIN;
           if (lane == 0) ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-          TW_END(tw_pw);
           if (!ok) break;
         }
-        TW_BEGIN;
         const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
         const uint32_t b_dst = a_dst + p.a_stage_bytes;
         const int x0 = px * p.patch_w, y0 = py * p.patch_h;
@@ -526,10 +499,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
         ++it;
         if (++s == stages) { s = 0; ++fill; }
-        TW_END(tw_pi);
       }
     }
-    if (lane == 0) { TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it); }
     // drain: every copy issued must have landed in this CTA's shared memory before it exits
     if (lane == 0)
       for (long i = max(0L, it - stages); i < it; ++i)
@@ -541,7 +512,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int s = 0;
       long fill = 0, it = 0;
       bool ok = true;
-      long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
       const int hrows = p.patch_h >> 1;    // image rows per half
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
@@ -553,12 +523,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int ks = 2 * p.pad + 1, dy = w.tap / ks - p.pad, dx = w.tap % ks - p.pad;
         for (int i = 0; i < 2 * w.nkb; ++i) {
           if (fill > 0) {
-            TW_BEGIN;
             ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
-            TW_END(tw_pw);
             if (!ok) break;
           }
-          TW_BEGIN;
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes, b_dst = a_dst + p.a_half_bytes;
           const int x0 = px * p.patch_w, y0 = py * p.patch_h + (i & 1) * hrows;
           mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
@@ -567,10 +534,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if ((i & 1) && ++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
           ++it;
           if (++s == slots) { s = 0; ++fill; }
-          TW_END(tw_pi);
         }
       }
-      TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it);
       for (long i = max(0L, it - slots); i < it; ++i)
         if (!mbar_wait(&full_bar[i % slots], (uint32_t)((i / slots) & 1), p.status, p.tag)) break;
     }
@@ -590,14 +555,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int s = 0;                           // half-slot of the next first half (always even)
       uint32_t parity = 0;
       bool ok = true;
-      long long tw_mw = 0, tw_mi = 0; (void)tw_mw; (void)tw_mi;
-      const long long t_start = clock64(); (void)t_start;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
         if (w.nkb == 0) continue;
         const uint32_t d = tmem_base;      // one unit per CTA and accumulator set (acc_bufs = 1)
         uint32_t acc = 0;
-#ifndef XC_TIMELINE
         if (p.ks_h0 == 3 && p.ks_x == 1 && p.ks_h1 == 3) {      // halves of 56 pixels (28-wide images): unrolled
           ok = two ? umma_halves_items<3, 1, 3, true>(w.nkb, s, parity, acc, p.stages, full_bar, empty_bar, base16, slot16,
                                                        a_lo0, b_lo0, a_half16, a_sub, step, p.sbo >> 4, hi, hi_x, idesc, d,
@@ -608,15 +570,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (ok) umma_commit(&tmem_full_bar[0]);
           continue;
         }
-#endif
         for (int i = 0; i < w.nkb; ++i) {
           const uint32_t h0 = base16 + (uint32_t)s * slot16, h1 = h0 + slot16;
-          { TW_BEGIN; ok = mbar_wait(&full_bar[s], parity, p.status, p.tag); TW_END(tw_mw); }
+          ok = mbar_wait(&full_bar[s], parity, p.status, p.tag);
           if (!ok) break;
-#ifdef XC_TIMELINE
-          if (i == 0) TT(2);
-#endif
-          TW_BEGIN;
           tc_fence_after();
           uint32_t a = a_lo0 | h0, b = b_lo0 | (h0 + a_half16);
           for (int k = 0; k < p.ks_h0; ++k) {
@@ -624,10 +581,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (two) umma_bf16(d + tile_n, a + a_sub, hi, b, hi, idesc, acc);
             acc = 1u; a += step; b += step;
           }
-          TW_END(tw_mi);
-          { TW_BEGIN; ok = mbar_wait(&full_bar[s + 1], parity, p.status, p.tag); TW_END(tw_mw); }
+          ok = mbar_wait(&full_bar[s + 1], parity, p.status, p.tag);
           if (!ok) break;
-          { TW_BEGIN;
           tc_fence_after();
           if (p.ks_x) {                     // rows [16 ks_h0, +8) of the first half and [0, 8) of the second
             umma_bf16(d, a, hi_x, b, hi_x, idesc, acc);
@@ -645,11 +600,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           umma_commit(&empty_bar[s + 1]);
           s += 2;
           if (s == p.stages) { s = 0; parity ^= 1u; }
-          TW_END(tw_mi); }
         }
         if (ok) umma_commit(&tmem_full_bar[0]);
-        TT(3);
-        TW_STORE(2, tw_mw); TW_STORE(3, tw_mi); TW_STORE(4, clock64() - t_start);
       }
     }
   } else if (warp == 0) {
@@ -661,7 +613,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       long fill = 0;                       // how often the ring has wrapped
       long it = 0;                         // stages filled so far, across units
       bool ok = true;
-      long long tw_pw = 0, tw_pi = 0; (void)tw_pw; (void)tw_pi;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
         const int row0 = w.tm * p.m_sub * TILE_M;
@@ -682,12 +633,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int i = 0; i < w.nkb; ++i) {
           if (fill > 0) {
-            TW_BEGIN;
             ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
-            TW_END(tw_pw);
             if (!ok) break;
           }
-          TW_BEGIN;
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
           const uint32_t b_dst = a_dst + p.a_stage_bytes;
           mbar_arrive_expect_tx(&full_bar[s], p.mode == MODE_BACKPROBE
@@ -726,10 +674,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
           ++it;
           if (++s == stages) { s = 0; ++fill; }
-          TW_END(tw_pi);
         }
       }
-      TW_STORE(0, tw_pw); TW_STORE(1, tw_pi); TW_STORE(6, (long long)it);
       // drain: every copy issued must have landed in this CTA's shared memory before it exits
       // (immediate on the normal path, bounded on the failure path)
       for (long i = max(0L, it - stages); i < it; ++i)
@@ -763,8 +709,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t full_a = full_a0, empty_a = empty_a0;
       long lu = 0;
       bool ok = true;
-      long long tw_mw = 0, tw_mi = 0; (void)tw_mw; (void)tw_mi;
-      const long long t_start = clock64(); (void)t_start;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
         const Unit w = decode_unit(p, u);
         if (w.nkb == 0) continue;
@@ -781,14 +725,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t idesc_u = p.mode == MODE_BACKPROBE
                                      ? (idesc & ~(0x3Fu << 17)) | ((uint32_t)(w.nblk * 8) << 17) : idesc;
         for (int i = 0; i < w.nkb; ++i) {
-          { TW_BEGIN;
           if (!mbar_try_wait_a(full_a, full_parity)) ok = mbar_wait_slow(&full_bar[s], full_parity, p.status, p.tag);
-          TW_END(tw_mw); }
           if (!ok) break;
-#ifdef XC_TIMELINE
-          if (lu == 0 && i == 0) TT(2);
-#endif
-          TW_BEGIN;
           tc_fence_after();
           uint32_t a_lo = a_lo0 | s16;
           uint32_t b_lo = b_lo0 | (s16 + a_stage16);
@@ -854,11 +792,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           umma_commit_a(empty_a);            // stage s may be refilled once these MMAs have read it
           s16 += stage16; full_a += 8; empty_a += 8;
           if (++s == stages) { s = 0; s16 = base16; full_a = full_a0; empty_a = empty_a0; full_parity ^= 1u; }
-          TW_END(tw_mi);
         }
         if (ok) umma_commit(&tmem_full_bar[buf]);
-        TT(3);
-        TW_STORE(2, tw_mw); TW_STORE(3, tw_mi); TW_STORE(4, clock64() - t_start);
       }
     }
   } else {
@@ -928,10 +863,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!ok) break;
         tc_fence_after();
       }
-#ifdef XC_TIMELINE
-      const long long t_epi0 = clock64();
-      if (warp == 2 && lane == 0) TT(4);
-#endif
       const long col0 = (long)w.tn * p.tile_n;
       if (p.mode == MODE_BACKPROBE) {
         // D[j, q] -> L[j][q].  Each warp stages 32 rows x 64 positions at a time in the layout the tensor store
@@ -1041,13 +972,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&tmem_empty_bar[buf]);
-#ifdef XC_TIMELINE
-      if (warp == 2 && lane == 0 && blockIdx.x < 1024) {
-        g_waits[blockIdx.x * 8 + 5] += clock64() - t_epi0;
-        g_waits[blockIdx.x * 8 + 7] = clock64() - t_kernel0;
-        TT(5);
-      }
-#endif
     }
     // the tensor stores read this CTA's shared memory: they must be done before it exits
     if (p.mode == MODE_BACKPROBE && lane == 0) bulk_wait_all();
@@ -1059,7 +983,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
-  if (threadIdx.x == 0) TT(6);
 }
 
 // S[j][b] = sum over splits of the partial tiles, which are stored in accumulator order (see the
@@ -1746,11 +1669,3 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
 
 }  // namespace xconv
 
-#ifdef XC_TIMELINE
-extern "C" int xconv_debug_waits(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, xconv::g_waits, sizeof(long long) * 1024 * 8);
-}
-extern "C" int xconv_debug_times(long long* out) {
-  return (int)cudaMemcpyFromSymbol(out, xconv::g_times, sizeof(long long) * 4 * 1024 * 8);
-}
-#endif

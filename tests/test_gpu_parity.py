@@ -12,7 +12,7 @@ import __graft_entry__ as entry
 from oracle import xconv_oracle as O
 from paper_2106_06998_b200 import binding as xb
 from paper_2106_06998_b200 import inputs
-from tests._util import TOL, check, dev, host, sketch_oracle_chunked
+from tests._util import TOL, TOL_SKETCH, check, dev, host, sketch_oracle_chunked
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +33,7 @@ def _full_layer_parity(lay, K=3):
     torch.cuda.synchronize()
     assert torch.equal(S, S2)
     Yo, So, dWo, dXo = O.xconv_layer(lay["X"], lay["W"], lay["dY"], lay["Z"])
-    errs = dict(Y=check("Y", host(Y), Yo, tol), S=check("sketch", host(S), So, tol),
+    errs = dict(Y=check("Y", host(Y), Yo, tol), S=check("sketch", host(S), So, TOL_SKETCH),
                 dX=check("dX", host(dX), dXo, tol))
     # the estimator alone, from the oracle's own sketch (float), so that its error is not inherited
     So32 = torch.from_numpy(So.astype(np.float32)).cuda()
@@ -112,7 +112,7 @@ def test_sketch_tensor_path_k_blocking(shape):
     d = dev(lay)
     S = xb.xconv_sketch(d["X"], d["Z"])
     torch.cuda.synchronize()
-    check("sketch", host(S), O.sketch(lay["X"], lay["Z"]), TOL["bf16"])
+    check("sketch", host(S), O.sketch(lay["X"], lay["Z"]), TOL_SKETCH)
 
 
 @pytest.mark.parametrize("shape", [
@@ -179,7 +179,7 @@ def test_config_recipes_reduced_all_elements(cfg, r, shrink):
 
 # ------------------------------------------------------------------ full sizes, sampled outputs
 
-FULL = [(2, 16), (2, 64), (3, 32), (3, 128), (4, 64), (5, 16), (5, 64), (5, 256), (5, 1024)]
+FULL = [(2, 16), (2, 64), (3, 32), (3, 128), (4, 64), (4, 256), (5, 16), (5, 64), (5, 256), (5, 1024)]
 
 
 @pytest.mark.parametrize("cfg,r", FULL)
@@ -196,17 +196,25 @@ def test_full_size_sampled(cfg, r):
     torch.cuda.synchronize()
     assert xb.workspace_status(xb.workspace(256, S.device)) == 0
     So = sketch_oracle_chunked(lay["X"], lay["Z"])
-    check("sketch", host(S), So, tol)
+    check("sketch", host(S), So, TOL_SKETCH)
     g = np.random.Generator(np.random.PCG64(cfg * 1000 + r))
-    ms = np.sort(g.choice(lay["Cout"], size=min(4, lay["Cout"]), replace=False))
-    ns = np.sort(g.choice(lay["Cin"], size=min(6, lay["Cin"]), replace=False))
+    # output / input channels at the ends of the channel range, either side of the 128-row tile boundary, and at random
+    ms = np.unique(np.concatenate([[0, lay["Cout"] - 1, min(127, lay["Cout"] - 1), min(128, lay["Cout"] - 1)],
+                                   g.choice(lay["Cout"], size=min(2, lay["Cout"]), replace=False)]))
+    ns = np.unique(np.concatenate([[0, lay["Cin"] - 1], g.choice(lay["Cin"], size=min(4, lay["Cin"]), replace=False)]))
     dWo = O.wgrad_estimate(So, lay["dY"][:, ms], lay["Z"][:, ns])
     check("dW block", host(dW)[np.ix_(ms, ns)], dWo, tol)
-    # the two halves as the benchmark calls them (Algorithm 1's order, which xconv_wgrad leaves when r > B)
-    L = xb.xconv_backprobe(S, d["dY"])
+    # the two halves as the benchmark calls them (Algorithm 1's order, which xconv_wgrad leaves when r > B),
+    # fed the oracle's own sketch rounded to float
+    So32 = So.astype(np.float32)
+    L = xb.xconv_backprobe(torch.from_numpy(So32).cuda(), d["dY"])
     dW2 = xb.xconv_contract(L, d["Z"])
     torch.cuda.synchronize()
     check("dW block (back-probe + contraction)", host(dW2)[np.ix_(ms, ns)], dWo, tol)
+    # L itself (Algorithm 1 backward step 3) on a few probes x output channels, all pixels
+    js = np.sort(g.choice(r, size=min(5, r), replace=False))
+    Lo = O.backprobe(So32[js], lay["dY"][:, ms])
+    check("L rows", host(L[torch.from_numpy(js).cuda()][:, torch.from_numpy(ms).cuda()]), Lo, tol)
     del L, dW2
     bs = np.sort(g.choice(lay["B"], size=min(2, lay["B"]), replace=False))
     check("Y samples", host(Y[bs]), O.conv_forward(lay["X"][bs], lay["W"]), tol)
@@ -241,6 +249,42 @@ def test_block_sparse_probes_with_channel_scale(dtype):
     want = O.wgrad_estimate(O.sketch(lay["X"], lay["Z"]), lay["dY"], lay["Z"], scale=sc)
     check("dW nnz-scaled", host(dW), want, TOL[dtype])
     assert float(dW[:, 3].abs().max()) == 0.0
+
+
+@pytest.mark.parametrize("shape", [
+    # B, Cin, Cout, H, W, r
+    (16, 64, 128, 12, 20, 24),        # r > B is false: back-probe, contraction and its reduce kernel on tcgen05
+    (8, 32, 32, 40, 24, 72),          # r > B: xconv_wgrad sums over the probes first; 64-byte-swizzle tiles
+    (32, 256, 256, 8, 28, 16),        # wide layer: contraction in half-stages
+])
+def test_block_sparse_probes_with_channel_scale_on_the_tensor_path(shape):
+    """Eq. (7) probes (whole channel blocks of a probing vector zero with probability 1 - p_n) and the
+    1/nnz(Z_n) scale of Eq. (8) on layers the tcgen05 kernels serve, in both orders of summation."""
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="bf16", seed=sum(shape) + 1, z="rademacher", x="relu")
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, torch.bfloat16)
+    assert xb.engine_for(desc, xb.OP_CONTRACT) == "tcgen05_bf16" and xb.engine_for(desc, xb.OP_BACKPROBE) == "tcgen05_bf16"
+    g = np.random.Generator(np.random.PCG64(sum(shape)))
+    mask = (g.random((r, Cin, 1, 1)) < 0.5).astype(np.float32)
+    mask[:, 5] = 0                                     # one channel never probed: estimate must be exactly 0
+    mask[0, 6] = 1                                     # and its neighbours probed at least once
+    lay["Z"] = lay["Z"] * mask
+    sc = O.channel_scale(lay["Z"])
+    assert sc[5] == 0.0 and sc[6] > 0.0
+    d = dev(lay)
+    cs = torch.from_numpy(sc.astype(np.float32)).cuda()
+    S = xb.xconv_sketch(d["X"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"], chan_scale=cs)
+    So = O.sketch(lay["X"], lay["Z"])
+    want = O.wgrad_estimate(So, lay["dY"], lay["Z"], scale=sc)
+    check("sketch (block-sparse probes)", host(S), So, TOL_SKETCH)
+    check("dW nnz-scaled", host(dW), want, TOL["bf16"])
+    assert float(dW[:, 5].abs().max()) == 0.0
+    # the paper's order of summation as well (back-probe, then the contraction with the scale)
+    L = xb.xconv_backprobe(S, d["dY"])
+    dW2 = xb.xconv_contract(L, d["Z"], chan_scale=cs)
+    check("dW nnz-scaled (back-probe + contraction)", host(dW2), want, TOL["bf16"])
+    assert float(dW2[:, 5].abs().max()) == 0.0
 
 
 def test_orthogonal_probe_basis_recovers_exact_gradient_on_gpu():
@@ -294,7 +338,7 @@ def test_bounded_wait_reports_timeout_and_next_call_recovers():
     S = torch.empty((16, 128), dtype=torch.float32, device="cuda")
     xb.sketch_into(desc, d["X"], d["Z"], S, ws)
     assert xb.workspace_status(ws) == 0
-    check("sketch after a timed-out call", host(S), O.sketch(lay["X"], lay["Z"]), 1e-2)
+    check("sketch after a timed-out call", host(S), O.sketch(lay["X"], lay["Z"]), TOL_SKETCH)
 
 
 def test_engines_reported():

@@ -426,3 +426,16 @@ def test_estimator_on_redrawn_probes_is_unbiased():
     err = np.abs(acc / T - exact).max()
     single = np.std([O.wgrad_estimate(O.sketch(X, Z), dY, Z) for Z in (O.rademacher_probes(s, r, Cin, H, W) for s in range(50))], axis=0).max()
     assert err < 5.0 * single / np.sqrt(T)
+
+
+def test_rel_fro_on_a_hand_computed_pair():
+    """The parity metric itself: ||a - b||_F / ||b||_F on values worked out by hand.
+    a - b = (3, 4, 0, 0) has norm 5; b = (1, 2, 2, 4) has norm 5; a shifted copy gives a different value, so
+    the arguments are not interchangeable and the denominator is the second one."""
+    a = np.array([[4.0, 6.0], [2.0, 4.0]])
+    b = np.array([[1.0, 2.0], [2.0, 4.0]])
+    assert O.rel_fro(a, b) == pytest.approx(1.0, abs=1e-15)
+    assert O.rel_fro(b, a) == pytest.approx(5.0 / np.sqrt(72.0), abs=1e-15)
+    assert O.rel_fro(b, b) == 0.0
+    assert O.rel_fro(2 * b, b) == pytest.approx(1.0, abs=1e-15)          # scale of the error, not of the data
+    assert O.rel_fro(np.array([3.0, 4.0]), np.zeros(2)) == pytest.approx(5.0)   # zero reference: absolute norm

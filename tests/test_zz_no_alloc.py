@@ -12,9 +12,10 @@ import pytest
 import torch
 
 import __graft_entry__ as entry
+from oracle import xconv_oracle as O
 from paper_2106_06998_b200 import binding as xb
 from paper_2106_06998_b200 import inputs
-from tests._util import TOL
+from tests._util import TOL_SKETCH, check, host
 
 pytestmark = pytest.mark.gpu
 
@@ -46,8 +47,30 @@ def test_static_scratch_sketch_matches_workspace_sketch_twice_in_a_row(dtype):
                                                   torch.cuda.current_stream().cuda_stream)
                 assert st == 0, xb.lib().xconv_status_string(st)
                 torch.cuda.synchronize()
-                assert _rel(got, want) <= TOL[dtype], (dtype, rep, call, _rel(got, want))
+                assert _rel(got, want) <= TOL_SKETCH, (dtype, rep, call, _rel(got, want))
             assert torch.equal(xb.xconv_sketch_static(X, Z), got)     # binding wrapper, and reproducible
+            # and against the definition itself (Algorithm 1 forward step 3), not only the other entry point
+            check("static-scratch sketch", host(got), O.sketch(lay["X"], lay["Z"]), TOL_SKETCH)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [
+    # B, Cin, H, W, r
+    (512, 8, 16, 16, 1024),      # r*B = 2^19: the fixed array holds two slabs, so four k-splits shrink to two
+    (1024, 8, 16, 16, 1024),     # r*B = 2^20 exactly: one slab fills the array, a single split
+])
+def test_static_scratch_at_and_near_its_limit(shape, dtype):
+    """The fixed array bounds the number of k-splits; at r*B equal to its size one slab fills it to the last float."""
+    B, Cin, H, W, r = shape
+    assert r * B <= xb.STATIC_SCRATCH_FLOATS
+    lay = inputs.make_custom(B, Cin, 8, H, W, r, dtype=dtype, seed=sum(shape), z="rademacher")
+    X, Z = xb.to_device(lay["X"], dtype), xb.to_device(lay["Z"], dtype)
+    want = xb.xconv_sketch(X, Z)
+    for call in range(2):
+        got = xb.xconv_sketch_static(X, Z)
+        torch.cuda.synchronize()
+        assert _rel(got, want) <= TOL_SKETCH, (dtype, call, _rel(got, want))
+    check("static-scratch sketch", host(got), O.sketch(lay["X"], lay["Z"]), TOL_SKETCH)
 
 
 def test_static_scratch_rejects_layers_beyond_its_fixed_size():
