@@ -29,9 +29,11 @@
  *   W, dW        : element (m,n,ky,kx) at ((m*KH + ky)*KW + kx)*Cin + n
  *   S            : element (j,b) at j*B + b, always float
  * (This is torch's channels_last memory format of the logical NCHW / OIHW tensors.)
- * X, W, dY, Z, Y, dX are stored in desc.dtype (float or bfloat16); S and dW are always float.
- * With bfloat16 storage all sums are accumulated in float; L is kept in bfloat16 and S is rounded to
- * bfloat16 where it feeds the tensor cores.
+ * X, W, dY, Z, Y, dX are stored in desc.dtype (float, bfloat16, or float16 -- the "half precision" of
+ * the paper's Section 5.2); S and dW are always float.
+ * With 16-bit storage all sums are accumulated in float; L is kept in the storage type and S is rounded to
+ * it where it feeds the tensor cores.  (float16 storage: values beyond 65504 in magnitude overflow, as in
+ * any half-precision pipeline; the library does not rescale.)
  *
  * OWNERSHIP AND EXECUTION.  All pointers are device pointers owned by the caller, 16-byte aligned,
  * unless a parameter is documented as a host pointer.  The library allocates no device memory and
@@ -62,7 +64,7 @@
 extern "C" {
 #endif
 
-typedef enum { XCONV_F32 = 0, XCONV_BF16 = 1 } xconv_dtype;
+typedef enum { XCONV_F32 = 0, XCONV_BF16 = 1, XCONV_F16 = 2 } xconv_dtype;
 
 typedef enum {
   XCONV_OK = 0,
@@ -79,10 +81,11 @@ typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCO
                XCONV_OP_WGRAD_SEEDED = 7 } xconv_op;
 
 /* Which arithmetic engine a call will use for its dominant kernel. */
-typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2 } xconv_engine;
+typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2,
+               XCONV_ENGINE_TCGEN05_F16 = 3 } xconv_engine;
 
 /* One convolutional layer: stride 1, dilation 1, one group, no bias, "same" output size
- * (2*pad_h = KH-1, 2*pad_w = KW-1; KH = KW in {1, 3}). */
+ * (2*pad_h = KH-1, 2*pad_w = KW-1; KH = KW in {1, 3, 5}). */
 typedef struct {
   int32_t B, Cin, Cout, H, W;
   int32_t KH, KW, pad_h, pad_w;

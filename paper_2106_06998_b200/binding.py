@@ -2,7 +2,7 @@
 
 Tensors are torch CUDA tensors of logical shape (batch, channel, H, W) / (Cout, Cin, KH, KW) /
 (r, Cin, H, W) held in ``torch.channels_last`` memory format (the library's layout), in float32 or
-bfloat16.  torch is used for device memory and streams only.  There is no fallback: if the shared
+bfloat16 or float16.  torch is used for device memory and streams only.  There is no fallback: if the shared
 library is missing or a layer has no kernel, a RuntimeError is raised.
 """
 from __future__ import annotations
@@ -16,9 +16,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxconv.so")
 
-XCONV_F32, XCONV_BF16 = 0, 1
+XCONV_F32, XCONV_BF16, XCONV_F16 = 0, 1, 2
 OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT, OP_SKETCH_SEEDED, OP_WGRAD_SEEDED = 0, 1, 2, 3, 4, 5, 6, 7
-ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16"}
+ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16", 3: "tcgen05_f16"}
 STATUS_OK = 0
 
 # every symbol include/xconv.h declares
@@ -99,7 +99,9 @@ def _dtype_code(t: torch.dtype) -> int:
         return XCONV_F32
     if t == torch.bfloat16:
         return XCONV_BF16
-    raise TypeError(f"libxconv stores float32 or bfloat16, got {t}")
+    if t == torch.float16:
+        return XCONV_F16
+    raise TypeError(f"libxconv stores float32, bfloat16 or float16, got {t}")
 
 
 def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None) -> XConvDesc:
@@ -373,4 +375,6 @@ def to_device(a, dtype: str, device="cuda") -> torch.Tensor:
     t = torch.from_numpy(a).to(device)
     if dtype == "bf16":
         t = t.to(torch.bfloat16)
+    elif dtype == "f16":
+        t = t.to(torch.float16)
     return t.contiguous(memory_format=torch.channels_last)

@@ -39,10 +39,10 @@ static xconv_status validate(const xconv_desc* d) {
   if (!d) return XCONV_ERR_INVALID_ARG;
   if (d->B <= 0 || d->Cin <= 0 || d->Cout <= 0 || d->H <= 0 || d->W <= 0 || d->r <= 0 || d->KH <= 0 || d->KW <= 0)
     return XCONV_ERR_INVALID_ARG;
-  if (d->dtype != XCONV_F32 && d->dtype != XCONV_BF16) return XCONV_ERR_INVALID_ARG;
+  if (d->dtype != XCONV_F32 && d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return XCONV_ERR_INVALID_ARG;
   if (d->pad_h < 0 || d->pad_w < 0) return XCONV_ERR_INVALID_ARG;
   if (d->circular != 0) return XCONV_ERR_UNSUPPORTED;
-  if (d->KH != d->KW || (d->KH != 1 && d->KH != 3)) return XCONV_ERR_UNSUPPORTED;
+  if (d->KH != d->KW || (d->KH != 1 && d->KH != 3 && d->KH != 5)) return XCONV_ERR_UNSUPPORTED;
   if (2 * d->pad_h != d->KH - 1 || 2 * d->pad_w != d->KW - 1) return XCONV_ERR_UNSUPPORTED;
   // 32-bit grid and index limits of the kernels.  r, B and the channel counts land on the y axis of a
   // grid (at most 65535 blocks of 16 or more) in the FP32-FMA kernels, and r and B trade places when
@@ -113,7 +113,7 @@ static WgradPlan plan_wgrad_core(const xconv_desc* d) {
     return p;
   }
   const long items = (long)d->r * d->H * cdiv(d->W, 32);
-  const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32);
+  const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32) * (d->KH == 5 ? 5 : 1);   // 5 x 5: one offset row per block
   // one wave of the grid: two blocks of this kernel fit an SM (its 72 accumulators per thread)
   long splits = std::max(1L, std::min(std::max(1L, 2L * 148 / tiles), cdiv(items, 2)));
   splits = std::min(splits, 4096L);
@@ -198,6 +198,8 @@ static xconv_status run_probes_from_seed(const xconv_desc* d, unsigned long long
   const uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFull), k1 = (uint32_t)(seed >> 32);
   cudaError_t e = d->dtype == XCONV_F32
       ? launch_pdl(probes_from_seed_kernel<float>, dim3(grid), dim3(256), 0, st, static_cast<float*>(Z), total, k0, k1)
+      : d->dtype == XCONV_F16
+      ? launch_pdl(probes_from_seed_kernel<f16>, dim3(grid), dim3(256), 0, st, static_cast<f16*>(Z), total, k0, k1)
       : launch_pdl(probes_from_seed_kernel<bf16>, dim3(grid), dim3(256), 0, st, static_cast<bf16*>(Z), total, k0, k1);
   ++g_launches;
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
@@ -244,7 +246,8 @@ static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z
   }
   if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st, redraw ? seed : nullptr);
   return d->dtype == XCONV_F32 ? run_sketch_simt<float>(d, p, X, Z, S, w, st)
-                               : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
+         : d->dtype == XCONV_F16 ? run_sketch_simt<f16>(d, p, X, Z, S, w, st)
+                                 : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
 }
 
 template <typename T, typename TL>
@@ -262,16 +265,18 @@ static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, c
                                       float* dW, float alpha, float* part, cudaStream_t st) {
   const int T9 = d->KH * d->KW;
   const TL* L = static_cast<const TL*>(Lv);
-  dim3 g2((unsigned)cdiv(d->Cin, 64), (unsigned)cdiv(d->Cout, 32), (unsigned)p.splits);
   const T* Zt = static_cast<const T*>(Z);
   const bool vec = d->Cin % 4 == 0 && d->Cout % 4 == 0;      // rows of L and Z then start on 4-element boundaries
-  if (d->KH == 3) {
-    if (vec) contract_simt<TL, T, 3, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
-    else contract_simt<TL, T, 3, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
-  } else {
-    if (vec) contract_simt<TL, T, 1, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
-    else contract_simt<TL, T, 1, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split);
-  }
+  const unsigned gx = (unsigned)cdiv(d->Cin, 64), gy = (unsigned)cdiv(d->Cout, 32), gz = (unsigned)p.splits;
+#define XC_CONTRACT(KS, DYS) do { \
+    dim3 g2(gx * (KS / DYS), gy, gz); \
+    if (vec) contract_simt<TL, T, KS, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+    else contract_simt<TL, T, KS, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+  } while (0)
+  if (d->KH == 3) XC_CONTRACT(3, 3);
+  else if (d->KH == 5) XC_CONTRACT(5, 1);
+  else XC_CONTRACT(1, 1);
+#undef XC_CONTRACT
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
   const long count = (long)d->Cout * T9 * d->Cin;
@@ -290,6 +295,9 @@ static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* i
   if (d->KH == 3) {
     if (dgrad) conv_simt<T, 3, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
     else       conv_simt<T, 3, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+  } else if (d->KH == 5) {
+    if (dgrad) conv_simt<T, 5, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
+    else       conv_simt<T, 5, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
   } else {
     if (dgrad) conv_simt<T, 1, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
     else       conv_simt<T, 1, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
@@ -309,7 +317,8 @@ static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, co
   TcConvPlan t;
   if (tc_plan_conv(d, dgrad, &t)) return tc_run_conv(d, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
   return d->dtype == XCONV_F32 ? run_conv_simt<float>(d, dgrad, in, Wt, out, st)
-                               : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
+         : d->dtype == XCONV_F16 ? run_conv_simt<f16>(d, dgrad, in, Wt, out, st)
+                                 : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
 }
 
 // L = S dY^T into `L`; `Sb` receives the bfloat16 copy of S that the tensor-core kernel reads.
@@ -317,14 +326,16 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
                                   void* L, void* Sb_, char* w, cudaStream_t st) {
   if (p.tc_bp) {
     const long n = (long)d->r * d->B;
-    bf16* Sb = static_cast<bf16*>(Sb_);
-    cudaError_t e = launch_pdl(cast_f32_to_bf16, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, Sb, n);
+    cudaError_t e = d->dtype == XCONV_F16
+        ? launch_pdl(cast_f32_to_16<f16>, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, static_cast<f16*>(Sb_), n)
+        : launch_pdl(cast_f32_to_16<bf16>, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, static_cast<bf16*>(Sb_), n);
     ++g_launches;
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
-    return tc_run_backprobe(d, p.t, Sb, dY, L, w, st);
+    return tc_run_backprobe(d, p.t, Sb_, dY, L, w, st);
   }
   return d->dtype == XCONV_F32 ? run_backprobe_simt<float, float>(d, S, dY, L, st)
-                               : run_backprobe_simt<bf16, bf16>(d, S, dY, L, st);
+         : d->dtype == XCONV_F16 ? run_backprobe_simt<f16, f16>(d, S, dY, L, st)
+                                 : run_backprobe_simt<bf16, bf16>(d, S, dY, L, st);
 }
 
 static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const void* L, const void* Z,
@@ -332,6 +343,8 @@ static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const 
   if (p.tc_ct) return tc_run_contract(d, p.t, L, Z, dW, alpha, w, part, st);
   return d->dtype == XCONV_F32
              ? run_contract_simt<float, float>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st)
+         : d->dtype == XCONV_F16
+             ? run_contract_simt<f16, f16>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st)
              : run_contract_simt<bf16, bf16>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st);
 }
 
@@ -413,15 +426,16 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
 
 int xconv_engine_for(const xconv_desc* desc, int op) {
   if (validate(desc) != XCONV_OK) return XCONV_ENGINE_NONE;
+  const int tc = desc->dtype == XCONV_F16 ? XCONV_ENGINE_TCGEN05_F16 : XCONV_ENGINE_TCGEN05_BF16;
   switch (op) {
-    case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_SKETCH: return plan_sketch(desc).tc ? tc : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_WGRAD:
-    case XCONV_OP_CONTRACT: return plan_wgrad(desc).tc_ct ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
-    case XCONV_OP_BACKPROBE: return plan_wgrad(desc).tc_bp ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_CONTRACT: return plan_wgrad(desc).tc_ct ? tc : XCONV_ENGINE_SIMT_F32;
+    case XCONV_OP_BACKPROBE: return plan_wgrad(desc).tc_bp ? tc : XCONV_ENGINE_SIMT_F32;
     case XCONV_OP_FORWARD:
     case XCONV_OP_DGRAD: {
       TcConvPlan t;
-      return tc_plan_conv(desc, op == XCONV_OP_DGRAD, &t) ? XCONV_ENGINE_TCGEN05_BF16 : XCONV_ENGINE_SIMT_F32;
+      return tc_plan_conv(desc, op == XCONV_OP_DGRAD, &t) ? tc : XCONV_ENGINE_SIMT_F32;
     }
     default: return XCONV_ENGINE_NONE;
   }

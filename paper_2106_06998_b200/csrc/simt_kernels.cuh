@@ -169,18 +169,22 @@ __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ 
 // Offset contraction (Algorithm 1 backward step 4; Eq. 6 block by block):
 //   part[s][m][tap][n] = sum over the (j, y, x) of split s of L[j,y,x,m] * Z[j,y+ky-p,x+kx-p,n].
 // The shift of each kernel offset is an index offset into a haloed probe tile in shared memory, so
-// no shifted or im2col copy of Z exists.  A block owns 32 output x 64 input channels and all KS*KS
-// offsets; work items are (probe, row, 32-pixel chunk) triples dealt to grid.z splits in order.
+// no shifted or im2col copy of Z exists.  A block owns 32 output x 64 input channels and DYS rows of
+// the KS x KS offsets (all of them for 3 x 3; one row at a time for 5 x 5, whose 25 x 8 sums per thread
+// would not fit the registers); work items are (probe, row, 32-pixel chunk) triples dealt to grid.z
+// splits in order.  grid.x = (blocks of 64 input channels) x (KS / DYS groups of offset rows).
 // ---------------------------------------------------------------------------------------------
-template <typename TL, typename TZ, int KS, bool VEC>
+template <typename TL, typename TZ, int KS, int DYS, bool VEC>
 __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, const TZ* __restrict__ Z,
                                                      float* __restrict__ part, int r, int H, int W, int Cin,
                                                      int Cout, long items_per_split) {
-  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS;
+  constexpr int P = (KS - 1) / 2, XC = 32, T = DYS * KS, TALL = KS * KS;
   __shared__ __align__(16) float Ls[XC][32];
-  __shared__ __align__(16) float Zs[KS][XC + KS - 1][64];
+  __shared__ __align__(16) float Zs[DYS][XC + KS - 1][64];
   const int tid = threadIdx.x;
-  const int n0 = blockIdx.x * 64, m0 = blockIdx.y * 32;
+  const int nblocks = (Cin + 63) / 64;
+  const int dy0 = (blockIdx.x / nblocks) * DYS;          // first offset row of this block
+  const int n0 = (blockIdx.x % nblocks) * 64, m0 = blockIdx.y * 32;
   const int tx = tid & 15, ty = tid >> 4;
   const int chunks = (W + XC - 1) / XC;
   const long items = (long)r * H * chunks;
@@ -209,11 +213,11 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
         if (x0 + px < W && m0 + mm < Cout) v = ld4(L + (((long)j * H + y) * W + x0 + px) * Cout + m0 + mm);
         *reinterpret_cast<float4*>(&Ls[px][mm]) = v;
       }
-      for (int idx = tid; idx < KS * (XC + KS - 1) * 16; idx += 256) {
+      for (int idx = tid; idx < DYS * (XC + KS - 1) * 16; idx += 256) {
         const int nn = (idx & 15) * 4;
         const int px = (idx >> 4) % (XC + KS - 1);
         const int dy = (idx >> 4) / (XC + KS - 1);
-        const int yy = y + dy - P, xx = x0 + px - P;
+        const int yy = y + dy0 + dy - P, xx = x0 + px - P;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
           v = ld4(Z + (((long)j * H + yy) * W + xx) * Cin + n0 + nn);
@@ -226,11 +230,11 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
       if (x0 + px < W && m0 + mm < Cout) v = to_f(L[(((long)j * H + y) * W + x0 + px) * Cout + m0 + mm]);
       Ls[px][mm] = v;
     }
-    for (int idx = tid; idx < KS * (XC + KS - 1) * 64; idx += 256) {
+    for (int idx = tid; idx < DYS * (XC + KS - 1) * 64; idx += 256) {
       const int nn = idx & 63;
       const int px = (idx >> 6) % (XC + KS - 1);
       const int dy = (idx >> 6) / (XC + KS - 1);
-      const int yy = y + dy - P, xx = x0 + px - P;
+      const int yy = y + dy0 + dy - P, xx = x0 + px - P;
       float v = 0.f;
       if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
         v = to_f(Z[(((long)j * H + yy) * W + xx) * Cin + n0 + nn]);
@@ -242,7 +246,7 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
     for (int px = 0; px < XC; ++px) {
       const float2 l = *reinterpret_cast<const float2*>(&Ls[px][ty * 2]);
 #pragma unroll
-      for (int dy = 0; dy < KS; ++dy)
+      for (int dy = 0; dy < DYS; ++dy)
 #pragma unroll
         for (int dx = 0; dx < KS; ++dx) {
           const float4 z = *reinterpret_cast<const float4*>(&Zs[dy][px + dx][tx * 4]);
@@ -256,7 +260,7 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
     }
     __syncthreads();
   }
-  float* out = part + (long)blockIdx.z * Cout * T * Cin;
+  float* out = part + (long)blockIdx.z * Cout * TALL * Cin;
 #pragma unroll
   for (int i = 0; i < 2; ++i) {
     const int m = m0 + ty * 2 + i;
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const int n = n0 + tx * 4 + k;
-        if (n < Cin) out[((long)m * T + t) * Cin + n] = acc[t][i][k];
+        if (n < Cin) out[((long)m * TALL + dy0 * KS + t) * Cin + n] = acc[t][i][k];
       }
   }
 }
@@ -277,13 +281,14 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
 //   out[b,y,x,co] = sum_{tap,ci} w(co,ci,tap) * in[b,y+dy-p,x+dx-p,ci]
 //   forward: w(co,ci,tap) = Wt[co][tap][ci]          (Wt is [Cout][T][Cin])
 //   dgrad  : w(co,ci,tap) = Wt[ci][T-1-tap][co]
-// A block owns 32 pixels of one image row and 64 output channels; input channels go by 16.
+// A block owns 32 pixels of one image row and 64 output channels; input channels go by 16 (by 4 for
+// 5 x 5 kernels, whose weight tile would not fit the static shared memory otherwise).
 // ---------------------------------------------------------------------------------------------
 template <typename T_, int KS, bool DGRAD>
 __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, const T_* __restrict__ Wt,
                                                  T_* __restrict__ out, int B, int H, int W, int Ci, int Co,
                                                  int Cin_w) {
-  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS, CK = 16;
+  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS, CK = KS >= 5 ? 4 : 16;
   __shared__ __align__(16) float Xs[KS][XC + KS - 1][CK];
   __shared__ __align__(16) float Ws[T][CK][64];
   const int tid = threadIdx.x;
@@ -363,12 +368,13 @@ static __global__ void transpose_f32(const float* __restrict__ in, float* __rest
   out[(long)b * rows + j] = in[i];
 }
 
-// float -> bfloat16 copy (the sketch as tensor-core operand).
-static __global__ void cast_f32_to_bf16(const float* __restrict__ in, bf16* __restrict__ out, long n) {
+// float -> 16-bit storage type copy (the sketch as tensor-core operand).
+template <typename T>
+static __global__ void cast_f32_to_16(const float* __restrict__ in, T* __restrict__ out, long n) {
   pdl_trigger();
   pdl_wait();
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = __float2bfloat16_rn(in[i]);
+  if (i < n) out[i] = from_f<T>(in[i]);
 }
 
 }  // namespace xconv

@@ -83,7 +83,7 @@ extern "C" xconv_status xconv_sketch_static(const xconv_desc* desc, const void* 
                                             void* cuda_stream) {
   if (!desc || !X || !Z || !sketch) return XCONV_ERR_INVALID_ARG;
   if (desc->B <= 0 || desc->Cin <= 0 || desc->H <= 0 || desc->W <= 0 || desc->r <= 0) return XCONV_ERR_INVALID_ARG;
-  if (desc->dtype != XCONV_F32 && desc->dtype != XCONV_BF16) return XCONV_ERR_INVALID_ARG;
+  if (desc->dtype != XCONV_F32 && desc->dtype != XCONV_BF16 && desc->dtype != XCONV_F16) return XCONV_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(Z) | reinterpret_cast<uintptr_t>(sketch)) & 15u)
     return XCONV_ERR_ALIGNMENT;
   // the one partial-sum slab [r][B] must fit the fixed array; beyond that there is nowhere to put it
@@ -94,5 +94,6 @@ extern "C" xconv_status xconv_sketch_static(const xconv_desc* desc, const void* 
   if (s != XCONV_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   return desc->dtype == XCONV_F32 ? sketch_static_run<float>(desc, X, Z, sketch, scratch, st)
-                                  : sketch_static_run<bf16>(desc, X, Z, sketch, scratch, st);
+         : desc->dtype == XCONV_F16 ? sketch_static_run<f16>(desc, X, Z, sketch, scratch, st)
+                                    : sketch_static_run<bf16>(desc, X, Z, sketch, scratch, st);
 }

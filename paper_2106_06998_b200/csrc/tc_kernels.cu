@@ -100,6 +100,7 @@ struct TcParams {
   int z_is_a;              // SKETCH: Z is the A operand (probes on the MMA rows) instead of the B operand
   long z_row_len;          // entries of one probing vector, H*W*Cin
   long rows_z;             // probing vectors (rows of Z)
+  int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
 };
@@ -213,7 +214,8 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem], bfloat16 inputs, float accumulate; issued by one thread.  The two
+// D[tmem] (+)= A[smem] * B[smem], 16-bit inputs (bfloat16 or float16, per the instruction descriptor), float
+// accumulate; issued by one thread.  The two
 // shared-memory descriptors come as 32-bit halves: only the low half (start address) changes between
 // k-steps, so the issuing thread -- whose own instruction stream is the critical path of the CTA when
 // the tiles are small -- spends one 32-bit add per operand and k-step.
@@ -301,31 +303,31 @@ __device__ __forceinline__ uint2 z_sign_bits64(long e0, uint32_t k0, uint32_t k1
   const uint4 w = philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), k0, k1);
   return (e0 & 64) ? make_uint2(w.z, w.w) : make_uint2(w.x, w.y);
 }
-// Eight consecutive entries as bfloat16 (+1 = 0x3F80, -1 = 0xBF80) from bits 0..7 of `t` (higher bits are
-// ignored).  Two sign bits b0, b1 at positions 2i, 2i+1 go to bits 15 and 31 of a word: the product of
+// Eight consecutive entries as bfloat16 (+1 = 0x3F80, -1 = 0xBF80; `ones` = 0x3F803F80) or float16 (+1 = 0x3C00,
+// `ones` = 0x3C003C00) from bits 0..7 of `t` (higher bits are ignored).  Two sign bits b0, b1 at positions 2i, 2i+1 go to bits 15 and 31 of a word: the product of
 // (t & (3 << 2i)) with (0x40008000 >> 2i) holds b0 at bits 15 and 30 and b1 at bits 16 and 31.
-__device__ __forceinline__ uint4 z_pack8(uint32_t t) {
+__device__ __forceinline__ uint4 z_pack8(uint32_t t, uint32_t ones) {
   uint4 o;
-  o.x = (((t & 0x03u) * 0x40008000u) & 0x80008000u) | 0x3F803F80u;
-  o.y = (((t & 0x0Cu) * 0x10002000u) & 0x80008000u) | 0x3F803F80u;
-  o.z = (((t & 0x30u) * 0x04000800u) & 0x80008000u) | 0x3F803F80u;
-  o.w = (((t & 0xC0u) * 0x01000200u) & 0x80008000u) | 0x3F803F80u;
+  o.x = (((t & 0x03u) * 0x40008000u) & 0x80008000u) | ones;
+  o.y = (((t & 0x0Cu) * 0x10002000u) & 0x80008000u) | ones;
+  o.z = (((t & 0x30u) * 0x04000800u) & 0x80008000u) | ones;
+  o.w = (((t & 0xC0u) * 0x01000200u) & 0x80008000u) | ones;
   return o;
 }
 
 // 64 entries of one row of a K-major, 128-byte-swizzled tile (row base `rbase`): eight 16-byte pieces.
-__device__ __forceinline__ void z_store64(uint32_t rbase, int row, uint2 bits) {
+__device__ __forceinline__ void z_store64(uint32_t rbase, int row, uint2 bits, uint32_t ones) {
 #pragma unroll
   for (int c = 0; c < 8; ++c) {
-    const uint4 o = z_pack8((c < 4 ? bits.x : bits.y) >> ((c & 3) * 8));
+    const uint4 o = z_pack8((c < 4 ? bits.x : bits.y) >> ((c & 3) * 8), ones);
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (((uint32_t)c ^ ((uint32_t)row & 7u)) << 4)),
                  "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
   }
 }
 // 128 entries: the same row of two consecutive k-block tiles, `tile_bytes` apart.
-__device__ __forceinline__ void z_store128(uint32_t rbase, uint32_t tile_bytes, int row, uint4 w) {
-  z_store64(rbase, row, make_uint2(w.x, w.y));
-  z_store64(rbase + tile_bytes, row, make_uint2(w.z, w.w));
+__device__ __forceinline__ void z_store128(uint32_t rbase, uint32_t tile_bytes, int row, uint4 w, uint32_t ones) {
+  z_store64(rbase, row, make_uint2(w.x, w.y), ones);
+  z_store64(rbase + tile_bytes, row, make_uint2(w.z, w.w), ones);
 }
 
 // The MMAs of `nkb` k-blocks that arrive in two halves (see TcParams::halves), with the numbers of k-steps known at
@@ -369,6 +371,13 @@ __device__ __forceinline__ bool umma_halves_items(int nkb, int& s, uint32_t& par
     if (s == slots) { s = 0; parity ^= 1u; }
   }
   return true;
+}
+
+// Two floats rounded to the 16-bit storage type, packed (first in the low half).
+__device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, int f16) {
+  if (f16) { __half2 h = __floats2half2_rn(__uint_as_float(a), __uint_as_float(b)); return *reinterpret_cast<uint32_t*>(&h); }
+  __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
+  return *reinterpret_cast<uint32_t*>(&h);
 }
 
 constexpr int TILE_M = 128;
@@ -542,7 +551,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1 && p.mode == MODE_CONTRACT && p.halves) {
     // ------------------------------------------------------------------ MMA issuer, k-blocks in two halves
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) |
+      const uint32_t idesc = (1u << 4) | (p.f16 ? 0u : (1u << 7) | (1u << 10)) | (1u << 15) | (1u << 16) |
                              ((uint32_t)(p.tile_n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
       const uint32_t step = p.mn_step >> 4;                                   // 16 rows
       const uint32_t a_lo0 = (p.a_lbo >> 4) << 16, b_lo0 = (p.b_lbo >> 4) << 16;
@@ -686,7 +695,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // One thread.  With small tiles the time between two tcgen05.mma is set by this thread's own
     // instruction stream, so the loop carries descriptors as 32-bit halves and does no division.
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn_major << 15) |
+      // instruction descriptor: float accumulator (bit 4), A and B formats (bits 7-9, 10-12: 0 = float16, 1 = bfloat16,
+      // always the same for both), operand majorness (bits 15, 16), N >> 3 (bits 17-22), M >> 4 (bits 24-28)
+      const uint32_t idesc = (1u << 4) | (p.f16 ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)p.a_mn_major << 15) |
                              ((uint32_t)p.b_mn_major << 16) | ((uint32_t)(p.tile_n >> 3) << 17) |
                              ((uint32_t)(TILE_M >> 4) << 24);
       // Shared-memory descriptor (128-byte swizzle): start address >> 4 | (lbo >> 4) << 16 in the low
@@ -818,6 +829,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
         const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
         const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
+        const uint32_t z_ones = p.f16 ? 0x3C003C00u : 0x3F803F80u;
         long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
         for (int i = 0; i < w.nkb && ok; ++i) {
           if (gen_fill > 0) {
@@ -839,14 +851,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
               const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
               const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
-              z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0);
-              if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1);
+              z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0, z_ones);
+              if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
             }
           } else {
             for (int item = gtid; item < nrows * p.kgroup; item += 128) {
               const int row = item % nrows, g = item / nrows;
               const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
-              z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits);
+              z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
             }
           }
           fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
@@ -885,14 +897,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             (uint32_t)(buf * acc_cols + mt * unit_cols + b * 64 + half * 32), v);
 #pragma unroll
               for (int i = 0; i < 32; i += 8) {
-                __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
-                __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-                __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
                 const uint32_t sdst = rowbase + ((((uint32_t)half * 4u + (uint32_t)(i >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sdst),
-                             "r"(*reinterpret_cast<uint32_t*>(&h0)), "r"(*reinterpret_cast<uint32_t*>(&h1)),
-                             "r"(*reinterpret_cast<uint32_t*>(&h2)), "r"(*reinterpret_cast<uint32_t*>(&h3)) : "memory");
+                             "r"(pack2(v[i + 0], v[i + 1], p.f16)), "r"(pack2(v[i + 2], v[i + 3], p.f16)),
+                             "r"(pack2(v[i + 4], v[i + 5], p.f16)), "r"(pack2(v[i + 6], v[i + 7], p.f16)) : "memory");
               }
             }
             fence_async_smem();
@@ -936,18 +944,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
                   uint4 o;
-                  __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(v[i + 0]), __uint_as_float(v[i + 1]));
-                  __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
-                  __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[i + 4]), __uint_as_float(v[i + 5]));
-                  __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(v[i + 6]), __uint_as_float(v[i + 7]));
-                  o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
-                  o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+                  o.x = pack2(v[i + 0], v[i + 1], p.f16); o.y = pack2(v[i + 2], v[i + 3], p.f16);
+                  o.z = pack2(v[i + 4], v[i + 5], p.f16); o.w = pack2(v[i + 6], v[i + 7], p.f16);
                   *reinterpret_cast<uint4*>(dst + i) = o;
                 }
               } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
-                  if (i < nc && col0 + c + i < p.cols) dst[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                  if (i < nc && col0 + c + i < p.cols)
+                    reinterpret_cast<unsigned short*>(dst)[i] = (unsigned short)(pack2(v[i], v[i], p.f16) & 0xFFFFu);
               }
             }
           } else {
@@ -1090,9 +1095,10 @@ static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   return fn;
 }
 
-// bfloat16 tensor map, 128-byte swizzle unless told otherwise; dims/strides innermost first, strides in bytes for dims 1..rank-1.
+// Tensor map over 16-bit elements (bfloat16, or float16 if `f16`), 128-byte swizzle unless told otherwise;
+// dims/strides innermost first, strides in bytes for dims 1..rank-1.
 static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
-                     const uint32_t* box, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+                     const uint32_t* box, bool f16, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
   if (!fn) return false;
   cuuint32_t estr[5] = {1, 1, 1, 1, 1};
@@ -1100,7 +1106,7 @@ static bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t*
   cuuint32_t bx[5];
   for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, bx, estr,
+  CUresult r = fn(m, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, bx, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -1135,7 +1141,7 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
 // ---- sketch --------------------------------------------------------------------------------
 
 bool tc_plan_sketch(const xconv_desc* d, TcSketchPlan* p, bool redraw) {
-  if (d->dtype != XCONV_BF16) return false;
+  if (d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return false;
   const long K = (long)d->H * d->W * d->Cin;
   if (K % 8 != 0 || K < 2048 || K > 2000000000L) return false;
   p->swap = d->B >= d->r ? 1 : 0;
@@ -1179,6 +1185,7 @@ bool tc_sketch_can_redraw(const xconv_desc* d) {
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const void* X, const void* Z, float* S,
                            char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed) {
   const long K = (long)d->H * d->W * d->Cin;
+  const bool f16 = d->dtype == XCONV_F16;
   const int rows = pl.swap ? d->B : d->r, cols = pl.swap ? d->r : d->B;
   if (seed) Z = X;                                   // the map of Z is built but never used: any valid base
   const void* A = pl.swap ? X : Z;
@@ -1194,15 +1201,16 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
     const uint64_t sa[2] = {(uint64_t)K * 2, 128};
     const uint32_t box_a[3] = {64, rows_box, (uint32_t)pl.kgroup};
     const uint32_t box_b[3] = {64, (uint32_t)pl.tile_n, (uint32_t)pl.kgroup};
-    if (!make_map(&ma, A, 3, da, sa, box_a) || !make_map(&mb, Bm, 3, db, sa, box_b)) return XCONV_ERR_CUDA;
+    if (!make_map(&ma, A, 3, da, sa, box_a, f16) || !make_map(&mb, Bm, 3, db, sa, box_b, f16)) return XCONV_ERR_CUDA;
   } else {
     const uint64_t da[2] = {(uint64_t)K, (uint64_t)rows}, db[2] = {(uint64_t)K, (uint64_t)cols};
     const uint64_t sa[1] = {(uint64_t)K * 2};
     const uint32_t box_a[2] = {64, rows_box};
     const uint32_t box_b[2] = {64, (uint32_t)pl.tile_n};
-    if (!make_map(&ma, A, 2, da, sa, box_a) || !make_map(&mb, Bm, 2, db, sa, box_b)) return XCONV_ERR_CUDA;
+    if (!make_map(&ma, A, 2, da, sa, box_a, f16) || !make_map(&mb, Bm, 2, db, sa, box_b, f16)) return XCONV_ERR_CUDA;
   }
   TcParams p{};
+  p.f16 = f16 ? 1 : 0;
   p.mode = MODE_SKETCH;
   p.tile_n = pl.tile_n;
   p.m_sub = pl.m_sub;
@@ -1276,7 +1284,7 @@ static void pick_patch(int H, int W, int* pw, int* ph) {
 }
 
 int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
-  if (d->dtype != XCONV_BF16) return 0;
+  if (d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return 0;
   int mask = 0;
   const long Q = (long)d->H * d->W * d->Cout;
   // back-probe: D[j, q], rows = r, cols = Q, k = B
@@ -1372,6 +1380,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
                               void* L, char* ws_head, cudaStream_t st) {
   const long Q = (long)d->H * d->W * d->Cout;
   const int bk = pl.bp_ksteps * 16;
+  const bool f16 = d->dtype == XCONV_F16;
   CUtensorMap ma, mb;
   // A = S (bfloat16) [r][B], k = b contiguous; B operand = dY [B][Q], q contiguous (MN-major tile)
   // dY as (64 positions, B rows, Q/64 blocks of 64 positions): one box fetches the [bk x 64] piece of one
@@ -1381,14 +1390,15 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[2] = {(uint64_t)Q * 2, 128};
   const uint32_t box_a[2] = {64, (uint32_t)pl.bp_rows_box};           // 128-byte rows whatever bk is (zero fill past B)
   const uint32_t box_b[3] = {64, (uint32_t)bk, 1};
-  if (!make_map(&ma, S_bf16, 2, da, sa, box_a) || !make_map(&mb, dY, 3, db, sb, box_b)) return XCONV_ERR_CUDA;
+  if (!make_map(&ma, S_bf16, 2, da, sa, box_a, f16) || !make_map(&mb, dY, 3, db, sb, box_b, f16)) return XCONV_ERR_CUDA;
   // L [r][Q] for the epilogue's stores, as (64 positions, r rows, Q/64 groups): one box = the 32 rows of one
   // epilogue warp x one block of positions
   CUtensorMap mc;
   const uint64_t dc[3] = {64, (uint64_t)d->r, (uint64_t)(Q / 64)};
   const uint32_t box_c[3] = {64, 32, 1};
-  if (!make_map(&mc, L, 3, dc, sb, box_c)) return XCONV_ERR_CUDA;
+  if (!make_map(&mc, L, 3, dc, sb, box_c, f16)) return XCONV_ERR_CUDA;
   TcParams p{};
+  p.f16 = f16 ? 1 : 0;
   p.mode = MODE_BACKPROBE;
   p.tile_n = pl.bp_tile_n;
   p.m_sub = pl.bp_m_sub;
@@ -1429,6 +1439,7 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
                              float alpha, char* ws_head, char* part, cudaStream_t st) {
   const int T = d->KH * d->KW;
   const int bk = pl.patch_w * pl.patch_h;
+  const bool f16 = d->dtype == XCONV_F16;
   CUtensorMap ma, mb;
   // (cw channels, x, y, groups of cw channels, probe), cw = 64 or 32: one box = a whole
   // [patch x channels] tile laid out as consecutive blocks of (2*cw)-byte rows, one block per channel
@@ -1449,8 +1460,9 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   const uint32_t box_h = (uint32_t)(pl.ct_halves ? pl.patch_h / 2 : pl.patch_h);   // image rows per copy
   const uint32_t box_a[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, box_h, (uint32_t)groups_a, 1};
   const uint32_t box_b[5] = {(uint32_t)cw, (uint32_t)pl.patch_w, box_h, (uint32_t)groups_b, 1};
-  if (!make_map(&ma, L, 5, da, sa, box_a, swz) || !make_map(&mb, Z, 5, db, sb, box_b, swz)) return XCONV_ERR_CUDA;
+  if (!make_map(&ma, L, 5, da, sa, box_a, f16, swz) || !make_map(&mb, Z, 5, db, sb, box_b, f16, swz)) return XCONV_ERR_CUDA;
   TcParams p{};
+  p.f16 = f16 ? 1 : 0;
   p.mode = MODE_CONTRACT;
   p.tile_n = pl.ct_tile_n;
   p.m_sub = pl.ct_m_sub;
@@ -1578,7 +1590,7 @@ static void pick_patch_conv(int H, int W, int* pw, int* ph) {
 }
 
 bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
-  if (d->dtype != XCONV_BF16) return false;
+  if (d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return false;
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
   if (Ci % 32 != 0 || Co % 8 != 0 || Co < 16) return false;
   p->tile_n = std::min(256, round_up(Co, 16));
@@ -1605,6 +1617,7 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
                          void* out, char* ws_head, char* wt, cudaStream_t st) {
   const int T = d->KH * d->KW;
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
+  const bool f16 = d->dtype == XCONV_F16;
   const void* Wk = W;
   if (dgrad) {
     const long count = (long)d->Cout * T * d->Cin;
@@ -1624,8 +1637,9 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   const uint64_t db[2] = {(uint64_t)T * Ci, (uint64_t)Co};
   const uint64_t sb[1] = {(uint64_t)T * Ci * 2};
   const uint32_t box_b[2] = {cw, (uint32_t)pl.tile_n};
-  if (!make_map(&ma, in, 5, da, sa, box_a, swz) || !make_map(&mb, Wk, 2, db, sb, box_b, swz)) return XCONV_ERR_CUDA;
+  if (!make_map(&ma, in, 5, da, sa, box_a, f16, swz) || !make_map(&mb, Wk, 2, db, sb, box_b, f16, swz)) return XCONV_ERR_CUDA;
   TcParams p{};
+  p.f16 = f16 ? 1 : 0;
   p.mode = MODE_CONV;
   p.tile_n = pl.tile_n;
   const uint32_t px = (uint32_t)(pl.patch_w * pl.patch_h);

@@ -5,7 +5,7 @@ arithmetic, so that the float64 oracle and the CUDA path can both be fed from
 it without sharing anything else.
 
 Every array is generated on the host from ``numpy.random.Generator(PCG64(seed))``
-as float32, rounded once to the storage type (float32 or bfloat16,
+as float32, rounded once to the storage type (float32, bfloat16 or float16,
 round-to-nearest-even) and handed out as a float32 array holding exactly the
 stored values.  Logical index order is (batch, channel, y, x) for X and dY,
 (Cout, Cin, ky, kx) for W and (probe, channel, y, x) for Z.
@@ -65,6 +65,8 @@ def round_to_storage(a: np.ndarray, dtype: str) -> np.ndarray:
         return np.ascontiguousarray(a, dtype=np.float32)
     if dtype == "bf16":
         return round_bf16(a)
+    if dtype == "f16":      # IEEE half precision, round to nearest even (numpy's conversion)
+        return np.ascontiguousarray(a, dtype=np.float32).astype(np.float16).astype(np.float32)
     raise ValueError(f"unknown storage dtype {dtype!r}")
 
 

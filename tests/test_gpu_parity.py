@@ -165,6 +165,49 @@ def test_pointwise_kernel(dtype):
     _full_layer_parity(lay, K=1)
 
 
+# 5 x 5 kernels: the layers of the paper's CIFAR-10 network (appendix, network tables): 3 -> 16 and
+# 16 -> 32 channels on 32 x 32 images, 32 -> 32 on 16 x 16, plus a wide layer for the tcgen05 kernels.
+@pytest.mark.parametrize("dtype,shape", [
+    # B, Cin, Cout, H, W, r
+    ("f32", (4, 3, 16, 32, 32, 8)),
+    ("f32", (4, 16, 32, 32, 32, 8)),
+    ("bf16", (4, 16, 32, 32, 32, 16)),
+    ("f32", (6, 32, 32, 16, 16, 12)),
+    ("bf16", (16, 32, 32, 16, 16, 12)),       # 32-channel groups: tcgen05, 64-byte-swizzle tiles
+    ("bf16", (16, 128, 64, 9, 11, 24)),       # tcgen05, ragged patches, 25 offsets
+    ("bf16", (8, 64, 64, 12, 12, 40)),        # r > B: the probes are summed first
+    ("f32", (2, 5, 7, 6, 9, 5)),              # odd everything
+])
+def test_five_by_five_kernels(dtype, shape):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape) + 5, KH=5, KW=5,
+                             z="rademacher", x="relu")
+    _full_layer_parity(lay, K=5)
+
+
+# float16 storage (the paper's "half precision", Section 5.2).  Tolerance 2e-3: S and L are each rounded once
+# to float16 (2^-11 / sqrt(3) = 2.8e-4 relative rms each, about 4e-4 together); five times that.
+@pytest.mark.parametrize("shape,K", [
+    # B, Cin, Cout, H, W, r
+    ((3, 5, 7, 9, 11, 5), 3),              # FP32-FMA kernels, odd sizes
+    ((16, 128, 128, 28, 28, 32), 3),       # the ImageNet-stage recipe, shrunk: tcgen05 with float16 operands
+    ((16, 128, 128, 28, 28, 128), 3),      # r > B
+    ((24, 192, 320, 9, 13, 40), 3),        # ragged tiles
+    ((8, 32, 32, 40, 24, 72), 3),          # 32-channel groups (64-byte swizzle)
+    ((16, 32, 32, 16, 16, 12), 5),         # 5 x 5 kernel
+    ((16, 64, 128, 8, 12, 32), 1),         # pointwise kernel
+])
+def test_float16_storage(shape, K):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="f16", seed=sum(shape) + 16, KH=K, KW=K,
+                             z="rademacher", x="relu")
+    lay["dY"] = inputs.round_to_storage(lay["dY"] * np.float32(0.1), "f16")     # the recipe's N(0, 1e-2)
+    if Cin >= 32:
+        desc = xb.make_desc(B, Cin, Cout, H, W, r, torch.float16, K)
+        assert xb.engine_for(desc, xb.OP_CONTRACT) == "tcgen05_f16" and xb.engine_for(desc, xb.OP_SKETCH) == "tcgen05_f16"
+    _full_layer_parity(lay, K=K)
+
+
 @pytest.mark.parametrize("cfg,r,shrink", [
     (1, 8, {}),                                   # the small configuration at full size
     (2, 16, dict(B=32)), (2, 64, dict(B=32)),

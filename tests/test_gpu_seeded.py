@@ -21,7 +21,7 @@ def _built():
     torch.cuda.set_device(0)
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float16])
 @pytest.mark.parametrize("shape", [(1, 1, 1, 1), (3, 5, 4, 7), (8, 16, 9, 9), (5, 64, 6, 12), (130, 8, 5, 13)])
 def test_probes_from_seed_match_the_oracle_generator_bit_for_bit(shape, dtype):
     r, Cin, H, W = shape
@@ -55,6 +55,18 @@ def test_seeded_sketch_matches_oracle_and_the_stored_probe_path(shape):
     torch.cuda.synchronize()
     # the same sum in a possibly different order (the seeded plan may take more k-blocks per stage)
     check("seeded sketch against the stored-probe sketch", host(S), host(S_stored), 1e-5)
+    check("seeded sketch", host(S), O.sketch(lay["X"], O.rademacher_probes(seed, r, Cin, H, W)), TOL_SKETCH)
+
+
+@pytest.mark.parametrize("shape", [(24, 8, 16, 16, 8), (8, 64, 6, 35, 40)])
+def test_seeded_sketch_float16_storage_redraws_float16_signs(shape):
+    B, Cin, H, W, r = shape
+    seed = 31 * sum(shape)
+    lay = inputs.make_custom(B, Cin, 8, H, W, r, dtype="f16", seed=sum(shape), z="rademacher", x="normal")
+    X = xb.to_device(lay["X"], "f16")
+    assert xb.engine_for(xb.make_desc(B, Cin, 8, H, W, r, torch.float16), xb.OP_SKETCH) == "tcgen05_f16"
+    S = xb.xconv_sketch_seeded(X, seed, r)
+    torch.cuda.synchronize()
     check("seeded sketch", host(S), O.sketch(lay["X"], O.rademacher_probes(seed, r, Cin, H, W)), TOL_SKETCH)
 
 

@@ -48,7 +48,7 @@ def test_invalid_descriptors_are_rejected(lib):
     d = _desc()
     d.circular = 1                       # the paper's circular shift has no kernel
     assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
-    d = _desc(K=5)                       # 5x5 kernels have no kernel yet
+    d = _desc(K=7)                       # kernel sizes beyond 5 x 5 have no kernel
     assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
     d = _desc()
     d.pad_h = 0                          # not a "same" convolution
