@@ -36,6 +36,9 @@ literal block-matrix estimator of Eq. (6) (sketch, backprobe, wgrad_estimate).
 philox4x32_10 and rademacher_probes (probing vectors redrawn from a stored seed, Algorithm 1) are pinned
 by the generator's published known-answer vectors (tests/golden/philox4x32_10_kat.txt), by the
 balance and independence of the signs, and by the unbiasedness of the estimator run on them.
+sketch_independent and wgrad_estimate_independent (the estimator applied to each channel pair on its own) are
+pinned by exact recovery with one orthogonal basis per channel, by unbiasedness with the crosstalk-free
+Hutchinson variance, and by their reduction to the multi-channel functions for a single input channel.
 rel_fro, the metric every parity verdict passes through, is pinned on a hand-computed pair.
 No function here is "parity unpinned".
 """
@@ -180,6 +183,32 @@ def xconv_layer(X, W, dY, Z, pad=None, circular=False, scale=None):
     dW = wgrad_estimate(S, dY, Z, KH, KW, pad, circular, scale)
     dX = dx_exact(dY, W, pad, circular)
     return Y, S, dW, dX
+
+
+# --- trace estimation applied to every input/output channel pair on its own ---------------------------
+
+def sketch_independent(X, Z):
+    """The per-channel sketch X-bar^n = Z_n^T X^n in R^{r x B} for every input channel n: what has to be kept
+    when the single-channel estimator (Eq. 4) is applied to each channel pair independently (first sentence
+    of the multi-channel case, Section 3) instead of probing the stacked matrix.
+
+    S[j,n,b] = sum_{y,x} Z[j,n,y,x] X[b,n,y,x]; summing it over n gives the multi-channel sketch."""
+    X = np.asarray(X, F64)
+    Z = np.asarray(Z, F64)
+    return np.stack([sketch(X[:, n:n + 1], Z[:, n:n + 1]) for n in range(X.shape[1])], axis=1)
+
+
+def wgrad_estimate_independent(S, dY, Z, KH=3, KW=3, pad=None, circular=False):
+    """dw_i^{n,m} ~ (1/r) sum_j (z_{n,j}^T X^n) ((dY^m)^T T_{-k(i)} z_{n,j}): Eq. (4) for the pair (n, m), with the
+    n-th block of the probing vectors and the n-th per-channel sketch.  No other channel enters the estimate
+    of a pair, so there is no crosstalk.  S [r, Cin, B] from ``sketch_independent``."""
+    S = np.asarray(S, F64)
+    Z = np.asarray(Z, F64)
+    Cin = Z.shape[1]
+    dW = np.zeros((np.asarray(dY).shape[1], Cin, KH, KW), F64)
+    for n in range(Cin):
+        dW[:, n:n + 1] = wgrad_estimate(S[:, n, :], dY, Z[:, n:n + 1], KH, KW, pad, circular)
+    return dW
 
 
 # --- the literal block-matrix form of Eq. (6), for tiny layers only ---------------------------

@@ -439,3 +439,54 @@ def test_rel_fro_on_a_hand_computed_pair():
     assert O.rel_fro(b, b) == 0.0
     assert O.rel_fro(2 * b, b) == pytest.approx(1.0, abs=1e-15)          # scale of the error, not of the data
     assert O.rel_fro(np.array([3.0, 4.0]), np.zeros(2)) == pytest.approx(5.0)   # zero reference: absolute norm
+
+
+# ---------------------------------------------------------------- independent probing (per channel pair)
+
+def test_independent_sketch_sums_to_the_multichannel_sketch_and_reduces_for_one_channel():
+    X, Wt, dY = _tiny(seed=40, B=3, Cin=3, Cout=2, H=4, W=5)
+    Z = _rng(41).standard_normal((7, 3, 4, 5))
+    Si = O.sketch_independent(X, Z)
+    assert Si.shape == (7, 3, 3)
+    np.testing.assert_allclose(Si.sum(axis=1), O.sketch(X, Z), atol=1e-12)
+    # brute force for one entry
+    j, n, b = 4, 2, 1
+    assert abs(Si[j, n, b] - sum(Z[j, n, y, x] * X[b, n, y, x] for y in range(4) for x in range(5))) < 1e-12
+    # a single input channel: both estimators coincide (Eq. 4 is the Cin = Cout = 1 case of Eq. 6)
+    X1, Z1 = X[:, :1], Z[:, :1]
+    np.testing.assert_allclose(O.wgrad_estimate_independent(O.sketch_independent(X1, Z1), dY, Z1),
+                               O.wgrad_estimate(O.sketch(X1, Z1), dY, Z1), atol=1e-12)
+
+
+def test_independent_probing_recovers_the_exact_gradient_with_one_orthogonal_basis_per_channel():
+    """r = N and (1/r) Z_n Z_n^T = I_N for every channel n (a different basis each): every pair's trace is exact."""
+    X, Wt, dY = _tiny(seed=42, B=3, Cin=3, Cout=2, H=3, W=4)
+    N = 12
+    Z = np.stack([np.sqrt(N) * np.linalg.qr(_rng(50 + n).standard_normal((N, N)))[0].T.reshape(N, 3, 4)
+                  for n in range(3)], axis=1)                     # [r = N, Cin, H, W]
+    est = O.wgrad_estimate_independent(O.sketch_independent(X, Z), dY, Z)
+    np.testing.assert_allclose(est, _loops_dw(X, dY, 3, 3, False), atol=1e-10)
+    # the multi-channel estimator on the same probes is NOT exact (r = N < N*Cin: crosstalk remains)
+    assert O.rel_fro(O.wgrad_estimate(O.sketch(X, Z), dY, Z), _loops_dw(X, dY, 3, 3, False)) > 1e-2
+
+
+def test_independent_probing_is_unbiased_with_the_crosstalk_free_variance():
+    """Per pair the variance is the single-channel Hutchinson expression: the sum over the other channels'
+    blocks, which the multi-channel estimator carries, is absent."""
+    X, Wt, dY = _tiny(seed=20, B=3, Cin=2, Cout=2, H=4, W=4)
+    exact = _loops_dw(X, dY, 3, 3, False)
+    T = 6000
+    Zall = _rng(43).standard_normal((T, 2, 4, 4))
+    ests = np.stack([O.wgrad_estimate_independent(O.sketch_independent(X, Zall[t:t + 1]), dY, Zall[t:t + 1])
+                     for t in range(T)])
+    mean, var = ests.mean(0), ests.var(0, ddof=1)
+    for m in range(2):
+        for ky in range(3):
+            for kx in range(3):
+                C = _C_blocks(X, dY, m, ky, kx)
+                for n in range(2):
+                    v = np.sum(C[n] ** 2) + np.trace(C[n] @ C[n])
+                    z = (mean[m, n, ky, kx] - exact[m, n, ky, kx]) / math.sqrt(v / T)
+                    assert abs(z) < 4.5, (m, n, ky, kx, z)
+                    assert 0.8 < var[m, n, ky, kx] / v < 1.25, (m, n, ky, kx, var[m, n, ky, kx], v)
+                    assert v < _closed_form_variance(C, n, False)
