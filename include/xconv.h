@@ -78,7 +78,7 @@ typedef enum {
 
 typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3,
                XCONV_OP_BACKPROBE = 4, XCONV_OP_CONTRACT = 5, XCONV_OP_SKETCH_SEEDED = 6,
-               XCONV_OP_WGRAD_SEEDED = 7 } xconv_op;
+               XCONV_OP_WGRAD_SEEDED = 7, XCONV_OP_WGRAD_INDEPENDENT = 8 } xconv_op;
 
 /* Which arithmetic engine a call will use for its dominant kernel. */
 typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2,
@@ -154,6 +154,22 @@ xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const 
                              void* ws, size_t ws_bytes, void* cuda_stream);
 xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z, float* dW,
                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Trace estimation applied to every input/output channel pair on its own ("independent" probing: first
+ * sentence of the multi-channel case in Section 3; Eq. 4 per pair).  The probing vectors have the same shape
+ * as for the multi-channel estimator, Z [r,H,W,Cin], but block n of a vector only ever meets channel n:
+ *   sketch[j,n,b]  = sum_{y,x} Z[j,n,y,x] * X[b,n,y,x]                  (r*Cin*B floats, element (j,n,b) at (j*Cin + n)*B + b)
+ *   dW[m,n,ky,kx]  = (1/r) * sum_{j,b,y,x} sketch[j,n,b] * dY[b,m,y,x] * Z[j,n,y+ky-pad_h,x+kx-pad_w]
+ * No other input channel enters the estimate of a pair (no crosstalk), at the price of a sketch Cin times
+ * larger: the memory factor per sample is N/r instead of N*Cin/r.  xconv_sketch_independent needs no scratch.
+ * xconv_wgrad_independent takes xconv_workspace_bytes(desc, XCONV_OP_WGRAD_INDEPENDENT) bytes; it sums over
+ * the probes first (the activation rebuilt channel by channel from its sketch, held in `ws` in desc.dtype) and
+ * then runs the offset contraction over the batch -- the same sum as the formula above in another order.
+ * desc.chan_scale is ignored (the scale is 1/r). */
+xconv_status xconv_sketch_independent(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
+                                      void* cuda_stream);
+xconv_status xconv_wgrad_independent(const xconv_desc* desc, const float* sketch, const void* dY, const void* Z,
+                                     float* dW, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Exact input gradient (the transposed convolution; the method leaves it as in standard
  * back-propagation, Section 1).  dY [B,H,W,Cout], W [Cout,KH,KW,Cin]; dX [B,H,W,Cin] in desc.dtype. */

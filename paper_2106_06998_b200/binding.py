@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libxconv.so")
 
 XCONV_F32, XCONV_BF16, XCONV_F16 = 0, 1, 2
-OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT, OP_SKETCH_SEEDED, OP_WGRAD_SEEDED = 0, 1, 2, 3, 4, 5, 6, 7
+OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT, OP_SKETCH_SEEDED, OP_WGRAD_SEEDED, OP_WGRAD_INDEPENDENT = 0, 1, 2, 3, 4, 5, 6, 7, 8
 ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16", 3: "tcgen05_f16"}
 STATUS_OK = 0
 
@@ -25,6 +25,7 @@ STATUS_OK = 0
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
            "xconv_dgrad", "xconv_probes_from_seed", "xconv_sketch_seeded", "xconv_wgrad_seeded", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
            "xconv_workspace_status", "xconv_selftest_wait_limit", "xconv_measure_fma_rate",
+           "xconv_sketch_independent", "xconv_wgrad_independent",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
     L.xconv_wgrad_seeded.restype = c_int
     L.xconv_wgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad.restype = c_int
+    L.xconv_sketch_independent.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
+    L.xconv_sketch_independent.restype = c_int
+    L.xconv_wgrad_independent.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    L.xconv_wgrad_independent.restype = c_int
     L.xconv_backprobe_bytes.argtypes = [P]; L.xconv_backprobe_bytes.restype = c_size_t
     L.xconv_backprobe.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_backprobe.restype = c_int
@@ -312,6 +317,39 @@ def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_
     dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
     wgrad_into(desc, sketch, dY, Z, dW, ws)
+    return dW
+
+
+def xconv_sketch_independent(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
+    """Per-channel sketch S[j, n, b] = <Z[j, n], X[b, n]> (estimator applied to each channel pair on its own):
+    float32 tensor [r, Cin, B]."""
+    _cl(X, "X"); _cl(Z, "Z")
+    B, Cin, H, W = X.shape
+    r = Z.shape[0]
+    if tuple(Z.shape[1:]) != (Cin, H, W) or Z.dtype != X.dtype:
+        raise ValueError("Z must be (r, Cin, H, W) in X's dtype")
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    S = torch.empty((r, Cin, B), dtype=torch.float32, device=X.device)
+    _check(lib().xconv_sketch_independent(ctypes.byref(desc), X.data_ptr(), Z.data_ptr(), S.data_ptr(), _stream()),
+           "xconv_sketch_independent")
+    return S
+
+
+def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3) -> torch.Tensor:
+    """dW estimate per channel pair from the per-channel sketch: float32 (Cout, Cin, K, K), channels_last."""
+    _cl(dY, "dY"); _cl(Z, "Z")
+    B, Cout, H, Wd = dY.shape
+    r, Cin = Z.shape[0], Z.shape[1]
+    if tuple(sketch.shape) != (r, Cin, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
+        raise ValueError("sketch must be a contiguous float32 [r, Cin, B] tensor")
+    if tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != dY.dtype:
+        raise ValueError("shape or dtype mismatch between dY and Z")
+    K = kernel_size
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K)
+    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    ws = workspace(workspace_bytes(desc, OP_WGRAD_INDEPENDENT), dY.device)
+    _check(lib().xconv_wgrad_independent(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), Z.data_ptr(),
+                                         dW.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_independent")
     return dW
 
 

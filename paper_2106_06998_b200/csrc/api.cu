@@ -396,6 +396,47 @@ __global__ void __launch_bounds__(256) fma_rate_kernel(float* __restrict__ sink,
   sink[(long)blockIdx.x * blockDim.x + threadIdx.x] = t;
 }
 
+// ----------------------------------------------------------------------------------- per-pair ("independent") probing
+
+// Layout of the scratch of xconv_wgrad_independent: header | Xr (the activation rebuilt per channel) | partial sums
+struct IndepPlan { xconv_desc d2; WgradPlan p2; size_t x_off, part_off, bytes; };
+
+static IndepPlan plan_indep(const xconv_desc* d) {
+  IndepPlan ip{};
+  ip.d2 = *d; ip.d2.r = d->B; ip.d2.chan_scale = nullptr;     // the contraction runs over the batch
+  ip.p2 = plan_wgrad_core(&ip.d2);
+  const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
+  const int T = d->KH * d->KW;
+  ip.x_off = WS_HEADER;
+  ip.part_off = ip.x_off + align_up((size_t)d->B * d->H * d->W * d->Cin * es, 256);
+  const size_t part = ip.p2.tc_ct ? ip.p2.t.part_bytes : (size_t)ip.p2.splits * d->Cout * T * d->Cin * sizeof(float);
+  ip.bytes = ip.part_off + align_up(part, 256);
+  return ip;
+}
+
+static xconv_status validate_indep(const xconv_desc* d) {
+  xconv_status s = validate(d);
+  if (s != XCONV_OK) return s;
+  if (d->r > 65535L * IS_JT || d->B > 65535L * IR_BT) return XCONV_ERR_UNSUPPORTED;     // grid z axes
+  return XCONV_OK;
+}
+
+template <typename T>
+static xconv_status run_sketch_indep(const xconv_desc* d, const void* X, const void* Z, float* S, cudaStream_t st) {
+  const long N = (long)d->H * d->W;
+  dim3 grid((unsigned)cdiv(d->B, IS_BT), (unsigned)cdiv(d->Cin, 32), (unsigned)cdiv(d->r, IS_JT));
+  sketch_indep_simt<T><<<grid, 256, 0, st>>>(static_cast<const T*>(X), static_cast<const T*>(Z), S, d->r, d->B, N, d->Cin);
+  return check_launch();
+}
+
+template <typename T>
+static xconv_status run_rebuild_indep(const xconv_desc* d, const float* S, const void* Z, void* Xr, cudaStream_t st) {
+  const long N = (long)d->H * d->W;
+  dim3 grid((unsigned)cdiv(N, 8), (unsigned)cdiv(d->Cin, 32), (unsigned)cdiv(d->B, IR_BT));
+  rebuild_indep_simt<T><<<grid, 256, 0, st>>>(S, static_cast<const T*>(Z), static_cast<T*>(Xr), d->r, d->B, N, d->Cin);
+  return check_launch();
+}
+
 int launches() { return g_launches; }
 void count_launch() { ++g_launches; }
 void set_cuda_error(int e) { g_last_cuda_error = e; }
@@ -420,6 +461,7 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
     case XCONV_OP_BACKPROBE:
     case XCONV_OP_CONTRACT: return plan_wgrad(desc).bytes;
     case XCONV_OP_DGRAD: return conv_ws_bytes(desc, true);
+    case XCONV_OP_WGRAD_INDEPENDENT: return validate_indep(desc) == XCONV_OK ? plan_indep(desc).bytes : 0;
     default: return 0;
   }
 }
@@ -486,6 +528,39 @@ xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, con
   s = run_probes_from_seed(desc, seed, Z, st);
   if (s != XCONV_OK) return s;
   return run_wgrad(desc, sketch, dY, Z, dW, ws, base, st);
+}
+
+xconv_status xconv_sketch_independent(const xconv_desc* desc, const void* X, const void* Z, float* sketch,
+                                      void* cuda_stream) {
+  xconv_status s = validate_indep(desc);
+  if (s != XCONV_OK) return s;
+  if (!X || !Z || !sketch) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(Z) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  return desc->dtype == XCONV_F32 ? run_sketch_indep<float>(desc, X, Z, sketch, st)
+         : desc->dtype == XCONV_F16 ? run_sketch_indep<f16>(desc, X, Z, sketch, st)
+                                    : run_sketch_indep<bf16>(desc, X, Z, sketch, st);
+}
+
+xconv_status xconv_wgrad_independent(const xconv_desc* desc, const float* sketch, const void* dY, const void* Z,
+                                     float* dW, void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate_indep(desc);
+  if (s != XCONV_OK) return s;
+  if (!sketch || !dY || !Z || !dW) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(sketch) || !aligned16(dY) || !aligned16(Z) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
+  const IndepPlan ip = plan_indep(desc);
+  if ((s = validate(&ip.d2)) != XCONV_OK) return s;
+  s = check_ws(ws, ws_bytes, ip.bytes);
+  if (s != XCONV_OK) return s;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* w = static_cast<char*>(ws);
+  s = desc->dtype == XCONV_F32 ? run_rebuild_indep<float>(desc, sketch, Z, w + ip.x_off, st)
+      : desc->dtype == XCONV_F16 ? run_rebuild_indep<f16>(desc, sketch, Z, w + ip.x_off, st)
+                                 : run_rebuild_indep<bf16>(desc, sketch, Z, w + ip.x_off, st);
+  if (s != XCONV_OK) return s;
+  return run_contract(&ip.d2, ip.p2, dY, w + ip.x_off, dW, 1.0f / (float)desc->r, w + ip.part_off, w, st);
 }
 
 xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W, const void* Z, void* Y,

@@ -360,6 +360,94 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Trace estimation per channel pair ("independent" probing, first sentence of the multi-channel case in
+// Section 3): the sketch keeps the input channels apart,
+//   S[j][n][b] = sum_{pixels q} Z[j,q,n] * X[b,q,n],
+// and the estimate of dW[m,n,k] uses only block n of the probing vectors.  Its cheapest order of summation
+// rebuilds every channel of the activation from its own sketch,
+//   Xr[b,q,n] = sum_j S[j][n][b] * Z[j,q,n],
+// and then runs the offset contraction over the batch (dY in the place of L, Xr in the place of Z).
+// Both kernels below put 32 consecutive channels on the lanes of a warp, so every load is one row of
+// channels-last memory.
+// ---------------------------------------------------------------------------------------------
+constexpr int IS_JT = 4, IS_BT = 8;      // probes x samples per thread in the sketch
+template <typename T>
+__global__ void __launch_bounds__(256) sketch_indep_simt(const T* __restrict__ X, const T* __restrict__ Z,
+                                                         float* __restrict__ S, int r, int B, long N, int Cin) {
+  __shared__ float red[8][IS_JT * IS_BT][33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n = blockIdx.y * 32 + lane, b0 = blockIdx.x * IS_BT, j0 = blockIdx.z * IS_JT;
+  const bool live = n < Cin;
+  float acc[IS_JT][IS_BT];
+#pragma unroll
+  for (int j = 0; j < IS_JT; ++j)
+#pragma unroll
+    for (int b = 0; b < IS_BT; ++b) acc[j][b] = 0.f;
+  // the eight warps take the pixels in turn; their sums are added below in warp order
+  for (long q = warp; q < N; q += 8) {
+    float z[IS_JT], x[IS_BT];
+#pragma unroll
+    for (int j = 0; j < IS_JT; ++j) z[j] = (live && j0 + j < r) ? to_f(Z[((long)(j0 + j) * N + q) * Cin + n]) : 0.f;
+#pragma unroll
+    for (int b = 0; b < IS_BT; ++b) x[b] = (live && b0 + b < B) ? to_f(X[((long)(b0 + b) * N + q) * Cin + n]) : 0.f;
+#pragma unroll
+    for (int j = 0; j < IS_JT; ++j)
+#pragma unroll
+      for (int b = 0; b < IS_BT; ++b) acc[j][b] = fmaf(z[j], x[b], acc[j][b]);
+  }
+#pragma unroll
+  for (int j = 0; j < IS_JT; ++j)
+#pragma unroll
+    for (int b = 0; b < IS_BT; ++b) red[warp][j * IS_BT + b][lane] = acc[j][b];
+  __syncthreads();
+  // thread t sums output (t / 32, lane) ... over the eight warps, in order
+  for (int o = warp; o < IS_JT * IS_BT; o += 8) {
+    float t = red[0][o][lane];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) t += red[w][o][lane];
+    const int j = j0 + o / IS_BT, b = b0 + o % IS_BT;
+    if (live && j < r && b < B) S[((long)j * Cin + n) * B + b] = t;
+  }
+}
+
+// Xr[b,q,n] = sum_j S[j][n][b] Z[j,q,n], written in the storage type.  A block owns 32 channels x 8 pixels
+// x 8 samples; the sketch entries of 16 probes at a time are staged in shared memory.
+constexpr int IR_BT = 8, IR_JC = 16;
+template <typename T>
+__global__ void __launch_bounds__(256) rebuild_indep_simt(const float* __restrict__ S, const T* __restrict__ Z,
+                                                          T* __restrict__ Xr, int r, int B, long N, int Cin) {
+  __shared__ float Ss[IR_JC][32][IR_BT + 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int n0 = blockIdx.y * 32, n = n0 + lane, b0 = blockIdx.z * IR_BT;
+  const long q = (long)blockIdx.x * 8 + warp;
+  const bool live = n < Cin && q < N;
+  float acc[IR_BT];
+#pragma unroll
+  for (int b = 0; b < IR_BT; ++b) acc[b] = 0.f;
+  for (int jc = 0; jc < r; jc += IR_JC) {
+    for (int idx = threadIdx.x; idx < IR_JC * 32 * IR_BT; idx += 256) {
+      const int bb = idx % IR_BT, nn = (idx / IR_BT) % 32, jj = idx / (IR_BT * 32);
+      Ss[jj][nn][bb] = (jc + jj < r && n0 + nn < Cin && b0 + bb < B) ? S[((long)(jc + jj) * Cin + n0 + nn) * B + b0 + bb] : 0.f;
+    }
+    __syncthreads();
+    if (live) {
+      const int nj = min(IR_JC, r - jc);
+      for (int jj = 0; jj < nj; ++jj) {
+        const float z = to_f(Z[((long)(jc + jj) * N + q) * Cin + n]);
+#pragma unroll
+        for (int b = 0; b < IR_BT; ++b) acc[b] = fmaf(Ss[jj][lane][b], z, acc[b]);
+      }
+    }
+    __syncthreads();
+  }
+  if (live) {
+#pragma unroll
+    for (int b = 0; b < IR_BT; ++b)
+      if (b0 + b < B) Xr[((long)(b0 + b) * N + q) * Cin + n] = from_f<T>(acc[b]);
+  }
+}
+
 // out[b][j] = in[j][b] for a small [rows][cols] float matrix (the sketch, transposed).
 static __global__ void transpose_f32(const float* __restrict__ in, float* __restrict__ out, int rows, int cols) {
   const long i = (long)blockIdx.x * blockDim.x + threadIdx.x;
