@@ -39,6 +39,8 @@ balance and independence of the signs, and by the unbiasedness of the estimator 
 sketch_independent and wgrad_estimate_independent (the estimator applied to each channel pair on its own) are
 pinned by exact recovery with one orthogonal basis per channel, by unbiasedness with the crosstalk-free
 Hutchinson variance, and by their reduction to the multi-channel functions for a single input channel.
+The functions for volumes (shift3, conv_forward3d, dw_exact3d, dx_exact3d, wgrad_contract3d, wgrad_estimate3d) are
+pinned by brute-force loops, by their reduction to the two-dimensional functions at depth 1, and by exact recovery.
 rel_fro, the metric every parity verdict passes through, is pinned on a hand-computed pair.
 No function here is "parity unpinned".
 """
@@ -183,6 +185,91 @@ def xconv_layer(X, W, dY, Z, pad=None, circular=False, scale=None):
     dW = wgrad_estimate(S, dY, Z, KH, KW, pad, circular, scale)
     dX = dx_exact(dY, W, pad, circular)
     return Y, S, dW, dX
+
+
+# --- three-dimensional layers (volumes): the same method with one more shift axis ---------------------
+# Arrays are (batch, channel, z, y, x); kernels (Cout, Cin, KD, KH, KW).  The sketch and the back-probe do not
+# see the geometry (``sketch`` and ``backprobe`` above flatten every pixel axis), only the shifts do.
+
+def shift3(A, dz, dy, dx, circular=False):
+    """(shift3 A)[..., z, y, x] = A[..., z+dz, y+dy, x+dx]; zero outside the volume unless ``circular``
+    (the shift T_k(i) of Section 3 for a three-dimensional offset k(i))."""
+    A = np.asarray(A, dtype=F64)
+    if circular:
+        return np.roll(A, shift=(-dz, -dy, -dx), axis=(-3, -2, -1))
+    D = A.shape[-3]
+    out = np.zeros_like(A)
+    z0, z1 = max(0, -dz), min(D, D - dz)
+    if z0 < z1:
+        out[..., z0:z1, :, :] = shift(A[..., z0 + dz:z1 + dz, :, :], dy, dx, False)
+    return out
+
+
+def _pads3(K, pad):
+    return tuple((k - 1) // 2 for k in K) if pad is None else tuple(pad)
+
+
+def conv_forward3d(X, W, pad=None, circular=False):
+    """Eq. (5) for volumes: Y[b,m,z,y,x] = sum_{n,kz,ky,kx} W[m,n,kz,ky,kx] X[b,n,z+kz-pd,y+ky-ph,x+kx-pw]."""
+    X = np.asarray(X, F64)
+    W = np.asarray(W, F64)
+    Cout, Cin, KD, KH, KW = W.shape
+    pd, ph, pw = _pads3((KD, KH, KW), pad)
+    Y = np.zeros((X.shape[0], Cout) + X.shape[2:], F64)
+    for kz in range(KD):
+        for ky in range(KH):
+            for kx in range(KW):
+                Y += np.einsum("mn,bnzyx->bmzyx", W[:, :, kz, ky, kx], shift3(X, kz - pd, ky - ph, kx - pw, circular))
+    return Y
+
+
+def dw_exact3d(X, dY, K=(3, 3, 3), pad=None, circular=False):
+    """Eq. (2) for volumes: dW[m,n,kz,ky,kx] = sum_{b,z,y,x} dY[b,m,z,y,x] X[b,n,z+kz-pd,y+ky-ph,x+kx-pw]."""
+    X = np.asarray(X, F64)
+    dY = np.asarray(dY, F64)
+    pd, ph, pw = _pads3(K, pad)
+    dW = np.zeros((dY.shape[1], X.shape[1]) + tuple(K), F64)
+    for kz in range(K[0]):
+        for ky in range(K[1]):
+            for kx in range(K[2]):
+                dW[:, :, kz, ky, kx] = np.einsum("bmzyx,bnzyx->mn", dY, shift3(X, kz - pd, ky - ph, kx - pw, circular))
+    return dW
+
+
+def dx_exact3d(dY, W, pad=None, circular=False):
+    """Adjoint of ``conv_forward3d`` in X: dX[b,n,u] = sum_{m,k} W[m,n,k] dY[b,m,u-k+p] (standard back-propagation)."""
+    dY = np.asarray(dY, F64)
+    W = np.asarray(W, F64)
+    Cout, Cin, KD, KH, KW = W.shape
+    pd, ph, pw = _pads3((KD, KH, KW), pad)
+    dX = np.zeros((dY.shape[0], Cin) + dY.shape[2:], F64)
+    for kz in range(KD):
+        for ky in range(KH):
+            for kx in range(KW):
+                dX += np.einsum("mn,bmzyx->bnzyx", W[:, :, kz, ky, kx], shift3(dY, -(kz - pd), -(ky - ph), -(kx - pw), circular))
+    return dX
+
+
+def wgrad_contract3d(L, Z, K=(3, 3, 3), pad=None, circular=False, scale=None):
+    """Algorithm 1 backward step 4 for volumes:
+    dW[m,n,kz,ky,kx] = scale[n] * sum_{j,z,y,x} L[j,m,z,y,x] Z[j,n,z+kz-pd,y+ky-ph,x+kx-pw], scale = 1/r unless given."""
+    L = np.asarray(L, F64)
+    Z = np.asarray(Z, F64)
+    pd, ph, pw = _pads3(K, pad)
+    if scale is None:
+        scale = np.full(Z.shape[1], 1.0 / Z.shape[0])
+    dW = np.zeros((L.shape[1], Z.shape[1]) + tuple(K), F64)
+    for kz in range(K[0]):
+        for ky in range(K[1]):
+            for kx in range(K[2]):
+                Zs = shift3(Z, kz - pd, ky - ph, kx - pw, circular)
+                dW[:, :, kz, ky, kx] = np.einsum("jmzyx,jnzyx->mn", L, Zs) * scale[None, :]
+    return dW
+
+
+def wgrad_estimate3d(S, dY, Z, K=(3, 3, 3), pad=None, circular=False, scale=None):
+    """Algorithm 1 backward steps 3-4 for volumes (``sketch`` and ``backprobe`` serve any number of pixel axes)."""
+    return wgrad_contract3d(backprobe(S, dY), Z, K, pad, circular, scale)
 
 
 # --- trace estimation applied to every input/output channel pair on its own ---------------------------

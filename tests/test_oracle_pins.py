@@ -490,3 +490,69 @@ def test_independent_probing_is_unbiased_with_the_crosstalk_free_variance():
                     assert abs(z) < 4.5, (m, n, ky, kx, z)
                     assert 0.8 < var[m, n, ky, kx] / v < 1.25, (m, n, ky, kx, var[m, n, ky, kx], v)
                     assert v < _closed_form_variance(C, n, False)
+
+
+# ---------------------------------------------------------------- volumes (three-dimensional layers)
+
+def _tiny3(seed, B=2, Cin=2, Cout=3, D=3, H=4, W=3, K=(3, 3, 3)):
+    g = _rng(seed)
+    return (g.standard_normal((B, Cin, D, H, W)), g.standard_normal((Cout, Cin) + K), g.standard_normal((B, Cout, D, H, W)))
+
+
+@pytest.mark.parametrize("circular", [False, True])
+@pytest.mark.parametrize("K", [(3, 3, 3), (1, 3, 3), (3, 1, 5)])
+def test_volume_functions_against_brute_force_loops(K, circular):
+    X, Wt, dY = _tiny3(60, K=K)
+    B, Cin, D, H, W = X.shape
+    Cout = Wt.shape[0]
+    pd, ph, pw = [(k - 1) // 2 for k in K]
+    Y = np.zeros((B, Cout, D, H, W)); dW = np.zeros_like(Wt); dX = np.zeros_like(X)
+
+    def src(z, y, x, kz, ky, kx):
+        zz, yy, xx = z + kz - pd, y + ky - ph, x + kx - pw
+        if circular:
+            return zz % D, yy % H, xx % W
+        return (zz, yy, xx) if (0 <= zz < D and 0 <= yy < H and 0 <= xx < W) else None
+
+    for b in range(B):
+        for m in range(Cout):
+            for n in range(Cin):
+                for z in range(D):
+                    for y in range(H):
+                        for x in range(W):
+                            for kz in range(K[0]):
+                                for ky in range(K[1]):
+                                    for kx in range(K[2]):
+                                        s_ = src(z, y, x, kz, ky, kx)
+                                        if s_ is None:
+                                            continue
+                                        Y[b, m, z, y, x] += Wt[m, n, kz, ky, kx] * X[(b, n) + s_]
+                                        dW[m, n, kz, ky, kx] += dY[b, m, z, y, x] * X[(b, n) + s_]
+                                        dX[(b, n) + s_] += Wt[m, n, kz, ky, kx] * dY[b, m, z, y, x]
+    np.testing.assert_allclose(O.conv_forward3d(X, Wt, circular=circular), Y, atol=1e-11)
+    np.testing.assert_allclose(O.dw_exact3d(X, dY, K, circular=circular), dW, atol=1e-11)
+    np.testing.assert_allclose(O.dx_exact3d(dY, Wt, circular=circular), dX, atol=1e-11)
+
+
+def test_volume_functions_reduce_to_the_planar_ones_at_depth_one():
+    X, Wt, dY = _tiny(seed=61, B=2, Cin=3, Cout=2, H=5, W=4)
+    Z = _rng(62).standard_normal((6, 3, 5, 4))
+    X3, W3, dY3, Z3 = X[:, :, None], Wt[:, :, None], dY[:, :, None], Z[:, :, None]
+    np.testing.assert_allclose(O.conv_forward3d(X3, W3)[:, :, 0], O.conv_forward(X, Wt), atol=1e-12)
+    np.testing.assert_allclose(O.dx_exact3d(dY3, W3)[:, :, 0], O.dx_exact(dY, Wt), atol=1e-12)
+    np.testing.assert_allclose(O.dw_exact3d(X3, dY3, (1, 3, 3))[:, :, 0], O.dw_exact(X, dY), atol=1e-12)
+    S = O.sketch(X3, Z3)
+    np.testing.assert_allclose(S, O.sketch(X, Z), atol=1e-12)
+    np.testing.assert_allclose(O.wgrad_estimate3d(S, dY3, Z3, (1, 3, 3))[:, :, 0], O.wgrad_estimate(S, dY, Z), atol=1e-12)
+
+
+def test_volume_estimator_recovers_the_exact_gradient_with_an_orthogonal_basis():
+    X, Wt, dY = _tiny3(63, B=2, Cin=2, Cout=2, D=2, H=3, W=2)
+    n = 2 * 2 * 3 * 2
+    Q, _ = np.linalg.qr(_rng(64).standard_normal((n, n)))
+    Z = (np.sqrt(n) * Q.T).reshape(n, 2, 2, 3, 2)
+    est = O.wgrad_estimate3d(O.sketch(X, Z), dY, Z)
+    np.testing.assert_allclose(est, O.dw_exact3d(X, dY), atol=1e-10)
+    # a wrong sign of the depth shift would not recover it
+    wrong = O.wgrad_contract3d(O.backprobe(O.sketch(X, Z), dY), Z[:, :, ::-1])
+    assert O.rel_fro(wrong, O.dw_exact3d(X, dY)) > 0.1
