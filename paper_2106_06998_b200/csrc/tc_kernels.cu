@@ -27,6 +27,7 @@
 #include <cudaTypedefs.h>
 
 #include <algorithm>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -100,6 +101,7 @@ struct TcParams {
   int z_is_a;              // SKETCH: Z is the A operand (probes on the MMA rows) instead of the B operand
   long z_row_len;          // entries of one probing vector, H*W*Cin
   long rows_z;             // probing vectors (rows of Z)
+  int pf_ahead;            // BACKPROBE: stages by which L2 prefetches of the dY tiles run ahead of their copies (0: none)
   int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
@@ -199,6 +201,11 @@ __device__ __forceinline__ void bulk_wait_read_upto(int pending) {
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// Ask L2 for a box ahead of its copy into shared memory (a hint: no completion, no shared memory).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -374,7 +381,7 @@ __device__ __forceinline__ bool umma_halves_items(int nkb, int& s, uint32_t& par
 }
 
 // Two floats rounded to the 16-bit storage type, packed (first in the low half).
-__device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, int f16) {
+__device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, bool f16) {
   if (f16) { __half2 h = __floats2half2_rn(__uint_as_float(a), __uint_as_float(b)); return *reinterpret_cast<uint32_t*>(&h); }
   __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
   return *reinterpret_cast<uint32_t*>(&h);
@@ -426,6 +433,9 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
 
 // ------------------------------------------------------------------------------------ the kernel
 
+// F16: the 16-bit storage type is float16 instead of bfloat16 (a compile-time constant, so that the epilogues'
+// conversions carry no selection between the two).
+template <bool F16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const TcParams p) {
@@ -551,7 +561,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   } else if (warp == 1 && p.mode == MODE_CONTRACT && p.halves) {
     // ------------------------------------------------------------------ MMA issuer, k-blocks in two halves
     if (lane == 0) {
-      const uint32_t idesc = (1u << 4) | (p.f16 ? 0u : (1u << 7) | (1u << 10)) | (1u << 15) | (1u << 16) |
+      const uint32_t idesc = (1u << 4) | (F16 ? 0u : (1u << 7) | (1u << 10)) | (1u << 15) | (1u << 16) |
                              ((uint32_t)(p.tile_n >> 3) << 17) | ((uint32_t)(TILE_M >> 4) << 24);
       const uint32_t step = p.mn_step >> 4;                                   // 16 rows
       const uint32_t a_lo0 = (p.a_lbo >> 4) << 16, b_lo0 = (p.b_lbo >> 4) << 16;
@@ -667,6 +677,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // dY tile: one box (64 positions x k rows) per block of the column tile, one behind the other
             for (int b = 0; b < w.nblk; ++b)
               tma_load_3d(b_dst + (uint32_t)b * p.b_box_bytes, &map_b, 0, kc, w.blk0 + b, &full_bar[s]);
+            if (p.pf_ahead > 0) {            // the dY boxes of the stage pf_ahead stages on, into L2
+              const long ita = it + p.pf_ahead;
+              const long ua = blockIdx.x + (long)gridDim.x * (ita / p.kblocks);
+              if (ua < p.units) {
+                const Unit wa = decode_unit(p, ua);
+                const int kca = (int)(ita % p.kblocks) * p.ksteps * 16;
+                for (int b = 0; b < wa.nblk; ++b) tma_prefetch_3d(&map_b, 0, kca, wa.blk0 + b);
+              }
+            }
             kc += p.ksteps * 16;
           } else if (p.mode == MODE_CONV) {
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
@@ -697,7 +716,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       // instruction descriptor: float accumulator (bit 4), A and B formats (bits 7-9, 10-12: 0 = float16, 1 = bfloat16,
       // always the same for both), operand majorness (bits 15, 16), N >> 3 (bits 17-22), M >> 4 (bits 24-28)
-      const uint32_t idesc = (1u << 4) | (p.f16 ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)p.a_mn_major << 15) |
+      const uint32_t idesc = (1u << 4) | (F16 ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)p.a_mn_major << 15) |
                              ((uint32_t)p.b_mn_major << 16) | ((uint32_t)(p.tile_n >> 3) << 17) |
                              ((uint32_t)(TILE_M >> 4) << 24);
       // Shared-memory descriptor (128-byte swizzle): start address >> 4 | (lbo >> 4) << 16 in the low
@@ -829,7 +848,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
         const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
         const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
-        const uint32_t z_ones = p.f16 ? 0x3C003C00u : 0x3F803F80u;
+        const uint32_t z_ones = F16 ? 0x3C003C00u : 0x3F803F80u;
         long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
         for (int i = 0; i < w.nkb && ok; ++i) {
           if (gen_fill > 0) {
@@ -899,8 +918,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               for (int i = 0; i < 32; i += 8) {
                 const uint32_t sdst = rowbase + ((((uint32_t)half * 4u + (uint32_t)(i >> 3)) ^ ((uint32_t)lane & 7u)) << 4);
                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sdst),
-                             "r"(pack2(v[i + 0], v[i + 1], p.f16)), "r"(pack2(v[i + 2], v[i + 3], p.f16)),
-                             "r"(pack2(v[i + 4], v[i + 5], p.f16)), "r"(pack2(v[i + 6], v[i + 7], p.f16)) : "memory");
+                             "r"(pack2(v[i + 0], v[i + 1], F16)), "r"(pack2(v[i + 2], v[i + 3], F16)),
+                             "r"(pack2(v[i + 4], v[i + 5], F16)), "r"(pack2(v[i + 6], v[i + 7], F16)) : "memory");
               }
             }
             fence_async_smem();
@@ -944,15 +963,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
                   uint4 o;
-                  o.x = pack2(v[i + 0], v[i + 1], p.f16); o.y = pack2(v[i + 2], v[i + 3], p.f16);
-                  o.z = pack2(v[i + 4], v[i + 5], p.f16); o.w = pack2(v[i + 6], v[i + 7], p.f16);
+                  o.x = pack2(v[i + 0], v[i + 1], F16); o.y = pack2(v[i + 2], v[i + 3], F16);
+                  o.z = pack2(v[i + 4], v[i + 5], F16); o.w = pack2(v[i + 6], v[i + 7], F16);
                   *reinterpret_cast<uint4*>(dst + i) = o;
                 }
               } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i)
                   if (i < nc && col0 + c + i < p.cols)
-                    reinterpret_cast<unsigned short*>(dst)[i] = (unsigned short)(pack2(v[i], v[i], p.f16) & 0xFFFFu);
+                    reinterpret_cast<unsigned short*>(dst)[i] = (unsigned short)(pack2(v[i], v[i], F16) & 0xFFFFu);
               }
             }
           } else {
@@ -1127,12 +1146,13 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
                            cudaStream_t st, const CUtensorMap* mc = nullptr) {
   const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_bytes + p.smem_pad;
   if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
-  cudaError_t e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
+  void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, TcParams) = p.f16 ? tc_gemm_kernel<true> : tc_gemm_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   TcParams q = p;
   q.tag = call_tag();
   if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
-  e = launch_pdl(tc_gemm_kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, mc ? *mc : ma, q);
+  e = launch_pdl(kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, mc ? *mc : ma, q);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
@@ -1432,7 +1452,10 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st, &mc);
+  long grid = std::min<long>(p.units, (long)NUM_SMS);
+  if (const char* e = getenv("XC_BP_GRID")) grid = std::max(1L, std::min(grid, atol(e)));
+  if (const char* e = getenv("XC_BP_PF")) p.pf_ahead = atoi(e);
+  return launch(ma, mb, p, (unsigned)grid, st, &mc);
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,

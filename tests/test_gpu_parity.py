@@ -12,7 +12,7 @@ import __graft_entry__ as entry
 from oracle import xconv_oracle as O
 from paper_2106_06998_b200 import binding as xb
 from paper_2106_06998_b200 import inputs
-from tests._util import TOL, TOL_SKETCH, check, dev, host, sketch_oracle_chunked
+from tests._util import TOL, TOL_SKETCH, check, dev, host, sketch_oracle_chunked, sketch_tol
 
 pytestmark = pytest.mark.gpu
 
@@ -239,7 +239,7 @@ def test_full_size_sampled(cfg, r):
     torch.cuda.synchronize()
     assert xb.workspace_status(xb.workspace(256, S.device)) == 0
     So = sketch_oracle_chunked(lay["X"], lay["Z"])
-    check("sketch", host(S), So, TOL_SKETCH)
+    check("sketch", host(S), So, sketch_tol(lay["Cin"] * lay["H"] * lay["width"]))
     g = np.random.Generator(np.random.PCG64(cfg * 1000 + r))
     # output / input channels at the ends of the channel range, either side of the 128-row tile boundary, and at random
     ms = np.unique(np.concatenate([[0, lay["Cout"] - 1, min(127, lay["Cout"] - 1), min(128, lay["Cout"] - 1)],
