@@ -85,7 +85,14 @@ typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TC
                XCONV_ENGINE_TCGEN05_F16 = 3 } xconv_engine;
 
 /* One convolutional layer: stride 1, dilation 1, one group, no bias, "same" output size
- * (2*pad_h = KH-1, 2*pad_w = KW-1; KH = KW in {1, 3, 5}). */
+ * (2*pad_h = KH-1, 2*pad_w = KW-1; KH = KW in {1, 3, 5}).
+ *
+ * Volumes (three-dimensional layers, as in the paper's 3-D segmentation experiment, Section 5.5): set D > 1.
+ * Every tensor gains a depth axis between the sample (or probe) index and the rows: X, dY, Y, dX
+ * [B,D,H,W,C], Z [r,D,H,W,Cin], W and dW [Cout,KD,KH,KW,Cin] (torch's channels_last_3d of NCDHW / OIDHW),
+ * and every formula above gains the matching sum over kz and shift z + kz - pad_d.  KD = 3 (with KH = KW = 3,
+ * pad_d = 1) is a 3 x 3 x 3 kernel; KD = 1 (pad_d = 0) applies a planar kernel to every plane.  D, KD and
+ * pad_d of 0 (a zero-initialised tail) mean a planar layer, the same as D = KD = 1. */
 typedef struct {
   int32_t B, Cin, Cout, H, W;
   int32_t KH, KW, pad_h, pad_w;
@@ -93,6 +100,7 @@ typedef struct {
   int32_t dtype;            /* xconv_dtype: storage of X, W, dY, Z, Y, dX */
   int32_t circular;         /* must be 0 (truncating shifts) */
   const float* chan_scale;  /* NULL: scale 1/r.  Else device pointer to Cin floats (Eq. 8). */
+  int32_t D, KD, pad_d;     /* depth of the volume and of the kernel; 0 or 1: planar layer */
 } xconv_desc;
 
 /* Scratch bytes `op` needs for this layer (0 is possible).  Returns 0 for an invalid descriptor. */

@@ -32,7 +32,8 @@ EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_
 class XConvDesc(Structure):
     _fields_ = [("B", c_int32), ("Cin", c_int32), ("Cout", c_int32), ("H", c_int32), ("W", c_int32),
                 ("KH", c_int32), ("KW", c_int32), ("pad_h", c_int32), ("pad_w", c_int32), ("r", c_int32),
-                ("dtype", c_int32), ("circular", c_int32), ("chan_scale", c_void_p)]
+                ("dtype", c_int32), ("circular", c_int32), ("chan_scale", c_void_p),
+                ("D", c_int32), ("KD", c_int32), ("pad_d", c_int32)]
 
 
 class XConvError(RuntimeError):
@@ -109,18 +110,34 @@ def _dtype_code(t: torch.dtype) -> int:
     raise TypeError(f"libxconv stores float32, bfloat16 or float16, got {t}")
 
 
-def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None) -> XConvDesc:
+def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1) -> XConvDesc:
+    """Layer descriptor; D > 1 describes a volume (tensors gain a depth axis), KD its kernel depth (1 or 3)."""
     code = dtype if isinstance(dtype, int) else _dtype_code(dtype)
     cs = chan_scale.data_ptr() if chan_scale is not None else None
-    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs)
+    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs, D, KD, (KD - 1) // 2)
 
 
 def _cl(t: torch.Tensor, name: str) -> torch.Tensor:
+    """Checks the layout: 4-d tensors in channels_last, 5-d tensors (volumes) in channels_last_3d."""
     if not t.is_cuda:
         raise ValueError(f"{name} must be a CUDA tensor")
-    if t.dim() != 4 or not t.is_contiguous(memory_format=torch.channels_last):
-        raise ValueError(f"{name} must be a 4-d tensor in torch.channels_last memory format")
+    fmt = {4: torch.channels_last, 5: torch.channels_last_3d}.get(t.dim())
+    if fmt is None or not t.is_contiguous(memory_format=fmt):
+        raise ValueError(f"{name} must be a 4-d tensor in torch.channels_last or a 5-d tensor in "
+                         "torch.channels_last_3d memory format")
     return t
+
+
+def _geo(t: torch.Tensor):
+    """(D, H, W) of a 4-d (planar, D = 1) or 5-d (volume) tensor."""
+    return (1, t.shape[2], t.shape[3]) if t.dim() == 4 else (t.shape[2], t.shape[3], t.shape[4])
+
+
+def _like(shape_head, geo, dim, **kw):
+    """An empty tensor (head..., [D,] H, W) in the channels-last format of a `dim`-d tensor."""
+    D, H, W = geo
+    shape = tuple(shape_head) + ((H, W) if dim == 4 else (D, H, W))
+    return torch.empty(shape, memory_format=torch.channels_last if dim == 4 else torch.channels_last_3d, **kw)
 
 
 def _stream() -> int:
@@ -215,13 +232,14 @@ def last_launch_count() -> int:
 # ------------------------------------------------------------------ same names as the C ABI
 
 def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
-    """S = Z^T X (Algorithm 1 forward step 3): float32 tensor [r, B]."""
+    """S = Z^T X (Algorithm 1 forward step 3): float32 tensor [r, B].  X (B, Cin, [D,] H, W), Z (r, Cin, [D,] H, W)."""
     _cl(X, "X"); _cl(Z, "Z")
-    B, Cin, H, W = X.shape
+    B, Cin = X.shape[:2]
+    D, H, W = _geo(X)
     r = Z.shape[0]
-    if tuple(Z.shape[1:]) != (Cin, H, W) or Z.dtype != X.dtype:
-        raise ValueError("Z must be (r, Cin, H, W) in X's dtype")
-    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    if tuple(Z.shape[1:]) != tuple(X.shape[1:]) or Z.dtype != X.dtype:
+        raise ValueError("Z must be (r, Cin, [D,] H, W) in X's dtype")
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype, D=D)
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
     ws = workspace(workspace_bytes(desc, OP_SKETCH), X.device)
     sketch_into(desc, X, Z, S, ws)
@@ -285,15 +303,18 @@ def xconv_sketch_static(X: torch.Tensor, Z: torch.Tensor, out: torch.Tensor | No
 
 
 def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
-    """Y = conv(X, W) and the sketch S = Z^T X (Algorithm 1 forward steps 1 and 3)."""
+    """Y = conv(X, W) and the sketch S = Z^T X (Algorithm 1 forward steps 1 and 3).  5-d tensors are volumes."""
     _cl(X, "X"); _cl(W, "W"); _cl(Z, "Z")
-    B, Cin, H, Wd = X.shape
-    Cout, _, K, _ = W.shape
+    B, Cin = X.shape[:2]
+    D, H, Wd = _geo(X)
+    Cout, K = W.shape[0], W.shape[-1]
+    KD = W.shape[2] if W.dim() == 5 else 1
     r = Z.shape[0]
-    if W.shape[1] != Cin or tuple(Z.shape[1:]) != (Cin, H, Wd) or W.dtype != X.dtype or Z.dtype != X.dtype:
+    if (W.shape[1] != Cin or W.dim() != X.dim() or tuple(Z.shape[1:]) != tuple(X.shape[1:]) or W.dtype != X.dtype
+            or Z.dtype != X.dtype):
         raise ValueError("shape or dtype mismatch between X, W and Z")
-    desc = make_desc(B, Cin, Cout, H, Wd, r, X.dtype, K)
-    Y = torch.empty((B, Cout, H, Wd), dtype=X.dtype, device=X.device, memory_format=torch.channels_last)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, X.dtype, K, D=D, KD=KD)
+    Y = _like((B, Cout), (D, H, Wd), X.dim(), dtype=X.dtype, device=X.device)
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
     ws = workspace(workspace_bytes(desc, OP_FORWARD), X.device)
     forward_into(desc, X, W, Z, Y, S, ws)
@@ -301,20 +322,21 @@ def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
 
 
 def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
-                chan_scale: torch.Tensor | None = None) -> torch.Tensor:
-    """dW estimate (Algorithm 1 backward steps 3-4): float32 (Cout, Cin, K, K), channels_last."""
+                chan_scale: torch.Tensor | None = None, kernel_depth: int = 1) -> torch.Tensor:
+    """dW estimate (Algorithm 1 backward steps 3-4): float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY"); _cl(Z, "Z")
-    B, Cout, H, Wd = dY.shape
+    B, Cout = dY.shape[:2]
+    D, H, Wd = _geo(dY)
     r, Cin = Z.shape[0], Z.shape[1]
     if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
         raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
-    if tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != dY.dtype:
+    if tuple(Z.shape[2:]) != tuple(dY.shape[2:]) or Z.dtype != dY.dtype:
         raise ValueError("shape or dtype mismatch between dY and Z")
     if chan_scale is not None and (chan_scale.dtype != torch.float32 or chan_scale.numel() != Cin):
         raise ValueError("chan_scale must hold Cin float32 values")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale)
-    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale, D=D, KD=kernel_depth)
+    dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
     wgrad_into(desc, sketch, dY, Z, dW, ws)
     return dW
@@ -324,29 +346,32 @@ def xconv_sketch_independent(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
     """Per-channel sketch S[j, n, b] = <Z[j, n], X[b, n]> (estimator applied to each channel pair on its own):
     float32 tensor [r, Cin, B]."""
     _cl(X, "X"); _cl(Z, "Z")
-    B, Cin, H, W = X.shape
+    B, Cin = X.shape[:2]
+    D, H, W = _geo(X)
     r = Z.shape[0]
-    if tuple(Z.shape[1:]) != (Cin, H, W) or Z.dtype != X.dtype:
-        raise ValueError("Z must be (r, Cin, H, W) in X's dtype")
-    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    if tuple(Z.shape[1:]) != tuple(X.shape[1:]) or Z.dtype != X.dtype:
+        raise ValueError("Z must be (r, Cin, [D,] H, W) in X's dtype")
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype, D=D)
     S = torch.empty((r, Cin, B), dtype=torch.float32, device=X.device)
     _check(lib().xconv_sketch_independent(ctypes.byref(desc), X.data_ptr(), Z.data_ptr(), S.data_ptr(), _stream()),
            "xconv_sketch_independent")
     return S
 
 
-def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3) -> torch.Tensor:
-    """dW estimate per channel pair from the per-channel sketch: float32 (Cout, Cin, K, K), channels_last."""
+def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
+                            kernel_depth: int = 1) -> torch.Tensor:
+    """dW estimate per channel pair from the per-channel sketch: float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY"); _cl(Z, "Z")
-    B, Cout, H, Wd = dY.shape
+    B, Cout = dY.shape[:2]
+    D, H, Wd = _geo(dY)
     r, Cin = Z.shape[0], Z.shape[1]
     if tuple(sketch.shape) != (r, Cin, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
         raise ValueError("sketch must be a contiguous float32 [r, Cin, B] tensor")
-    if tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != dY.dtype:
+    if tuple(Z.shape[2:]) != tuple(dY.shape[2:]) or Z.dtype != dY.dtype:
         raise ValueError("shape or dtype mismatch between dY and Z")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K)
-    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth)
+    dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD_INDEPENDENT), dY.device)
     _check(lib().xconv_wgrad_independent(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), Z.data_ptr(),
                                          dW.data_ptr(), ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_independent")
@@ -354,30 +379,32 @@ def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Ten
 
 
 def xconv_backprobe(sketch: torch.Tensor, dY: torch.Tensor) -> torch.Tensor:
-    """L = S dY^T (Algorithm 1 backward step 3): (r, Cout, H, W) in dY's dtype, channels_last."""
+    """L = S dY^T (Algorithm 1 backward step 3): (r, Cout, [D,] H, W) in dY's dtype, channels-last."""
     _cl(dY, "dY")
-    B, Cout, H, Wd = dY.shape
+    B, Cout = dY.shape[:2]
+    D, H, Wd = _geo(dY)
     r = sketch.shape[0]
     if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
         raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
-    desc = make_desc(B, 1, Cout, H, Wd, r, dY.dtype)
-    L = torch.empty((r, Cout, H, Wd), dtype=dY.dtype, device=dY.device, memory_format=torch.channels_last)
+    desc = make_desc(B, 1, Cout, H, Wd, r, dY.dtype, D=D)
+    L = _like((r, Cout), (D, H, Wd), dY.dim(), dtype=dY.dtype, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
     backprobe_into(desc, sketch, dY, L, ws)
     return L
 
 
 def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
-                   chan_scale: torch.Tensor | None = None) -> torch.Tensor:
+                   chan_scale: torch.Tensor | None = None, kernel_depth: int = 1) -> torch.Tensor:
     """dW[m,n,k] = scale[n] * sum L[j,m,.] Z[j,n,.+k] (Algorithm 1 backward step 4)."""
     _cl(L, "L"); _cl(Z, "Z")
-    r, Cout, H, Wd = L.shape
+    r, Cout = L.shape[:2]
+    D, H, Wd = _geo(L)
     Cin = Z.shape[1]
-    if Z.shape[0] != r or tuple(Z.shape[2:]) != (H, Wd) or Z.dtype != L.dtype:
+    if Z.shape[0] != r or tuple(Z.shape[2:]) != tuple(L.shape[2:]) or Z.dtype != L.dtype:
         raise ValueError("shape or dtype mismatch between L and Z")
     K = kernel_size
-    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale)
-    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=L.device, memory_format=torch.channels_last)
+    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale, D=D, KD=kernel_depth)
+    dW = _like((Cout, Cin), (kernel_depth, K, K), L.dim(), dtype=torch.float32, device=L.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), L.device)
     contract_into(desc, L, Z, dW, ws)
     return dW
@@ -386,12 +413,14 @@ def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
 def xconv_dgrad(dY: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
     """Exact dX (transposed convolution)."""
     _cl(dY, "dY"); _cl(W, "W")
-    B, Cout, H, Wd = dY.shape
-    _, Cin, K, _ = W.shape
-    if W.shape[0] != Cout or W.dtype != dY.dtype:
+    B, Cout = dY.shape[:2]
+    D, H, Wd = _geo(dY)
+    Cin, K = W.shape[1], W.shape[-1]
+    KD = W.shape[2] if W.dim() == 5 else 1
+    if W.shape[0] != Cout or W.dtype != dY.dtype or W.dim() != dY.dim():
         raise ValueError("shape or dtype mismatch between dY and W")
-    desc = make_desc(B, Cin, Cout, H, Wd, 1, dY.dtype, K)
-    dX = torch.empty((B, Cin, H, Wd), dtype=dY.dtype, device=dY.device, memory_format=torch.channels_last)
+    desc = make_desc(B, Cin, Cout, H, Wd, 1, dY.dtype, K, D=D, KD=KD)
+    dX = _like((B, Cin), (D, H, Wd), dY.dim(), dtype=dY.dtype, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_DGRAD), dY.device)
     dgrad_into(desc, dY, W, dX, ws)
     return dX
@@ -409,10 +438,10 @@ def xconv_sketch_wgrad_host(desc: XConvDesc, hX, hdY, hZ, hS, hdW, arena: torch.
 
 
 def to_device(a, dtype: str, device="cuda") -> torch.Tensor:
-    """Host float32 array (logical NCHW, already rounded to ``dtype``) -> channels_last device tensor."""
+    """Host float32 array (logical NCHW or NCDHW, already rounded to ``dtype``) -> channels-last device tensor."""
     t = torch.from_numpy(a).to(device)
     if dtype == "bf16":
         t = t.to(torch.bfloat16)
     elif dtype == "f16":
         t = t.to(torch.float16)
-    return t.contiguous(memory_format=torch.channels_last)
+    return t.contiguous(memory_format=torch.channels_last if t.dim() == 4 else torch.channels_last_3d)

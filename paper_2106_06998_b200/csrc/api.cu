@@ -35,27 +35,60 @@ static void new_call() {
 }
 unsigned int call_tag() { return g_tag; }
 
+// Depth of the volume and of the kernel (0 and 1 both mean a planar layer).
+static inline int depth(const xconv_desc* d) { return d->D > 1 ? d->D : 1; }
+static inline int kdepth(const xconv_desc* d) { return d->KD > 1 ? d->KD : 1; }
+
 static xconv_status validate(const xconv_desc* d) {
   if (!d) return XCONV_ERR_INVALID_ARG;
   if (d->B <= 0 || d->Cin <= 0 || d->Cout <= 0 || d->H <= 0 || d->W <= 0 || d->r <= 0 || d->KH <= 0 || d->KW <= 0)
     return XCONV_ERR_INVALID_ARG;
   if (d->dtype != XCONV_F32 && d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return XCONV_ERR_INVALID_ARG;
-  if (d->pad_h < 0 || d->pad_w < 0) return XCONV_ERR_INVALID_ARG;
+  if (d->pad_h < 0 || d->pad_w < 0 || d->D < 0 || d->KD < 0 || d->pad_d < 0) return XCONV_ERR_INVALID_ARG;
   if (d->circular != 0) return XCONV_ERR_UNSUPPORTED;
   if (d->KH != d->KW || (d->KH != 1 && d->KH != 3 && d->KH != 5)) return XCONV_ERR_UNSUPPORTED;
   if (2 * d->pad_h != d->KH - 1 || 2 * d->pad_w != d->KW - 1) return XCONV_ERR_UNSUPPORTED;
+  // kernels over volumes: 3 x 3 x 3, or planar kernels (1 x K x K) applied to every plane
+  if (kdepth(d) != 1 && !(kdepth(d) == 3 && d->KH == 3)) return XCONV_ERR_UNSUPPORTED;
+  if (2 * d->pad_d != kdepth(d) - 1) return XCONV_ERR_UNSUPPORTED;
   // 32-bit grid and index limits of the kernels.  r, B and the channel counts land on the y axis of a
   // grid (at most 65535 blocks of 16 or more) in the FP32-FMA kernels, and r and B trade places when
   // xconv_wgrad sums over the probes first.
-  const long Kdim = (long)d->H * d->W * d->Cin, Q = (long)d->H * d->W * d->Cout;
-  if (Kdim > (1L << 40) || Q > (1L << 40) || (long)d->B * d->H * cdiv(d->W, 32) > 2000000000L)
+  const long px = (long)depth(d) * d->H * d->W;
+  const long Kdim = px * d->Cin, Q = px * d->Cout;
+  if (Kdim > (1L << 40) || Q > (1L << 40) || (long)d->B * depth(d) * d->H * cdiv(d->W, 32) > 2000000000L ||
+      (long)depth(d) * d->H > 2000000000L)
     return XCONV_ERR_UNSUPPORTED;
   const long axis_limit = 65535L * 16;
   if (d->r > axis_limit || d->B > axis_limit || d->Cin > axis_limit || d->Cout > axis_limit ||
-      (long)d->r * d->B > (1L << 40))
+      (long)d->r * d->B > (1L << 40) || (long)d->r * depth(d) > 2000000000L || (long)d->B * depth(d) > 2000000000L)
     return XCONV_ERR_UNSUPPORTED;
   return XCONV_OK;
 }
+
+// The sketch, the back-probe and the per-channel kernels see the pixels of a sample as one flat axis: for
+// them a volume is an image with D*H rows.
+static xconv_desc flat(const xconv_desc* d) {
+  xconv_desc f = *d;
+  f.H = d->H * depth(d);
+  f.D = 1; f.KD = 1; f.pad_d = 0;
+  return f;
+}
+// A planar kernel on a volume treats every plane as an image of its own: D times the probes for the
+// contraction, D times the batch for the convolutions.  (Only for kdepth(d) == 1.)
+static xconv_desc planes_ct(const xconv_desc* d) {
+  xconv_desc f = *d;
+  f.r = d->r * depth(d);
+  f.D = 1; f.KD = 1; f.pad_d = 0;
+  return f;
+}
+static xconv_desc planes_cv(const xconv_desc* d) {
+  xconv_desc f = *d;
+  f.B = d->B * depth(d);
+  f.D = 1; f.KD = 1; f.pad_d = 0;
+  return f;
+}
+static inline bool volumetric(const xconv_desc* d) { return kdepth(d) == 3; }
 
 // ----------------------------------------------------------------------------------- plans
 // A plan fixes every launch shape and workspace offset from the descriptor alone, so that
@@ -70,7 +103,9 @@ struct SketchPlan {
   size_t part_off, bytes;
 };
 
-static SketchPlan plan_sketch(const xconv_desc* d, bool seeded = false) {
+static SketchPlan plan_sketch(const xconv_desc* d_, bool seeded = false) {
+  const xconv_desc fl = flat(d_);
+  const xconv_desc* d = &fl;
   SketchPlan p{};
   const long K = (long)d->H * d->W * d->Cin;
   p.part_off = WS_HEADER;
@@ -93,27 +128,32 @@ static SketchPlan plan_sketch(const xconv_desc* d, bool seeded = false) {
 struct WgradPlan {
   bool tc_bp, tc_ct;
   int splits; long items_per_split;    // simt contraction
-  TcWgradPlan t;                       // tcgen05
+  TcWgradPlan t;                       // tcgen05: contraction fields (planned on the per-plane layer)
+  TcWgradPlan tb;                      // tcgen05: back-probe fields (planned on the flattened layer)
   size_t l_off, sb_off, part_off, bytes;
 };
 
 static WgradPlan plan_wgrad_core(const xconv_desc* d) {
   WgradPlan p{};
-  const long Q = (long)d->H * d->W * d->Cout;
-  const int T = d->KH * d->KW;
+  const long Q = (long)depth(d) * d->H * d->W * d->Cout;
+  const int T = kdepth(d) * d->KH * d->KW;
   const size_t lsz = d->dtype == XCONV_F32 ? 4 : 2;
   p.l_off = WS_HEADER;
   p.sb_off = p.l_off + align_up((size_t)d->r * Q * lsz, 256);
   p.part_off = p.sb_off + align_up((size_t)d->r * d->B * 2, 256);
-  const int mask = tc_plan_wgrad(d, &p.t);
-  p.tc_bp = (mask & 1) != 0;
-  p.tc_ct = (mask & 2) != 0;
+  const xconv_desc f = flat(d);
+  p.tc_bp = (tc_plan_wgrad(&f, &p.tb) & 1) != 0;
+  if (!volumetric(d)) {                 // the tensor-core contraction works plane by plane
+    const xconv_desc c = planes_ct(d);
+    p.tc_ct = (tc_plan_wgrad(&c, &p.t) & 2) != 0;
+  }
   if (p.tc_ct) {
     p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
     return p;
   }
-  const long items = (long)d->r * d->H * cdiv(d->W, 32);
-  const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32) * (d->KH == 5 ? 5 : 1);   // 5 x 5: one offset row per block
+  const long items = (long)d->r * depth(d) * d->H * cdiv(d->W, 32);
+  // blocks per split: 5 x 5 kernels take one offset row per block, 3 x 3 x 3 kernels three
+  const long tiles = cdiv(d->Cin, 64) * cdiv(d->Cout, 32) * (d->KH == 5 ? 5 : volumetric(d) ? 3 : 1);
   // one wave of the grid: two blocks of this kernel fit an SM (its 72 accumulators per thread)
   long splits = std::max(1L, std::min(std::max(1L, 2L * 148 / tiles), cdiv(items, 2)));
   splits = std::min(splits, 4096L);
@@ -147,9 +187,9 @@ static SwappedWgrad plan_wgrad_swapped(const xconv_desc* d) {
   w.p1 = plan_wgrad_core(&w.d1);
   w.p2 = plan_wgrad_core(&w.d2);
   const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
-  const int T = d->KH * d->KW;
+  const int T = kdepth(d) * d->KH * d->KW;
   w.x_off = WS_HEADER;
-  w.st_off = w.x_off + align_up((size_t)d->B * d->H * d->W * d->Cin * es, 256);
+  w.st_off = w.x_off + align_up((size_t)d->B * depth(d) * d->H * d->W * d->Cin * es, 256);
   w.sb_off = w.st_off + align_up((size_t)d->r * d->B * 4, 256);
   w.part_off = w.sb_off + align_up((size_t)d->r * d->B * 2, 256);
   const size_t part = w.p2.tc_ct ? w.p2.t.part_bytes : (size_t)w.p2.splits * d->Cout * T * d->Cin * sizeof(float);
@@ -193,7 +233,7 @@ __global__ void __launch_bounds__(256) probes_from_seed_kernel(T* __restrict__ Z
 }
 
 static xconv_status run_probes_from_seed(const xconv_desc* d, unsigned long long seed, void* Z, cudaStream_t st) {
-  const long total = (long)d->r * d->H * d->W * d->Cin;
+  const long total = (long)d->r * depth(d) * d->H * d->W * d->Cin;
   const unsigned grid = (unsigned)cdiv(cdiv(total, 8), 256);
   const uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFull), k1 = (uint32_t)(seed >> 32);
   cudaError_t e = d->dtype == XCONV_F32
@@ -207,7 +247,7 @@ static xconv_status run_probes_from_seed(const xconv_desc* d, unsigned long long
 }
 
 static size_t probes_bytes(const xconv_desc* d) {
-  return align_up((size_t)d->r * d->H * d->W * d->Cin * (d->dtype == XCONV_F32 ? 4 : 2), 256);
+  return align_up((size_t)d->r * depth(d) * d->H * d->W * d->Cin * (d->dtype == XCONV_F32 ? 4 : 2), 256);
 }
 
 // ----------------------------------------------------------------------------------- launchers
@@ -229,10 +269,15 @@ static xconv_status run_sketch_simt(const xconv_desc* d, const SketchPlan& p, co
 
 // Whether the sketch kernel of this layer redraws Z itself; otherwise the seeded call first writes Z
 // into the workspace (behind the regular scratch) and runs the regular kernels on it.
-static bool sketch_redraws(const xconv_desc* d, const SketchPlan& p) { return p.tc && tc_sketch_can_redraw(d); }
+static bool sketch_redraws(const xconv_desc* d, const SketchPlan& p) {
+  const xconv_desc fl = flat(d);
+  return p.tc && tc_sketch_can_redraw(&fl);
+}
 
-static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z, float* S, void* ws,
+static xconv_status run_sketch(const xconv_desc* d_, const void* X, const void* Z, float* S, void* ws,
                                size_t ws_bytes, cudaStream_t st, const unsigned long long* seed = nullptr) {
+  const xconv_desc fl = flat(d_);
+  const xconv_desc* d = &fl;
   const SketchPlan p = plan_sketch(d, seed != nullptr);
   const bool redraw = seed && sketch_redraws(d, p);
   const size_t need = p.bytes + (seed && !redraw ? probes_bytes(d) : 0);
@@ -253,7 +298,7 @@ static xconv_status run_sketch(const xconv_desc* d, const void* X, const void* Z
 template <typename T, typename TL>
 static xconv_status run_backprobe_simt(const xconv_desc* d, const float* S, const void* dY, void* Lv,
                                        cudaStream_t st) {
-  const long Q = (long)d->H * d->W * d->Cout;
+  const long Q = (long)depth(d) * d->H * d->W * d->Cout;
   dim3 g1((unsigned)cdiv(Q, 1024), (unsigned)cdiv(d->r, 16));
   backprobe_simt<T, TL><<<g1, 256, 0, st>>>(S, static_cast<const T*>(dY), static_cast<TL*>(Lv), d->r, d->B, Q,
                                             (Q % 4 == 0) ? 1 : 0);
@@ -263,19 +308,20 @@ static xconv_status run_backprobe_simt(const xconv_desc* d, const float* S, cons
 template <typename T, typename TL>
 static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, const void* Lv, const void* Z,
                                       float* dW, float alpha, float* part, cudaStream_t st) {
-  const int T9 = d->KH * d->KW;
+  const int T9 = kdepth(d) * d->KH * d->KW;
   const TL* L = static_cast<const TL*>(Lv);
   const T* Zt = static_cast<const T*>(Z);
   const bool vec = d->Cin % 4 == 0 && d->Cout % 4 == 0;      // rows of L and Z then start on 4-element boundaries
   const unsigned gx = (unsigned)cdiv(d->Cin, 64), gy = (unsigned)cdiv(d->Cout, 32), gz = (unsigned)p.splits;
-#define XC_CONTRACT(KS, DYS) do { \
-    dim3 g2(gx * (KS / DYS), gy, gz); \
-    if (vec) contract_simt<TL, T, KS, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
-    else contract_simt<TL, T, KS, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+#define XC_CONTRACT(KS, KD, DYS) do { \
+    dim3 g2(gx * (KD * KS / DYS), gy, gz); \
+    if (vec) contract_simt<TL, T, KS, KD, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+    else contract_simt<TL, T, KS, KD, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
   } while (0)
-  if (d->KH == 3) XC_CONTRACT(3, 3);
-  else if (d->KH == 5) XC_CONTRACT(5, 1);
-  else XC_CONTRACT(1, 1);
+  if (volumetric(d)) XC_CONTRACT(3, 3, 3);
+  else if (d->KH == 3) XC_CONTRACT(3, 1, 3);
+  else if (d->KH == 5) XC_CONTRACT(5, 1, 1);
+  else XC_CONTRACT(1, 1, 1);
 #undef XC_CONTRACT
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
@@ -288,34 +334,36 @@ template <typename T>
 static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* in, const void* Wt, void* out,
                                   cudaStream_t st) {
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
-  dim3 grid((unsigned)((long)d->B * d->H * cdiv(d->W, 32)), (unsigned)cdiv(Co, 64));
+  const int D = depth(d), planes = d->B * D;
+  dim3 grid((unsigned)((long)planes * d->H * cdiv(d->W, 32)), (unsigned)cdiv(Co, 64));
   const T* i_ = static_cast<const T*>(in);
   const T* w_ = static_cast<const T*>(Wt);
   T* o_ = static_cast<T*>(out);
-  if (d->KH == 3) {
-    if (dgrad) conv_simt<T, 3, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-    else       conv_simt<T, 3, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-  } else if (d->KH == 5) {
-    if (dgrad) conv_simt<T, 5, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-    else       conv_simt<T, 5, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-  } else {
-    if (dgrad) conv_simt<T, 1, true><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-    else       conv_simt<T, 1, false><<<grid, 256, 0, st>>>(i_, w_, o_, d->B, d->H, d->W, Ci, Co, d->Cin);
-  }
+#define XC_CONV(KS, KD) do { \
+    if (dgrad) conv_simt<T, KS, KD, true><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin); \
+    else       conv_simt<T, KS, KD, false><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin); \
+  } while (0)
+  if (volumetric(d)) XC_CONV(3, 3);
+  else if (d->KH == 3) XC_CONV(3, 1);
+  else if (d->KH == 5) XC_CONV(5, 1);
+  else XC_CONV(1, 1);
+#undef XC_CONV
   return check_launch();
 }
 
 // Scratch of the convolution calls: the header, and for the tensor-core dgrad the transposed weights.
 static size_t conv_ws_bytes(const xconv_desc* d, bool dgrad) {
   TcConvPlan t;
-  if (tc_plan_conv(d, dgrad, &t)) return WS_HEADER + align_up(t.wt_bytes, 256);
+  const xconv_desc c = planes_cv(d);
+  if (!volumetric(d) && tc_plan_conv(&c, dgrad, &t)) return WS_HEADER + align_up(t.wt_bytes, 256);
   return WS_HEADER;
 }
 
 static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, const void* Wt, void* out,
                              char* ws, cudaStream_t st) {
   TcConvPlan t;
-  if (tc_plan_conv(d, dgrad, &t)) return tc_run_conv(d, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
+  const xconv_desc c = planes_cv(d);
+  if (!volumetric(d) && tc_plan_conv(&c, dgrad, &t)) return tc_run_conv(&c, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
   return d->dtype == XCONV_F32 ? run_conv_simt<float>(d, dgrad, in, Wt, out, st)
          : d->dtype == XCONV_F16 ? run_conv_simt<f16>(d, dgrad, in, Wt, out, st)
                                  : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
@@ -331,7 +379,8 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
         : launch_pdl(cast_f32_to_16<bf16>, dim3((unsigned)cdiv(n, 256)), dim3(256), 0, st, S, static_cast<bf16*>(Sb_), n);
     ++g_launches;
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
-    return tc_run_backprobe(d, p.t, Sb_, dY, L, w, st);
+    const xconv_desc f = flat(d);
+    return tc_run_backprobe(&f, p.tb, Sb_, dY, L, w, st);
   }
   return d->dtype == XCONV_F32 ? run_backprobe_simt<float, float>(d, S, dY, L, st)
          : d->dtype == XCONV_F16 ? run_backprobe_simt<f16, f16>(d, S, dY, L, st)
@@ -340,7 +389,10 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
 
 static xconv_status run_contract(const xconv_desc* d, const WgradPlan& p, const void* L, const void* Z,
                                  float* dW, float alpha, char* part, char* w, cudaStream_t st) {
-  if (p.tc_ct) return tc_run_contract(d, p.t, L, Z, dW, alpha, w, part, st);
+  if (p.tc_ct) {
+    const xconv_desc c = planes_ct(d);
+    return tc_run_contract(&c, p.t, L, Z, dW, alpha, w, part, st);
+  }
   return d->dtype == XCONV_F32
              ? run_contract_simt<float, float>(d, p, L, Z, dW, alpha, reinterpret_cast<float*>(part), st)
          : d->dtype == XCONV_F16
@@ -406,9 +458,9 @@ static IndepPlan plan_indep(const xconv_desc* d) {
   ip.d2 = *d; ip.d2.r = d->B; ip.d2.chan_scale = nullptr;     // the contraction runs over the batch
   ip.p2 = plan_wgrad_core(&ip.d2);
   const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
-  const int T = d->KH * d->KW;
+  const int T = kdepth(d) * d->KH * d->KW;
   ip.x_off = WS_HEADER;
-  ip.part_off = ip.x_off + align_up((size_t)d->B * d->H * d->W * d->Cin * es, 256);
+  ip.part_off = ip.x_off + align_up((size_t)d->B * depth(d) * d->H * d->W * d->Cin * es, 256);
   const size_t part = ip.p2.tc_ct ? ip.p2.t.part_bytes : (size_t)ip.p2.splits * d->Cout * T * d->Cin * sizeof(float);
   ip.bytes = ip.part_off + align_up(part, 256);
   return ip;
@@ -423,7 +475,7 @@ static xconv_status validate_indep(const xconv_desc* d) {
 
 template <typename T>
 static xconv_status run_sketch_indep(const xconv_desc* d, const void* X, const void* Z, float* S, cudaStream_t st) {
-  const long N = (long)d->H * d->W;
+  const long N = (long)depth(d) * d->H * d->W;
   dim3 grid((unsigned)cdiv(d->B, IS_BT), (unsigned)cdiv(d->Cin, 32), (unsigned)cdiv(d->r, IS_JT));
   sketch_indep_simt<T><<<grid, 256, 0, st>>>(static_cast<const T*>(X), static_cast<const T*>(Z), S, d->r, d->B, N, d->Cin);
   return check_launch();
@@ -431,7 +483,7 @@ static xconv_status run_sketch_indep(const xconv_desc* d, const void* X, const v
 
 template <typename T>
 static xconv_status run_rebuild_indep(const xconv_desc* d, const float* S, const void* Z, void* Xr, cudaStream_t st) {
-  const long N = (long)d->H * d->W;
+  const long N = (long)depth(d) * d->H * d->W;
   dim3 grid((unsigned)cdiv(N, 8), (unsigned)cdiv(d->Cin, 32), (unsigned)cdiv(d->B, IR_BT));
   rebuild_indep_simt<T><<<grid, 256, 0, st>>>(S, static_cast<const T*>(Z), static_cast<T*>(Xr), d->r, d->B, N, d->Cin);
   return check_launch();
@@ -477,7 +529,8 @@ int xconv_engine_for(const xconv_desc* desc, int op) {
     case XCONV_OP_FORWARD:
     case XCONV_OP_DGRAD: {
       TcConvPlan t;
-      return tc_plan_conv(desc, op == XCONV_OP_DGRAD, &t) ? tc : XCONV_ENGINE_SIMT_F32;
+      const xconv_desc c = planes_cv(desc);
+      return !volumetric(desc) && tc_plan_conv(&c, op == XCONV_OP_DGRAD, &t) ? tc : XCONV_ENGINE_SIMT_F32;
     }
     default: return XCONV_ENGINE_NONE;
   }
@@ -593,7 +646,7 @@ xconv_status xconv_wgrad(const xconv_desc* desc, const float* sketch, const void
 
 size_t xconv_backprobe_bytes(const xconv_desc* desc) {
   if (validate(desc) != XCONV_OK) return 0;
-  return (size_t)desc->r * desc->H * desc->W * desc->Cout * (desc->dtype == XCONV_F32 ? 4 : 2);
+  return (size_t)desc->r * depth(desc) * desc->H * desc->W * desc->Cout * (desc->dtype == XCONV_F32 ? 4 : 2);
 }
 
 xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const void* dY, void* L, void* ws,
@@ -643,12 +696,12 @@ struct HostArena { size_t x, dy, z, s, dw, ws, ws_bytes, total, xb, dyb, zb, sb,
 static HostArena host_arena(const xconv_desc* d) {
   HostArena a{};
   const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
-  const size_t px = (size_t)d->H * d->W;
+  const size_t px = (size_t)depth(d) * d->H * d->W;
   a.xb = (size_t)d->B * px * d->Cin * es;
   a.dyb = (size_t)d->B * px * d->Cout * es;
   a.zb = (size_t)d->r * px * d->Cin * es;
   a.sb = (size_t)d->r * d->B * 4;
-  a.dwb = (size_t)d->Cout * d->KH * d->KW * d->Cin * 4;
+  a.dwb = (size_t)d->Cout * kdepth(d) * d->KH * d->KW * d->Cin * 4;
   a.x = 0;
   a.dy = a.x + align_up(a.xb, 256);
   a.z = a.dy + align_up(a.dyb, 256);

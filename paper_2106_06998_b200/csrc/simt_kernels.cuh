@@ -172,22 +172,24 @@ __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ 
 // no shifted or im2col copy of Z exists.  A block owns 32 output x 64 input channels and DYS rows of
 // the KS x KS offsets (all of them for 3 x 3; one row at a time for 5 x 5, whose 25 x 8 sums per thread
 // would not fit the registers); work items are (probe, row, 32-pixel chunk) triples dealt to grid.z
-// splits in order.  grid.x = (blocks of 64 input channels) x (KS / DYS groups of offset rows).
+// splits in order.  grid.x = (blocks of 64 input channels) x (KD * KS / DYS groups of offset rows).
+// Volumes (D planes per probe, KD planes per kernel): an "offset row" is a (dz, dy) pair, rho = kz * KS + ky,
+// and a work item carries its plane z; a row whose plane z + dz lies outside the volume reads zeros.
 // ---------------------------------------------------------------------------------------------
-template <typename TL, typename TZ, int KS, int DYS, bool VEC>
+template <typename TL, typename TZ, int KS, int KD, int DYS, bool VEC>
 __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, const TZ* __restrict__ Z,
-                                                     float* __restrict__ part, int r, int H, int W, int Cin,
+                                                     float* __restrict__ part, int r, int D, int H, int W, int Cin,
                                                      int Cout, long items_per_split) {
-  constexpr int P = (KS - 1) / 2, XC = 32, T = DYS * KS, TALL = KS * KS;
+  constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = DYS * KS, TALL = KD * KS * KS;
   __shared__ __align__(16) float Ls[XC][32];
   __shared__ __align__(16) float Zs[DYS][XC + KS - 1][64];
   const int tid = threadIdx.x;
   const int nblocks = (Cin + 63) / 64;
-  const int dy0 = (blockIdx.x / nblocks) * DYS;          // first offset row of this block
+  const int dy0 = (blockIdx.x / nblocks) * DYS;          // first offset row (kz * KS + ky) of this block
   const int n0 = (blockIdx.x % nblocks) * 64, m0 = blockIdx.y * 32;
   const int tx = tid & 15, ty = tid >> 4;
   const int chunks = (W + XC - 1) / XC;
-  const long items = (long)r * H * chunks;
+  const long items = (long)r * D * H * chunks;
   const long ib = (long)blockIdx.z * items_per_split;
   const long ie = min(items, ib + items_per_split);
 
@@ -202,7 +204,8 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
   for (long it = ib; it < ie; ++it) {
     const int xc = (int)(it % chunks);
     const int y = (int)((it / chunks) % H);
-    const int j = (int)(it / ((long)chunks * H));
+    const long jz = it / ((long)chunks * H);              // plane index j * D + z
+    const int z = (int)(jz % D);
     const int x0 = xc * XC;
     if (VEC) {
       // channel counts are multiples of 4: four consecutive channels per load (the tiles fill in a quarter
@@ -210,34 +213,36 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
       {
         const int mm = (tid & 7) * 4, px = tid >> 3;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (x0 + px < W && m0 + mm < Cout) v = ld4(L + (((long)j * H + y) * W + x0 + px) * Cout + m0 + mm);
+        if (x0 + px < W && m0 + mm < Cout) v = ld4(L + ((jz * H + y) * W + x0 + px) * Cout + m0 + mm);
         *reinterpret_cast<float4*>(&Ls[px][mm]) = v;
       }
       for (int idx = tid; idx < DYS * (XC + KS - 1) * 16; idx += 256) {
         const int nn = (idx & 15) * 4;
         const int px = (idx >> 4) % (XC + KS - 1);
         const int dy = (idx >> 4) / (XC + KS - 1);
-        const int yy = y + dy0 + dy - P, xx = x0 + px - P;
+        const int rho = dy0 + dy, dz = rho / KS - PD;
+        const int yy = y + rho % KS - P, xx = x0 + px - P;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
-          v = ld4(Z + (((long)j * H + yy) * W + xx) * Cin + n0 + nn);
+        if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
+          v = ld4(Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn);
         *reinterpret_cast<float4*>(&Zs[dy][px][nn]) = v;
       }
     } else {
     for (int idx = tid; idx < XC * 32; idx += 256) {
       const int mm = idx & 31, px = idx >> 5;
       float v = 0.f;
-      if (x0 + px < W && m0 + mm < Cout) v = to_f(L[(((long)j * H + y) * W + x0 + px) * Cout + m0 + mm]);
+      if (x0 + px < W && m0 + mm < Cout) v = to_f(L[((jz * H + y) * W + x0 + px) * Cout + m0 + mm]);
       Ls[px][mm] = v;
     }
     for (int idx = tid; idx < DYS * (XC + KS - 1) * 64; idx += 256) {
       const int nn = idx & 63;
       const int px = (idx >> 6) % (XC + KS - 1);
       const int dy = (idx >> 6) / (XC + KS - 1);
-      const int yy = y + dy0 + dy - P, xx = x0 + px - P;
+      const int rho = dy0 + dy, dz = rho / KS - PD;
+      const int yy = y + rho % KS - P, xx = x0 + px - P;
       float v = 0.f;
-      if (yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
-        v = to_f(Z[(((long)j * H + yy) * W + xx) * Cin + n0 + nn]);
+      if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
+        v = to_f(Z[(((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn]);
       Zs[dy][px][nn] = v;
     }
     }
@@ -282,20 +287,22 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
 //   forward: w(co,ci,tap) = Wt[co][tap][ci]          (Wt is [Cout][T][Cin])
 //   dgrad  : w(co,ci,tap) = Wt[ci][T-1-tap][co]
 // A block owns 32 pixels of one image row and 64 output channels; input channels go by 16 (by 4 for
-// 5 x 5 kernels, whose weight tile would not fit the static shared memory otherwise).
+// 5 x 5 and 3 x 3 x 3 kernels, whose weight tile would not fit the static shared memory otherwise).
+// Volumes: `B` counts planes (images x depth D), KD planes per kernel, offset rows rho = kz * KS + ky.
 // ---------------------------------------------------------------------------------------------
-template <typename T_, int KS, bool DGRAD>
+template <typename T_, int KS, int KD, bool DGRAD>
 __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, const T_* __restrict__ Wt,
-                                                 T_* __restrict__ out, int B, int H, int W, int Ci, int Co,
+                                                 T_* __restrict__ out, int B, int D, int H, int W, int Ci, int Co,
                                                  int Cin_w) {
-  constexpr int P = (KS - 1) / 2, XC = 32, T = KS * KS, CK = KS >= 5 ? 4 : 16;
-  __shared__ __align__(16) float Xs[KS][XC + KS - 1][CK];
+  constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = KD * KS * KS, CK = T >= 25 ? 4 : 16, R = KD * KS;
+  __shared__ __align__(16) float Xs[R][XC + KS - 1][CK];
   __shared__ __align__(16) float Ws[T][CK][64];
   const int tid = threadIdx.x;
   const int chunks = (W + XC - 1) / XC;
   const int xc = blockIdx.x % chunks;
   const int y = (blockIdx.x / chunks) % H;
-  const int b = blockIdx.x / (chunks * H);
+  const int b = blockIdx.x / (chunks * H);              // plane index: image * D + z
+  const int z = b % D;
   const int x0 = xc * XC, co0 = blockIdx.y * 64;
   const int cp = tid & 31, pg = tid >> 5;
   float acc[4][2];
@@ -303,15 +310,15 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
   for (int p = 0; p < 4; ++p) acc[p][0] = acc[p][1] = 0.f;
 
   for (int ci0 = 0; ci0 < Ci; ci0 += CK) {
-    for (int idx = tid; idx < KS * (XC + KS - 1) * CK; idx += 256) {
+    for (int idx = tid; idx < R * (XC + KS - 1) * CK; idx += 256) {
       const int cc = idx % CK;
       const int px = (idx / CK) % (XC + KS - 1);
-      const int dy = idx / (CK * (XC + KS - 1));
-      const int yy = y + dy - P, xx = x0 + px - P;
+      const int rho = idx / (CK * (XC + KS - 1)), dz = rho / KS - PD;
+      const int yy = y + rho % KS - P, xx = x0 + px - P;
       float v = 0.f;
-      if (yy >= 0 && yy < H && xx >= 0 && xx < W && ci0 + cc < Ci)
-        v = to_f(in[(((long)b * H + yy) * W + xx) * Ci + ci0 + cc]);
-      Xs[dy][px][cc] = v;
+      if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && ci0 + cc < Ci)
+        v = to_f(in[(((long)(b + dz) * H + yy) * W + xx) * Ci + ci0 + cc]);
+      Xs[rho][px][cc] = v;
     }
     for (int idx = tid; idx < T * CK * 64; idx += 256) {
       int cc, tap, co;
@@ -330,7 +337,7 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
 #pragma unroll 4
     for (int cc = 0; cc < CK; ++cc) {
 #pragma unroll
-      for (int dy = 0; dy < KS; ++dy) {
+      for (int dy = 0; dy < R; ++dy) {
         float xv[4 + KS - 1];
 #pragma unroll
         for (int p = 0; p < 4 + KS - 1; ++p) xv[p] = Xs[dy][pg * 4 + p][cc];

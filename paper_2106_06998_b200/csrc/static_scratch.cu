@@ -54,7 +54,7 @@ static xconv_status static_scratch_address(float** out) {
 template <typename T>
 static xconv_status sketch_static_run(const xconv_desc* d, const void* X, const void* Z, float* S, float* scratch,
                                       cudaStream_t st) {
-  const long K = (long)d->H * d->W * d->Cin;
+  const long K = (long)(d->D > 1 ? d->D : 1) * d->H * d->W * d->Cin;
   const long out_elems = (long)d->r * d->B;
   // as many k-splits as fill the GPU, capped by what the fixed array can hold
   const long tiles = ((d->r + 63) / 64) * (long)((d->B + 63) / 64);
@@ -88,7 +88,7 @@ extern "C" xconv_status xconv_sketch_static(const xconv_desc* desc, const void* 
     return XCONV_ERR_ALIGNMENT;
   // the one partial-sum slab [r][B] must fit the fixed array; beyond that there is nowhere to put it
   if ((long)desc->r * desc->B > (long)XCONV_STATIC_SCRATCH_FLOATS) return XCONV_ERR_WORKSPACE;
-  if ((long)desc->H * desc->W * desc->Cin > (1L << 40)) return XCONV_ERR_UNSUPPORTED;
+  if (desc->D < 0 || (long)(desc->D > 1 ? desc->D : 1) * desc->H * desc->W * desc->Cin > (1L << 40)) return XCONV_ERR_UNSUPPORTED;
   float* scratch = nullptr;
   xconv_status s = static_scratch_address(&scratch);
   if (s != XCONV_OK) return s;
