@@ -27,7 +27,6 @@
 #include <cudaTypedefs.h>
 
 #include <algorithm>
-#include <cstdlib>
 
 #include "common.cuh"
 
@@ -101,7 +100,6 @@ struct TcParams {
   int z_is_a;              // SKETCH: Z is the A operand (probes on the MMA rows) instead of the B operand
   long z_row_len;          // entries of one probing vector, H*W*Cin
   long rows_z;             // probing vectors (rows of Z)
-  int pf_ahead;            // BACKPROBE: stages by which L2 prefetches of the dY tiles run ahead of their copies (0: none)
   int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
@@ -201,11 +199,6 @@ __device__ __forceinline__ void bulk_wait_read_upto(int pending) {
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// Ask L2 for a box ahead of its copy into shared memory (a hint: no completion, no shared memory).
-__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2) {
-  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -677,15 +670,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // dY tile: one box (64 positions x k rows) per block of the column tile, one behind the other
             for (int b = 0; b < w.nblk; ++b)
               tma_load_3d(b_dst + (uint32_t)b * p.b_box_bytes, &map_b, 0, kc, w.blk0 + b, &full_bar[s]);
-            if (p.pf_ahead > 0) {            // the dY boxes of the stage pf_ahead stages on, into L2
-              const long ita = it + p.pf_ahead;
-              const long ua = blockIdx.x + (long)gridDim.x * (ita / p.kblocks);
-              if (ua < p.units) {
-                const Unit wa = decode_unit(p, ua);
-                const int kca = (int)(ita % p.kblocks) * p.ksteps * 16;
-                for (int b = 0; b < wa.nblk; ++b) tma_prefetch_3d(&map_b, 0, kca, wa.blk0 + b);
-              }
-            }
             kc += p.ksteps * 16;
           } else if (p.mode == MODE_CONV) {
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
@@ -1452,10 +1436,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
   p.status = reinterpret_cast<unsigned int*>(ws_head);
-  long grid = std::min<long>(p.units, (long)NUM_SMS);
-  if (const char* e = getenv("XC_BP_GRID")) grid = std::max(1L, std::min(grid, atol(e)));
-  if (const char* e = getenv("XC_BP_PF")) p.pf_ahead = atoi(e);
-  return launch(ma, mb, p, (unsigned)grid, st, &mc);
+  return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st, &mc);
 }
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
