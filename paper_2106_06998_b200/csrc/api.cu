@@ -4,7 +4,6 @@
 #include <algorithm>
 #include <atomic>
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 
 #include "common.cuh"
@@ -205,40 +204,6 @@ static WgradPlan plan_wgrad(const xconv_desc* d) {
   return p;
 }
 
-// ----------------------------------------------------------------------------------- forward pass in batch chunks
-// xconv_forward reads X twice, once for the convolution and once for the sketch.  Columns of S belong to
-// samples, so the two steps can alternate over chunks of the batch: the sketch of a chunk then finds the
-// chunk's X (which the convolution has just read) in the L2 cache instead of HBM.  A chunk is sized so
-// that its X and Y together stay well inside L2; layers whose whole X and Y fit, whose batch is too small
-// to cut, or whose sketch does not run on the tensor cores are done in one piece.
-static const size_t FORWARD_CHUNK_BYTES = 80u << 20;
-
-struct ForwardPlan { int chunk; size_t bytes; };      // chunk == B: one piece
-
-static ForwardPlan plan_forward(const xconv_desc* d) {
-  ForwardPlan f{};
-  f.chunk = d->B;
-  f.bytes = plan_sketch(d).bytes;
-  const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
-  const size_t per_sample = (size_t)depth(d) * d->H * d->W * (d->Cin + d->Cout) * es;
-  TcConvPlan t;
-  const xconv_desc cv = planes_cv(d);
-  if (es != 2 || volumetric(d) || !tc_plan_conv(&cv, false, &t) || !plan_sketch(d).tc) return f;
-  if (per_sample * d->B <= FORWARD_CHUNK_BYTES) return f;
-  int chunk = (int)(FORWARD_CHUNK_BYTES / per_sample) / 16 * 16;
-  if (const char* e = getenv("XC_FWD_CHUNK")) chunk = atoi(e);
-  if (chunk < 32 || chunk * 2 > d->B) return f;
-  xconv_desc c = *d;
-  c.B = chunk;
-  xconv_desc tail = *d;
-  tail.B = d->B % chunk ? d->B % chunk : chunk;
-  const SketchPlan pc = plan_sketch(&c), pt = plan_sketch(&tail);
-  if (!pc.tc || !pt.tc) return f;
-  f.chunk = chunk;
-  f.bytes = std::max(f.bytes, std::max(pc.bytes, pt.bytes));
-  return f;
-}
-
 // ----------------------------------------------------------------------------------- probes from a seed
 
 // Z redrawn from a seed: entry e (in memory order) is +1 if bit (e mod 128) of Philox block (e div 128) is 0,
@@ -310,8 +275,7 @@ static bool sketch_redraws(const xconv_desc* d, const SketchPlan& p) {
 }
 
 static xconv_status run_sketch(const xconv_desc* d_, const void* X, const void* Z, float* S, void* ws,
-                               size_t ws_bytes, cudaStream_t st, const unsigned long long* seed = nullptr,
-                               int ldS = 0) {
+                               size_t ws_bytes, cudaStream_t st, const unsigned long long* seed = nullptr) {
   const xconv_desc fl = flat(d_);
   const xconv_desc* d = &fl;
   const SketchPlan p = plan_sketch(d, seed != nullptr);
@@ -325,8 +289,7 @@ static xconv_status run_sketch(const xconv_desc* d_, const void* X, const void* 
     if (s != XCONV_OK) return s;
     Z = w + p.bytes;
   }
-  if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st, redraw ? seed : nullptr, ldS);
-  if (ldS > 0 && ldS != d->B) return XCONV_ERR_UNSUPPORTED;      // column blocks of S: tensor-core path only
+  if (p.tc) return tc_run_sketch(d, p.t, X, Z, S, w, w + p.part_off, st, redraw ? seed : nullptr);
   return d->dtype == XCONV_F32 ? run_sketch_simt<float>(d, p, X, Z, S, w, st)
          : d->dtype == XCONV_F16 ? run_sketch_simt<f16>(d, p, X, Z, S, w, st)
                                  : run_sketch_simt<bf16>(d, p, X, Z, S, w, st);
@@ -539,7 +502,7 @@ extern "C" {
 size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
   if (validate(desc) != XCONV_OK) return 0;
   switch (op) {
-    case XCONV_OP_FORWARD: return plan_forward(desc).bytes;
+    case XCONV_OP_FORWARD:
     case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
     case XCONV_OP_WGRAD_SEEDED: return plan_wgrad(desc).bytes + probes_bytes(desc);
     case XCONV_OP_SKETCH_SEEDED: {
@@ -660,28 +623,14 @@ xconv_status xconv_forward(const xconv_desc* desc, const void* X, const void* W,
   if (!X || !W || !Z || !Y || !sketch) return XCONV_ERR_INVALID_ARG;
   if (!aligned16(X) || !aligned16(W) || !aligned16(Z) || !aligned16(Y) || !aligned16(sketch))
     return XCONV_ERR_ALIGNMENT;
-  const ForwardPlan fp = plan_forward(desc);
-  if (!ws || ws_bytes < fp.bytes) return XCONV_ERR_WORKSPACE;
+  const SketchPlan p = plan_sketch(desc);
+  if (!ws || ws_bytes < p.bytes) return XCONV_ERR_WORKSPACE;
   if (!aligned16(ws)) return XCONV_ERR_ALIGNMENT;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   new_call();
-  if (fp.chunk >= desc->B) {
-    s = run_conv(desc, false, X, W, Y, static_cast<char*>(ws), st);
-    if (s != XCONV_OK) return s;
-    return run_sketch(desc, X, Z, sketch, ws, ws_bytes, st);
-  }
-  // convolution and sketch alternate over chunks of the batch (see plan_forward)
-  const size_t px = (size_t)depth(desc) * desc->H * desc->W * 2;          // bytes per sample and channel
-  for (int b0 = 0; b0 < desc->B; b0 += fp.chunk) {
-    xconv_desc c = *desc;
-    c.B = std::min(fp.chunk, desc->B - b0);
-    const char* Xc = static_cast<const char*>(X) + (size_t)b0 * px * desc->Cin;
-    s = run_conv(&c, false, Xc, W, static_cast<char*>(Y) + (size_t)b0 * px * desc->Cout, static_cast<char*>(ws), st);
-    if (s != XCONV_OK) return s;
-    s = run_sketch(&c, Xc, Z, sketch + b0, ws, ws_bytes, st, nullptr, desc->B);
-    if (s != XCONV_OK) return s;
-  }
-  return XCONV_OK;
+  s = run_conv(desc, false, X, W, Y, static_cast<char*>(ws), st);
+  if (s != XCONV_OK) return s;
+  return run_sketch(desc, X, Z, sketch, ws, ws_bytes, st);
 }
 
 xconv_status xconv_wgrad(const xconv_desc* desc, const float* sketch, const void* dY, const void* Z, float* dW,

@@ -49,10 +49,8 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& p, bool dgrad, c
 
 // `seed` != nullptr: Z is not read; its tiles are redrawn inside the kernel from the Philox stream of *seed
 // (Rademacher entries; see xconv_probes_from_seed).  Only for layers tc_sketch_can_redraw accepts.
-// `ldS` > 0: S is a column block of a wider matrix whose rows lie ldS floats apart (a batch chunk's sketch).
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const void* X, const void* Z, float* S,
-                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed = nullptr,
-                           int ldS = 0);
+                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed = nullptr);
 bool tc_sketch_can_redraw(const xconv_desc* d);
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const void* S_bf16, const void* dY,
                               void* L, char* ws_head, cudaStream_t st);

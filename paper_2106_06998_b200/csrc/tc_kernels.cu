@@ -1187,7 +1187,7 @@ bool tc_sketch_can_redraw(const xconv_desc* d) {
 }
 
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const void* X, const void* Z, float* S,
-                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed, int ldS) {
+                           char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed) {
   const long K = (long)d->H * d->W * d->Cin;
   const bool f16 = d->dtype == XCONV_F16;
   const int rows = pl.swap ? d->B : d->r, cols = pl.swap ? d->r : d->B;
@@ -1262,8 +1262,8 @@ xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& pl, const vo
   const long groups = split_stride / 4;
   cudaError_t e = launch_pdl(reduce_sketch_partials, dim3((unsigned)cdivl(groups, RS_GROUPS)),
                              dim3(RS_LANES * RS_GROUPS), 0, st, p.part, S,
-                             groups, split_stride, pl.splits, pl.tiles_n, pl.m_sub, pl.tile_n, rows, cols,
-                             ldS > 0 ? ldS : d->B, pl.swap);
+                             groups, split_stride, pl.splits, pl.tiles_n, pl.m_sub, pl.tile_n, rows, cols, d->B,
+                             pl.swap);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
