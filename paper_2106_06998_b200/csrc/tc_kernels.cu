@@ -16,8 +16,8 @@
 //             patch per work unit; both tiles K-major (channels contiguous), the reduction runs over
 //             (offset, 64-channel block), and the offset again moves the TMA box of the input.
 //
-// Structure of a CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (one TMEM lane quadrant each).  A ring of shared-memory stages is handed
+// Structure of a CTA (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..9 = epilogue (two per TMEM lane quadrant, sharing the columns of a tile).  A ring of shared-memory stages is handed
 // from producer to issuer with mbarriers; tcgen05.commit returns stages and signals the epilogue.
 // Every wait is bounded: on expiry the CTA records the call's tag in the workspace header, drains
 // its outstanding copies (bounded again), frees its tensor memory and returns.
@@ -54,7 +54,7 @@ struct TcParams {
   uint32_t sbo, mn_step, layout;
   int cw_shift;            // log2 of the channels per tile block (6 or 5)
   // BACKPROBE: behind the stages every epilogue warp owns a ring of epi_slots staging slots of 4 KB (32 rows x
-  // 64 positions) from which it stores L with tensor stores; epi_bytes = 4 warps x epi_slots x 4 KB (0 elsewhere).
+  // 64 positions) from which it stores L with tensor stores; epi_bytes = epilogue warps x epi_slots x 4 KB (0 elsewhere).
   // Column tiles have bp_base blocks of 64 positions, the first bp_rem tiles one more (at most 4).
   uint32_t epi_bytes;
   int epi_slots;
@@ -382,7 +382,9 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, bool f16) {
 
 constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
-constexpr int TC_THREADS = 192;
+constexpr int EPI_GROUPS = 2;                       // epilogue warps per tensor-memory lane quadrant
+constexpr int EPI_WARPS = 4 * EPI_GROUPS;
+constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -429,7 +431,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
 // F16: the 16-bit storage type is float16 instead of bfloat16 (a compile-time constant, so that the epilogues'
 // conversions carry no selection between the two).
 template <bool F16>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, 2)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -448,8 +450,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 5 : 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 1 + EPI_WARPS : 1); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], EPI_WARPS); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     prefetch_tmap(&map_a);
@@ -811,8 +813,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..)
+    // A warp reads the 32 tensor-memory lanes of its quadrant (warp index mod 4); the EPI_GROUPS warps of a
+    // quadrant deal the column chunks (back-probe: the 64-position blocks) of a tile among themselves.
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
+    const int eg = (warp - 2) >> 2;             // which of the quadrant's warps
     const uint32_t epi_base = tiles_base + (uint32_t)p.stages * stage_bytes;
     uint32_t epi_slot = 0;                    // BACKPROBE: next staging slot of this warp's ring
     int gen_s = 0;                            // seeded: stage the generator fills next, and how often the ring wrapped
@@ -827,7 +832,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
         // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
         // copy would have produced, hand the stage over with one arrival per warp.
-        const int gtid = (int)threadIdx.x - 64;                       // 0..127
+        const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
+        constexpr int GEN = 32 * EPI_WARPS;
         const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
         const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
         const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
@@ -846,8 +852,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
             // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
             const int nitems = nrows * (p.kgroup >> 1);
-            for (int it0 = gtid; it0 < nitems; it0 += 256) {
-              const int it1 = it0 + 128;
+            for (int it0 = gtid; it0 < nitems; it0 += 2 * GEN) {
+              const int it1 = it0 + GEN;
               const bool two = it1 < nitems;
               const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
               const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
@@ -858,7 +864,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
             }
           } else {
-            for (int item = gtid; item < nrows * p.kgroup; item += 128) {
+            for (int item = gtid; item < nrows * p.kgroup; item += GEN) {
               const int row = item % nrows, g = item / nrows;
               const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
               z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
@@ -887,11 +893,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int mt = 0; mt < p.m_sub; ++mt) {
           const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;
           if (row_w >= p.rows) continue;                                       // warp-uniform
-          for (int b = 0; b < w.nblk; ++b) {
+          for (int b = eg; b < w.nblk; b += EPI_GROUPS) {
             // the store that used this slot epi_slots blocks ago must have read it
             if (lane == 0) bulk_wait_read_upto(p.epi_slots - 1);
             __syncwarp();
-            const uint32_t slot_base = epi_base + ((uint32_t)quad * p.epi_slots + epi_slot) * 4096u;
+            const uint32_t slot_base = epi_base + ((uint32_t)(quad * EPI_GROUPS + eg) * p.epi_slots + epi_slot) * 4096u;
             const uint32_t rowbase = slot_base + (uint32_t)lane * 128u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -922,11 +928,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (row_w >= p.rows) continue;                                         // warp-uniform
         if (p.mode == MODE_CONV && w.img + mt >= p.nimg) continue;
         const long row = row_w + lane;
-        for (int cu = 0; cu < unit_cols; cu += 32) {
+        for (int cu = eg * 32; cu < unit_cols; cu += 32 * EPI_GROUPS) {
           // several offsets per unit (CONTRACT): tile_n is then a multiple of 32 and a chunk lies in one offset
           const int tap_l = unit_cols > p.tile_n ? cu / p.tile_n : 0;
           const int c = cu - tap_l * p.tile_n;
-          if (col0 + c >= p.cols) break;
+          if (col0 + c >= p.cols) continue;
           uint32_t v[32];
 #pragma unroll
           for (int i = 0; i < 32; ++i) v[i] = 0u;
@@ -1084,7 +1090,7 @@ static inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 static const int SMEM_LIMIT = 227 * 1024;
 static const int STATIC_SMEM_SLACK = 2048;     // barriers + alignment slack
 static const int NUM_SMS = 148;
-static const int BP_SLOT_BYTES = 4 * 32 * 128;      // back-probe output staging: per slot, 4 warps x 32 rows x 64 positions
+static const int BP_SLOT_BYTES = EPI_WARPS * 32 * 128;   // back-probe output staging: per slot, one block of 32 rows x 64 positions per epilogue warp
 
 static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;

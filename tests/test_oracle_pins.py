@@ -556,3 +556,55 @@ def test_volume_estimator_recovers_the_exact_gradient_with_an_orthogonal_basis()
     # a wrong sign of the depth shift would not recover it
     wrong = O.wgrad_contract3d(O.backprobe(O.sketch(X, Z), dY), Z[:, :, ::-1])
     assert O.rel_fro(wrong, O.dw_exact3d(X, dY)) > 0.1
+
+
+# ---------------------------------------------------------------- Theorem 1: dependence on the block probabilities p_n
+
+def _masked_estimates(X, dY, r, probs, T, seed):
+    """T estimates with Eq. (7) probes (block n of a probing vector non-zero with probability probs[n]) and
+    the 1/nnz(Z_n) scale of Eq. (8); trials in which a channel was never probed are dropped."""
+    g = _rng(seed)
+    Cin, H, W = X.shape[1:]
+    out = []
+    while len(out) < T:
+        mask = g.random((r, Cin, 1, 1)) < np.asarray(probs).reshape(1, Cin, 1, 1)
+        if not mask.any(axis=0).all():
+            continue
+        Z = g.standard_normal((r, Cin, H, W)) * mask
+        out.append(O.wgrad_estimate(O.sketch(X, Z), dY, Z, scale=O.channel_scale(Z)))
+    return np.stack(out)
+
+
+def test_theorem1_own_block_error_scales_like_inverse_sqrt_of_p_times_r():
+    """Single input channel, so that only the first term of Theorem 1's bound is there: ||A^{n,m}||_F / sqrt(p_n r).
+    Quartering p_n doubles the rms error (the estimate then averages nnz(Z_n) ~ p_n r probes instead of r)."""
+    X, Wt, dY = _tiny(seed=70, B=3, Cin=1, Cout=2, H=4, W=4)
+    exact = _loops_dw(X, dY, 3, 3, False)
+    r, T = 64, 600
+    rms = {}
+    for p_ in (1.0, 0.25):
+        est = _masked_estimates(X, dY, r, [p_], T, seed=71)
+        rms[p_] = np.sqrt(np.mean((est - exact) ** 2))
+    ratio = rms[0.25] / rms[1.0]
+    assert 1.75 < ratio < 2.4, ratio            # sqrt(1 / 0.25) = 2, a little more because nnz fluctuates
+    # and against r at fixed p: four times the probes halve it
+    est4 = _masked_estimates(X, dY, 4 * r, [0.25], T, seed=72)
+    assert 1.75 < rms[0.25] / np.sqrt(np.mean((est4 - exact) ** 2)) < 2.3
+
+
+def test_theorem1_crosstalk_from_channel_j_scales_like_sqrt_p_j():
+    """Two input channels; the estimate of block (m, n = 0) carries the crosstalk term sqrt(p_1 / p_0) ||A^{.,1}||_F of
+    Theorem 1.  With p_0 = 1 fixed, its variance is the single-channel Hutchinson variance plus p_1 ||C_1||_F^2 / r:
+    making the other channel's blocks sparser removes crosstalk in proportion."""
+    X, Wt, dY = _tiny(seed=73, B=3, Cin=2, Cout=1, H=3, W=3)
+    X[:, 1] *= 3.0                                   # make the crosstalk term the larger one
+    r, T = 16, 4000
+    var = {p1: _masked_estimates(X, dY, r, [1.0, p1], T, seed=74).var(axis=0, ddof=1) for p1 in (1.0, 0.25)}
+    for ky in range(3):
+        for kx in range(3):
+            C = _C_blocks(X, dY, 0, ky, kx)
+            own = (np.sum(C[0] ** 2) + np.trace(C[0] @ C[0])) / r
+            cross = np.sum(C[1] ** 2) / r
+            for p1 in (1.0, 0.25):
+                want = own + p1 * cross
+                assert 0.8 < var[p1][0, 0, ky, kx] / want < 1.25, (ky, kx, p1, var[p1][0, 0, ky, kx], want)
