@@ -74,18 +74,19 @@ static xconv_desc flat(const xconv_desc* d) {
   f.D = 1; f.KD = 1; f.pad_d = 0;
   return f;
 }
-// A planar kernel on a volume treats every plane as an image of its own: D times the probes for the
-// contraction, D times the batch for the convolutions.  (Only for kdepth(d) == 1.)
+// The tensor-core contraction and convolution work plane by plane: D times the probes for the contraction,
+// D times the batch for the convolutions.  A planar kernel on a volume treats every plane as an image of its
+// own (D = 1 from there on); a 3 x 3 x 3 kernel keeps D, so that the kernels know where a volume ends.
 static xconv_desc planes_ct(const xconv_desc* d) {
   xconv_desc f = *d;
   f.r = d->r * depth(d);
-  f.D = 1; f.KD = 1; f.pad_d = 0;
+  if (kdepth(d) == 1) { f.D = 1; f.KD = 1; f.pad_d = 0; }
   return f;
 }
 static xconv_desc planes_cv(const xconv_desc* d) {
   xconv_desc f = *d;
   f.B = d->B * depth(d);
-  f.D = 1; f.KD = 1; f.pad_d = 0;
+  if (kdepth(d) == 1) { f.D = 1; f.KD = 1; f.pad_d = 0; }
   return f;
 }
 static inline bool volumetric(const xconv_desc* d) { return kdepth(d) == 3; }
@@ -143,10 +144,8 @@ static WgradPlan plan_wgrad_core(const xconv_desc* d) {
   p.part_off = p.sb_off + align_up((size_t)d->r * d->B * 2, 256);
   const xconv_desc f = flat(d);
   p.tc_bp = (tc_plan_wgrad(&f, &p.tb) & 1) != 0;
-  if (!volumetric(d)) {                 // the tensor-core contraction works plane by plane
-    const xconv_desc c = planes_ct(d);
-    p.tc_ct = (tc_plan_wgrad(&c, &p.t) & 2) != 0;
-  }
+  const xconv_desc c = planes_ct(d);    // the tensor-core contraction works plane by plane
+  p.tc_ct = (tc_plan_wgrad(&c, &p.t) & 2) != 0;
   if (p.tc_ct) {
     p.bytes = p.part_off + align_up(p.t.part_bytes, 256);
     return p;
@@ -355,7 +354,7 @@ static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* i
 static size_t conv_ws_bytes(const xconv_desc* d, bool dgrad) {
   TcConvPlan t;
   const xconv_desc c = planes_cv(d);
-  if (!volumetric(d) && tc_plan_conv(&c, dgrad, &t)) return WS_HEADER + align_up(t.wt_bytes, 256);
+  if (tc_plan_conv(&c, dgrad, &t)) return WS_HEADER + align_up(t.wt_bytes, 256);
   return WS_HEADER;
 }
 
@@ -363,7 +362,7 @@ static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, co
                              char* ws, cudaStream_t st) {
   TcConvPlan t;
   const xconv_desc c = planes_cv(d);
-  if (!volumetric(d) && tc_plan_conv(&c, dgrad, &t)) return tc_run_conv(&c, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
+  if (tc_plan_conv(&c, dgrad, &t)) return tc_run_conv(&c, t, dgrad, in, Wt, out, ws, ws + WS_HEADER, st);
   return d->dtype == XCONV_F32 ? run_conv_simt<float>(d, dgrad, in, Wt, out, st)
          : d->dtype == XCONV_F16 ? run_conv_simt<f16>(d, dgrad, in, Wt, out, st)
                                  : run_conv_simt<bf16>(d, dgrad, in, Wt, out, st);
@@ -530,7 +529,7 @@ int xconv_engine_for(const xconv_desc* desc, int op) {
     case XCONV_OP_DGRAD: {
       TcConvPlan t;
       const xconv_desc c = planes_cv(desc);
-      return !volumetric(desc) && tc_plan_conv(&c, op == XCONV_OP_DGRAD, &t) ? tc : XCONV_ENGINE_SIMT_F32;
+      return tc_plan_conv(&c, op == XCONV_OP_DGRAD, &t) ? tc : XCONV_ENGINE_SIMT_F32;
     }
     default: return XCONV_ENGINE_NONE;
   }

@@ -100,6 +100,10 @@ struct TcParams {
   int z_is_a;              // SKETCH: Z is the A operand (probes on the MMA rows) instead of the B operand
   long z_row_len;          // entries of one probing vector, H*W*Cin
   long rows_z;             // probing vectors (rows of Z)
+  // Volumes: the planes (probe x depth for CONTRACT, image x depth for CONV) are the outermost tensor axis; a
+  // kernel offset with a depth component dz reads plane + dz, and where that leaves the volume the box is
+  // sent to row H of the plane instead, which lies outside the image: the copy engine fills it with zeros.
+  int depth, pad_d;        // planes per probe or image (1: planar layer), depth padding of the kernel
   int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
   unsigned int tag;        // tag of this call
@@ -534,7 +538,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int px = (int)(q % p.patches_x); q /= p.patches_x;
         int py = (int)(q % p.patches_y); q /= p.patches_y;
         int pj = (int)q;
-        const int ks = 2 * p.pad + 1, dy = w.tap / ks - p.pad, dx = w.tap % ks - p.pad;
+        const int ks = 2 * p.pad + 1, tp = w.tap % (ks * ks), dy = tp / ks - p.pad, dx = tp % ks - p.pad;
+        const int dz = w.tap / (ks * ks) - p.pad_d;
+        int pz = pj % p.depth;               // depth of plane pj inside its volume
         for (int i = 0; i < 2 * w.nkb; ++i) {
           if (fill > 0) {
             ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
@@ -544,8 +550,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int x0 = px * p.patch_w, y0 = py * p.patch_h + (i & 1) * hrows;
           mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
           tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
-          tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
-          if ((i & 1) && ++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
+          const bool inside = (unsigned)(pz + dz) < (unsigned)p.depth;
+          tma_load_5d(b_dst, &map_b, 0, x0 + dx, inside ? y0 + dy : p.H, col0 >> p.cw_shift, pj + dz, &full_bar[s]);
+          if ((i & 1) && ++px == p.patches_x) {
+            px = 0;
+            if (++py == p.patches_y) { py = 0; ++pj; if (++pz == p.depth) pz = 0; }
+          }
           ++it;
           if (++s == slots) { s = 0; ++fill; }
         }
@@ -632,18 +642,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int row0 = w.tm * p.m_sub * TILE_M;
         const int col0 = w.tn * p.tile_n;
         // running coordinates of the k-block
-        int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0;
+        int kc = 0, px = 0, py = 0, pj = 0, dx = 0, dy = 0, dz = 0, pz = 0;
         if (p.mode == MODE_SKETCH) kc = (int)((p.k_weave ? w.split : w.kb0) * 64 * p.kgroup);
         else if (p.mode == MODE_BACKPROBE) kc = (int)w.kb0 * p.ksteps * 16;
-        else if (p.mode == MODE_CONV) { dx = dy = -p.pad; }     // pj counts channel blocks, kc = offset * Cin
-        else {
+        else if (p.mode == MODE_CONV) {      // pj counts channel blocks, kc = offset * Cin; w.img is a plane
+          dx = dy = -p.pad;
+          dz = -p.pad_d;
+          pz = w.img % p.depth;
+        } else {
           long q = w.kb0;
           px = (int)(q % p.patches_x); q /= p.patches_x;
           py = (int)(q % p.patches_y); q /= p.patches_y;
           pj = (int)q;
-          const int ks = 2 * p.pad + 1;
-          dy = w.tap / ks - p.pad;
-          dx = w.tap % ks - p.pad;
+          pz = pj % p.depth;
+          const int ks = 2 * p.pad + 1, tp = w.tap % (ks * ks);
+          dz = w.tap / (ks * ks) - p.pad_d;
+          dy = tp / ks - p.pad;
+          dx = tp % ks - p.pad;
         }
         for (int i = 0; i < w.nkb; ++i) {
           if (fill > 0) {
@@ -676,15 +691,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else if (p.mode == MODE_CONV) {
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
             // [tile_n output channels x 64 input channels] block of the weights
-            tma_load_5d(a_dst, &map_a, 0, w.px * p.patch_w + dx, w.py * p.patch_h + dy, pj, w.img, &full_bar[s]);
+            const bool inside = (unsigned)(pz + dz) < (unsigned)p.depth;
+            tma_load_5d(a_dst, &map_a, 0, w.px * p.patch_w + dx, inside ? w.py * p.patch_h + dy : p.H, pj, w.img + dz,
+                        &full_bar[s]);
             tma_load_2d(b_dst, &map_b, kc + (pj << p.cw_shift), col0, &full_bar[s]);
-            if (++pj == p.cgroups) { pj = 0; kc += p.Cin; if (++dx > p.pad) { dx = -p.pad; ++dy; } }
+            if (++pj == p.cgroups) {
+              pj = 0; kc += p.Cin;
+              if (++dx > p.pad) { dx = -p.pad; if (++dy > p.pad) { dy = -p.pad; ++dz; } }
+            }
           } else {
             // one 5-d box per operand: (64 channels, patch x, patch y, channel groups of 64, probe)
             const int x0 = px * p.patch_w, y0 = py * p.patch_h;
             tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, pj, &full_bar[s]);
-            tma_load_5d(b_dst, &map_b, 0, x0 + dx, y0 + dy, col0 >> p.cw_shift, pj, &full_bar[s]);
-            if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; } }
+            const bool inside = (unsigned)(pz + dz) < (unsigned)p.depth;
+            tma_load_5d(b_dst, &map_b, 0, x0 + dx, inside ? y0 + dy : p.H, col0 >> p.cw_shift, pj + dz, &full_bar[s]);
+            if (++px == p.patches_x) { px = 0; if (++py == p.patches_y) { py = 0; ++pj; if (++pz == p.depth) pz = 0; } }
           }
           ++it;
           if (++s == stages) { s = 0; ++fill; }
@@ -1142,6 +1163,7 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
   TcParams q = p;
   q.tag = call_tag();
   if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
+  if (q.depth < 1) q.depth = 1;
   e = launch_pdl(kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, mc ? *mc : ma, q);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
@@ -1329,8 +1351,8 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
       if ((budget - slots * BP_SLOT_BYTES) / stage >= want) { p->bp_slots = slots; break; }
     p->bp_stages = std::max(1, std::min(MAX_STAGES, (budget - p->bp_slots * BP_SLOT_BYTES) / stage));
   }
-  // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch)
-  const int T = d->KH * d->KW;
+  // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch); volumes: d->r counts planes
+  const int T = d->KH * d->KW * (d->KD > 1 ? d->KD : 1);
   p->ct_cw = (d->Cout % 64 == 0 && d->Cin % 64 == 0) ? 64 : ((d->Cout % 32 == 0 && d->Cin % 32 == 0) ? 32 : 0);
   if (p->ct_cw && (long)d->H * d->W >= 16) {
     mask |= 2;
@@ -1447,7 +1469,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
 
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const void* L, const void* Z, float* dW,
                              float alpha, char* ws_head, char* part, cudaStream_t st) {
-  const int T = d->KH * d->KW;
+  const int T = d->KH * d->KW * (d->KD > 1 ? d->KD : 1);
   const int bk = pl.patch_w * pl.patch_h;
   const bool f16 = d->dtype == XCONV_F16;
   CUtensorMap ma, mb;
@@ -1530,6 +1552,9 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.patches_x = pl.patches_x;
   p.patches_y = pl.patches_y;
   p.pad = (d->KH - 1) / 2;
+  p.depth = d->D > 1 ? d->D : 1;
+  p.pad_d = d->KD > 1 ? (d->KD - 1) / 2 : 0;
+  p.H = d->H;
   p.rows = d->Cout;
   p.cols = d->Cin;
   p.T = T;
@@ -1612,20 +1637,21 @@ bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
   // second image's rows then start on a group boundary): the traffic into the SM per MMA cycle falls
   // from 94 to 62.5 bytes, which is what bounded the convolution.
   const int px = p->patch_w * p->patch_h;
-  p->m_sub = (px % 8 == 0 && d->B >= 2) ? 2 : 1;
+  // (a kernel with a depth component shifts every plane on its own: one plane per unit then)
+  p->m_sub = (px % 8 == 0 && d->B >= 2 && d->KD <= 1) ? 2 : 1;
   // Input channels go by 64 per stage (128-byte tile rows); layers whose channel count is a multiple of 32
   // only take 32 per stage (64-byte rows, 64-byte swizzle).  (32 per stage everywhere, for more and smaller
   // stages, was slower: 557 against 485 us on the 256-channel layer.)
   const uint32_t rows = (uint32_t)(p->m_sub == 2 ? px + TILE_M : TILE_M) + (uint32_t)p->tile_n;
   p->cw = Ci % 64 == 0 ? 64 : 32;
   p->stages = pick_stages(rows * 2 * (uint32_t)p->cw, 1);
-  p->wt_bytes = dgrad ? (size_t)d->Cout * d->KH * d->KW * d->Cin * 2 : 0;
+  p->wt_bytes = dgrad ? (size_t)d->Cout * d->KH * d->KW * (d->KD > 1 ? d->KD : 1) * d->Cin * 2 : 0;
   return true;
 }
 
 xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, const void* in, const void* W,
                          void* out, char* ws_head, char* wt, cudaStream_t st) {
-  const int T = d->KH * d->KW;
+  const int T = d->KH * d->KW * (d->KD > 1 ? d->KD : 1);
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
   const bool f16 = d->dtype == XCONV_F16;
   const void* Wk = W;
@@ -1679,6 +1705,8 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& pl, bool dgrad, 
   p.patches_x = pl.patches_x;
   p.patches_y = pl.patches_y;
   p.pad = (d->KH - 1) / 2;
+  p.depth = d->D > 1 ? d->D : 1;
+  p.pad_d = d->KD > 1 ? (d->KD - 1) / 2 : 0;
   p.rows = (long)pl.patch_w * pl.patch_h;
   p.cols = Co;
   p.L = static_cast<bf16*>(out);

@@ -32,7 +32,10 @@ SHAPES = [
     ("f32", (2, 3, 4, 3, 5, 4, 5), 3, 3),             # odd everything
     ("f32", (1, 1, 1, 1, 1, 1, 1), 3, 3),             # a single voxel: only the centre weight sees data
     ("f32", (3, 16, 8, 4, 6, 6, 6), 3, 3),
-    ("bf16", (4, 32, 32, 4, 8, 8, 8), 3, 3),          # sketch and back-probe on tcgen05 (flat pixel axis)
+    ("bf16", (4, 32, 32, 4, 8, 8, 8), 3, 3),          # tcgen05 throughout: planes moved by the depth offset, 32-channel groups
+    ("bf16", (2, 64, 128, 6, 12, 12, 16), 3, 3),      # tcgen05, 27 offsets, r > B (contraction over image planes)
+    ("f16", (6, 64, 64, 3, 10, 7, 4), 3, 3),          # tcgen05, r < B (contraction over probe planes), ragged patches
+    ("bf16", (3, 64, 64, 1, 9, 9, 8), 3, 3),          # a volume one plane deep: two thirds of the offsets see only padding
     ("bf16", (8, 64, 64, 3, 6, 12, 16), 1, 3),        # planar kernel on every plane: tcgen05 throughout
     ("f16", (8, 64, 32, 2, 8, 8, 24), 1, 3),          # the same with r > B
     ("bf16", (4, 32, 16, 5, 6, 6, 12), 3, 3),         # r > B on a volume
@@ -46,6 +49,10 @@ def test_volume_layers_match_the_oracle(dtype, shape, KD, K):
     B, Cin, Cout, D, H, W, r = shape
     lay = _volume_layer(B, Cin, Cout, D, H, W, r, KD, K, dtype, seed=sum(shape) + KD)
     tol = TOL[dtype]
+    if dtype != "f32" and Cin % 32 == 0 and Cout % 32 == 0:
+        desc = xb.make_desc(B, Cin, Cout, H, W, r, {"bf16": torch.bfloat16, "f16": torch.float16}[dtype], K, D=D, KD=KD)
+        tc = "tcgen05_" + dtype
+        assert xb.engine_for(desc, xb.OP_CONTRACT) == tc and xb.engine_for(desc, xb.OP_FORWARD) == tc
     d = {k: xb.to_device(v, dtype) for k, v in lay.items()}
     Y, S = xb.xconv_forward(d["X"], d["W"], d["Z"])
     dW = xb.xconv_wgrad(S, d["dY"], d["Z"], kernel_size=K, kernel_depth=KD)
