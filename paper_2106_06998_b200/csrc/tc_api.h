@@ -21,6 +21,7 @@ struct TcSketchPlan {
 struct TcWgradPlan {
   // back-probe
   int bp_tile_n, bp_m_sub, bp_acc_bufs, bp_tiles_q, bp_tiles_r, bp_stages, bp_ksteps, bp_rows_box, bp_slots;
+  int bp_groups;             // epilogue warps per tensor-memory lane quadrant
   long bp_base, bp_rem;      // column tiles: bp_base blocks of 64 positions each, the first bp_rem one more
   // contraction
   int ct_cw, ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;

@@ -16,8 +16,8 @@
 //             patch per work unit; both tiles K-major (channels contiguous), the reduction runs over
 //             (offset, 64-channel block), and the offset again moves the TMA box of the input.
 //
-// Structure of a CTA (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..9 = epilogue (two per TMEM lane quadrant, sharing the columns of a tile).  A ring of shared-memory stages is handed
+// Structure of a CTA (192 or 320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 (2..9) = epilogue, one (two) per TMEM lane quadrant; two share the columns of a tile.  A ring of shared-memory stages is handed
 // from producer to issuer with mbarriers; tcgen05.commit returns stages and signals the epilogue.
 // Every wait is bounded: on expiry the CTA records the call's tag in the workspace header, drains
 // its outstanding copies (bounded again), frees its tensor memory and returns.
@@ -103,6 +103,7 @@ struct TcParams {
   // Volumes: the planes (probe x depth for CONTRACT, image x depth for CONV) are the outermost tensor axis; a
   // kernel offset with a depth component dz reads plane + dz, and where that leaves the volume the box is
   // sent to row H of the plane instead, which lies outside the image: the copy engine fills it with zeros.
+  int epi_groups;          // epilogue warps per tensor-memory lane quadrant (1 or 2): the launch has 64 + 128 * epi_groups threads
   int depth, pad_d;        // planes per probe or image (1: planar layer), depth padding of the kernel
   int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
   unsigned int* status;    // workspace header: [0] tag of a timed-out call, [1] tag of the last call
@@ -386,9 +387,11 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, bool f16) {
 
 constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
-constexpr int EPI_GROUPS = 2;                       // epilogue warps per tensor-memory lane quadrant
-constexpr int EPI_WARPS = 4 * EPI_GROUPS;
-constexpr int TC_THREADS = 64 + 32 * EPI_WARPS;
+// Epilogue warps per tensor-memory lane quadrant: one, or two where a tile's epilogue outlasts its mainloop (the
+// back-probe of small batches).  More epilogue warps than needed only take issue slots from the two
+// single-thread roles: with two everywhere the wide layers lost 10-25 %.
+constexpr int MAX_EPI_GROUPS = 2;
+constexpr int TC_THREADS = 64 + 128 * MAX_EPI_GROUPS;     // launch bound; a launch has 64 + 128 * epi_groups threads
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -435,7 +438,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
 // F16: the 16-bit storage type is float16 instead of bfloat16 (a compile-time constant, so that the epilogues'
 // conversions carry no selection between the two).
 template <bool F16>
-__global__ void __launch_bounds__(TC_THREADS, 2)
+__global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_c, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -454,8 +457,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 1 + EPI_WARPS : 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], EPI_WARPS); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 1 + 4 * p.epi_groups : 1); mbar_init(&empty_bar[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4 * p.epi_groups); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     prefetch_tmap(&map_a);
@@ -835,7 +838,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------------------------------------------ epilogue (warps 2..)
-    // A warp reads the 32 tensor-memory lanes of its quadrant (warp index mod 4); the EPI_GROUPS warps of a
+    // A warp reads the 32 tensor-memory lanes of its quadrant (warp index mod 4); the epi_groups warps of a
     // quadrant deal the column chunks (back-probe: the 64-position blocks) of a tile among themselves.
     const int quad = warp & 3;                  // TMEM lanes [32*quad, 32*quad+32)
     const int eg = (warp - 2) >> 2;             // which of the quadrant's warps
@@ -854,7 +857,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
         // copy would have produced, hand the stage over with one arrival per warp.
         const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
-        constexpr int GEN = 32 * EPI_WARPS;
+        const int GEN = 128 * p.epi_groups;
         const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
         const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
         const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
@@ -914,11 +917,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int mt = 0; mt < p.m_sub; ++mt) {
           const long row_w = ((long)w.tm * p.m_sub + mt) * TILE_M + quad * 32;
           if (row_w >= p.rows) continue;                                       // warp-uniform
-          for (int b = eg; b < w.nblk; b += EPI_GROUPS) {
+          for (int b = eg; b < w.nblk; b += p.epi_groups) {
             // the store that used this slot epi_slots blocks ago must have read it
             if (lane == 0) bulk_wait_read_upto(p.epi_slots - 1);
             __syncwarp();
-            const uint32_t slot_base = epi_base + ((uint32_t)(quad * EPI_GROUPS + eg) * p.epi_slots + epi_slot) * 4096u;
+            const uint32_t slot_base = epi_base + ((uint32_t)(quad * p.epi_groups + eg) * p.epi_slots + epi_slot) * 4096u;
             const uint32_t rowbase = slot_base + (uint32_t)lane * 128u;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
@@ -949,7 +952,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (row_w >= p.rows) continue;                                         // warp-uniform
         if (p.mode == MODE_CONV && w.img + mt >= p.nimg) continue;
         const long row = row_w + lane;
-        for (int cu = eg * 32; cu < unit_cols; cu += 32 * EPI_GROUPS) {
+        for (int cu = eg * 32; cu < unit_cols; cu += 32 * p.epi_groups) {
           // several offsets per unit (CONTRACT): tile_n is then a multiple of 32 and a chunk lies in one offset
           const int tap_l = unit_cols > p.tile_n ? cu / p.tile_n : 0;
           const int c = cu - tap_l * p.tile_n;
@@ -1111,7 +1114,7 @@ static inline int round_up(int v, int a) { return (v + a - 1) / a * a; }
 static const int SMEM_LIMIT = 227 * 1024;
 static const int STATIC_SMEM_SLACK = 2048;     // barriers + alignment slack
 static const int NUM_SMS = 148;
-static const int BP_SLOT_BYTES = EPI_WARPS * 32 * 128;   // back-probe output staging: per slot, one block of 32 rows x 64 positions per epilogue warp
+static const int BP_SLOT_BYTES = 4 * 32 * 128;      // back-probe output staging: per slot and epilogue group, 4 warps x 32 rows x 64 positions
 
 static PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
   static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
@@ -1164,7 +1167,8 @@ static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const T
   q.tag = call_tag();
   if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
   if (q.depth < 1) q.depth = 1;
-  e = launch_pdl(kernel, dim3(grid), dim3(TC_THREADS), smem, st, ma, mb, mc ? *mc : ma, q);
+  if (q.epi_groups < 1) q.epi_groups = 1;
+  e = launch_pdl(kernel, dim3(grid), dim3(64 + 128 * q.epi_groups), smem, st, ma, mb, mc ? *mc : ma, q);
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
@@ -1346,10 +1350,13 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
     // be in flight, but a unit's k-blocks should all fit the stage ring (at least four stages otherwise).
     const int budget = SMEM_LIMIT - STATIC_SMEM_SLACK;
     const int want = std::min(4, (int)cdivl(d->B, p->bp_ksteps * 16) + 1);
+    // a tile whose reduction over the batch is one or two stages long is over before its epilogue: two warps per quadrant
+    p->bp_groups = cdivl(d->B, p->bp_ksteps * 16) <= 2 ? 2 : 1;
+    const int slot_bytes = BP_SLOT_BYTES * p->bp_groups;
     p->bp_slots = 2;
     for (int slots = 8; slots >= 2; slots /= 2)
-      if ((budget - slots * BP_SLOT_BYTES) / stage >= want) { p->bp_slots = slots; break; }
-    p->bp_stages = std::max(1, std::min(MAX_STAGES, (budget - p->bp_slots * BP_SLOT_BYTES) / stage));
+      if ((budget - slots * slot_bytes) / stage >= want) { p->bp_slots = slots; break; }
+    p->bp_stages = std::max(1, std::min(MAX_STAGES, (budget - p->bp_slots * slot_bytes) / stage));
   }
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch); volumes: d->r counts planes
   const int T = d->KH * d->KW * (d->KD > 1 ? d->KD : 1);
@@ -1449,7 +1456,8 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.a_mn_major = 0;
   p.b_mn_major = 1;
   p.b_lbo = p.b_box_bytes;
-  p.epi_bytes = (uint32_t)pl.bp_slots * BP_SLOT_BYTES;
+  p.epi_groups = pl.bp_groups;
+  p.epi_bytes = (uint32_t)pl.bp_slots * BP_SLOT_BYTES * pl.bp_groups;
   p.epi_slots = pl.bp_slots;
   p.bp_base = pl.bp_base;
   p.bp_rem = pl.bp_rem;
