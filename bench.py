@@ -476,21 +476,6 @@ def run_xconv(args):
                                    "note": "of the two units of the method (sketch; estimator = back-probe + "
                                            "contraction with L not counted), the one furthest below its roofline"}}
 
-    # ---- the other probe counts of this workload's sweep (shorter runs), same step and timing
-    sweep = []
-    if not args.no_sweep and world == 1:
-        for r2 in c["r"]:
-            if r2 == r:
-                continue
-            Z2 = xb.to_device(inputs.make_layer(cfg, r2, tensors=("Z",))["Z"], c["dtype"], dev)
-            lay2 = Layer(r2, Z2)
-            n2 = max(5, min(args.steps, 30))
-            tot2, _, _ = lay2.measure(n2, 3, None, phase_events=False)
-            ph2, _ = lay2.measure_phases(n2)
-            sweep.append({"r": r2, "ms_per_step": tot2 / n2, "value": 1e3 * n2 / tot2, "phases": phase_table(r2, lay2.desc, ph2)})
-            del lay2, Z2
-            torch.cuda.empty_cache()
-
     # ---- the rest of the layer API on the same tensors: forward (conv + sketch) and exact dX
     full = None
     if not args.no_context:
@@ -501,8 +486,8 @@ def run_xconv(args):
         wsf = torch.empty(max(xb.workspace_bytes(desc, xb.OP_FORWARD), xb.workspace_bytes(desc, xb.OP_DGRAD)),
                           dtype=torch.uint8, device=dev)
 
-        def _time(f, n=5):
-            for _ in range(2):
+        def _time(f, n=20):
+            for _ in range(3):
                 f()
             a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a_.record()
@@ -525,6 +510,21 @@ def run_xconv(args):
                 "note": "xconv_forward = conv + sketch; xconv_dgrad = exact dX; xconv_wgrad = back-probe + contraction "
                         "in one call; *_seeded: probes redrawn from a seed instead of read from memory; not part of the metric"}
         del Y, dX, wsf, wss
+
+    # ---- the other probe counts of this workload's sweep (shorter runs), same step and timing
+    sweep = []
+    if not args.no_sweep and world == 1:
+        for r2 in c["r"]:
+            if r2 == r:
+                continue
+            Z2 = xb.to_device(inputs.make_layer(cfg, r2, tensors=("Z",))["Z"], c["dtype"], dev)
+            lay2 = Layer(r2, Z2)
+            n2 = max(5, min(args.steps, 30))
+            tot2, _, _ = lay2.measure(n2, 3, None, phase_events=False)
+            ph2, _ = lay2.measure_phases(n2)
+            sweep.append({"r": r2, "ms_per_step": tot2 / n2, "value": 1e3 * n2 / tot2, "phases": phase_table(r2, lay2.desc, ph2)})
+            del lay2, Z2
+            torch.cuda.empty_cache()
 
     cpu = None
     if not args.no_cpu:

@@ -1074,17 +1074,38 @@ reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S, lo
 }
 
 // out[m][offset][n] = scale(n) * sum_s block_s[...]: walks one split's blocks in their stored order (see the
-// epilogue of MODE_CONTRACT), four consecutive input channels per thread, splits added in ascending order.
+// epilogue of MODE_CONTRACT), four consecutive input channels per group.  LANES threads share a group and take the
+// splits in turn (one thread per group would walk a chain of `splits` dependent loads: 41 us for the 296 splits
+// of a 32-channel layer); their sums are added in lane order, so the result is reproducible.
+template <int LANES>
 __global__ void __launch_bounds__(256) reduce_contract_partials(const float* __restrict__ part, float* __restrict__ out,
                                                                 long groups, long split_stride, int splits, int T,
                                                                 int tiles_m, int tiles_n, int m_sub, int tile_n,
                                                                 int Cout, int Cin, float alpha,
                                                                 const float* __restrict__ chan_scale) {
+  constexpr int GROUPS = 256 / LANES;
+  __shared__ float4 acc[LANES][GROUPS];
   pdl_trigger();
   pdl_wait();
-  long t = (long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= groups) return;
-  const long idx = t;
+  const int o = threadIdx.x % GROUPS, g = threadIdx.x / GROUPS;
+  const long idx = (long)blockIdx.x * GROUPS + o;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (idx < groups) {
+#pragma unroll 4
+    for (int k = g; k < splits; k += LANES) {
+      const float4 v = *reinterpret_cast<const float4*>(part + (long)k * split_stride + idx * 4);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+  }
+  if (LANES > 1) {
+    acc[g][o] = s;
+    __syncthreads();
+    if (g != 0) return;
+#pragma unroll
+    for (int l = 1; l < LANES; ++l) { s.x += acc[l][o].x; s.y += acc[l][o].y; s.z += acc[l][o].z; s.w += acc[l][o].w; }
+  }
+  if (idx >= groups) return;
+  long t = idx;
   const int row = (int)(t % TILE_M); t /= TILE_M;
   const int q = (int)(t % 8); t /= 8;
   const int chunks = tile_n >> 5;
@@ -1096,12 +1117,6 @@ __global__ void __launch_bounds__(256) reduce_contract_partials(const float* __r
   const int m = (tm * m_sub + mt) * TILE_M + row;
   const int n = tn * tile_n + chunk * 32 + q * 4;
   if (m >= Cout || n >= Cin) return;
-  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-  for (int k = 0; k < splits; ++k) {
-    const float4 v = *reinterpret_cast<const float4*>(part + (long)k * split_stride + idx * 4);
-    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
-  }
   float4 sc = make_float4(alpha, alpha, alpha, alpha);
   if (chan_scale) sc = make_float4(chan_scale[n], chan_scale[n + 1], chan_scale[n + 2], chan_scale[n + 3]);
   *reinterpret_cast<float4*>(out + ((long)m * T + tap) * Cin + n) = make_float4(s.x * sc.x, s.y * sc.y, s.z * sc.z, s.w * sc.w);
@@ -1573,9 +1588,14 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   if (s != XCONV_OK) return s;
   const long split_stride = (long)T * pl.ct_tiles_m * pl.ct_tiles_n * pl.ct_m_sub * TILE_M * pl.ct_tile_n;
   const long groups = split_stride / 4;
-  cudaError_t e = launch_pdl(reduce_contract_partials, dim3((unsigned)cdivl(groups, 256)), dim3(256), 0, st, p.part,
-                             dW, groups, split_stride, pl.ct_splits, T, pl.ct_tiles_m, pl.ct_tiles_n, pl.ct_m_sub,
-                             pl.ct_tile_n, d->Cout, d->Cin, alpha, d->chan_scale);
+  cudaError_t e;
+#define XC_REDUCE(LANES) launch_pdl(reduce_contract_partials<LANES>, dim3((unsigned)cdivl(groups, 256 / LANES)), dim3(256), 0, st, \
+                                    p.part, dW, groups, split_stride, pl.ct_splits, T, pl.ct_tiles_m, pl.ct_tiles_n, \
+                                    pl.ct_m_sub, pl.ct_tile_n, d->Cout, d->Cin, alpha, d->chan_scale)
+  if (pl.ct_splits >= 64) e = XC_REDUCE(16);
+  else if (pl.ct_splits >= 12) e = XC_REDUCE(4);
+  else e = XC_REDUCE(1);
+#undef XC_REDUCE
   count_launch();
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
   return XCONV_OK;
