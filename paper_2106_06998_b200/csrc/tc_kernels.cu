@@ -399,32 +399,38 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 
 struct Unit { int tm, tn, tap; long split, kb0; int nkb; int px, py, img; int blk0, nblk; };
 
-__device__ __forceinline__ Unit decode_unit(const TcParams& p, long u) {
+// Work unit u -> tile, offset, k-split.  32-bit divisions throughout (a launch has far fewer than 2^31 units):
+// every role of a CTA decodes each of its units on its own critical path, one instruction per ~6 clocks, and a
+// 64-bit division is a 100-instruction routine -- with one-stage tiles the decode alone was half the time per tile.
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, long u_) {
   Unit w;
+  const uint32_t u = (uint32_t)u_;
   w.px = w.py = w.img = 0;
   w.blk0 = w.nblk = 0;
   if (p.mode == MODE_CONV) {                 // channel tiles innermost, then patches of one image
-    long q = u;
-    w.tn = (int)(q % p.tiles_n); q /= p.tiles_n;
-    w.px = (int)(q % p.patches_x); q /= p.patches_x;
-    w.py = (int)(q % p.patches_y); q /= p.patches_y;
+    uint32_t q = u;
+    const uint32_t tn = (uint32_t)p.tiles_n, px = (uint32_t)p.patches_x, py = (uint32_t)p.patches_y;
+    w.tn = (int)(q % tn); q /= tn;
+    w.px = (int)(q % px); q /= px;
+    w.py = (int)(q % py); q /= py;
     w.img = (int)q * p.m_sub;
     w.tm = 0; w.tap = 0; w.split = 0;
   } else if (p.mode == MODE_BACKPROBE) {     // probe tiles innermost: the dY tile is re-read while hot in L2
-    w.tm = (int)(u % p.tiles_m);
-    w.tn = (int)(u / p.tiles_m);
+    const uint32_t tm = (uint32_t)p.tiles_m;
+    w.tm = tm == 1 ? 0 : (int)(u % tm);
+    w.tn = tm == 1 ? (int)u : (int)(u / tm);
     w.tap = 0;
     w.split = 0;
     // column tile tn covers blocks [blk0, blk0 + nblk) of 64 positions
-    w.blk0 = (int)(w.tn * p.bp_base + min((long)w.tn, p.bp_rem));
-    w.nblk = (int)p.bp_base + (w.tn < p.bp_rem ? 1 : 0);
+    w.blk0 = w.tn * (int)p.bp_base + min(w.tn, (int)p.bp_rem);
+    w.nblk = (int)p.bp_base + (w.tn < (int)p.bp_rem ? 1 : 0);
   } else {                                   // tiles of one k-split are adjacent: they share operands in L2
     const int tpu = p.mode == MODE_CONTRACT ? p.tpu : 1;
-    const long tiles = (long)(p.taps / tpu) * p.tiles_m * p.tiles_n;
-    long t = u % tiles;
+    const uint32_t tiles = (uint32_t)((p.taps / tpu) * p.tiles_m * p.tiles_n);
+    uint32_t t = u % tiles;
     w.split = u / tiles;
-    w.tn = (int)(t % p.tiles_n); t /= p.tiles_n;
-    w.tm = (int)(t % p.tiles_m); t /= p.tiles_m;
+    w.tn = (int)(t % (uint32_t)p.tiles_n); t /= (uint32_t)p.tiles_n;
+    w.tm = (int)(t % (uint32_t)p.tiles_m); t /= (uint32_t)p.tiles_m;
     w.tap = (int)t * tpu;                      // first offset of the unit
   }
   w.kb0 = w.split * p.kblocks_per_split + min(w.split, p.kb_rem);
@@ -494,9 +500,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const Unit w = decode_unit(p, u);
       const int row0 = w.tm * p.m_sub * TILE_M;
       const int col0 = w.tn * p.tile_n;
-      long q = w.kb0;
-      int px = (int)(q % p.patches_x); q /= p.patches_x;
-      int py = (int)(q % p.patches_y); q /= p.patches_y;
+      uint32_t q = (uint32_t)w.kb0;
+      int px = (int)(q % (uint32_t)p.patches_x); q /= (uint32_t)p.patches_x;
+      int py = (int)(q % (uint32_t)p.patches_y); q /= (uint32_t)p.patches_y;
       int pj = (int)q;
       const int tap = w.tap + max(0, min(lane - 1, p.tpu - 1));          // this lane's offset
       const int dy = tap / ks - p.pad, dx = tap % ks - p.pad;
@@ -537,9 +543,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
         const int row0 = w.tm * p.m_sub * TILE_M, col0 = w.tn * p.tile_n;
-        long q = w.kb0;
-        int px = (int)(q % p.patches_x); q /= p.patches_x;
-        int py = (int)(q % p.patches_y); q /= p.patches_y;
+        uint32_t q = (uint32_t)w.kb0;
+        int px = (int)(q % (uint32_t)p.patches_x); q /= (uint32_t)p.patches_x;
+        int py = (int)(q % (uint32_t)p.patches_y); q /= (uint32_t)p.patches_y;
         int pj = (int)q;
         const int ks = 2 * p.pad + 1, tp = w.tap % (ks * ks), dy = tp / ks - p.pad, dx = tp % ks - p.pad;
         const int dz = w.tap / (ks * ks) - p.pad_d;
@@ -653,9 +659,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           dz = -p.pad_d;
           pz = w.img % p.depth;
         } else {
-          long q = w.kb0;
-          px = (int)(q % p.patches_x); q /= p.patches_x;
-          py = (int)(q % p.patches_y); q /= p.patches_y;
+          uint32_t q = (uint32_t)w.kb0;
+          px = (int)(q % (uint32_t)p.patches_x); q /= (uint32_t)p.patches_x;
+          py = (int)(q % (uint32_t)p.patches_y); q /= (uint32_t)p.patches_y;
           pj = (int)q;
           pz = pj % p.depth;
           const int ks = 2 * p.pad + 1, tp = w.tap % (ks * ks);
@@ -752,8 +758,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
         const Unit w = decode_unit(p, u);
         if (w.nkb == 0) continue;
-        const int buf = (int)(lu % p.acc_bufs);
-        const long use = lu / p.acc_bufs;
+        const int buf = p.acc_bufs == 2 ? (int)(lu & 1) : 0;          // (no division: this thread's stream is the critical path)
+        const long use = p.acc_bufs == 2 ? lu >> 1 : lu;
         if (use > 0) {                      // the epilogue must have emptied this accumulator set
           ok = mbar_wait(&tmem_empty_bar[buf], (uint32_t)((use - 1) & 1), p.status, p.tag);
           if (!ok) break;
@@ -850,8 +856,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     bool ok = true;
     for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
       const Unit w = decode_unit(p, u);
-      const int buf = (int)(lu % p.acc_bufs);
-      const long use = lu / p.acc_bufs;
+      const int buf = p.acc_bufs == 2 ? (int)(lu & 1) : 0;
+      const long use = p.acc_bufs == 2 ? lu >> 1 : lu;
       if (p.seeded && p.mode == MODE_SKETCH) {
         // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
         // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
