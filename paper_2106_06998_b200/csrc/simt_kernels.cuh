@@ -201,11 +201,12 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
 #pragma unroll
       for (int k = 0; k < 4; ++k) acc[t][i][k] = 0.f;
 
+  // (x chunk, row, plane) of the first item, then stepped along: a 64-bit division per item costs as much as a
+  // sixth of the item's arithmetic
+  int xc = (int)(ib % chunks), y = (int)((ib / chunks) % H);
+  long jz = ib / ((long)chunks * H);                      // plane index j * D + z
+  int z = (int)(jz % D);
   for (long it = ib; it < ie; ++it) {
-    const int xc = (int)(it % chunks);
-    const int y = (int)((it / chunks) % H);
-    const long jz = it / ((long)chunks * H);              // plane index j * D + z
-    const int z = (int)(jz % D);
     const int x0 = xc * XC;
     if (VEC) {
       // channel counts are multiples of 4: four consecutive channels per load (the tiles fill in a quarter
@@ -264,6 +265,7 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
         }
     }
     __syncthreads();
+    if (++xc == chunks) { xc = 0; if (++y == H) { y = 0; ++jz; if (++z == D) z = 0; } }
   }
   float* out = part + (long)blockIdx.z * Cout * TALL * Cin;
 #pragma unroll

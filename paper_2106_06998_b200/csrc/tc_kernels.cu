@@ -1058,14 +1058,14 @@ reduce_sketch_partials(const float* __restrict__ part, float* __restrict__ S, lo
   for (int l = 1; l < RS_LANES; ++l) {
     t4[0] += acc[l][o].x; t4[1] += acc[l][o].y; t4[2] += acc[l][o].z; t4[3] += acc[l][o].w;
   }
-  long t = idx;
-  const int qn = tile_n < 32 ? tile_n >> 2 : 8;
+  uint32_t t = (uint32_t)idx;                   // (32-bit divisions: far fewer than 2^31 groups)
+  const uint32_t qn = tile_n < 32 ? tile_n >> 2 : 8;
   const int row = (int)(t % TILE_M); t /= TILE_M;
   const int q = (int)(t % qn); t /= qn;
-  const int chunks = (tile_n + 31) >> 5;
+  const uint32_t chunks = (uint32_t)(tile_n + 31) >> 5;
   const int chunk = (int)(t % chunks); t /= chunks;
-  const int mt = (int)(t % m_sub); t /= m_sub;
-  const int tn = (int)(t % tiles_n); t /= tiles_n;
+  const int mt = (int)(t % (uint32_t)m_sub); t /= (uint32_t)m_sub;
+  const int tn = (int)(t % (uint32_t)tiles_n); t /= (uint32_t)tiles_n;
   const int tm = (int)t;
   const long rr = (long)(tm * m_sub + mt) * TILE_M + row;
   const int cl = chunk * 32 + q * 4;
@@ -1111,14 +1111,14 @@ __global__ void __launch_bounds__(256) reduce_contract_partials(const float* __r
     for (int l = 1; l < LANES; ++l) { s.x += acc[l][o].x; s.y += acc[l][o].y; s.z += acc[l][o].z; s.w += acc[l][o].w; }
   }
   if (idx >= groups) return;
-  long t = idx;
+  uint32_t t = (uint32_t)idx;                   // (32-bit divisions: far fewer than 2^31 groups)
   const int row = (int)(t % TILE_M); t /= TILE_M;
-  const int q = (int)(t % 8); t /= 8;
-  const int chunks = tile_n >> 5;
+  const int q = (int)(t % 8u); t /= 8u;
+  const uint32_t chunks = (uint32_t)tile_n >> 5;
   const int chunk = (int)(t % chunks); t /= chunks;
-  const int mt = (int)(t % m_sub); t /= m_sub;
-  const int tn = (int)(t % tiles_n); t /= tiles_n;
-  const int tm = (int)(t % tiles_m); t /= tiles_m;
+  const int mt = (int)(t % (uint32_t)m_sub); t /= (uint32_t)m_sub;
+  const int tn = (int)(t % (uint32_t)tiles_n); t /= (uint32_t)tiles_n;
+  const int tm = (int)(t % (uint32_t)tiles_m); t /= (uint32_t)tiles_m;
   const int tap = (int)t;
   const int m = (tm * m_sub + mt) * TILE_M + row;
   const int n = tn * tile_n + chunk * 32 + q * 4;
