@@ -41,7 +41,7 @@ pinned by exact recovery with one orthogonal basis per channel, by unbiasedness 
 Hutchinson variance, and by their reduction to the multi-channel functions for a single input channel.
 The functions for volumes (shift3, conv_forward3d, dw_exact3d, dx_exact3d, wgrad_contract3d, wgrad_estimate3d) are
 pinned by brute-force loops, by their reduction to the two-dimensional functions at depth 1, and by exact recovery.
-rel_fro, the metric every parity verdict passes through, is pinned on a hand-computed pair.
+rel_fro, the metric every parity check passes through, is pinned on a hand-computed pair.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
