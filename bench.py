@@ -265,9 +265,10 @@ def run_xconv(args):
         the 126 MB L2 is held in several copies at different addresses and the steps rotate through them,
         so that every step finds its inputs in HBM, not in L2."""
 
-        def __init__(self, r_, Z_):
+        def __init__(self, r_, Z_, zero_blocks=None):
             self.r = r_
-            self.desc = xb.make_desc(B, Cin, Cout, H, W, r_, tdt)
+            self.zero_blocks = zero_blocks        # kept alive: the descriptor holds its address
+            self.desc = xb.make_desc(B, Cin, Cout, H, W, r_, tdt, zero_blocks=zero_blocks)
             self.S = torch.empty((r_, B), dtype=torch.float32, device=dev)
             self.dW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device=dev, memory_format=torch.channels_last)
             set_bytes = X.element_size() * (X.numel() + dY.numel() + Z_.numel() + r_ * Cout * H * W)
@@ -532,6 +533,43 @@ def run_xconv(args):
             del lay2, Z2
             torch.cuda.empty_cache()
 
+    # ---- block-sparse probes (Eq. 7) on this workload: the contraction told which 64-channel blocks of Z are zero
+    block_sparse = None
+    if (not args.no_sweep and world == 1 and tdt != torch.float32 and Cin % 64 == 0 and Cout % 64 == 0
+            and Cin % min(256, Cin) == 0 and r <= B):
+        block_sparse = []
+        n3 = max(5, min(args.steps, 30))
+        tile = min(256, Cin) // 64          # 64-channel blocks per column tile of the contraction
+
+        def sparse_case(r3, Z3, pg, whole_tiles):
+            gen = torch.Generator(device="cpu").manual_seed(inputs.seed_for(cfg, r3, "Z") + int(1000 * pg) + whole_tiles)
+            if whole_tiles:                 # the blocks of a probing vector inside a column tile are kept or dropped together
+                keep = (torch.rand((r3, Cin // 64 // tile), generator=gen) < pg).repeat_interleave(tile, dim=1).to(dev)
+            else:
+                keep = (torch.rand((r3, Cin // 64), generator=gen) < pg).to(dev)
+            Zs = (Z3 * keep.repeat_interleave(64, dim=1)[:, :, None, None].to(tdt)).contiguous(memory_format=torch.channels_last)
+            zb = xb.xconv_zero_blocks(Zs)
+            lay3 = Layer(r3, Zs, zero_blocks=zb)
+            used = xb.zero_blocks_used(lay3.desc)
+            xb.sketch_into(lay3.desc, X, Zs, lay3.S, lay3.ws)
+            t3, _ = lay3.measure_phase("contract", n3)
+            listed = float((zb.view(r3, -1, tile) == 0).any(dim=2).float().mean())
+            del lay3
+            torch.cuda.empty_cache()
+            return {"r": r3, "p_block": pg, "blocks": "256 channels" if whole_tiles else "64 channels",
+                    "zero_share": float(zb.float().mean()), "probes_read_share": listed, "skipping": used, "contract_ms": t3}
+
+        for pg in (1.0, 0.5, 0.25, 0.125):
+            block_sparse.append(sparse_case(r, Z, pg, True))
+        for pg in (0.5, 0.125):
+            block_sparse.append(sparse_case(r, Z, pg, False))
+        if 256 in c["r"] and r != 256:
+            Z256 = xb.to_device(inputs.make_layer(cfg, 256, tensors=("Z",))["Z"], c["dtype"], dev)
+            for pg in (1.0, 0.5):
+                block_sparse.append(sparse_case(256, Z256, pg, True))
+            del Z256
+            torch.cuda.empty_cache()
+
     cpu = None
     if not args.no_cpu:
         t, ts, tw, sample = oracle_sample_time(cfg, r, frac=args.oracle_frac)
@@ -570,6 +608,14 @@ def run_xconv(args):
                                      "three calls, which keeps a kernel's preamble from overlapping the previous "
                                      "kernel's tail (diagnostic)"},
             "sweep": sweep, "layer_api": full,
+            "block_sparse": None if block_sparse is None else {
+                "cases": block_sparse,
+                "dense_contract_ms": {str(r): phases["contract"]["ms"],
+                                      **{str(e["r"]): e["phases"]["contract"]["ms"] for e in sweep if e["r"] == 256}},
+                "note": "xconv_contract with desc.zero_blocks (Eq. 7): blocks of Z kept with probability p_block and named "
+                        "to the contraction when zero; per column tile of 256 channels it reads and multiplies only the "
+                        "probing vectors with a non-zero block there (probes_read_share), so blocks of 256 channels are "
+                        "skipped in proportion and independent 64-channel blocks only where all four of a tile are zero"},
             "memory_ratio": {"elements": Cin * H * W / r, "stored_bytes": Cin * H * W * es / (4.0 * r)},
             "context": context}
     print(json.dumps(line))

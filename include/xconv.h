@@ -92,7 +92,20 @@ typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TC
  * [B,D,H,W,C], Z [r,D,H,W,Cin], W and dW [Cout,KD,KH,KW,Cin] (torch's channels_last_3d of NCDHW / OIDHW),
  * and every formula above gains the matching sum over kz and shift z + kz - pad_d.  KD = 3 (with KH = KW = 3,
  * pad_d = 1) is a 3 x 3 x 3 kernel; KD = 1 (pad_d = 0) applies a planar kernel to every plane.  D, KD and
- * pad_d of 0 (a zero-initialised tail) mean a planar layer, the same as D = KD = 1. */
+ * pad_d of 0 (a zero-initialised tail) mean a planar layer, the same as D = KD = 1.
+ *
+ * zero_blocks (block-sparse probes, Eq. 7: block n of probing vector j is zero with probability 1 - p_n, so a
+ * share of the terms of Eq. 8's sum over j vanishes and need not be formed).  Byte [j*(Cin/64) + g] non-zero is the
+ * caller's promise that Z[j, ..., 64g .. 64g+63] is identically zero.  On the layers for which
+ * xconv_zero_blocks_used returns 1 -- wide layers on the tensor cores (Cin and Cout multiples of 64, the whole
+ * contraction one work unit per SM), planar or 3 x 3 x 3 volumes -- xconv_contract and xconv_wgrad (in the paper's
+ * order of summation, r <= B) then work on column tiles of up to 256 input channels and, for each tile, neither
+ * fetch nor multiply the probing vectors whose blocks in that tile are all named zero; their work falls in
+ * proportion.  Everywhere else the field is ignored, which gives the same result since the blocks are zero.
+ * The mask is read, never written; xconv_zero_blocks computes it from Z.  A block that is named zero but is not
+ * either enters the sum or drops out of it (it drops out when all blocks of its probing vector in its tile are
+ * named zero); no error is raised.  The workspace an op needs depends on whether the field is NULL: ask
+ * xconv_workspace_bytes with the descriptor the call will get.  A zero-initialised tail means no mask. */
 typedef struct {
   int32_t B, Cin, Cout, H, W;
   int32_t KH, KW, pad_h, pad_w;
@@ -101,6 +114,7 @@ typedef struct {
   int32_t circular;         /* must be 0 (truncating shifts) */
   const float* chan_scale;  /* NULL: scale 1/r.  Else device pointer to Cin floats (Eq. 8). */
   int32_t D, KD, pad_d;     /* depth of the volume and of the kernel; 0 or 1: planar layer */
+  const unsigned char* zero_blocks;  /* NULL, or device pointer to r * (Cin/64) bytes: see below */
 } xconv_desc;
 
 /* Scratch bytes `op` needs for this layer (0 is possible).  Returns 0 for an invalid descriptor. */
@@ -162,6 +176,17 @@ xconv_status xconv_backprobe(const xconv_desc* desc, const float* sketch, const 
                              void* ws, size_t ws_bytes, void* cuda_stream);
 xconv_status xconv_contract(const xconv_desc* desc, const void* L, const void* Z, float* dW,
                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* mask[j*(Cin/64) + g] = 1 if every element of Z[j, ..., 64g .. 64g+63] is +0 or -0, else 0 (the mask
+ * desc.zero_blocks takes).  Z [r,H,W,Cin] (volumes [r,D,H,W,Cin])
+ * in desc.dtype, mask r*(Cin/64) bytes, both device pointers.  Cin must be a multiple of 64
+ * (XCONV_ERR_UNSUPPORTED otherwise).  One pass over Z; no scratch. */
+xconv_status xconv_zero_blocks(const xconv_desc* desc, const void* Z, unsigned char* mask, void* cuda_stream);
+
+/* 1 if xconv_contract skips the blocks that desc.zero_blocks names on this layer (and with it xconv_wgrad,
+ * unless r > B makes that call sum over the probes first), 0 if the field is ignored there (or NULL, or the
+ * descriptor invalid).  Host-side arithmetic only. */
+int xconv_zero_blocks_used(const xconv_desc* desc);
 
 /* Trace estimation applied to every input/output channel pair on its own ("independent" probing: first
  * sentence of the multi-channel case in Section 3; Eq. 4 per pair).  The probing vectors have the same shape

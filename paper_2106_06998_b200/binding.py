@@ -25,7 +25,7 @@ STATUS_OK = 0
 EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_sketch", "xconv_wgrad",
            "xconv_dgrad", "xconv_probes_from_seed", "xconv_sketch_seeded", "xconv_wgrad_seeded", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
            "xconv_workspace_status", "xconv_selftest_wait_limit", "xconv_measure_fma_rate",
-           "xconv_sketch_independent", "xconv_wgrad_independent",
+           "xconv_sketch_independent", "xconv_wgrad_independent", "xconv_zero_blocks", "xconv_zero_blocks_used",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -33,7 +33,7 @@ class XConvDesc(Structure):
     _fields_ = [("B", c_int32), ("Cin", c_int32), ("Cout", c_int32), ("H", c_int32), ("W", c_int32),
                 ("KH", c_int32), ("KW", c_int32), ("pad_h", c_int32), ("pad_w", c_int32), ("r", c_int32),
                 ("dtype", c_int32), ("circular", c_int32), ("chan_scale", c_void_p),
-                ("D", c_int32), ("KD", c_int32), ("pad_d", c_int32)]
+                ("D", c_int32), ("KD", c_int32), ("pad_d", c_int32), ("zero_blocks", c_void_p)]
 
 
 class XConvError(RuntimeError):
@@ -75,6 +75,9 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_independent.restype = c_int
     L.xconv_wgrad_independent.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad_independent.restype = c_int
+    L.xconv_zero_blocks.argtypes = [P, c_void_p, c_void_p, c_void_p]
+    L.xconv_zero_blocks.restype = c_int
+    L.xconv_zero_blocks_used.argtypes = [P]; L.xconv_zero_blocks_used.restype = c_int
     L.xconv_backprobe_bytes.argtypes = [P]; L.xconv_backprobe_bytes.restype = c_size_t
     L.xconv_backprobe.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_backprobe.restype = c_int
@@ -110,11 +113,37 @@ def _dtype_code(t: torch.dtype) -> int:
     raise TypeError(f"libxconv stores float32, bfloat16 or float16, got {t}")
 
 
-def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1) -> XConvDesc:
-    """Layer descriptor; D > 1 describes a volume (tensors gain a depth axis), KD its kernel depth (1 or 3)."""
+def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1, zero_blocks=None) -> XConvDesc:
+    """Layer descriptor; D > 1 describes a volume (tensors gain a depth axis), KD its kernel depth (1 or 3);
+    zero_blocks: uint8 CUDA tensor [r, Cin/64] marking the all-zero 64-channel blocks of the probing vectors."""
     code = dtype if isinstance(dtype, int) else _dtype_code(dtype)
     cs = chan_scale.data_ptr() if chan_scale is not None else None
-    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs, D, KD, (KD - 1) // 2)
+    zb = None
+    if zero_blocks is not None:
+        if (zero_blocks.dtype != torch.uint8 or not zero_blocks.is_cuda or not zero_blocks.is_contiguous()
+                or Cin % 64 != 0 or tuple(zero_blocks.shape) != (r, Cin // 64)):
+            raise ValueError("zero_blocks must be a contiguous uint8 CUDA tensor [r, Cin/64] (Cin a multiple of 64)")
+        zb = zero_blocks.data_ptr()
+    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs, D, KD, (KD - 1) // 2, zb)
+
+
+def zero_blocks_used(desc: XConvDesc) -> bool:
+    """Whether the contraction of this layer skips the blocks desc.zero_blocks names (else the field is ignored)."""
+    return bool(lib().xconv_zero_blocks_used(ctypes.byref(desc)))
+
+
+def xconv_zero_blocks(Z: torch.Tensor) -> torch.Tensor:
+    """uint8 [r, Cin/64]: 1 where the 64-channel block of a probing vector holds only zeros (the mask that
+    xconv_contract / xconv_wgrad take as zero_blocks)."""
+    _cl(Z, "Z")
+    r, Cin = Z.shape[:2]
+    D, H, W = _geo(Z)
+    if Cin % 64 != 0:
+        raise ValueError("Cin must be a multiple of 64")
+    desc = make_desc(1, Cin, 64, H, W, r, Z.dtype, D=D)
+    mask = torch.empty((r, Cin // 64), dtype=torch.uint8, device=Z.device)
+    _check(lib().xconv_zero_blocks(ctypes.byref(desc), Z.data_ptr(), mask.data_ptr(), _stream()), "xconv_zero_blocks")
+    return mask
 
 
 def _cl(t: torch.Tensor, name: str) -> torch.Tensor:
@@ -322,7 +351,8 @@ def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
 
 
 def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
-                chan_scale: torch.Tensor | None = None, kernel_depth: int = 1) -> torch.Tensor:
+                chan_scale: torch.Tensor | None = None, kernel_depth: int = 1,
+                zero_blocks: torch.Tensor | None = None) -> torch.Tensor:
     """dW estimate (Algorithm 1 backward steps 3-4): float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY"); _cl(Z, "Z")
     B, Cout = dY.shape[:2]
@@ -335,7 +365,7 @@ def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_
     if chan_scale is not None and (chan_scale.dtype != torch.float32 or chan_scale.numel() != Cin):
         raise ValueError("chan_scale must hold Cin float32 values")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale, D=D, KD=kernel_depth)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks)
     dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
     wgrad_into(desc, sketch, dY, Z, dW, ws)
@@ -394,7 +424,8 @@ def xconv_backprobe(sketch: torch.Tensor, dY: torch.Tensor) -> torch.Tensor:
 
 
 def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
-                   chan_scale: torch.Tensor | None = None, kernel_depth: int = 1) -> torch.Tensor:
+                   chan_scale: torch.Tensor | None = None, kernel_depth: int = 1,
+                   zero_blocks: torch.Tensor | None = None) -> torch.Tensor:
     """dW[m,n,k] = scale[n] * sum L[j,m,.] Z[j,n,.+k] (Algorithm 1 backward step 4)."""
     _cl(L, "L"); _cl(Z, "Z")
     r, Cout = L.shape[:2]
@@ -403,7 +434,7 @@ def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
     if Z.shape[0] != r or tuple(Z.shape[2:]) != tuple(L.shape[2:]) or Z.dtype != L.dtype:
         raise ValueError("shape or dtype mismatch between L and Z")
     K = kernel_size
-    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale, D=D, KD=kernel_depth)
+    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks)
     dW = _like((Cout, Cin), (kernel_depth, K, K), L.dim(), dtype=torch.float32, device=L.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), L.device)
     contract_into(desc, L, Z, dW, ws)

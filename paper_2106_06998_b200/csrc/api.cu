@@ -72,6 +72,7 @@ static xconv_desc flat(const xconv_desc* d) {
   xconv_desc f = *d;
   f.H = d->H * depth(d);
   f.D = 1; f.KD = 1; f.pad_d = 0;
+  f.zero_blocks = nullptr;
   return f;
 }
 // The tensor-core contraction and convolution work plane by plane: D times the probes for the contraction,
@@ -80,7 +81,10 @@ static xconv_desc flat(const xconv_desc* d) {
 static xconv_desc planes_ct(const xconv_desc* d) {
   xconv_desc f = *d;
   f.r = d->r * depth(d);
-  if (kdepth(d) == 1) { f.D = 1; f.KD = 1; f.pad_d = 0; }
+  if (kdepth(d) == 1) {
+    f.D = 1; f.KD = 1; f.pad_d = 0;
+    if (depth(d) > 1) f.zero_blocks = nullptr;      // the mask is per probe, and r now counts planes
+  }
   return f;
 }
 static xconv_desc planes_cv(const xconv_desc* d) {
@@ -183,6 +187,7 @@ static SwappedWgrad plan_wgrad_swapped(const xconv_desc* d) {
   if (!w.on) return w;
   w.d1 = *d; w.d1.B = d->r; w.d1.r = d->B; w.d1.Cout = d->Cin; w.d1.chan_scale = nullptr;
   w.d2 = *d; w.d2.r = d->B;
+  w.d1.zero_blocks = w.d2.zero_blocks = nullptr;      // neither step sums over the probes block by block
   w.p1 = plan_wgrad_core(&w.d1);
   w.p2 = plan_wgrad_core(&w.d2);
   const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
@@ -430,6 +435,25 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
   return run_contract(d, p, w + p.l_off, Z, dW, alpha, w + p.part_off, w, st);
 }
 
+// One block per (probe, 64-channel group): do the H*W (volumes: D*H*W) rows of 64 channels hold anything but +-0?
+template <typename T>
+__global__ void __launch_bounds__(256) zero_blocks_kernel(const T* __restrict__ Z, unsigned char* __restrict__ mask,
+                                                           long pixels, int Cin) {
+  constexpr int PER_ROW = 64 * (int)sizeof(T) / 16;          // 16-byte pieces of one row of the block
+  constexpr uint32_t ABS = sizeof(T) == 4 ? 0x7FFFFFFFu : 0x7FFF7FFFu;      // a negative zero is a zero
+  const int groups = Cin / 64;
+  const long j = blockIdx.x / groups;
+  const int g = (int)(blockIdx.x % groups);
+  const T* base = Z + j * pixels * Cin + (long)g * 64;
+  int any = 0;
+  for (long i = threadIdx.x; i < pixels * PER_ROW; i += blockDim.x) {
+    const uint4 v = *reinterpret_cast<const uint4*>(base + (i / PER_ROW) * Cin + (i % PER_ROW) * (16 / (int)sizeof(T)));
+    any |= ((v.x | v.y | v.z | v.w) & ABS) != 0u;
+  }
+  any = __syncthreads_or(any);
+  if (threadIdx.x == 0) mask[blockIdx.x] = any ? 0 : 1;
+}
+
 // FP32 FMA throughput probe: every thread runs 16 independent chains of dependent FMAs on registers (no
 // memory traffic), 4 blocks of 256 threads per SM's worth of grid; the result is stored so that the
 // compiler keeps the arithmetic.
@@ -455,6 +479,7 @@ struct IndepPlan { xconv_desc d2; WgradPlan p2; size_t x_off, part_off, bytes; }
 static IndepPlan plan_indep(const xconv_desc* d) {
   IndepPlan ip{};
   ip.d2 = *d; ip.d2.r = d->B; ip.d2.chan_scale = nullptr;     // the contraction runs over the batch
+  ip.d2.zero_blocks = nullptr;
   ip.p2 = plan_wgrad_core(&ip.d2);
   const size_t es = d->dtype == XCONV_F32 ? 4 : 2;
   const int T = kdepth(d) * d->KH * d->KW;
@@ -767,6 +792,30 @@ xconv_status xconv_workspace_status(const void* ws, void* cuda_stream) {
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
   return (word[0] != WS_OK && word[0] == word[1]) ? XCONV_ERR_TIMEOUT : XCONV_OK;
+}
+
+int xconv_zero_blocks_used(const xconv_desc* desc) {
+  if (validate(desc) != XCONV_OK || desc->zero_blocks == nullptr) return 0;
+  const WgradPlan p = plan_wgrad(desc);
+  return (p.tc_ct && p.t.ct_masked) ? 1 : 0;
+}
+
+xconv_status xconv_zero_blocks(const xconv_desc* desc, const void* Z, unsigned char* mask, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!Z || !mask) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(Z)) return XCONV_ERR_ALIGNMENT;
+  if (desc->Cin % 64 != 0 || (long)desc->r * (desc->Cin / 64) > 2000000000L) return XCONV_ERR_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const long pixels = (long)depth(desc) * desc->H * desc->W;
+  const unsigned blocks = (unsigned)((long)desc->r * (desc->Cin / 64));
+  new_call();
+  if (desc->dtype == XCONV_F32) zero_blocks_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(Z), mask, pixels, desc->Cin);
+  else zero_blocks_kernel<unsigned short><<<blocks, 256, 0, st>>>(static_cast<const unsigned short*>(Z), mask, pixels, desc->Cin);
+  ++g_launches;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return XCONV_OK;
 }
 
 xconv_status xconv_measure_fma_rate(void* scratch, size_t scratch_bytes, double* tflops, void* cuda_stream) {

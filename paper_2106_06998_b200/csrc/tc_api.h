@@ -27,6 +27,9 @@ struct TcWgradPlan {
   int ct_cw, ct_tile_n, ct_m_sub, ct_tiles_m, ct_tiles_n, ct_splits, ct_stages;
   int ct_tpu;                // kernel offsets per work unit (they share the L tile of every stage)
   int ct_halves;             // k-blocks copied and released in two halves; ct_stages then counts half-slots
+  int ct_masked;             // block-sparse probes whose zero blocks are named: the contraction walks a list of the
+                             // probes with a non-zero block per column tile (ct_list_bytes at the end of the partials)
+  size_t ct_list_bytes;
   int patch_h, patch_w, patches_y, patches_x;
   long ct_items, ct_items_per_split, ct_items_rem;   // the first ct_items_rem splits take one item more
   size_t part_bytes;

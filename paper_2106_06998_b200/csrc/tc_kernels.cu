@@ -103,6 +103,14 @@ struct TcParams {
   // Volumes: the planes (probe x depth for CONTRACT, image x depth for CONV) are the outermost tensor axis; a
   // kernel offset with a depth component dz reads plane + dz, and where that leaves the volume the box is
   // sent to row H of the plane instead, which lies outside the image: the copy engine fills it with zeros.
+  // CONTRACT in halves with block-sparse probes (Eq. 7) whose all-zero 64-channel blocks the caller has named.  Row tn of
+  // `zlist` (zlist_ld words apart) serves column tile tn: word 0 = number n of probing vectors with at least one non-zero
+  // block in that tile, words 1..n = their indices in rising order, word n+1 = 0.  The k-blocks of a tile are those of
+  // its n listed probes only, dealt evenly to the zsplits k-splits; the others are neither copied nor multiplied.
+  // (A listed probe takes whole k-blocks, zero blocks included: an MMA into columns that the MMA before it wrote waits
+  // some 250 clocks for it whatever its width, so narrower MMAs for the non-zero blocks alone took as long.)  Null: dense.
+  const uint32_t* zlist;
+  int zlist_ld, zsplits;
   int epi_groups;          // epilogue warps per tensor-memory lane quadrant (1 or 2): the launch has 64 + 128 * epi_groups threads
   int depth, pad_d;        // planes per probe or image (1: planar layer), depth padding of the kernel
   int f16;                 // storage type of the 16-bit operands: 0 = bfloat16, 1 = float16 (both operands alike)
@@ -387,6 +395,7 @@ __device__ __forceinline__ uint32_t pack2(uint32_t a, uint32_t b, bool f16) {
 
 constexpr int TILE_M = 128;
 constexpr int MAX_STAGES = 8;
+constexpr int ZLIST_SMEM = 128;      // list entries of a unit held in shared memory (the rest are read from global memory)
 // Epilogue warps per tensor-memory lane quadrant: one, or two where a tile's epilogue outlasts its mainloop (the
 // back-probe of small batches).  More epilogue warps than needed only take issue slots from the two
 // single-thread roles: with two everywhere the wide layers lost 10-25 %.
@@ -433,6 +442,14 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, long u_) {
     w.tm = (int)(t % (uint32_t)p.tiles_m); t /= (uint32_t)p.tiles_m;
     w.tap = (int)t * tpu;                      // first offset of the unit
   }
+  if (p.zlist != nullptr) {                  // k-blocks of the listed probes only, dealt evenly to the k-splits
+    const uint32_t n = p.zlist[(uint32_t)w.tn * (uint32_t)p.zlist_ld];
+    const uint32_t K = n * (uint32_t)(p.patches_x * p.patches_y * p.depth), zs = (uint32_t)p.zsplits;
+    const uint32_t q = K / zs, rem = K % zs, sp = (uint32_t)w.split;
+    w.kb0 = (long)(sp * q + min(sp, rem));
+    w.nkb = (int)(q + (sp < rem ? 1u : 0u));
+    return w;
+  }
   w.kb0 = w.split * p.kblocks_per_split + min(w.split, p.kb_rem);
   const long kb1 = min(p.kblocks, w.kb0 + p.kblocks_per_split + (w.split < p.kb_rem ? 1 : 0));
   w.nkb = (int)max(0L, kb1 - w.kb0);
@@ -454,6 +471,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_slot;
   __shared__ int go;
+  __shared__ uint32_t zl[ZLIST_SMEM];        // block-sparse probes: the list entries of this CTA's one work unit
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // 128B swizzle wants 1024B alignment
@@ -474,6 +492,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
   pdl_trigger();
   pdl_wait();                              // from here on the previous kernel's results are visible
+  // Block-sparse probes (one unit per CTA): the unit's stretch of its tile's list, zl_len entries (and the entry behind
+  // the last, which the producer may fetch but never uses), goes to shared memory.
+  const uint32_t* zl_row = nullptr;
+  int zl_len = 0;
+  if (p.zlist != nullptr) {
+    const Unit w0 = decode_unit(p, blockIdx.x);
+    const uint32_t per_probe = (uint32_t)(p.patches_x * p.patches_y * p.depth);
+    const uint32_t first = (uint32_t)w0.kb0 / per_probe;
+    zl_len = w0.nkb > 0 ? (int)(((uint32_t)w0.kb0 + (uint32_t)w0.nkb - 1u) / per_probe - first) + 1 : 0;
+    zl_row = p.zlist + (size_t)w0.tn * p.zlist_ld + 1 + first;
+    for (int i = threadIdx.x; i <= zl_len && i < ZLIST_SMEM; i += blockDim.x) zl[i] = zl_row[i];
+  }
+  auto zent = [&](int i) -> uint32_t { return i < ZLIST_SMEM ? zl[i] : zl_row[i]; };
   if (threadIdx.x == 0) {
     // a CTA of this call gave up earlier: skip the work (one thread reads so that the whole CTA agrees)
     go = (*reinterpret_cast<volatile unsigned int*>(p.status) != p.tag) ? 1 : 0;
@@ -550,6 +581,34 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int ks = 2 * p.pad + 1, tp = w.tap % (ks * ks), dy = tp / ks - p.pad, dx = tp % ks - p.pad;
         const int dz = w.tap / (ks * ks) - p.pad_d;
         int pz = pj % p.depth;               // depth of plane pj inside its volume
+        if (p.zlist != nullptr) {
+          // block-sparse probes: pj counted the planes of the listed probes; the plane in memory is that of the probe
+          // the list entry names
+          int li = 0;
+          int plane = (int)zent(0) * p.depth + pz;
+          for (int i = 0; i < 2 * w.nkb; ++i) {
+            if (fill > 0) {
+              ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
+              if (!ok) break;
+            }
+            const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes, b_dst = a_dst + p.a_half_bytes;
+            const int x0 = px * p.patch_w, y0 = py * p.patch_h + (i & 1) * hrows;
+            mbar_arrive_expect_tx(&full_bar[s], stage_bytes);
+            tma_load_5d(a_dst, &map_a, 0, x0, y0, row0 >> p.cw_shift, plane, &full_bar[s]);
+            const bool inside = (unsigned)(pz + dz) < (unsigned)p.depth;
+            tma_load_5d(b_dst, &map_b, 0, x0 + dx, inside ? y0 + dy : p.H, col0 >> p.cw_shift, plane + dz, &full_bar[s]);
+            ++it;
+            if (++s == slots) { s = 0; ++fill; }
+            if ((i & 1) && ++px == p.patches_x) {
+              px = 0;
+              if (++py == p.patches_y) {
+                py = 0;
+                if (++pz == p.depth) { pz = 0; ++li; }
+                plane = (int)zent(li) * p.depth + pz;
+              }
+            }
+          }
+        } else
         for (int i = 0; i < 2 * w.nkb; ++i) {
           if (fill > 0) {
             ok = mbar_wait(&empty_bar[s], (uint32_t)((fill - 1) & 1), p.status, p.tag);
@@ -590,7 +649,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
         const Unit w = decode_unit(p, u);
-        if (w.nkb == 0) continue;
+        if (w.nkb == 0) { mbar_arrive(&tmem_full_bar[0]); continue; }      // nothing to multiply: the epilogue stores zeros
         const uint32_t d = tmem_base;      // one unit per CTA and accumulator set (acc_bufs = 1)
         uint32_t acc = 0;
         if (p.ks_h0 == 3 && p.ks_x == 1 && p.ks_h1 == 3) {      // halves of 56 pixels (28-wide images): unrolled
@@ -757,7 +816,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       bool ok = true;
       for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
         const Unit w = decode_unit(p, u);
-        if (w.nkb == 0) continue;
         const int buf = p.acc_bufs == 2 ? (int)(lu & 1) : 0;          // (no division: this thread's stream is the critical path)
         const long use = p.acc_bufs == 2 ? lu >> 1 : lu;
         if (use > 0) {                      // the epilogue must have emptied this accumulator set
@@ -765,6 +823,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!ok) break;
           tc_fence_after();
         }
+        // Nothing to multiply: the barriers still take their turn, so that their phases keep counting units, and the
+        // epilogue stores zeros without reading the accumulator.
+        if (w.nkb == 0) { mbar_arrive(&tmem_full_bar[buf]); continue; }
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * acc_cols);
         uint32_t acc = 0;
         // BACKPROBE: the MMA spans the blocks this column tile has
@@ -908,12 +969,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         if (!ok) break;
       }
-      if (w.nkb > 0) {
-        if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status, p.tag);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) break;
-        tc_fence_after();
-      }
+      if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status, p.tag);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
       const long col0 = (long)w.tn * p.tile_n;
       if (p.mode == MODE_BACKPROBE) {
         // D[j, q] -> L[j][q].  Each warp stages 32 rows x 64 positions at a time in the layout the tensor store
@@ -1432,8 +1491,49 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
       p->ct_stages = std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK) / half) & ~1;      // half-slots, an even number
       if (p->ct_stages < 4) p->ct_halves = 0, p->ct_stages = pick_stages(stage, ct_ctas);
     }
+    // Block-sparse probes whose zero blocks are named (one work unit per CTA, which the halves guarantee): a list of
+    // the probes with a non-zero block, per column tile, behind the partial sums
+    p->ct_masked = (d->zero_blocks != nullptr && p->ct_halves && p->ct_tile_n % 64 == 0) ? 1 : 0;
+    p->ct_list_bytes = 0;
+    if (p->ct_masked) {
+      const long probes = d->r / (d->D > 1 ? d->D : 1);
+      p->part_bytes = (p->part_bytes + 255) & ~(size_t)255;
+      p->ct_list_bytes = (size_t)p->ct_tiles_n * (size_t)(probes + 2) * sizeof(uint32_t);
+      p->part_bytes += p->ct_list_bytes;
+    }
   }
   return mask;
+}
+
+// Block-sparse probes: the list TcParams::zlist describes, from the caller's mask (zmask[j * groups + g] != 0: channels
+// [64 g, 64 g + 64) of probing vector j are all zero).  One block per column tile of `gpt` channel groups; the probes
+// keep their order, so that the sums of the contraction are taken in the same order whenever the mask is the same.
+__global__ void __launch_bounds__(1024) list_nonzero_blocks(const unsigned char* __restrict__ zmask, int groups, int gpt,
+                                                            int probes, uint32_t* __restrict__ list, int ld) {
+  __shared__ int warp_count[32];
+  pdl_trigger();
+  pdl_wait();
+  const int tn = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t* row = list + (size_t)tn * ld;
+  int base = 0;
+  for (int j0 = 0; j0 < probes; j0 += 1024) {
+    const int j = j0 + (int)threadIdx.x;
+    uint32_t bits = 0;
+    if (j < probes)
+      for (int g = 0; g < gpt; ++g) {
+        const int gg = tn * gpt + g;
+        if (gg < groups && zmask[(size_t)j * groups + gg] == 0) bits |= 1u << g;
+      }
+    const unsigned vote = __ballot_sync(0xffffffffu, bits != 0u);
+    if (lane == 0) warp_count[warp] = __popc(vote);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < 32; ++w) { before += w < warp ? warp_count[w] : 0; total += warp_count[w]; }
+    if (bits != 0u) row[1 + base + before + __popc(vote & ((1u << lane) - 1u))] = (uint32_t)j;
+    base += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) { row[0] = (uint32_t)base; row[1 + base] = 0u; }
 }
 
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const void* S_bf16, const void* dY,
@@ -1590,6 +1690,17 @@ xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& pl, const v
   p.Cin = d->Cin;
   p.part = reinterpret_cast<float*>(part);
   p.status = reinterpret_cast<unsigned int*>(ws_head);
+  if (pl.ct_masked) {
+    const int probes = d->r / p.depth;
+    uint32_t* list = reinterpret_cast<uint32_t*>(part + (pl.part_bytes - pl.ct_list_bytes));
+    p.zlist = list;
+    p.zlist_ld = probes + 2;
+    p.zsplits = pl.ct_splits;
+    const cudaError_t el = launch_pdl(list_nonzero_blocks, dim3((unsigned)pl.ct_tiles_n), dim3(1024), 0, st, d->zero_blocks,
+                                      d->Cin / 64, pl.ct_tile_n / 64, probes, list, p.zlist_ld);
+    count_launch();
+    if (el != cudaSuccess) { set_cuda_error((int)el); return XCONV_ERR_CUDA; }
+  }
   xconv_status s = launch(ma, mb, p, (unsigned)std::min<long>(p.units, 4L * NUM_SMS), st);
   if (s != XCONV_OK) return s;
   const long split_stride = (long)T * pl.ct_tiles_m * pl.ct_tiles_n * pl.ct_m_sub * TILE_M * pl.ct_tile_n;
