@@ -533,6 +533,19 @@ def run_xconv(args):
             del lay2, Z2
             torch.cuda.empty_cache()
 
+    # ---- the same step with Gaussian probing vectors (the workload names no distribution; Rademacher is the primary run)
+    gaussian = None
+    if not args.no_sweep and world == 1 and c["z"] != "gaussian":
+        Zg = xb.to_device(inputs.draw("gaussian", (r, Cin, H, W), inputs.seed_for(cfg, r, "Z") + 17, c["dtype"]), c["dtype"], dev)
+        layg = Layer(r, Zg)
+        ng = max(5, min(args.steps, 30))
+        totg, _, _ = layg.measure(ng, 3, None, phase_events=False)
+        phg, _ = layg.measure_phases(ng)
+        gaussian = {"r": r, "z": "gaussian", "ms_per_step": totg / ng, "value": 1e3 * ng / totg,
+                    "phases_ms": {k: v for k, v in phg.items()}}
+        del layg, Zg
+        torch.cuda.empty_cache()
+
     # ---- block-sparse probes (Eq. 7) on this workload: the contraction told which 64-channel blocks of Z are zero
     block_sparse = None
     if (not args.no_sweep and world == 1 and tdt != torch.float32 and Cin % 64 == 0 and Cout % 64 == 0
@@ -607,7 +620,7 @@ def run_xconv(args):
                                      "CUDA events; with_events_between_calls_ms: the step with an event between its "
                                      "three calls, which keeps a kernel's preamble from overlapping the previous "
                                      "kernel's tail (diagnostic)"},
-            "sweep": sweep, "layer_api": full,
+            "sweep": sweep, "gaussian_probes": gaussian, "layer_api": full,
             "block_sparse": None if block_sparse is None else {
                 "cases": block_sparse,
                 "dense_contract_ms": {str(r): phases["contract"]["ms"],

@@ -80,3 +80,31 @@ def test_binding_refuses_host_tensors_and_wrong_layout(lib):
     Z = torch.zeros(3, 4, 5, 5)
     with pytest.raises(ValueError):
         xb.xconv_sketch(X, Z)
+
+
+def test_zero_block_mask_changes_the_plan_only_where_it_is_used(lib):
+    """Host arithmetic only (the mask pointer is never followed): the contraction of wide 16-bit layers plans a list
+    of non-zero probes behind its partial sums; everywhere else the field changes nothing."""
+    def pair(**kw):
+        plain = _desc(**kw)
+        masked = _desc(**kw)
+        masked.zero_blocks = 256
+        return plain, masked
+    plain, masked = pair(B=512, Cin=256, Cout=256, H=28, W=28, r=64, dtype=xb.XCONV_BF16)
+    assert not xb.zero_blocks_used(plain) and xb.zero_blocks_used(masked)
+    grown = xb.workspace_bytes(masked, xb.OP_WGRAD) - xb.workspace_bytes(plain, xb.OP_WGRAD)
+    assert 4 * (64 + 2) <= grown <= 4 * (64 + 2) + 512          # one column tile: count, 64 entries, terminator
+    plain, masked = pair(B=512, Cin=512, Cout=256, H=28, W=28, r=64, dtype=xb.XCONV_F16)
+    assert xb.zero_blocks_used(masked)
+    assert xb.workspace_bytes(masked, xb.OP_WGRAD) - xb.workspace_bytes(plain, xb.OP_WGRAD) >= 2 * 4 * (64 + 2)
+    for kw in (dict(B=8, Cin=64, Cout=32, H=8, W=8, r=4, dtype=xb.XCONV_F32),           # FP32-FMA kernels
+               dict(B=32, Cin=128, Cout=64, H=12, W=20, r=24, dtype=xb.XCONV_BF16),     # small 16-bit layer
+               dict(B=8, Cin=96, Cout=64, H=16, W=16, r=8, dtype=xb.XCONV_BF16)):       # not whole 64-channel blocks
+        plain, masked = pair(**kw)
+        assert not xb.zero_blocks_used(masked)
+        assert xb.workspace_bytes(masked, xb.OP_WGRAD) == xb.workspace_bytes(plain, xb.OP_WGRAD)
+    # a planar kernel on a volume: the mask is per probing vector, the contraction walks planes
+    plain, masked = pair(B=8, Cin=128, Cout=128, H=16, W=16, r=6, dtype=xb.XCONV_BF16, D=3, KD=1)
+    assert not xb.zero_blocks_used(masked)
+    plain, masked = pair(B=8, Cin=128, Cout=128, H=16, W=16, r=6, dtype=xb.XCONV_BF16, D=3, KD=3)
+    assert xb.zero_blocks_used(masked)
