@@ -148,10 +148,13 @@ xconv_status xconv_sketch(const xconv_desc* desc, const void* X, const void* Z, 
  * inside the kernel, so that only X leaves HBM; otherwise Z is first written into `ws` and the regular
  * kernels run on it (xconv_workspace_bytes(desc, XCONV_OP_SKETCH_SEEDED) covers both cases).  The result
  * equals xconv_sketch on xconv_probes_from_seed's Z up to the order of summation.
- * xconv_wgrad_seeded is Algorithm 1's backward pass from the stored seed: step 2 redraws Z[seed] into `ws`
- * (xconv_workspace_bytes(desc, XCONV_OP_WGRAD_SEEDED) = the scratch of xconv_wgrad plus one Z), steps 3-4
- * are xconv_wgrad on it; the estimate equals xconv_wgrad(sketch, dY, xconv_probes_from_seed(seed)) bit for
- * bit.  With these two calls a layer keeps S (r*B floats) and the 8-byte seed between its forward and its
+ * xconv_wgrad_seeded is Algorithm 1's backward pass from the stored seed.  Where r > B and the tensor-core
+ * kernels cover the layer, xconv_wgrad sums over the probes first (S^T Z, then the offset contraction over the
+ * batch), Z is the streamed operand of its first kernel, and that kernel redraws its tiles of Z on chip: Z
+ * neither enters nor leaves HBM.  Elsewhere step 2 redraws Z[seed] into `ws` and steps 3-4 are xconv_wgrad on
+ * it (xconv_workspace_bytes(desc, XCONV_OP_WGRAD_SEEDED) covers both cases: the scratch of xconv_wgrad, plus
+ * one Z in the second).  Either way the estimate equals xconv_wgrad(sketch, dY, xconv_probes_from_seed(seed))
+ * bit for bit.  With these two calls a layer keeps S (r*B floats) and the 8-byte seed between its forward and its
  * backward pass, the memory factor the paper quotes. */
 xconv_status xconv_probes_from_seed(const xconv_desc* desc, unsigned long long seed, void* Z, void* cuda_stream);
 xconv_status xconv_sketch_seeded(const xconv_desc* desc, const void* X, unsigned long long seed, float* sketch,

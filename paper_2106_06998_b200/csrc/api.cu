@@ -375,7 +375,7 @@ static xconv_status run_conv(const xconv_desc* d, bool dgrad, const void* in, co
 
 // L = S dY^T into `L`; `Sb` receives the bfloat16 copy of S that the tensor-core kernel reads.
 static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const float* S, const void* dY,
-                                  void* L, void* Sb_, char* w, cudaStream_t st) {
+                                  void* L, void* Sb_, char* w, cudaStream_t st, const unsigned long long* seed = nullptr) {
   if (p.tc_bp) {
     const long n = (long)d->r * d->B;
     cudaError_t e = d->dtype == XCONV_F16
@@ -384,7 +384,7 @@ static xconv_status run_backprobe(const xconv_desc* d, const WgradPlan& p, const
     ++g_launches;
     if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
     const xconv_desc f = flat(d);
-    return tc_run_backprobe(&f, p.tb, Sb_, dY, L, w, st);
+    return tc_run_backprobe(&f, p.tb, Sb_, dY, L, w, st, seed);
   }
   return d->dtype == XCONV_F32 ? run_backprobe_simt<float, float>(d, S, dY, L, st)
          : d->dtype == XCONV_F16 ? run_backprobe_simt<f16, f16>(d, S, dY, L, st)
@@ -410,8 +410,16 @@ static xconv_status check_ws(void* ws, size_t ws_bytes, size_t need) {
   return XCONV_OK;
 }
 
+// Whether xconv_wgrad_seeded redraws the probing vectors inside its first kernel (the estimator summed over the
+// probes first, r > B, with that step on the tensor cores) instead of writing them to the workspace first.
+static bool wgrad_redraws(const xconv_desc* d) {
+  const SwappedWgrad sw = plan_wgrad_swapped(d);
+  return sw.on && sw.p1.tc_bp;
+}
+
+// `seed` != nullptr (only where wgrad_redraws holds): Z is not read.
 static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* dY, const void* Z, float* dW,
-                              void* ws, size_t ws_bytes, cudaStream_t st) {
+                              void* ws, size_t ws_bytes, cudaStream_t st, const unsigned long long* seed = nullptr) {
   const WgradPlan p = plan_wgrad(d);
   xconv_status s = check_ws(ws, ws_bytes, p.bytes);
   if (s != XCONV_OK) return s;
@@ -426,7 +434,7 @@ static xconv_status run_wgrad(const xconv_desc* d, const float* S, const void* d
     transpose_f32<<<(unsigned)cdiv(n, 256), 256, 0, st>>>(S, St, d->r, d->B);
     s = check_launch();
     if (s != XCONV_OK) return s;
-    s = run_backprobe(&sw.d1, sw.p1, St, Z, w + sw.x_off, w + sw.sb_off, w, st);
+    s = run_backprobe(&sw.d1, sw.p1, St, Z, w + sw.x_off, w + sw.sb_off, w, st, seed);
     if (s != XCONV_OK) return s;
     return run_contract(&sw.d2, sw.p2, dY, w + sw.x_off, dW, alpha, w + sw.part_off, w, st);
   }
@@ -528,7 +536,7 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
   switch (op) {
     case XCONV_OP_FORWARD:
     case XCONV_OP_SKETCH: return plan_sketch(desc).bytes;
-    case XCONV_OP_WGRAD_SEEDED: return plan_wgrad(desc).bytes + probes_bytes(desc);
+    case XCONV_OP_WGRAD_SEEDED: return plan_wgrad(desc).bytes + (wgrad_redraws(desc) ? 0 : probes_bytes(desc));
     case XCONV_OP_SKETCH_SEEDED: {
       const SketchPlan p = plan_sketch(desc, true);
       return p.bytes + (sketch_redraws(desc, p) ? 0 : probes_bytes(desc));
@@ -596,10 +604,13 @@ xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, con
   if (!sketch || !dY || !dW) return XCONV_ERR_INVALID_ARG;
   if (!aligned16(sketch) || !aligned16(dY) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
   const size_t base = plan_wgrad(desc).bytes;
-  s = check_ws(ws, ws_bytes, base + probes_bytes(desc));
+  const bool redraw = wgrad_redraws(desc);
+  s = check_ws(ws, ws_bytes, base + (redraw ? 0 : probes_bytes(desc)));
   if (s != XCONV_OK) return s;
   new_call();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // r > B on the tensor cores: the first kernel of the estimator redraws its tiles of Z on chip
+  if (redraw) return run_wgrad(desc, sketch, dY, nullptr, dW, ws, base, st, &seed);
   // Algorithm 1 backward step 2: redraw Z from the seed (behind the regular scratch), then steps 3-4
   char* Z = static_cast<char*>(ws) + base;
   s = run_probes_from_seed(desc, seed, Z, st);

@@ -56,8 +56,10 @@ xconv_status tc_run_conv(const xconv_desc* d, const TcConvPlan& p, bool dgrad, c
 xconv_status tc_run_sketch(const xconv_desc* d, const TcSketchPlan& p, const void* X, const void* Z, float* S,
                            char* ws_head, char* part, cudaStream_t st, const unsigned long long* seed = nullptr);
 bool tc_sketch_can_redraw(const xconv_desc* d);
+// `seed` != nullptr: the streamed operand (`dY`) is a set of probing vectors that is not read but redrawn inside
+// the kernel from the Philox stream of *seed -- the first step of the estimator when it sums over the probes first.
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& p, const void* S_bf16, const void* dY,
-                              void* L, char* ws_head, cudaStream_t st);
+                              void* L, char* ws_head, cudaStream_t st, const unsigned long long* seed = nullptr);
 xconv_status tc_run_contract(const xconv_desc* d, const TcWgradPlan& p, const void* L, const void* Z, float* dW,
                              float alpha, char* ws_head, char* part, cudaStream_t st);
 

@@ -337,6 +337,23 @@ __device__ __forceinline__ void z_store64(uint32_t rbase, int row, uint2 bits, u
                  "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
   }
 }
+// The same with every piece looked up by its eight sign bits in the table at shared-memory address `lut` (256 x 16
+// bytes: z_pack8 of every byte): one load per piece instead of sixteen integer instructions.  Pays where a warp draws
+// a stage alone and its instruction stream is the limit (the back-probe: 260 -> 220 us on the 256 x 256 images); where
+// all warps draw together beside a copy engine and a tensor pipe that fill shared memory's bandwidth (the sketch) the
+// extra loads cost more than the instructions (63 -> 76 us there).
+__device__ __forceinline__ void z_store64_lut(uint32_t rbase, int row, uint2 bits, uint32_t lut) {
+  const uint32_t r7 = (uint32_t)row & 7u;
+#pragma unroll
+  for (int c = 0; c < 8; ++c) {
+    const uint32_t word = c < 4 ? bits.x : bits.y;
+    const uint32_t off = (c & 3) == 0 ? (word << 4) & 0xFF0u : (word >> ((c & 3) * 8 - 4)) & 0xFF0u;
+    uint4 o;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(o.x), "=r"(o.y), "=r"(o.z), "=r"(o.w) : "r"(lut + off));
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(rbase + (((uint32_t)c ^ r7) << 4)),
+                 "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+  }
+}
 // 128 entries: the same row of two consecutive k-block tiles, `tile_bytes` apart.
 __device__ __forceinline__ void z_store128(uint32_t rbase, uint32_t tile_bytes, int row, uint4 w, uint32_t ones) {
   z_store64(rbase, row, make_uint2(w.x, w.y), ones);
@@ -479,16 +496,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int unit_cols = p.mode == MODE_CONTRACT ? p.tile_n * p.tpu : p.tile_n;  // columns of one row tile's accumulator
   const int acc_cols = unit_cols * p.m_sub;                                   // columns of one accumulator set
 
+  // Seeded calls: the epilogue warps redraw the tiles of Z, all of them together stage by stage -- except in a
+  // back-probe with one tile of at most 96 rows: there the warps of the lane quadrants that hold rows (below
+  // gen_quad0) are busy with the epilogue of every unit, the slowest role of that kernel, and the warps of the
+  // other quadrants, which have nothing to store, do nothing but draw, each whole stages by itself in turn.
+  const int gen_quad0 = (p.seeded && p.mode == MODE_BACKPROBE && p.tiles_m == 1 && p.m_sub == 1 && p.rows <= 96)
+                            ? (int)((p.rows + 31) / 32) : 0;
   // preamble: touches no global memory, so it may overlap the tail of the previous kernel
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full_bar[s], p.seeded ? 1 + 4 * p.epi_groups : 1); mbar_init(&empty_bar[s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&tmem_full_bar[b], 1); mbar_init(&tmem_empty_bar[b], 4 * p.epi_groups); }
+    // a stage is full when the producer's copies have landed and (seeded) the drawing warps have arrived: all epilogue
+    // warps, or the one drawing warp whose turn the stage is; an accumulator set is free when the storing warps are done
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(&full_bar[s], !p.seeded ? 1 : gen_quad0 > 0 ? 2 : 1 + 4 * p.epi_groups);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full_bar[b], 1);
+      mbar_init(&tmem_empty_bar[b], (gen_quad0 > 0 ? gen_quad0 : 4) * p.epi_groups);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     prefetch_tmap(&map_a);
     prefetch_tmap(&map_b);
     if (p.mode == MODE_BACKPROBE) prefetch_tmap(&map_c);
   }
+  // seeded back-probe: the table of sign patterns behind everything else in shared memory
+  const uint32_t z_lut = tiles_base + (uint32_t)p.stages * stage_bytes + p.epi_bytes + p.smem_pad;
+  if (p.seeded && p.mode == MODE_BACKPROBE)
+    for (uint32_t i = threadIdx.x; i < 256u; i += blockDim.x) {
+      const uint4 o = z_pack8(i, F16 ? 0x3C003C00u : 0x3F803F80u);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(z_lut + (i << 4)), "r"(o.x), "r"(o.y), "r"(o.z), "r"(o.w) : "memory");
+    }
   if (warp == 1) tmem_alloc(&tmem_slot, (uint32_t)p.tmem_cols);
   pdl_trigger();
   pdl_wait();                              // from here on the previous kernel's results are visible
@@ -736,7 +774,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t a_dst = tiles_base + (uint32_t)s * stage_bytes;
           const uint32_t b_dst = a_dst + p.a_stage_bytes;
           mbar_arrive_expect_tx(&full_bar[s], p.mode == MODE_BACKPROBE
-                                                  ? p.a_stage_bytes + (uint32_t)w.nblk * p.b_box_bytes : p.tx_bytes);
+                                                  ? p.a_stage_bytes + (p.seeded ? 0u : (uint32_t)w.nblk * p.b_box_bytes)
+                                                  : p.tx_bytes);
           if (p.mode == MODE_SKETCH) {
             // one box per operand: 128*m_sub rows of A, tile_n rows of B, 64 k each
             const bool get_a = !(p.seeded && p.z_is_a), get_b = !(p.seeded && !p.z_is_a);
@@ -753,8 +792,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           } else if (p.mode == MODE_BACKPROBE) {
             tma_load_2d(a_dst, &map_a, kc, row0, &full_bar[s]);
             // dY tile: one box (64 positions x k rows) per block of the column tile, one behind the other
-            for (int b = 0; b < w.nblk; ++b)
-              tma_load_3d(b_dst + (uint32_t)b * p.b_box_bytes, &map_b, 0, kc, w.blk0 + b, &full_bar[s]);
+            // (seeded: the streamed operand is Z, and the epilogue warps write its tile themselves)
+            if (!p.seeded)
+              for (int b = 0; b < w.nblk; ++b)
+                tma_load_3d(b_dst + (uint32_t)b * p.b_box_bytes, &map_b, 0, kc, w.blk0 + b, &full_bar[s]);
             kc += p.ksteps * 16;
           } else if (p.mode == MODE_CONV) {
             // input patch moved by the kernel offset (zero fill outside the image) and the matching
@@ -915,58 +956,144 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     long gen_fill = 0;
     long lu = 0;
     bool ok = true;
-    for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
-      const Unit w = decode_unit(p, u);
-      const int buf = p.acc_bufs == 2 ? (int)(lu & 1) : 0;
-      const long use = p.acc_bufs == 2 ? lu >> 1 : lu;
-      if (p.seeded && p.mode == MODE_SKETCH) {
-        // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
-        // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
-        // copy would have produced, hand the stage over with one arrival per warp.
-        const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
-        const int GEN = 128 * p.epi_groups;
-        const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
-        const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
-        const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
-        const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
-        const uint32_t z_ones = F16 ? 0x3C003C00u : 0x3F803F80u;
-        long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
+    // BACKPROBE with Z as the streamed operand: the Z tile of one stage (probes kc .., the blocks of unit w), items
+    // t0, t0 + stride, ... of it.  An item is one Philox block = 128 entries = one row of an even 64-position block and
+    // of the odd block behind it; two items per round, so that their dependent chains interleave.
+    auto fill_bp_stage = [&](uint32_t zbase, long kc, const Unit& w, int t0, int stride) {
+            const int rows_k = p.ksteps * 16;
+      const int even0 = w.blk0 & ~1, n = rows_k * ((w.blk0 + w.nblk - even0 + 1) >> 1);
+      for (int i0 = t0; i0 < n; i0 += 2 * stride) {
+        const int i1 = i0 + stride;
+        const bool two = i1 < n;
+        const int row0_ = i0 % rows_k, blk0_ = even0 + 2 * (i0 / rows_k);
+        const int row1_ = two ? i1 % rows_k : row0_, blk1_ = two ? even0 + 2 * (i1 / rows_k) : blk0_;
+        const unsigned long long e0 = (unsigned long long)((kc + row0_) * p.z_row_len + (long)blk0_ * 64);
+        const unsigned long long e1 = (unsigned long long)((kc + row1_) * p.z_row_len + (long)blk1_ * 64);
+        const uint4 o0 = philox4x32_10((uint32_t)(e0 >> 7), (uint32_t)(e0 >> 39), p.seed_lo, p.seed_hi);
+        const uint4 o1 = philox4x32_10((uint32_t)(e1 >> 7), (uint32_t)(e1 >> 39), p.seed_lo, p.seed_hi);
+        const int b0 = blk0_ - w.blk0, b1 = blk1_ - w.blk0;       // block of the tile that takes the first 64 entries
+        const uint32_t r0 = zbase + (uint32_t)row0_ * 128u, r1 = zbase + (uint32_t)row1_ * 128u;
+        if (b0 >= 0) z_store64_lut(r0 + (uint32_t)b0 * p.b_box_bytes, row0_, make_uint2(o0.x, o0.y), z_lut);
+        if (b0 + 1 < w.nblk) z_store64_lut(r0 + (uint32_t)(b0 + 1) * p.b_box_bytes, row0_, make_uint2(o0.z, o0.w), z_lut);
+        if (two && b1 >= 0) z_store64_lut(r1 + (uint32_t)b1 * p.b_box_bytes, row1_, make_uint2(o1.x, o1.y), z_lut);
+        if (two && b1 + 1 < w.nblk) z_store64_lut(r1 + (uint32_t)(b1 + 1) * p.b_box_bytes, row1_, make_uint2(o1.z, o1.w), z_lut);
+      }
+    };
+    // Probing vectors redrawn from the seed: the tiles of Z of one work unit, written by these warps.
+    auto redraw_unit = [&](const Unit& w) {
+      if (p.mode == MODE_SKETCH) {
+          // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
+          // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
+          // copy would have produced, hand the stage over with one arrival per warp.
+          const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
+          const int GEN = 128 * p.epi_groups;
+          const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
+          const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
+          const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
+          const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
+          const uint32_t z_ones = F16 ? 0x3C003C00u : 0x3F803F80u;
+          long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
+          for (int i = 0; i < w.nkb && ok; ++i) {
+            if (gen_fill > 0) {
+              if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
+              ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+              if (!ok) break;
+            }
+            const uint32_t zbase = tiles_base + (uint32_t)gen_s * stage_bytes + z_off;
+            const uint32_t tile_bytes = (uint32_t)tile_rows * 128u;
+            if ((p.kgroup & 1) == 0 && (p.z_row_len & 127) == 0) {
+              // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
+              // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
+              const int nitems = nrows * (p.kgroup >> 1);
+              for (int it0 = gtid; it0 < nitems; it0 += 2 * GEN) {
+                const int it1 = it0 + GEN;
+                const bool two = it1 < nitems;
+                const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
+                const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
+                const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
+                const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
+                const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
+                z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0, z_ones);
+                if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
+              }
+            } else {
+              for (int item = gtid; item < nrows * p.kgroup; item += GEN) {
+                const int row = item % nrows, g = item / nrows;
+                const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
+                z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
+              }
+            }
+            fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[gen_s]);
+            kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
+            if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
+          }
+      } else {
+        // BACKPROBE with Z as the streamed operand (the estimator summed over the probes first): a stage holds, per
+        // 64-position block of the column tile, ksteps*16 rows (probes) of 128 bytes, swizzled by the row like the
+        // copy would have left them.  One Philox block = 128 entries = the same row of an even block and the odd
+        // block behind it.  Rows past the last probe are drawn too: their partners in the A tile are zero.
+        const int gtid = (quad * p.epi_groups + eg) * 32 + lane, GEN = 128 * p.epi_groups;
+        const int rows_k = p.ksteps * 16;
+        long kc = w.kb0 * rows_k;
         for (int i = 0; i < w.nkb && ok; ++i) {
           if (gen_fill > 0) {
             if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
           }
-          const uint32_t zbase = tiles_base + (uint32_t)gen_s * stage_bytes + z_off;
-          const uint32_t tile_bytes = (uint32_t)tile_rows * 128u;
-          if ((p.kgroup & 1) == 0 && (p.z_row_len & 127) == 0) {
-            // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
-            // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
-            const int nitems = nrows * (p.kgroup >> 1);
-            for (int it0 = gtid; it0 < nitems; it0 += 2 * GEN) {
-              const int it1 = it0 + GEN;
-              const bool two = it1 < nitems;
-              const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
-              const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
-              const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
-              const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
-              const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
-              z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0, z_ones);
-              if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
-            }
-          } else {
-            for (int item = gtid; item < nrows * p.kgroup; item += GEN) {
-              const int row = item % nrows, g = item / nrows;
-              const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
-              z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
-            }
-          }
-          fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
+          fill_bp_stage(tiles_base + (uint32_t)gen_s * stage_bytes + p.a_stage_bytes, kc, w, gtid, GEN);
+          fence_async_smem();
           __syncwarp();
           if (lane == 0) mbar_arrive(&full_bar[gen_s]);
-          kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
+          kc += rows_k;
           if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
         }
+      }
+    };
+    // SKETCH: a unit's tiles are drawn when its turn comes (its epilogue is a few stores).  BACKPROBE: one unit ahead, so
+    // that the MMAs of the next unit run during this unit's epilogue -- needs the second accumulator set: with one,
+    // the next unit's MMAs wait for this epilogue, which would wait behind stages only those MMAs can free.
+    const bool redraw_ahead = p.seeded && p.mode == MODE_BACKPROBE && p.acc_bufs == 2 && gen_quad0 == 0;
+    if (redraw_ahead && blockIdx.x < p.units) redraw_unit(decode_unit(p, blockIdx.x));
+    if (gen_quad0 > 0 && quad >= gen_quad0) {
+      // A warp that only draws: it walks the stages of this CTA's units like the producer does and fills, alone, those
+      // that fall into the slots of the ring it owns (slot mod n_gen), as far ahead of the MMAs as the ring allows.  The
+      // slots have fixed owners because a wait by parity is only right for a thread that has seen every earlier phase
+      // of the barrier: a warp that came to a slot two rounds late would take the phase before last for the last.
+      // (numbered so that the first warps, the ones a short ring keeps busy, sit on different schedulers)
+      const int n_gen = (4 - gen_quad0) * p.epi_groups, mine = eg * (4 - gen_quad0) + (quad - gen_quad0);
+      const int rows_k = p.ksteps * 16;
+      int turn = 0;                         // gen_s mod n_gen
+      for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x) {
+        const Unit w = decode_unit(p, u);
+        long kc = w.kb0 * rows_k;
+        for (int i = 0; i < w.nkb && ok; ++i) {
+          if (turn == mine) {
+            if (gen_fill > 0) {
+              if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
+              ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+              if (!ok) break;
+            }
+            fill_bp_stage(tiles_base + (uint32_t)gen_s * stage_bytes + p.a_stage_bytes, kc, w, lane, 32);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[gen_s]);
+          }
+          kc += rows_k;
+          if (++turn == n_gen) turn = 0;
+          if (++gen_s == p.stages) { gen_s = 0; turn = 0; ++gen_fill; }
+        }
+      }
+    } else
+    for (long u = blockIdx.x; u < p.units && ok; u += gridDim.x, ++lu) {
+      const Unit w = decode_unit(p, u);
+      const int buf = p.acc_bufs == 2 ? (int)(lu & 1) : 0;
+      const long use = p.acc_bufs == 2 ? lu >> 1 : lu;
+      if (p.seeded && gen_quad0 == 0) {
+        if (!redraw_ahead) redraw_unit(w);
+        else if (u + gridDim.x < p.units) redraw_unit(decode_unit(p, u + gridDim.x));
         if (!ok) break;
       }
       if (lane == 0) ok = mbar_wait(&tmem_full_bar[buf], (uint32_t)(use & 1), p.status, p.tag);
@@ -1238,12 +1365,16 @@ static int pick_stages(uint32_t stage_bytes, int want_ctas_per_sm) {
 
 static xconv_status launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, unsigned grid,
                            cudaStream_t st, const CUtensorMap* mc = nullptr) {
-  const size_t smem = (size_t)p.stages * (p.a_stage_bytes + p.b_stage_bytes) + 1024 + (size_t)p.epi_bytes + p.smem_pad;
+  TcParams q = p;
+  // the seeded back-probe keeps a 4 KB table of sign patterns behind the stages: a stage gives way if it has to
+  const size_t table = (p.seeded && p.mode == MODE_BACKPROBE) ? 4096 : 0;
+  auto bytes = [&]() { return (size_t)q.stages * (q.a_stage_bytes + q.b_stage_bytes) + 1024 + (size_t)q.epi_bytes + q.smem_pad + table; };
+  while (table && q.stages > 2 && bytes() > (size_t)(SMEM_LIMIT - 1024)) --q.stages;
+  const size_t smem = bytes();
   if (smem > (size_t)(SMEM_LIMIT - 1024) || p.tmem_cols > 512 || p.stages > MAX_STAGES) return XCONV_ERR_UNSUPPORTED;
   void (*kernel)(CUtensorMap, CUtensorMap, CUtensorMap, TcParams) = p.f16 ? tc_gemm_kernel<true> : tc_gemm_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_LIMIT - 1024);
   if (e != cudaSuccess) { set_cuda_error((int)e); return XCONV_ERR_CUDA; }
-  TcParams q = p;
   q.tag = call_tag();
   if (q.layout == 0) { q.sbo = 1024; q.mn_step = 2048; q.layout = 2; q.cw_shift = 6; }
   if (q.depth < 1) q.depth = 1;
@@ -1537,7 +1668,7 @@ __global__ void __launch_bounds__(1024) list_nonzero_blocks(const unsigned char*
 }
 
 xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const void* S_bf16, const void* dY,
-                              void* L, char* ws_head, cudaStream_t st) {
+                              void* L, char* ws_head, cudaStream_t st, const unsigned long long* seed) {
   const long Q = (long)d->H * d->W * d->Cout;
   const int bk = pl.bp_ksteps * 16;
   const bool f16 = d->dtype == XCONV_F16;
@@ -1550,7 +1681,8 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   const uint64_t sa[1] = {(uint64_t)d->B * 2}, sb[2] = {(uint64_t)Q * 2, 128};
   const uint32_t box_a[2] = {64, (uint32_t)pl.bp_rows_box};           // 128-byte rows whatever bk is (zero fill past B)
   const uint32_t box_b[3] = {64, (uint32_t)bk, 1};
-  if (!make_map(&ma, S_bf16, 2, da, sa, box_a, f16) || !make_map(&mb, dY, 3, db, sb, box_b, f16)) return XCONV_ERR_CUDA;
+  // (seeded: the streamed operand is never read, and its map stands in with the output's address)
+  if (!make_map(&ma, S_bf16, 2, da, sa, box_a, f16) || !make_map(&mb, seed ? L : dY, 3, db, sb, box_b, f16)) return XCONV_ERR_CUDA;
   // L [r][Q] for the epilogue's stores, as (64 positions, r rows, Q/64 groups): one box = the 32 rows of one
   // epilogue warp x one block of positions
   CUtensorMap mc;
@@ -1565,6 +1697,14 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.acc_bufs = pl.bp_acc_bufs;
   p.tmem_cols = pow2_cols(pl.bp_acc_bufs * pl.bp_m_sub * pl.bp_tile_n);
   p.stages = pl.bp_stages;
+  int slots = pl.bp_slots;
+  if (seed) {
+    // Z drawn on chip: a stage is filled by one warp alone, which takes longer than a copy, so the ring should hold a
+    // stage for every drawing warp; the staging rings of the epilogue give up the room
+    slots = 2;
+    const int stage = pl.bp_rows_box * 128 + bk * 128 * (pl.bp_tile_n / 64);
+    p.stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - slots * BP_SLOT_BYTES * pl.bp_groups) / stage));
+  }
   p.ksteps = pl.bp_ksteps;
   p.a_boxes = 1;
   p.b_boxes = pl.bp_tile_n / 64;
@@ -1578,8 +1718,8 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.b_mn_major = 1;
   p.b_lbo = p.b_box_bytes;
   p.epi_groups = pl.bp_groups;
-  p.epi_bytes = (uint32_t)pl.bp_slots * BP_SLOT_BYTES * pl.bp_groups;
-  p.epi_slots = pl.bp_slots;
+  p.epi_bytes = (uint32_t)slots * BP_SLOT_BYTES * pl.bp_groups;
+  p.epi_slots = slots;
   p.bp_base = pl.bp_base;
   p.bp_rem = pl.bp_rem;
   p.tiles_m = pl.bp_tiles_r;
@@ -1592,6 +1732,12 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.cols = Q;
   p.L = static_cast<bf16*>(L);
   p.Q = Q;
+  if (seed) {
+    p.seeded = 1;
+    p.seed_lo = (uint32_t)(*seed & 0xFFFFFFFFull);
+    p.seed_hi = (uint32_t)(*seed >> 32);
+    p.z_row_len = Q;
+  }
   p.status = reinterpret_cast<unsigned int*>(ws_head);
   return launch(ma, mb, p, (unsigned)std::min<long>(p.units, (long)NUM_SMS), st, &mc);
 }

@@ -79,8 +79,17 @@ def test_seeded_sketch_float_storage():
     check("seeded sketch", host(S), O.sketch(lay["X"], O.rademacher_probes(seed, r, Cin, H, W)), TOL_SKETCH)
 
 
-@pytest.mark.parametrize("shape,dtype", [((16, 64, 64, 12, 20, 24), "bf16"), ((8, 32, 32, 40, 24, 72), "bf16"),
-                                         ((3, 5, 7, 9, 11, 5), "f32"), ((2, 16, 16, 8, 8, 8), "f32")])
+@pytest.mark.parametrize("shape,dtype", [
+    ((16, 64, 64, 12, 20, 24), "bf16"),
+    # r > B on the tensor cores: the estimator sums over the probes first and its first kernel redraws Z on chip
+    ((8, 32, 32, 40, 24, 72), "bf16"),       # two k-blocks of probes, the second with 8 of 64 rows
+    ((4, 64, 64, 16, 16, 200), "f16"),       # float16 signs, four k-blocks
+    ((16, 32, 64, 64, 64, 64), "bf16"),      # one k-block per tile, a few tiles per CTA
+    ((16, 32, 32, 128, 128, 64), "bf16"),    # 14 tiles per CTA: the ring of stages wraps, six warps draw in turn
+    ((2, 128, 64, 16, 16, 520), "bf16"),     # nine k-blocks per tile: more than the ring holds
+    ((5, 64, 32, 8, 24, 24), "bf16"),        # one ragged k-block; an odd number of samples
+    ((5, 64, 32, 9, 24, 17), "bf16"),        # 17 probes (not a multiple of 8): Z goes through the workspace
+    ((3, 5, 7, 9, 11, 5), "f32"), ((2, 16, 16, 8, 8, 8), "f32")])
 def test_seeded_layer_matches_the_oracle_with_redrawn_probes(shape, dtype):
     """Algorithm 1 end to end with nothing but S and the seed kept between the passes."""
     B, Cin, Cout, H, W, r = shape
