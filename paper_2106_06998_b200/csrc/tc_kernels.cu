@@ -982,53 +982,53 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // Probing vectors redrawn from the seed: the tiles of Z of one work unit, written by these warps.
     auto redraw_unit = [&](const Unit& w) {
       if (p.mode == MODE_SKETCH) {
-          // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
-          // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
-          // copy would have produced, hand the stage over with one arrival per warp.
-          const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
-          const int GEN = 128 * p.epi_groups;
-          const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
-          const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
-          const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
-          const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
-          const uint32_t z_ones = F16 ? 0x3C003C00u : 0x3F803F80u;
-          long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
-          for (int i = 0; i < w.nkb && ok; ++i) {
-            if (gen_fill > 0) {
-              if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
-              ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-              if (!ok) break;
-            }
-            const uint32_t zbase = tiles_base + (uint32_t)gen_s * stage_bytes + z_off;
-            const uint32_t tile_bytes = (uint32_t)tile_rows * 128u;
-            if ((p.kgroup & 1) == 0 && (p.z_row_len & 127) == 0) {
-              // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
-              // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
-              const int nitems = nrows * (p.kgroup >> 1);
-              for (int it0 = gtid; it0 < nitems; it0 += 2 * GEN) {
-                const int it1 = it0 + GEN;
-                const bool two = it1 < nitems;
-                const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
-                const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
-                const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
-                const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
-                const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
-                z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0, z_ones);
-                if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
-              }
-            } else {
-              for (int item = gtid; item < nrows * p.kgroup; item += GEN) {
-                const int row = item % nrows, g = item / nrows;
-                const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
-                z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
-              }
-            }
-            fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&full_bar[gen_s]);
-            kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
-            if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
+        // Redraw this unit's tiles of Z, stage by stage, in step with the producer (same ring, same parity):
+        // wait until the MMAs have released the stage, write the signs in the K-major swizzled layout the
+        // copy would have produced, hand the stage over with one arrival per warp.
+        const int gtid = (int)threadIdx.x - 64;                       // 0 .. GEN-1
+        const int GEN = 128 * p.epi_groups;
+        const int tile_rows = p.z_is_a ? (int)(p.a_stage_bytes / (128u * p.kgroup)) : p.tile_n;
+        const long first = p.z_is_a ? (long)w.tm * p.m_sub * TILE_M : (long)w.tn * p.tile_n;
+        const int nrows = (int)max(0L, min((long)tile_rows, p.rows_z - first));
+        const uint32_t z_off = p.z_is_a ? 0u : p.a_stage_bytes;
+        const uint32_t z_ones = F16 ? 0x3C003C00u : 0x3F803F80u;
+        long kc = (p.k_weave ? w.split : w.kb0) * 64 * p.kgroup;
+        for (int i = 0; i < w.nkb && ok; ++i) {
+          if (gen_fill > 0) {
+            if (lane == 0) ok = mbar_wait(&empty_bar[gen_s], (uint32_t)((gen_fill - 1) & 1), p.status, p.tag);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
           }
+          const uint32_t zbase = tiles_base + (uint32_t)gen_s * stage_bytes + z_off;
+          const uint32_t tile_bytes = (uint32_t)tile_rows * 128u;
+          if ((p.kgroup & 1) == 0 && (p.z_row_len & 127) == 0) {
+            // one Philox block = 128 entries = the same row of two consecutive k-blocks; two blocks per
+            // round of the loop so that the two dependent chains interleave (a warp runs alone on its scheduler)
+            const int nitems = nrows * (p.kgroup >> 1);
+            for (int it0 = gtid; it0 < nitems; it0 += 2 * GEN) {
+              const int it1 = it0 + GEN;
+              const bool two = it1 < nitems;
+              const int row0_ = it0 % nrows, pr0 = it0 / nrows, row1_ = two ? it1 % nrows : 0, pr1 = two ? it1 / nrows : 0;
+              const unsigned long long b0 = (unsigned long long)((first + row0_) * p.z_row_len + kc + pr0 * 128) >> 7;
+              const unsigned long long b1 = (unsigned long long)((first + row1_) * p.z_row_len + kc + pr1 * 128) >> 7;
+              const uint4 w0 = philox4x32_10((uint32_t)b0, (uint32_t)(b0 >> 32), p.seed_lo, p.seed_hi);
+              const uint4 w1 = philox4x32_10((uint32_t)b1, (uint32_t)(b1 >> 32), p.seed_lo, p.seed_hi);
+              z_store128(zbase + (uint32_t)(2 * pr0) * tile_bytes + (uint32_t)row0_ * 128u, tile_bytes, row0_, w0, z_ones);
+              if (two) z_store128(zbase + (uint32_t)(2 * pr1) * tile_bytes + (uint32_t)row1_ * 128u, tile_bytes, row1_, w1, z_ones);
+            }
+          } else {
+            for (int item = gtid; item < nrows * p.kgroup; item += GEN) {
+              const int row = item % nrows, g = item / nrows;
+              const uint2 bits = z_sign_bits64((first + row) * p.z_row_len + kc + g * 64, p.seed_lo, p.seed_hi);
+              z_store64(zbase + (uint32_t)g * tile_bytes + (uint32_t)row * 128u, row, bits, z_ones);
+            }
+          }
+          fence_async_smem();                 // the MMA reads the stage through the asynchronous proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&full_bar[gen_s]);
+          kc += 64 * p.kgroup * (p.k_weave ? p.k_weave : 1);
+          if (++gen_s == p.stages) { gen_s = 0; ++gen_fill; }
+        }
       } else {
         // BACKPROBE with Z as the streamed operand (the estimator summed over the probes first): a stage holds, per
         // 64-position block of the column tile, ksteps*16 rows (probes) of 128 bytes, swizzled by the row like the
