@@ -106,3 +106,22 @@ def test_seeded_layer_matches_the_oracle_with_redrawn_probes(shape, dtype):
     So = O.sketch(lay["X"], Zo)
     check("sketch", host(S), So, TOL_SKETCH)
     check("dW", host(dW), O.wgrad_estimate(So, lay["dY"], Zo), TOL[dtype])
+
+
+def test_seeded_estimator_back_to_back_calls_give_the_same_bits():
+    """r > B, Z redrawn on chip, eight calls in a row on one stream through one workspace."""
+    B, Cin, Cout, H, W, r = 16, 32, 32, 96, 96, 64
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="bf16", seed=77, z="rademacher", x="relu")
+    dY = xb.to_device(lay["dY"], "bf16")
+    S = torch.from_numpy(O.sketch(lay["X"], O.rademacher_probes(5, r, Cin, H, W)).astype(np.float32)).cuda()
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, torch.bfloat16)
+    assert xb.workspace_bytes(desc, xb.OP_WGRAD_SEEDED) == xb.workspace_bytes(desc, xb.OP_WGRAD)     # no Z in the workspace
+    ws = xb.workspace(xb.workspace_bytes(desc, xb.OP_WGRAD_SEEDED), dY.device)
+    outs = [torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device="cuda", memory_format=torch.channels_last) for _ in range(8)]
+    for o in outs:
+        xb.wgrad_seeded_into(desc, S, dY, 5, o, ws)
+    torch.cuda.synchronize()
+    assert xb.workspace_status(ws) == 0
+    assert all(torch.equal(outs[0], o) for o in outs[1:])
+    Zo = O.rademacher_probes(5, r, Cin, H, W)
+    check("dW", host(outs[-1]), O.wgrad_estimate(host(S), lay["dY"], Zo), TOL["bf16"])

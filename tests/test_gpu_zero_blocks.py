@@ -177,3 +177,26 @@ def test_mask_shape_is_checked():
         xb.make_desc(4, 96, 64, 8, 8, 4, torch.bfloat16, zero_blocks=torch.zeros((4, 1), dtype=torch.uint8, device="cuda"))
     with pytest.raises(ValueError):
         xb.make_desc(4, 128, 64, 8, 8, 4, torch.bfloat16, zero_blocks=torch.zeros((4, 3), dtype=torch.uint8, device="cuda"))
+
+
+def test_back_to_back_calls_give_the_same_bits():
+    """Ten masked contractions in a row on one stream (each kernel's preamble overlaps the tail of the one before):
+    the list kernel, the main kernel and the reduce kernel of every call see the state their own call left."""
+    Cin, Cout, H, W, r = 256, 256, 28, 28, 16
+    g = np.random.Generator(np.random.PCG64(123))
+    keep = g.random((r, 4)) < 0.4
+    keep[0, 0] = True
+    Z = inputs.draw("rademacher", (r, Cin, H, W), 1231, "bf16") * np.repeat(keep, 64, axis=1)[:, :, None, None]
+    Zd = xb.to_device(Z, "bf16")
+    Ld = xb.to_device(inputs.draw("normal", (r, Cout, H, W), 1232, "bf16"), "bf16")
+    zb = torch.from_numpy((~keep).astype(np.uint8)).cuda()
+    desc = xb.make_desc(1, Cin, Cout, H, W, r, torch.bfloat16, zero_blocks=zb)
+    assert xb.zero_blocks_used(desc)
+    ws = xb.workspace(xb.workspace_bytes(desc, xb.OP_WGRAD), Ld.device)
+    outs = [torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device="cuda", memory_format=torch.channels_last) for _ in range(10)]
+    for o in outs:
+        xb.contract_into(desc, Ld, Zd, o, ws)
+    torch.cuda.synchronize()
+    assert xb.workspace_status(ws) == 0
+    assert all(torch.equal(outs[0], o) for o in outs[1:])
+    check("contraction, ten calls", host(outs[-1]), O.wgrad_contract(host(Ld), Z), 1e-5)
