@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "simt_kernels.cuh"
 #include "tc_api.h"
+#include <type_traits>
 
 namespace xconv {
 
@@ -319,7 +320,13 @@ static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, c
   const unsigned gx = (unsigned)cdiv(d->Cin, 64), gy = (unsigned)cdiv(d->Cout, 32), gz = (unsigned)p.splits;
 #define XC_CONTRACT(KS, KD, DYS) do { \
     dim3 g2(gx * (KD * KS / DYS), gy, gz); \
-    if (vec) contract_simt<TL, T, KS, KD, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+    if (vec && std::is_same<TL, float>::value && std::is_same<T, float>::value) { \
+      const size_t smem = 2 * contract_async_tile_floats<KS, DYS>() * sizeof(float); \
+      auto kern = contract_simt_async<KS, KD, DYS>; \
+      cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+      if (ea != cudaSuccess) { g_last_cuda_error = (int)ea; return XCONV_ERR_CUDA; } \
+      kern<<<g2, 256, smem, st>>>(reinterpret_cast<const float*>(L), reinterpret_cast<const float*>(Zt), part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+    } else if (vec) contract_simt<TL, T, KS, KD, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
     else contract_simt<TL, T, KS, KD, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
   } while (0)
   if (volumetric(d)) XC_CONTRACT(3, 3, 3);

@@ -282,6 +282,116 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
   }
 }
 
+// The same contraction for float storage with channel counts that are multiples of 4, tiles copied with cp.async
+// into two sets of buffers: the tiles of the next work item are on their way while this one is multiplied (the kernel
+// above loads, waits, multiplies, and leaves the overlap to the second block of the SM).  Dynamic shared memory:
+// 2 * contract_async_tile_floats<KS, DYS>() floats.
+template <int KS, int DYS>
+__host__ __device__ constexpr int contract_async_tile_floats() { return 32 * 32 + DYS * (32 + KS - 1) * 64; }
+
+__device__ __forceinline__ void cp_async16(float* dst, const float* src, bool valid) {
+  // src-size 0 fills the 16 bytes with zeros without reading (src is then any valid address)
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
+               "r"(valid ? 16 : 0) : "memory");
+}
+
+template <int KS, int KD, int DYS>
+__global__ void __launch_bounds__(256) contract_simt_async(const float* __restrict__ L, const float* __restrict__ Z,
+                                                           float* __restrict__ part, int r, int D, int H, int W, int Cin,
+                                                           int Cout, long items_per_split) {
+  constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = DYS * KS, TALL = KD * KS * KS, ZW = XC + KS - 1;
+  constexpr int TILE = contract_async_tile_floats<KS, DYS>();
+  extern __shared__ __align__(16) float tiles[];          // [2][ Ls[XC][32] | Zs[DYS][ZW][64] ]
+  const int tid = threadIdx.x;
+  const int nblocks = (Cin + 63) / 64;
+  const int dy0 = (blockIdx.x / nblocks) * DYS;
+  const int n0 = (blockIdx.x % nblocks) * 64, m0 = blockIdx.y * 32;
+  const int tx = tid & 15, ty = tid >> 4;
+  const int chunks = (W + XC - 1) / XC;
+  const long items = (long)r * D * H * chunks;
+  const long ib = (long)blockIdx.z * items_per_split;
+  const long ie = min(items, ib + items_per_split);
+
+  float acc[T][2][4];
+#pragma unroll
+  for (int t = 0; t < T; ++t)
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[t][i][k] = 0.f;
+
+  // coordinates of the item whose tiles are fetched next (one ahead of the item being multiplied)
+  int xc = (int)(ib % chunks), y = (int)((ib / chunks) % H);
+  long jz = ib / ((long)chunks * H);
+  int z = (int)(jz % D);
+  auto fetch = [&](int buf) {
+    float* Ls = tiles + buf * TILE;
+    float* Zs = Ls + XC * 32;
+    const int x0 = xc * XC;
+    {
+      const int mm = (tid & 7) * 4, px = tid >> 3;
+      const bool ok = x0 + px < W && m0 + mm < Cout;
+      cp_async16(Ls + px * 32 + mm, ok ? L + ((jz * H + y) * W + x0 + px) * Cout + m0 + mm : L, ok);
+    }
+    for (int idx = tid; idx < DYS * ZW * 16; idx += 256) {
+      const int nn = (idx & 15) * 4;
+      const int px = (idx >> 4) % ZW;
+      const int dy = (idx >> 4) / ZW;
+      const int rho = dy0 + dy, dz = rho / KS - PD;
+      const int yy = y + rho % KS - P, xx = x0 + px - P;
+      const bool ok = z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin;
+      cp_async16(Zs + (dy * ZW + px) * 64 + nn, ok ? Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn : Z, ok);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (++xc == chunks) { xc = 0; if (++y == H) { y = 0; ++jz; if (++z == D) z = 0; } }
+  };
+
+  int buf = 0;
+  if (ib < ie) fetch(0);
+  for (long it = ib; it < ie; ++it) {
+    if (it + 1 < ie) {
+      fetch(buf ^ 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // this item's copies have landed; the next item's may be in flight
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    const float* Ls = tiles + buf * TILE;
+    const float* Zs = Ls + XC * 32;
+#pragma unroll 4
+    for (int px = 0; px < XC; ++px) {
+      const float2 l = *reinterpret_cast<const float2*>(Ls + px * 32 + ty * 2);
+#pragma unroll
+      for (int dy = 0; dy < DYS; ++dy)
+#pragma unroll
+        for (int dx = 0; dx < KS; ++dx) {
+          const float4 zv = *reinterpret_cast<const float4*>(Zs + (dy * ZW + px + dx) * 64 + tx * 4);
+          float* a0 = acc[dy * KS + dx][0];
+          float* a1 = acc[dy * KS + dx][1];
+          a0[0] = fmaf(l.x, zv.x, a0[0]); a0[1] = fmaf(l.x, zv.y, a0[1]);
+          a0[2] = fmaf(l.x, zv.z, a0[2]); a0[3] = fmaf(l.x, zv.w, a0[3]);
+          a1[0] = fmaf(l.y, zv.x, a1[0]); a1[1] = fmaf(l.y, zv.y, a1[1]);
+          a1[2] = fmaf(l.y, zv.z, a1[2]); a1[3] = fmaf(l.y, zv.w, a1[3]);
+        }
+    }
+    __syncthreads();             // all reads of this buffer are done before the copies of the item after next land in it
+    buf ^= 1;
+  }
+  float* out = part + (long)blockIdx.z * Cout * TALL * Cin;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const int m = m0 + ty * 2 + i;
+    if (m >= Cout) continue;
+#pragma unroll
+    for (int t = 0; t < T; ++t)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int n = n0 + tx * 4 + k;
+        if (n < Cin) out[((long)m * TALL + dy0 * KS + t) * Cin + n] = acc[t][i][k];
+      }
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Direct convolution, used for Y (Algorithm 1 forward step 1; Eq. 5) and, with the weights read
 // transposed and flipped, for the exact input gradient dX:
