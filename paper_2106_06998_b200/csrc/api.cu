@@ -263,8 +263,16 @@ static xconv_status run_sketch_simt(const xconv_desc* d, const SketchPlan& p, co
   const long K = (long)d->H * d->W * d->Cin;
   float* part = reinterpret_cast<float*>(ws + p.part_off);
   dim3 grid((unsigned)cdiv(d->B, 64), (unsigned)cdiv(d->r, 64), (unsigned)p.splits);
-  gemm_tn_simt<T><<<grid, 256, 0, st>>>(static_cast<const T*>(Z), static_cast<const T*>(X), part, d->r, d->B, K,
-                                        p.k_per_split, (K % 4 == 0) ? 1 : 0);
+  if (std::is_same<T, float>::value && K % 4 == 0 && p.k_per_split % GT_KS == 0) {
+    const size_t smem = (size_t)GT_STAGES * 128 * GT_LD * sizeof(float);
+    cudaError_t ea = cudaFuncSetAttribute(gemm_tn_simt_async, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (ea != cudaSuccess) { g_last_cuda_error = (int)ea; return XCONV_ERR_CUDA; }
+    gemm_tn_simt_async<<<grid, 256, smem, st>>>(reinterpret_cast<const float*>(Z), reinterpret_cast<const float*>(X), part,
+                                                d->r, d->B, K, p.k_per_split);
+  } else {
+    gemm_tn_simt<T><<<grid, 256, 0, st>>>(static_cast<const T*>(Z), static_cast<const T*>(X), part, d->r, d->B, K,
+                                          p.k_per_split, (K % 4 == 0) ? 1 : 0);
+  }
   xconv_status s = check_launch();
   if (s != XCONV_OK) return s;
   const long count = (long)d->r * d->B;

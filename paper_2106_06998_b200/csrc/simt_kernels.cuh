@@ -83,6 +83,89 @@ __global__ void __launch_bounds__(256) gemm_tn_simt(const T* __restrict__ A, con
   }
 }
 
+// The same for float operands whose rows start on 16-byte boundaries (K a multiple of 4, k ranges multiples of 32):
+// the tiles are copied with cp.async straight into k-contiguous rows of shared memory, three stages deep, and the
+// arithmetic reads four consecutive k of a row with one 128-bit load (the kernel above transposes every tile
+// through registers with scalar stores, and its warps wait on those between the two barriers of a step).  A thread
+// owns rows tm + 16 i and columns tn + 16 j, i, j < 4: the sixteen lanes that differ in tn then read consecutive
+// rows, 36 floats apart, which spread over all banks.  Dynamic shared memory: GT_STAGES * 128 * GT_LD floats.
+constexpr int GT_KS = 32, GT_LD = 36, GT_STAGES = 3;
+__device__ __forceinline__ void cp_async16_f(float* dst, const float* src, bool valid) {
+  // src-size 0 fills the 16 bytes with zeros without reading (src is then any valid address)
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
+               "r"(valid ? 16 : 0) : "memory");
+}
+static __global__ void __launch_bounds__(256) gemm_tn_simt_async(const float* __restrict__ A, const float* __restrict__ Bm,
+                                                          float* __restrict__ part, int M, int N, long K, long k_per_split) {
+  extern __shared__ __align__(16) float gt_tiles[];       // [stage][A rows 0..63 | B rows 0..63][GT_LD]
+  const int tid = threadIdx.x;
+  const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+  const long kb = (long)blockIdx.z * k_per_split;
+  const long ke = min(K, kb + k_per_split);
+  const int tm = tid >> 4, tn = tid & 15;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  auto fetch = [&](int stage, long k0) {
+    float* t = gt_tiles + stage * 128 * GT_LD;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int idx = tid + 256 * i, row = idx >> 3, c = (idx & 7) * 4;       // rows 0..63: A, 64..127: B
+      const bool is_a = row < 64;
+      const int g = is_a ? m0 + row : n0 + row - 64;
+      const bool ok = (is_a ? g < M : g < N) && k0 + c < ke;
+      const float* src = (is_a ? A : Bm) + (long)g * K + k0 + c;
+      cp_async16_f(t + row * GT_LD + c, ok ? src : A, ok);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  const long steps = kb < ke ? (ke - kb + GT_KS - 1) / GT_KS : 0;
+  for (int s = 0; s < GT_STAGES - 1; ++s) {
+    if (s < steps) fetch(s, kb + (long)s * GT_KS);
+    else asm volatile("cp.async.commit_group;" ::: "memory");          // keeps the group count in step
+  }
+  for (long st = 0; st < steps; ++st) {
+    // the copies of step st are the oldest group but GT_STAGES - 2
+    asm volatile("cp.async.wait_group %0;" ::"n"(GT_STAGES - 2) : "memory");
+    __syncthreads();             // ... and every thread is done with the stage that the next fetch overwrites
+    if (st + GT_STAGES - 1 < steps) fetch((int)((st + GT_STAGES - 1) % GT_STAGES), kb + (st + GT_STAGES - 1) * GT_KS);
+    else asm volatile("cp.async.commit_group;" ::: "memory");
+    const float* ta = gt_tiles + (int)(st % GT_STAGES) * 128 * GT_LD;
+    const float* tb = ta + 64 * GT_LD;
+#pragma unroll
+    for (int k4 = 0; k4 < GT_KS; k4 += 4) {
+      float4 a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = *reinterpret_cast<const float4*>(ta + (tm + 16 * i) * GT_LD + k4);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = *reinterpret_cast<const float4*>(tb + (tn + 16 * j) * GT_LD + k4);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[i][j] = fmaf(a[i].x, b[j].x, acc[i][j]);
+          acc[i][j] = fmaf(a[i].y, b[j].y, acc[i][j]);
+          acc[i][j] = fmaf(a[i].z, b[j].z, acc[i][j]);
+          acc[i][j] = fmaf(a[i].w, b[j].w, acc[i][j]);
+        }
+    }
+  }
+  float* out = part + (long)blockIdx.z * M * N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = m0 + tm + 16 * i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = n0 + tn + 16 * j;
+      if (n < N) out[(long)m * N + n] = acc[i][j];
+    }
+  }
+}
+
 // out[i] = scale(i) * sum_s part[s][i].  Eight threads share an output and take the splits in turn (one
 // thread per output would walk a chain of `splits` dependent loads); their eight sums are added in a
 // fixed order, so results are reproducible.  scale(i) = chan_scale[i % period] if chan_scale else alpha.
@@ -289,12 +372,6 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
 template <int KS, int DYS>
 __host__ __device__ constexpr int contract_async_tile_floats() { return 32 * 32 + DYS * (32 + KS - 1) * 64; }
 
-__device__ __forceinline__ void cp_async16(float* dst, const float* src, bool valid) {
-  // src-size 0 fills the 16 bytes with zeros without reading (src is then any valid address)
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src),
-               "r"(valid ? 16 : 0) : "memory");
-}
-
 template <int KS, int KD, int DYS>
 __global__ void __launch_bounds__(256) contract_simt_async(const float* __restrict__ L, const float* __restrict__ Z,
                                                            float* __restrict__ part, int r, int D, int H, int W, int Cin,
@@ -331,7 +408,7 @@ __global__ void __launch_bounds__(256) contract_simt_async(const float* __restri
     {
       const int mm = (tid & 7) * 4, px = tid >> 3;
       const bool ok = x0 + px < W && m0 + mm < Cout;
-      cp_async16(Ls + px * 32 + mm, ok ? L + ((jz * H + y) * W + x0 + px) * Cout + m0 + mm : L, ok);
+      cp_async16_f(Ls + px * 32 + mm, ok ? L + ((jz * H + y) * W + x0 + px) * Cout + m0 + mm : L, ok);
     }
     for (int idx = tid; idx < DYS * ZW * 16; idx += 256) {
       const int nn = (idx & 15) * 4;
@@ -340,7 +417,7 @@ __global__ void __launch_bounds__(256) contract_simt_async(const float* __restri
       const int rho = dy0 + dy, dz = rho / KS - PD;
       const int yy = y + rho % KS - P, xx = x0 + px - P;
       const bool ok = z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin;
-      cp_async16(Zs + (dy * ZW + px) * 64 + nn, ok ? Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn : Z, ok);
+      cp_async16_f(Zs + (dy * ZW + px) * 64 + nn, ok ? Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn : Z, ok);
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     if (++xc == chunks) { xc = 0; if (++y == H) { y = 0; ++jz; if (++z == D) z = 0; } }
