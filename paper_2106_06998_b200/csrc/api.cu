@@ -312,9 +312,20 @@ template <typename T, typename TL>
 static xconv_status run_backprobe_simt(const xconv_desc* d, const float* S, const void* dY, void* Lv,
                                        cudaStream_t st) {
   const long Q = (long)depth(d) * d->H * d->W * d->Cout;
-  dim3 g1((unsigned)cdiv(Q, 1024), (unsigned)cdiv(d->r, 16));
-  backprobe_simt<T, TL><<<g1, 256, 0, st>>>(S, static_cast<const T*>(dY), static_cast<TL*>(Lv), d->r, d->B, Q,
-                                            (Q % 4 == 0) ? 1 : 0);
+  // Block size: the kernel holds about 126 registers per thread, so an SM runs floor(65536 / (126 t)) blocks of t
+  // threads; the time goes with (waves of the grid) x (threads an SM runs at once).  256 threads leave the last
+  // wave of a small layer part empty (256 blocks for 296 places on the 64-channel 32 x 32 layer; 224 threads fill it).
+  int threads = 256;
+  long best = -1;
+  for (int t = 256; t >= 128; t -= 32) {
+    const long per_sm = std::min<long>(65536 / (126L * t), 2048 / t);
+    const long blocks = cdiv(cdiv(Q, 4), t) * cdiv(d->r, 16);
+    const long cost = cdiv(blocks, 148 * per_sm) * per_sm * t;
+    if (best < 0 || cost < best) { best = cost; threads = t; }
+  }
+  dim3 g1((unsigned)cdiv(cdiv(Q, 4), threads), (unsigned)cdiv(d->r, 16));
+  backprobe_simt<T, TL><<<g1, threads, 0, st>>>(S, static_cast<const T*>(dY), static_cast<TL*>(Lv), d->r, d->B, Q,
+                                                (Q % 4 == 0) ? 1 : 0);
   return check_launch();
 }
 

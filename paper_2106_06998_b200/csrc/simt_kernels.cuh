@@ -193,21 +193,22 @@ reduce_partials(const float* __restrict__ part, float* __restrict__ out, long co
 
 // ---------------------------------------------------------------------------------------------
 // Back-probe, L = S dY^T (Algorithm 1 backward step 3): L[j][q] = sum_b S[j,b] * dY[b,q], q running
-// over the H*W*Cout positions of one sample.  A block owns 1024 q and 16 probes.
+// over the H*W*Cout positions of one sample.  A block owns 4 * blockDim.x q and 16 probes (the host picks the block
+// size, a multiple of 32 up to 256, so that the grid fills whole waves of the SMs).
 // ---------------------------------------------------------------------------------------------
 template <typename T, typename TL>
 __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ S, const T* __restrict__ dY,
                                                       TL* __restrict__ L, int r, int B, long Q, int vec) {
   __shared__ __align__(16) float Ss[128][16];
   const int tid = threadIdx.x;
-  const long q = ((long)blockIdx.x * 256 + tid) * 4;
+  const long q = ((long)blockIdx.x * blockDim.x + tid) * 4;
   const int j0 = blockIdx.y * 16;
   float4 acc[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
 
   for (int b0 = 0; b0 < B; b0 += 128) {
-    for (int idx = tid; idx < 128 * 16; idx += 256) {
+    for (int idx = tid; idx < 128 * 16; idx += blockDim.x) {
       const int jj = idx >> 7, bb = idx & 127;   // consecutive threads read consecutive b
       Ss[bb][jj] = (b0 + bb < B && j0 + jj < r) ? S[(long)(j0 + jj) * B + b0 + bb] : 0.f;
     }
