@@ -123,7 +123,10 @@ static SketchPlan plan_sketch(const xconv_desc* d_, bool seeded = false) {
   const long tiles = cdiv(d->r, 64) * cdiv(d->B, 64);
   // short chains: a block walks its k-range step by step with one step of loads in flight, so the time of a
   // sketch is (steps per block) x (load latency) unless the range is dealt to many blocks
-  long splits = std::max(1L, std::min(cdiv(4 * 148, tiles), cdiv(K, 128)));
+  // one full wave of the grid: four blocks of the transposing kernel fit an SM, three of the cp.async kernel that
+  // serves float rows on 16-byte boundaries (80 registers, 54 KB)
+  const long per_sm = (d->dtype == XCONV_F32 && K % 4 == 0) ? 3 : 4;
+  long splits = std::max(1L, std::min(cdiv(per_sm * 148, tiles), cdiv(K, 128)));
   splits = std::min(splits, 2048L);
   p.k_per_split = align_up((size_t)cdiv(K, splits), 32);
   p.splits = (int)cdiv(K, p.k_per_split);
