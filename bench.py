@@ -341,6 +341,36 @@ def run_xconv(args):
                       for k, n in enumerate(("sketch", "backprobe", "contract"))}
             return total, ph, clk
 
+        def measure_graph(self, steps):
+            """The same step captured once into a CUDA graph and replayed `steps` times (the library allocates nothing
+            and never synchronises, so its calls can be captured): ms per step, or None if capture is unavailable.
+            One tensor set: for layers below L2's size the replays find their inputs in L2, so only the launch-bound
+            layers gain from it."""
+            try:
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    self.count = 0
+                    self.step()
+                torch.cuda.current_stream().wait_stream(side)
+                graph = torch.cuda.CUDAGraph()
+                self.count = 0
+                with torch.cuda.graph(graph):
+                    self.step()
+                for _ in range(3):
+                    graph.replay()
+                a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a_.record()
+                for _ in range(steps):
+                    graph.replay()
+                b_.record()
+                torch.cuda.synchronize()
+                if xb.workspace_status(self.ws) != 0:
+                    return None
+                return a_.elapsed_time(b_) / steps
+            except Exception:
+                return None
+
         def phase_call(self, name, i):
             """One launch of one phase on the i-th tensor set (through the C ABI, as in the step)."""
             X_, dY_, Z_, L_ = self.sets[i % len(self.sets)]
@@ -408,6 +438,7 @@ def run_xconv(args):
     n_phase = max(5, min(args.steps, 100))
     phase_ms, phase_sets = layer.measure_phases(n_phase)
     total_ev_ms, phase_ev_ms, _ = layer.measure(n_phase, 3, None, phase_events=True)
+    graph_ms = layer.measure_graph(n_phase) if world == 1 else None
     desc, S, dW = layer.desc, layer.S, layer.dW
     launches = [n_launch]
 
@@ -616,6 +647,7 @@ def run_xconv(args):
             "phase_timing": {"launches_per_phase": n_phase, "tensor_sets_per_phase": phase_sets,
                              "fp32_fma_tflops_measured": fma_tflops,
                              "with_events_between_calls_ms": dict(phase_ev_ms, step=total_ev_ms / n_phase),
+                             "step_replayed_from_a_cuda_graph_ms": graph_ms,
                              "note": "phases and roofline: each call timed alone, K launches back to back between two "
                                      "CUDA events; with_events_between_calls_ms: the step with an event between its "
                                      "three calls, which keeps a kernel's preamble from overlapping the previous "

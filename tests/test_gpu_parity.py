@@ -394,3 +394,39 @@ def test_engines_reported():
     assert xb.engine_for(d4, xb.OP_SKETCH) == "tcgen05_bf16" and xb.engine_for(d4, xb.OP_WGRAD) == "tcgen05_bf16"
     d6 = xb.make_desc(16, 24, 40, 30, 30, 8, torch.bfloat16)         # channels not multiples of 32: FP32 FMA
     assert xb.engine_for(d6, xb.OP_WGRAD) == "simt_f32"
+
+
+def test_a_step_can_be_captured_into_a_cuda_graph():
+    """The library allocates nothing, keeps no per-call state on the host and never synchronises: sketch and
+    estimator are captured once and replayed, with the bits of the uncaptured calls."""
+    lay = inputs.make_layer(1, 8)
+    d = dev(lay)
+    B, Cin, H, W = d["X"].shape
+    Cout, r = d["dY"].shape[1], d["Z"].shape[0]
+    desc = xb.make_desc(B, Cin, Cout, H, W, r, d["X"].dtype)
+    S = torch.empty((r, B), dtype=torch.float32, device="cuda")
+    dW = torch.empty((Cout, Cin, 3, 3), dtype=torch.float32, device="cuda", memory_format=torch.channels_last)
+    ws = xb.workspace(max(xb.workspace_bytes(desc, xb.OP_SKETCH), xb.workspace_bytes(desc, xb.OP_WGRAD)), S.device)
+
+    def step():
+        xb.sketch_into(desc, d["X"], d["Z"], S, ws)
+        xb.wgrad_into(desc, S, d["dY"], d["Z"], dW, ws)
+
+    step()
+    torch.cuda.synchronize()
+    S0, W0 = S.clone(), dW.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for _ in range(3):
+        S.zero_(); dW.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(S, S0) and torch.equal(dW, W0)
+    assert xb.workspace_status(ws) == 0
+    check("dW replayed", host(dW), O.wgrad_estimate(O.sketch(lay["X"], lay["Z"]), lay["dY"], lay["Z"]), TOL["f32"])
