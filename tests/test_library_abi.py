@@ -108,3 +108,30 @@ def test_zero_block_mask_changes_the_plan_only_where_it_is_used(lib):
     assert not xb.zero_blocks_used(masked)
     plain, masked = pair(B=8, Cin=128, Cout=128, H=16, W=16, r=6, dtype=xb.XCONV_BF16, D=3, KD=3)
     assert xb.zero_blocks_used(masked)
+
+
+def test_planning_survives_random_descriptors(lib):
+    """Host arithmetic only: 3000 seeded random layers (odd sizes, all storage types, volumes, kernel sizes, with and
+    without a zero-block mask) through every size and engine query -- no crash, no absurd size, and an engine
+    answer for every layer that validates."""
+    import numpy as np
+    import torch
+    g = np.random.Generator(np.random.PCG64(20210612))
+    ops = [xb.OP_FORWARD, xb.OP_SKETCH, xb.OP_WGRAD, xb.OP_DGRAD, xb.OP_SKETCH_SEEDED, xb.OP_WGRAD_SEEDED]
+    for _ in range(3000):
+        B = int(g.choice([1, 2, 3, 8, 16, 17, 64, 100, 512, 1000]))
+        Cin = int(g.choice([1, 3, 8, 16, 32, 48, 64, 96, 128, 192, 256, 320, 512, 1024]))
+        Cout = int(g.choice([1, 3, 8, 16, 32, 48, 64, 96, 128, 192, 256, 320, 512]))
+        H, W = (int(g.choice([1, 2, 3, 4, 7, 8, 14, 16, 28, 31, 32, 56, 64, 100, 256])) for _ in range(2))
+        r = int(g.choice([1, 2, 5, 8, 16, 24, 64, 100, 256, 1000, 1024]))
+        K = int(g.choice([1, 3, 5]))
+        D = int(g.choice([1, 1, 1, 2, 3, 5]))
+        KD = 3 if (K == 3 and g.random() < 0.3) else 1
+        dt = [torch.float32, torch.bfloat16, torch.float16][int(g.integers(0, 3))]
+        d = xb.make_desc(B, Cin, Cout, H, W, r, dt, K, D=D, KD=KD)
+        if g.random() < 0.5:
+            d.zero_blocks = 256                      # never followed on the host
+        sizes = [xb.workspace_bytes(d, op) for op in ops]
+        assert all(0 < s < (1 << 46) for s in sizes), (B, Cin, Cout, H, W, r, K, D, KD, sizes)
+        assert all(xb.engine_for(d, op) != "none" for op in ops[:4])
+        assert xb.zero_blocks_used(d) in (False, True)
