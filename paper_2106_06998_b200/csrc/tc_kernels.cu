@@ -961,6 +961,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // of the odd block behind it; two items per round, so that their dependent chains interleave.
     auto fill_bp_stage = [&](uint32_t zbase, long kc, const Unit& w, int t0, int stride) {
             const int rows_k = p.ksteps * 16;
+      if ((p.z_row_len & 127) != 0) {
+        // rows of Z that start in the middle of a Philox block (their length is an odd multiple of 64): a row's even
+        // blocks are not the first halves of Philox blocks in every row, so each (row, block) takes its own half
+        for (int i = t0; i < rows_k * w.nblk; i += stride) {
+          const int row = i % rows_k, b = i / rows_k;
+          const uint2 bits = z_sign_bits64((kc + row) * p.z_row_len + (long)(w.blk0 + b) * 64, p.seed_lo, p.seed_hi);
+          z_store64_lut(zbase + (uint32_t)b * p.b_box_bytes + (uint32_t)row * 128u, row, bits, z_lut);
+        }
+        return;
+      }
       const int even0 = w.blk0 & ~1, n = rows_k * ((w.blk0 + w.nblk - even0 + 1) >> 1);
       for (int i0 = t0; i0 < n; i0 += 2 * stride) {
         const int i1 = i0 + stride;

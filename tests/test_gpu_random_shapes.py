@@ -79,3 +79,15 @@ def test_random_layer(seed):
     else:
         want = O.wgrad_estimate_independent(Sio, lay["dY"], lay["Z"], K, K)
     check("dW (independent) " + note, host(dWi), want, tol)
+    # planar layers: the same layer with its probing vectors redrawn from a seed (Algorithm 1 keeps the seed, not Z)
+    if D == 1:
+        zseed = 900000 + seed
+        Zo = O.rademacher_probes(zseed, r, Cin, H, W)
+        Ss = xb.xconv_sketch_seeded(d["X"], zseed, r)
+        Sso = O.sketch(lay["X"], Zo)
+        check("seeded sketch " + note, host(Ss), Sso, TOL_SKETCH)
+        dWs = xb.xconv_wgrad_seeded(Ss, d["dY"], zseed, Cin, kernel_size=K)
+        Zg = xb.xconv_probes_from_seed(zseed, r, Cin, H, W, d["X"].dtype)
+        assert np.array_equal(host(Zg), Zo)
+        assert torch.equal(dWs, xb.xconv_wgrad(Ss, d["dY"], Zg, kernel_size=K))
+        check("seeded dW " + note, host(dWs), O.wgrad_estimate(host(Ss), lay["dY"], Zo, K, K), tol)

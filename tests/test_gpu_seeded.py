@@ -88,6 +88,8 @@ def test_seeded_sketch_float_storage():
     ((16, 32, 32, 128, 128, 64), "bf16"),    # 14 tiles per CTA: the ring of stages wraps, six warps draw in turn
     ((2, 128, 64, 16, 16, 520), "bf16"),     # nine k-blocks per tile: more than the ring holds
     ((5, 64, 32, 8, 24, 24), "bf16"),        # one ragged k-block; an odd number of samples
+    ((4, 32, 32, 9, 22, 16), "bf16"),        # a probing vector is 99 x 64 entries long: odd rows start mid Philox block
+    ((6, 96, 32, 11, 6, 48), "f16"),         # the same with 96 channels, float16
     ((5, 64, 32, 9, 24, 17), "bf16"),        # 17 probes (not a multiple of 8): Z goes through the workspace
     ((3, 5, 7, 9, 11, 5), "f32"), ((2, 16, 16, 8, 8, 8), "f32")])
 def test_seeded_layer_matches_the_oracle_with_redrawn_probes(shape, dtype):
