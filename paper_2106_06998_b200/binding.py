@@ -275,10 +275,12 @@ def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
     return S
 
 
-def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=torch.bfloat16, device="cuda") -> torch.Tensor:
-    """Z[seed]: Rademacher probing vectors (r, Cin, H, W), channels_last, from the library's Philox stream."""
-    desc = make_desc(1, Cin, 1, H, W, r, dtype)
-    Z = torch.empty((r, Cin, H, W), dtype=dtype, device=device, memory_format=torch.channels_last)
+def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=torch.bfloat16, device="cuda",
+                           D: int = 1) -> torch.Tensor:
+    """Z[seed]: Rademacher probing vectors (r, Cin, H, W) (volumes, D > 1: (r, Cin, D, H, W)), channels-last, from the
+    library's Philox stream."""
+    desc = make_desc(1, Cin, 1, H, W, r, dtype, D=D)
+    Z = _like((r, Cin), (D, H, W), 5 if D > 1 else 4, dtype=dtype, device=device)
     _check(lib().xconv_probes_from_seed(ctypes.byref(desc), seed, Z.data_ptr(), _stream()), "xconv_probes_from_seed")
     return Z
 
@@ -286,25 +288,28 @@ def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=to
 def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int) -> torch.Tensor:
     """S = Z[seed]^T X without a stored Z (Algorithm 1 keeps the seed): float32 tensor [r, B]."""
     _cl(X, "X")
-    B, Cin, H, W = X.shape
-    desc = make_desc(B, Cin, 1, H, W, r, X.dtype)
+    B, Cin = X.shape[:2]
+    D, H, W = _geo(X)
+    desc = make_desc(B, Cin, 1, H, W, r, X.dtype, D=D)
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
     ws = workspace(workspace_bytes(desc, OP_SKETCH_SEEDED), X.device)
     sketch_seeded_into(desc, X, seed, S, ws)
     return S
 
 
-def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: int, kernel_size: int = 3) -> torch.Tensor:
-    """dW estimate from the sketch and the seed (Algorithm 1 backward steps 2-4): Z[seed] is redrawn into the
-    workspace, never passed in.  float32 (Cout, Cin, K, K), channels_last."""
+def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: int, kernel_size: int = 3,
+                       kernel_depth: int = 1) -> torch.Tensor:
+    """dW estimate from the sketch and the seed (Algorithm 1 backward steps 2-4): Z[seed] is redrawn on chip or into
+    the workspace, never passed in.  float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY")
-    B, Cout, H, Wd = dY.shape
+    B, Cout = dY.shape[:2]
+    D, H, Wd = _geo(dY)
     r = sketch.shape[0]
     if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
         raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K)
-    dW = torch.empty((Cout, Cin, K, K), dtype=torch.float32, device=dY.device, memory_format=torch.channels_last)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth)
+    dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD_SEEDED), dY.device)
     _check(lib().xconv_wgrad_seeded(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
                                     ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_seeded")

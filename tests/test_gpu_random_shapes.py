@@ -34,7 +34,7 @@ def _draw_case(seed):
     return dict(dtype=dtype, K=K, D=D, KD=KD, Cin=Cin, Cout=Cout, H=H, W=W, B=B, r=r)
 
 
-@pytest.mark.parametrize("seed", range(48))
+@pytest.mark.parametrize("seed", range(128))
 def test_random_layer(seed):
     c = _draw_case(1000 + seed)
     dtype, K, D, KD = c["dtype"], c["K"], c["D"], c["KD"]
@@ -79,15 +79,57 @@ def test_random_layer(seed):
     else:
         want = O.wgrad_estimate_independent(Sio, lay["dY"], lay["Z"], K, K)
     check("dW (independent) " + note, host(dWi), want, tol)
-    # planar layers: the same layer with its probing vectors redrawn from a seed (Algorithm 1 keeps the seed, not Z)
-    if D == 1:
-        zseed = 900000 + seed
-        Zo = O.rademacher_probes(zseed, r, Cin, H, W)
-        Ss = xb.xconv_sketch_seeded(d["X"], zseed, r)
-        Sso = O.sketch(lay["X"], Zo)
-        check("seeded sketch " + note, host(Ss), Sso, TOL_SKETCH)
-        dWs = xb.xconv_wgrad_seeded(Ss, d["dY"], zseed, Cin, kernel_size=K)
-        Zg = xb.xconv_probes_from_seed(zseed, r, Cin, H, W, d["X"].dtype)
-        assert np.array_equal(host(Zg), Zo)
-        assert torch.equal(dWs, xb.xconv_wgrad(Ss, d["dY"], Zg, kernel_size=K))
+    # the same layer with its probing vectors redrawn from a seed (Algorithm 1 keeps the seed, not Z); a volume's
+    # probing vector is numbered in memory order like an image of D*H rows
+    zseed = 900000 + seed
+    Zo = O.rademacher_probes(zseed, r, Cin, D * H, W)
+    if D > 1:
+        Zo = Zo.reshape(r, Cin, D, H, W)
+    Ss = xb.xconv_sketch_seeded(d["X"], zseed, r)
+    check("seeded sketch " + note, host(Ss), O.sketch(lay["X"], Zo), TOL_SKETCH)
+    dWs = xb.xconv_wgrad_seeded(Ss, d["dY"], zseed, Cin, kernel_size=K, kernel_depth=KD)
+    Zg = xb.xconv_probes_from_seed(zseed, r, Cin, H, W, d["X"].dtype, D=D)
+    assert np.array_equal(host(Zg), Zo)
+    assert torch.equal(dWs, xb.xconv_wgrad(Ss, d["dY"], Zg, kernel_size=K, kernel_depth=KD))
+    if D > 1:
+        check("seeded dW " + note, host(dWs), O.wgrad_estimate3d(host(Ss), lay["dY"], Zo, (KD, K, K)), tol)
+    else:
         check("seeded dW " + note, host(dWs), O.wgrad_estimate(host(Ss), lay["dY"], Zo, K, K), tol)
+
+
+def _draw_medium(seed):
+    g = np.random.Generator(np.random.PCG64(seed))
+    dtype = ["bf16", "f16"][int(g.integers(0, 2))]
+    Cin, Cout = int(g.choice([32, 64, 96])), int(g.choice([32, 64]))
+    H, W = int(g.integers(9, 41)), int(g.integers(9, 41))
+    B, r = int(g.choice([4, 8, 13, 24, 40])), int(g.choice([8, 16, 40, 72, 136, 200]))
+    return dict(dtype=dtype, Cin=Cin, Cout=Cout, H=H, W=W, B=B, r=r)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_medium_layer(seed):
+    """Larger images on the tensor-core tiles (several tiles per CTA, rings of stages that wrap, ragged tiles, probing
+    vectors of every length modulo 128), the estimator in both orders of summation, stored and redrawn probes."""
+    c = _draw_medium(5000 + seed)
+    dtype = c["dtype"]
+    B, Cin, Cout, H, W, r = c["B"], c["Cin"], c["Cout"], c["H"], c["W"], c["r"]
+    note = str(c)
+    lay = dict(X=inputs.draw("relu", (B, Cin, H, W), seed * 10 + 7, dtype),
+               dY=inputs.draw("normal", (B, Cout, H, W), seed * 10 + 8, dtype, 0.1 if dtype == "f16" else 1.0))
+    d = {k: xb.to_device(v, dtype) for k, v in lay.items()}
+    zseed = 7000 + seed
+    Zo = O.rademacher_probes(zseed, r, Cin, H, W)
+    Zg = xb.xconv_probes_from_seed(zseed, r, Cin, H, W, d["X"].dtype)
+    assert np.array_equal(host(Zg), Zo)
+    So = O.sketch(lay["X"], Zo)
+    S = xb.xconv_sketch(d["X"], Zg)
+    Ss = xb.xconv_sketch_seeded(d["X"], zseed, r)
+    check("sketch " + note, host(S), So, TOL_SKETCH)
+    check("seeded sketch " + note, host(Ss), So, TOL_SKETCH)
+    want = O.wgrad_estimate(host(S), lay["dY"], Zo)
+    dW = xb.xconv_wgrad(S, d["dY"], Zg)
+    check("dW " + note, host(dW), want, TOL[dtype])
+    assert torch.equal(dW, xb.xconv_wgrad_seeded(S, d["dY"], zseed, Cin))
+    L = xb.xconv_backprobe(S, d["dY"])
+    check("L " + note, host(L), O.backprobe(host(S), lay["dY"]), TOL[dtype])
+    check("dW (halves) " + note, host(xb.xconv_contract(L, Zg)), O.wgrad_contract(host(L), Zo), 1e-5)
