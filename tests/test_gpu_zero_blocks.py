@@ -200,3 +200,32 @@ def test_back_to_back_calls_give_the_same_bits():
     assert xb.workspace_status(ws) == 0
     assert all(torch.equal(outs[0], o) for o in outs[1:])
     check("contraction, ten calls", host(outs[-1]), O.wgrad_contract(host(Ld), Z), 1e-5)
+
+
+def _draw_masked(seed):
+    g = np.random.Generator(np.random.PCG64(seed))
+    return dict(dtype=["bf16", "f16"][int(g.integers(0, 2))], Cin=int(g.choice([128, 192, 256, 320, 512])),
+                Cout=int(g.choice([64, 128, 256])), H=int(g.choice([12, 14, 16, 20, 24, 28])),
+                W=int(g.choice([12, 14, 16, 20, 24, 28])), r=int(g.integers(4, 49)), K=int(g.choice([1, 3, 3])),
+                p=float(g.choice([0.1, 0.3, 0.6, 0.9])))
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_masked_contraction(seed):
+    """Seeded random wide layers and masks (some skip, some ignore the mask; whole probes, whole tiles and single
+    blocks zero): the contraction against the oracle, which gets the probes that are not zero altogether."""
+    c = _draw_masked(3000 + seed)
+    dtype, Cin, Cout, H, W, r, K = c["dtype"], c["Cin"], c["Cout"], c["H"], c["W"], c["r"], c["K"]
+    g = np.random.Generator(np.random.PCG64(4000 + seed))
+    keep = g.random((r, Cin // 64)) < c["p"]
+    keep[g.integers(0, r)] = False                          # one probe zero altogether
+    keep[g.integers(0, r), 0] = True                        # and at least one block that is not
+    Z = inputs.draw("rademacher", (r, Cin, H, W), seed * 10 + 1, dtype) * np.repeat(keep, 64, axis=1)[:, :, None, None]
+    Lh = inputs.draw("normal", (r, Cout, H, W), seed * 10 + 2, dtype)
+    Zd, Ld = xb.to_device(Z, dtype), xb.to_device(Lh, dtype)
+    zb = xb.xconv_zero_blocks(Zd)
+    assert np.array_equal(zb.cpu().numpy(), (~keep).astype(np.uint8))
+    got = xb.xconv_contract(Ld, Zd, kernel_size=K, zero_blocks=zb)
+    rows = np.flatnonzero(keep.any(axis=1))
+    want = O.wgrad_contract(Lh[rows], Z[rows], KH=K, KW=K, scale=np.full(Cin, 1.0 / r))
+    check("masked contraction " + str(c), host(got), want, 1e-5)
