@@ -130,7 +130,7 @@ class ClockSampler:
 _ORACLE_INPUTS = {}
 
 
-def oracle_sample_time(cfg, r, frac=8):
+def oracle_sample_time(cfg, r, frac=8, impl="numpy"):
     """The float64 oracle, as it stands, on a bounded sample of the workload: the sketch of B/frac
     samples plus the estimator for Cout/frac output channels (all probes, input channels and pixels).
     Both costs are linear in the sliced axis, so the layer time is frac x the sample time."""
@@ -152,6 +152,9 @@ def oracle_sample_time(cfg, r, frac=8):
                                inputs.draw(c["z"], (r, c["Cin"], c["H"], c["W"]), 13, c["dtype"]),
                                g.standard_normal((r, c["B"])))
     X, dY, Z, S = _ORACLE_INPUTS[key]
+    if impl == "c":                          # the same formulas as plain C loop nests (oracle/xconv_oracle.c)
+        from oracle import c_oracle as O
+        O.lib()
     t0 = time.perf_counter()
     O.sketch(X, Z)
     t1 = time.perf_counter()
@@ -617,7 +620,14 @@ def run_xconv(args):
     cpu = None
     if not args.no_cpu:
         t, ts, tw, sample = oracle_sample_time(cfg, r, frac=args.oracle_frac)
-        cpu = {"value": 1.0 / t, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample,
+        c_loops = None
+        try:                                 # the second statement of the oracle, timed on the same sample
+            tc_, _, _, _ = oracle_sample_time(cfg, r, frac=args.oracle_frac, impl="c")
+            from oracle import c_oracle
+            c_loops = {"value": 1.0 / tc_, "unit": UNIT, "cores": c_oracle.threads(), "kind": "oracle, plain C loop nests with OpenMP"}
+        except Exception as e:               # no gcc or no OpenMP on this host
+            c_loops = {"unavailable": type(e).__name__}
+        cpu = {"value": 1.0 / t, "unit": UNIT, "cores": host_threads(), "kind": "oracle", "sample": sample, "c_loops": c_loops,
                "sketch_s": ts, "wgrad_s": tw}
 
     context = {}

@@ -42,6 +42,8 @@ Hutchinson variance, and by their reduction to the multi-channel functions for a
 The functions for volumes (shift3, conv_forward3d, dw_exact3d, dx_exact3d, wgrad_contract3d, wgrad_estimate3d) are
 pinned by brute-force loops, by their reduction to the two-dimensional functions at depth 1, and by exact recovery.
 rel_fro, the metric every parity check passes through, is pinned on a hand-computed pair.
+oracle/xconv_oracle.c states the layer's formulas a second time as plain C loop nests (loader: oracle/c_oracle.py); the two
+are compared on random layers and the C one is pinned by the same brute-force loops and by exact recovery.
 No function here is "parity unpinned".
 """
 from __future__ import annotations

@@ -430,3 +430,20 @@ def test_a_step_can_be_captured_into_a_cuda_graph():
         assert torch.equal(S, S0) and torch.equal(dW, W0)
     assert xb.workspace_status(ws) == 0
     check("dW replayed", host(dW), O.wgrad_estimate(O.sketch(lay["X"], lay["Z"]), lay["dY"], lay["Z"]), TOL["f32"])
+
+
+@pytest.mark.parametrize("dtype,shape", [("f32", (5, 12, 10, 9, 11, 7)), ("bf16", (16, 64, 128, 12, 20, 24))])
+def test_against_the_plain_c_oracle(dtype, shape):
+    """The same layer against the second statement of the oracle (plain C loop nests, oracle/xconv_oracle.c)."""
+    from oracle import c_oracle as C
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape) + 5, z="rademacher", x="relu")
+    d = dev(lay)
+    Y, S = xb.xconv_forward(d["X"], d["W"], d["Z"])
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"])
+    dX = xb.xconv_dgrad(d["dY"], d["W"])
+    So = C.sketch(lay["X"], lay["Z"])
+    check("sketch", host(S), So, TOL_SKETCH)
+    check("Y", host(Y), C.conv_forward(lay["X"], lay["W"]), TOL[dtype])
+    check("dX", host(dX), C.dx_exact(lay["dY"], lay["W"]), TOL[dtype])
+    check("dW", host(dW), C.wgrad_estimate(So, lay["dY"], lay["Z"]), TOL[dtype])

@@ -608,3 +608,57 @@ def test_theorem1_crosstalk_from_channel_j_scales_like_sqrt_p_j():
             for p1 in (1.0, 0.25):
                 want = own + p1 * cross
                 assert 0.8 < var[p1][0, 0, ky, kx] / want < 1.25, (ky, kx, p1, var[p1][0, 0, ky, kx], want)
+
+
+# --- the plain-C statement of the oracle (oracle/xconv_oracle.c) -------------------------------------------------
+# Pinned by the same brute-force loops and by exact recovery (neither goes through the numpy oracle), and compared
+# with the numpy oracle on random layers.
+
+def _c():
+    from oracle import c_oracle
+    c_oracle.lib()
+    return c_oracle
+
+
+@pytest.mark.parametrize("K", [1, 3, 5])
+def test_c_oracle_against_brute_force_loops(K):
+    C = _c()
+    X, Wt, dY = _tiny(seed=10 + K, H=5, W=6 if K == 5 else 4, KH=K, KW=K)
+    np.testing.assert_allclose(C.conv_forward(X, Wt), _loops_conv(X, Wt, False), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(C.dw_exact(X, dY, K, K), _loops_dw(X, dY, K, K, False), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(C.dx_exact(dY, Wt), _loops_dx(dY, Wt, False), rtol=0, atol=1e-12)
+
+
+def test_c_oracle_recovers_the_exact_gradient_with_an_orthogonal_basis():
+    C = _c()
+    X, Wt, dY = _tiny(seed=13, B=3, Cin=2, Cout=3, H=4, W=3)
+    Z = _orth_probes(2, 4, 3, seed=19)
+    est = C.wgrad_estimate(C.sketch(X, Z), dY, Z)
+    np.testing.assert_allclose(est, _loops_dw(X, dY, 3, 3, False), rtol=0, atol=1e-11)
+
+
+def test_c_oracle_wrong_shift_sign_would_fail():
+    """The pin above has teeth for the C loops too: probing with the mirrored offset misses the gradient."""
+    C = _c()
+    X, Wt, dY = _tiny(seed=14, B=3, Cin=2, Cout=3, H=4, W=3)
+    Z = _orth_probes(2, 4, 3, seed=20)
+    est = C.wgrad_estimate(C.sketch(X, Z), dY, Z)
+    mirrored = est[:, :, ::-1, ::-1]
+    assert np.abs(mirrored - _loops_dw(X, dY, 3, 3, False)).max() > 1e-3
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_c_and_numpy_oracles_agree_on_random_layers(seed):
+    C = _c()
+    g = np.random.default_rng(100 + seed)
+    B, Cin, Cout, H, W, r = (int(g.integers(1, 6)) for _ in range(6))
+    K = int(g.choice([1, 3, 5]))
+    X, dY = g.standard_normal((B, Cin, H, W)), g.standard_normal((B, Cout, H, W))
+    Z, Wt = g.standard_normal((r, Cin, H, W)), g.standard_normal((Cout, Cin, K, K))
+    sc = g.random(Cin)
+    S = O.sketch(X, Z)
+    for got, want in ((C.conv_forward(X, Wt), O.conv_forward(X, Wt)), (C.dx_exact(dY, Wt), O.dx_exact(dY, Wt)),
+                      (C.dw_exact(X, dY, K, K), O.dw_exact(X, dY, K, K)), (C.sketch(X, Z), S),
+                      (C.backprobe(S, dY), O.backprobe(S, dY)),
+                      (C.wgrad_estimate(S, dY, Z, K, K, scale=sc), O.wgrad_estimate(S, dY, Z, K, K, scale=sc))):
+        np.testing.assert_allclose(got, want, rtol=0, atol=1e-11)
