@@ -79,6 +79,8 @@ def test_random_layer(seed):
     else:
         want = O.wgrad_estimate_independent(Sio, lay["dY"], lay["Z"], K, K)
     check("dW (independent) " + note, host(dWi), want, tol)
+    if D == 1:        # the sketch through the entry point that takes no workspace
+        check("sketch (no workspace) " + note, host(xb.xconv_sketch_static(d["X"], d["Z"])), So, TOL_SKETCH)
     # the same layer with its probing vectors redrawn from a seed (Algorithm 1 keeps the seed, not Z); a volume's
     # probing vector is numbered in memory order like an image of D*H rows
     zseed = 900000 + seed
