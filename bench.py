@@ -599,7 +599,9 @@ def run_xconv(args):
             lay3 = Layer(r3, Zs, zero_blocks=zb)
             used = xb.zero_blocks_used(lay3.desc)
             xb.sketch_into(lay3.desc, X, Zs, lay3.S, lay3.ws)
+            torch.cuda.nvtx.range_push(f"zb_r{r3}_p{pg}_w{int(whole_tiles)}")      # a handle for profilers
             t3, _ = lay3.measure_phase("contract", n3)
+            torch.cuda.nvtx.range_pop()
             listed = float((zb.view(r3, -1, tile) == 0).any(dim=2).float().mean())
             del lay3
             torch.cuda.empty_cache()
