@@ -527,7 +527,16 @@ def run_xconv(args):
         wsf = torch.empty(max(xb.workspace_bytes(desc, xb.OP_FORWARD), xb.workspace_bytes(desc, xb.OP_DGRAD)),
                           dtype=torch.uint8, device=dev)
 
-        def _time(f, n=20):
+        def _time(f, n=20, name=None):
+            if name:
+                torch.cuda.nvtx.range_push("api_" + name)          # a handle for profilers
+            try:
+                return _time_inner(f, n)
+            finally:
+                if name:
+                    torch.cuda.nvtx.range_pop()
+
+        def _time_inner(f, n):
             for _ in range(3):
                 f()
             a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -544,9 +553,9 @@ def run_xconv(args):
         S2 = torch.empty_like(S)
         full = {"forward_ms": _time(lambda: xb.forward_into(desc, X, Wt, Z, Y, S, wsf)),
                 "dgrad_ms": _time(lambda: xb.dgrad_into(desc, dY, Wt, dX, wsf)),
-                "wgrad_ms": _time(lambda: xb.wgrad_into(desc, S, dY, Z, dW, layer.ws)),
-                "sketch_seeded_ms": _time(lambda: xb.sketch_seeded_into(desc, X, 12345, S2, wss)),
-                "wgrad_seeded_ms": _time(lambda: xb.wgrad_seeded_into(desc, S, dY, 12345, dW, wss)),
+                "wgrad_ms": _time(lambda: xb.wgrad_into(desc, S, dY, Z, dW, layer.ws), name="wgrad"),
+                "sketch_seeded_ms": _time(lambda: xb.sketch_seeded_into(desc, X, 12345, S2, wss), name="sketch_seeded"),
+                "wgrad_seeded_ms": _time(lambda: xb.wgrad_seeded_into(desc, S, dY, 12345, dW, wss), name="wgrad_seeded"),
                 "conv_engine": xb.engine_for(desc, xb.OP_FORWARD),
                 "note": "xconv_forward = conv + sketch; xconv_dgrad = exact dX; xconv_wgrad = back-probe + contraction "
                         "in one call; *_seeded: probes redrawn from a seed instead of read from memory; not part of the metric"}
