@@ -1708,12 +1708,16 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.tmem_cols = pow2_cols(pl.bp_acc_bufs * pl.bp_m_sub * pl.bp_tile_n);
   p.stages = pl.bp_stages;
   int slots = pl.bp_slots;
+  int staging_quads = 4;                 // lane quadrants whose warps store (and own staging rings)
   if (seed) {
     // Z drawn on chip: a stage is filled by one warp alone, which takes longer than a copy, so the ring should hold a
-    // stage for every drawing warp; the staging rings of the epilogue give up the room
+    // stage for every drawing warp; the staging rings of the epilogue give up the room (and where only the first
+    // quadrants hold rows -- the others do nothing but draw -- only those have rings at all)
     slots = 2;
+    if (pl.bp_tiles_r == 1 && pl.bp_m_sub == 1 && d->r <= 96) staging_quads = (int)cdivl(d->r, 32);
     const int stage = pl.bp_rows_box * 128 + bk * 128 * (pl.bp_tile_n / 64);
-    p.stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - slots * BP_SLOT_BYTES * pl.bp_groups) / stage));
+    const int other = slots * (BP_SLOT_BYTES / 4) * staging_quads * pl.bp_groups + 4096;      // staging + table of signs
+    p.stages = std::max(1, std::min(MAX_STAGES, (SMEM_LIMIT - STATIC_SMEM_SLACK - other) / stage));
   }
   p.ksteps = pl.bp_ksteps;
   p.a_boxes = 1;
@@ -1728,7 +1732,7 @@ xconv_status tc_run_backprobe(const xconv_desc* d, const TcWgradPlan& pl, const 
   p.b_mn_major = 1;
   p.b_lbo = p.b_box_bytes;
   p.epi_groups = pl.bp_groups;
-  p.epi_bytes = (uint32_t)slots * BP_SLOT_BYTES * pl.bp_groups;
+  p.epi_bytes = (uint32_t)slots * (BP_SLOT_BYTES / 4) * staging_quads * pl.bp_groups;
   p.epi_slots = slots;
   p.bp_base = pl.bp_base;
   p.bp_rem = pl.bp_rem;
