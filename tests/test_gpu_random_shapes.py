@@ -135,3 +135,26 @@ def test_random_medium_layer(seed):
     L = xb.xconv_backprobe(S, d["dY"])
     check("L " + note, host(L), O.backprobe(host(S), lay["dY"]), TOL[dtype])
     check("dW (halves) " + note, host(xb.xconv_contract(L, Zg)), O.wgrad_contract(host(L), Zo), 1e-5)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_medium_convolution(seed):
+    """Forward convolution and exact input gradient on larger images (ragged patches, channel counts on and off the
+    tensor-core tiles, all kernel sizes and storage types), against the plain-C statement of the oracle."""
+    from oracle import c_oracle as C
+    g = np.random.Generator(np.random.PCG64(90000 + seed))
+    dtype = ["bf16", "f16", "f32"][int(g.integers(0, 3))]
+    K = int(g.choice([1, 3, 3, 5]))
+    Cin, Cout = int(g.choice([8, 32, 64, 96, 128, 160])), int(g.choice([8, 32, 64, 96, 128, 160]))
+    H, W = int(g.integers(5, 41)), int(g.integers(5, 41))
+    B = int(g.integers(1, 7))
+    note = str(dict(dtype=dtype, K=K, Cin=Cin, Cout=Cout, H=H, W=W, B=B))
+    X = inputs.draw("relu", (B, Cin, H, W), seed * 7 + 1, dtype)
+    Wt = inputs.draw("normal", (Cout, Cin, K, K), seed * 7 + 2, dtype, (2.0 / (Cin * K * K)) ** 0.5)
+    dY = inputs.draw("normal", (B, Cout, H, W), seed * 7 + 3, dtype, 0.1 if dtype == "f16" else 1.0)
+    Z = inputs.draw("rademacher", (4, Cin, H, W), seed * 7 + 4, dtype)
+    d = {k: xb.to_device(v, dtype) for k, v in dict(X=X, W=Wt, dY=dY, Z=Z).items()}
+    Y, _ = xb.xconv_forward(d["X"], d["W"], d["Z"])
+    dX = xb.xconv_dgrad(d["dY"], d["W"])
+    check("Y " + note, host(Y), C.conv_forward(X, Wt), TOL[dtype])
+    check("dX " + note, host(dX), C.dx_exact(dY, Wt), TOL[dtype])
