@@ -94,3 +94,34 @@ def test_independent_probing_on_a_volume():
     dW = xb.xconv_wgrad_independent(S, d["dY"], d["Z"], kernel_size=3, kernel_depth=3)
     want = np.concatenate([O.wgrad_estimate3d(So[:, n, :], lay["dY"], lay["Z"][:, n:n + 1]) for n in range(Cin)], axis=1)
     check("dW (independent, volume)", host(dW), want, TOL["f32"])
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_medium_volumes(seed):
+    """Seeded random volumes on the tensor-core tiles (depth 2-6, planar and 3 x 3 x 3 kernels, both orders of
+    summation), every entry point, stored and redrawn probes."""
+    g = np.random.Generator(np.random.PCG64(120000 + seed))
+    dtype = ["bf16", "f16"][int(g.integers(0, 2))]
+    D, KD = int(g.choice([2, 3, 4, 6])), int(g.choice([1, 3]))
+    Cin, Cout = int(g.choice([32, 64, 96])), int(g.choice([32, 64, 128]))
+    H, W = int(g.integers(5, 17)), int(g.integers(5, 17))
+    B, r = int(g.integers(1, 7)), int(g.choice([4, 8, 12, 24, 40]))
+    note = str(dict(dtype=dtype, D=D, KD=KD, Cin=Cin, Cout=Cout, H=H, W=W, B=B, r=r))
+    X = inputs.draw("relu", (B, Cin, D, H, W), seed * 7 + 1, dtype)
+    Wt = inputs.draw("normal", (Cout, Cin, KD, 3, 3), seed * 7 + 2, dtype, (2.0 / (Cin * KD * 9)) ** 0.5)
+    dY = inputs.draw("normal", (B, Cout, D, H, W), seed * 7 + 3, dtype, 0.1 if dtype == "f16" else 1.0)
+    zseed = 5 + seed
+    Zo = O.rademacher_probes(zseed, r, Cin, D * H, W).reshape(r, Cin, D, H, W)      # numbered like an image of D*H rows
+    d = {k: xb.to_device(v, dtype) for k, v in dict(X=X, W=Wt, dY=dY).items()}
+    Zg = xb.xconv_probes_from_seed(zseed, r, Cin, H, W, d["X"].dtype, D=D)
+    assert np.array_equal(host(Zg), Zo)
+    Y, S = xb.xconv_forward(d["X"], d["W"], Zg)
+    check("S " + note, host(S), O.sketch(X, Zo), TOL_SKETCH)
+    check("Y " + note, host(Y), O.conv_forward3d(X, Wt), TOL[dtype])
+    check("dX " + note, host(xb.xconv_dgrad(d["dY"], d["W"])), O.dx_exact3d(dY, Wt), TOL[dtype])
+    dW = xb.xconv_wgrad(S, d["dY"], Zg, kernel_depth=KD)
+    check("dW " + note, host(dW), O.wgrad_estimate3d(host(S), dY, Zo, (KD, 3, 3)), TOL[dtype])
+    assert torch.equal(dW, xb.xconv_wgrad_seeded(S, d["dY"], zseed, Cin, kernel_depth=KD))
+    L = xb.xconv_backprobe(S, d["dY"])
+    check("dW (halves) " + note, host(xb.xconv_contract(L, Zg, kernel_depth=KD)),
+          O.wgrad_contract3d(host(L), Zo, (KD, 3, 3)), 1e-5)
