@@ -71,6 +71,25 @@ def test_edge_shapes_all_elements(shape, dtype):
     _full_layer_parity(lay)
 
 
+# The 3 x 3 layers of the paper's two MNIST networks (appendix, network tables): 1 -> 16 on 28 x 28, 16 -> 32 on
+# 14 x 14, 32 -> 32 on 7 x 7 (the Julia network), 1 -> 32 and 32 -> 64 on 28 x 28 (the PyTorch network, whose
+# code figure in Section 4.2 uses 32 probing vectors).
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [
+    # B, Cin, Cout, H, W, r
+    (16, 1, 16, 28, 28, 8),
+    (16, 16, 32, 14, 14, 8),
+    (16, 32, 32, 7, 7, 8),
+    (8, 1, 32, 28, 28, 32),
+    (8, 32, 64, 28, 28, 32),
+])
+def test_layers_of_the_papers_mnist_networks(shape, dtype):
+    B, Cin, Cout, H, W, r = shape
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape) + 28, z="rademacher",
+                             x="normal" if Cin == 1 else "relu")
+    _full_layer_parity(lay)
+
+
 # Shapes that reach the tcgen05 kernels with ragged tiles: channel counts that are not powers of two
 # (several 64- or 32-channel groups, partial last tile), images that no patch tiles exactly, probe counts
 # and batches that are not multiples of the MMA tile, r > B (re-associated wgrad) and r < B.
