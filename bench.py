@@ -68,7 +68,7 @@ def layer_work(c, r):
 # DRAM bytes (read + write) of one launch of the dominant kernel, from the ncu capture summarised in
 # profiles/ (None where the kernel has changed since, or was never captured).
 NCU_TRAFFIC = {   # (config, r, phase): bytes; profiles/tc_gemm_kernel_config*.md, profiles/simt_kernels_config2_r64.md
-    (5, 64, "sketch"): 235.4e6, (5, 64, "backprobe"): 221.8e6, (5, 64, "contract"): 55.3e6,
+    (5, 64, "sketch"): 235.9e6, (5, 64, "backprobe"): 221.4e6, (5, 64, "contract"): 55.0e6,
     (5, 16, "contract"): 12.9e6, (5, 256, "contract"): 205.8e6,
     (4, 64, "sketch"): 339.6e6, (4, 64, "backprobe"): 277.1e6, (4, 64, "contract"): 545.5e6,
     (3, 32, "sketch"): 79.1e6, (3, 32, "backprobe"): 53.2e6, (3, 32, "contract"): 53.8e6,
