@@ -20,7 +20,9 @@
  *   dW[m,n,ky,kx]    = scale[n] * sum_{j,y,x} L[j,m,y,x] * Z[j,n,y+ky-pad_h,x+kx-pad_w]
  *   dX[b,n,u,v]      = sum_{m,ky,kx} W[m,n,ky,kx] * dY[b,m,u-ky+pad_h,v-kx+pad_w]
  * A pixel index outside [0,H)x[0,W) reads as zero (the truncating shift that matches a zero-padded
- * convolution; the paper's circular shift T_k is not implemented).  scale[n] = 1/r (Eq. 6) unless
+ * convolution), or, with desc.circular = 1, wraps around the image: the paper's circular shift T_k
+ * (Section 3), i.e. a convolution with circular padding, its exact dX and the estimator written with the
+ * same T_k.  scale[n] = 1/r (Eq. 6) unless
  * chan_scale is given (Eq. 8: 1/nnz(Z_n) for block-sparse probes).
  *
  * MEMORY LAYOUT.  Every tensor is dense and channels-last: the channel index is the fastest one.
@@ -69,7 +71,7 @@ typedef enum { XCONV_F32 = 0, XCONV_BF16 = 1, XCONV_F16 = 2 } xconv_dtype;
 typedef enum {
   XCONV_OK = 0,
   XCONV_ERR_INVALID_ARG = 1, /* NULL descriptor/pointer, non-positive size */
-  XCONV_ERR_UNSUPPORTED = 2, /* valid request without a kernel (stride, even kernel size, circular shifts ...) */
+  XCONV_ERR_UNSUPPORTED = 2, /* valid request without a kernel (stride, even kernel size, circular shifts over volumes ...) */
   XCONV_ERR_ALIGNMENT = 3,   /* a pointer is not 16-byte aligned */
   XCONV_ERR_WORKSPACE = 4,   /* ws is NULL or smaller than xconv_workspace_bytes */
   XCONV_ERR_CUDA = 5,        /* a CUDA runtime/driver call failed; see xconv_last_cuda_error */
@@ -111,7 +113,9 @@ typedef struct {
   int32_t KH, KW, pad_h, pad_w;
   int32_t r;                /* number of probing vectors */
   int32_t dtype;            /* xconv_dtype: storage of X, W, dY, Z, Y, dX */
-  int32_t circular;         /* must be 0 (truncating shifts) */
+  int32_t circular;         /* 0: truncating shifts (zero padding); 1: circular shifts T_k of Section 3 (planar layers
+                               only; the offset contraction and the convolutions then run on the FP32-FMA kernels,
+                               whatever the storage type: a copy-engine box cannot wrap around an image) */
   const float* chan_scale;  /* NULL: scale 1/r.  Else device pointer to Cin floats (Eq. 8). */
   int32_t D, KD, pad_d;     /* depth of the volume and of the kernel; 0 or 1: planar layer */
   const unsigned char* zero_blocks;  /* NULL, or device pointer to r * (Cin/64) bytes: see below */

@@ -113,9 +113,11 @@ def _dtype_code(t: torch.dtype) -> int:
     raise TypeError(f"libxconv stores float32, bfloat16 or float16, got {t}")
 
 
-def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1, zero_blocks=None) -> XConvDesc:
+def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1, zero_blocks=None,
+              circular=False) -> XConvDesc:
     """Layer descriptor; D > 1 describes a volume (tensors gain a depth axis), KD its kernel depth (1 or 3);
-    zero_blocks: uint8 CUDA tensor [r, Cin/64] marking the all-zero 64-channel blocks of the probing vectors."""
+    zero_blocks: uint8 CUDA tensor [r, Cin/64] marking the all-zero 64-channel blocks of the probing vectors;
+    circular: the paper's circular shifts T_k (circular padding) instead of zero padding, planar layers only."""
     code = dtype if isinstance(dtype, int) else _dtype_code(dtype)
     cs = chan_scale.data_ptr() if chan_scale is not None else None
     zb = None
@@ -124,7 +126,7 @@ def make_desc(B, Cin, Cout, H, W, r, dtype, K=3, chan_scale=None, D=1, KD=1, zer
                 or Cin % 64 != 0 or tuple(zero_blocks.shape) != (r, Cin // 64)):
             raise ValueError("zero_blocks must be a contiguous uint8 CUDA tensor [r, Cin/64] (Cin a multiple of 64)")
         zb = zero_blocks.data_ptr()
-    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 0, cs, D, KD, (KD - 1) // 2, zb)
+    return XConvDesc(B, Cin, Cout, H, W, K, K, (K - 1) // 2, (K - 1) // 2, r, code, 1 if circular else 0, cs, D, KD, (KD - 1) // 2, zb)
 
 
 def zero_blocks_used(desc: XConvDesc) -> bool:
@@ -298,7 +300,7 @@ def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int) -> torch.Tensor:
 
 
 def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: int, kernel_size: int = 3,
-                       kernel_depth: int = 1) -> torch.Tensor:
+                       kernel_depth: int = 1, circular: bool = False) -> torch.Tensor:
     """dW estimate from the sketch and the seed (Algorithm 1 backward steps 2-4): Z[seed] is redrawn on chip or into
     the workspace, never passed in.  float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY")
@@ -308,7 +310,7 @@ def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: i
     if tuple(sketch.shape) != (r, B) or sketch.dtype != torch.float32 or not sketch.is_contiguous():
         raise ValueError("sketch must be a contiguous float32 [r, B] tensor")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth, circular=circular)
     dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD_SEEDED), dY.device)
     _check(lib().xconv_wgrad_seeded(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
@@ -336,7 +338,7 @@ def xconv_sketch_static(X: torch.Tensor, Z: torch.Tensor, out: torch.Tensor | No
     return S
 
 
-def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
+def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor, circular: bool = False):
     """Y = conv(X, W) and the sketch S = Z^T X (Algorithm 1 forward steps 1 and 3).  5-d tensors are volumes."""
     _cl(X, "X"); _cl(W, "W"); _cl(Z, "Z")
     B, Cin = X.shape[:2]
@@ -347,7 +349,7 @@ def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
     if (W.shape[1] != Cin or W.dim() != X.dim() or tuple(Z.shape[1:]) != tuple(X.shape[1:]) or W.dtype != X.dtype
             or Z.dtype != X.dtype):
         raise ValueError("shape or dtype mismatch between X, W and Z")
-    desc = make_desc(B, Cin, Cout, H, Wd, r, X.dtype, K, D=D, KD=KD)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, X.dtype, K, D=D, KD=KD, circular=circular)
     Y = _like((B, Cout), (D, H, Wd), X.dim(), dtype=X.dtype, device=X.device)
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
     ws = workspace(workspace_bytes(desc, OP_FORWARD), X.device)
@@ -357,7 +359,7 @@ def xconv_forward(X: torch.Tensor, W: torch.Tensor, Z: torch.Tensor):
 
 def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
                 chan_scale: torch.Tensor | None = None, kernel_depth: int = 1,
-                zero_blocks: torch.Tensor | None = None) -> torch.Tensor:
+                zero_blocks: torch.Tensor | None = None, circular: bool = False) -> torch.Tensor:
     """dW estimate (Algorithm 1 backward steps 3-4): float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY"); _cl(Z, "Z")
     B, Cout = dY.shape[:2]
@@ -370,7 +372,8 @@ def xconv_wgrad(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_
     if chan_scale is not None and (chan_scale.dtype != torch.float32 or chan_scale.numel() != Cin):
         raise ValueError("chan_scale must hold Cin float32 values")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks,
+                     circular=circular)
     dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), dY.device)
     wgrad_into(desc, sketch, dY, Z, dW, ws)
@@ -394,7 +397,7 @@ def xconv_sketch_independent(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
 
 
 def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
-                            kernel_depth: int = 1) -> torch.Tensor:
+                            kernel_depth: int = 1, circular: bool = False) -> torch.Tensor:
     """dW estimate per channel pair from the per-channel sketch: float32 (Cout, Cin, [KD,] K, K), channels-last."""
     _cl(dY, "dY"); _cl(Z, "Z")
     B, Cout = dY.shape[:2]
@@ -405,7 +408,7 @@ def xconv_wgrad_independent(sketch: torch.Tensor, dY: torch.Tensor, Z: torch.Ten
     if tuple(Z.shape[2:]) != tuple(dY.shape[2:]) or Z.dtype != dY.dtype:
         raise ValueError("shape or dtype mismatch between dY and Z")
     K = kernel_size
-    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth)
+    desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth, circular=circular)
     dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD_INDEPENDENT), dY.device)
     _check(lib().xconv_wgrad_independent(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), Z.data_ptr(),
@@ -430,7 +433,7 @@ def xconv_backprobe(sketch: torch.Tensor, dY: torch.Tensor) -> torch.Tensor:
 
 def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
                    chan_scale: torch.Tensor | None = None, kernel_depth: int = 1,
-                   zero_blocks: torch.Tensor | None = None) -> torch.Tensor:
+                   zero_blocks: torch.Tensor | None = None, circular: bool = False) -> torch.Tensor:
     """dW[m,n,k] = scale[n] * sum L[j,m,.] Z[j,n,.+k] (Algorithm 1 backward step 4)."""
     _cl(L, "L"); _cl(Z, "Z")
     r, Cout = L.shape[:2]
@@ -439,14 +442,15 @@ def xconv_contract(L: torch.Tensor, Z: torch.Tensor, kernel_size: int = 3,
     if Z.shape[0] != r or tuple(Z.shape[2:]) != tuple(L.shape[2:]) or Z.dtype != L.dtype:
         raise ValueError("shape or dtype mismatch between L and Z")
     K = kernel_size
-    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks)
+    desc = make_desc(1, Cin, Cout, H, Wd, r, L.dtype, K, chan_scale, D=D, KD=kernel_depth, zero_blocks=zero_blocks,
+                     circular=circular)
     dW = _like((Cout, Cin), (kernel_depth, K, K), L.dim(), dtype=torch.float32, device=L.device)
     ws = workspace(workspace_bytes(desc, OP_WGRAD), L.device)
     contract_into(desc, L, Z, dW, ws)
     return dW
 
 
-def xconv_dgrad(dY: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
+def xconv_dgrad(dY: torch.Tensor, W: torch.Tensor, circular: bool = False) -> torch.Tensor:
     """Exact dX (transposed convolution)."""
     _cl(dY, "dY"); _cl(W, "W")
     B, Cout = dY.shape[:2]
@@ -455,7 +459,7 @@ def xconv_dgrad(dY: torch.Tensor, W: torch.Tensor) -> torch.Tensor:
     KD = W.shape[2] if W.dim() == 5 else 1
     if W.shape[0] != Cout or W.dtype != dY.dtype or W.dim() != dY.dim():
         raise ValueError("shape or dtype mismatch between dY and W")
-    desc = make_desc(B, Cin, Cout, H, Wd, 1, dY.dtype, K, D=D, KD=KD)
+    desc = make_desc(B, Cin, Cout, H, Wd, 1, dY.dtype, K, D=D, KD=KD, circular=circular)
     dX = _like((B, Cin), (D, H, Wd), dY.dim(), dtype=dY.dtype, device=dY.device)
     ws = workspace(workspace_bytes(desc, OP_DGRAD), dY.device)
     dgrad_into(desc, dY, W, dX, ws)

@@ -46,12 +46,14 @@ static xconv_status validate(const xconv_desc* d) {
     return XCONV_ERR_INVALID_ARG;
   if (d->dtype != XCONV_F32 && d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return XCONV_ERR_INVALID_ARG;
   if (d->pad_h < 0 || d->pad_w < 0 || d->D < 0 || d->KD < 0 || d->pad_d < 0) return XCONV_ERR_INVALID_ARG;
-  if (d->circular != 0) return XCONV_ERR_UNSUPPORTED;
+  if (d->circular != 0 && d->circular != 1) return XCONV_ERR_INVALID_ARG;
   if (d->KH != d->KW || (d->KH != 1 && d->KH != 3 && d->KH != 5)) return XCONV_ERR_UNSUPPORTED;
   if (2 * d->pad_h != d->KH - 1 || 2 * d->pad_w != d->KW - 1) return XCONV_ERR_UNSUPPORTED;
   // kernels over volumes: 3 x 3 x 3, or planar kernels (1 x K x K) applied to every plane
   if (kdepth(d) != 1 && !(kdepth(d) == 3 && d->KH == 3)) return XCONV_ERR_UNSUPPORTED;
   if (2 * d->pad_d != kdepth(d) - 1) return XCONV_ERR_UNSUPPORTED;
+  // circular shifts (the operator T_k of the paper's Section 3) are served for planar layers only
+  if (d->circular && (depth(d) > 1 || kdepth(d) > 1)) return XCONV_ERR_UNSUPPORTED;
   // 32-bit grid and index limits of the kernels.  r, B and the channel counts land on the y axis of a
   // grid (at most 65535 blocks of 16 or more) in the FP32-FMA kernels, and r and B trade places when
   // xconv_wgrad sums over the probes first.
@@ -347,9 +349,9 @@ static xconv_status run_contract_simt(const xconv_desc* d, const WgradPlan& p, c
       auto kern = contract_simt_async<KS, KD, DYS>; \
       cudaError_t ea = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
       if (ea != cudaSuccess) { g_last_cuda_error = (int)ea; return XCONV_ERR_CUDA; } \
-      kern<<<g2, 256, smem, st>>>(reinterpret_cast<const float*>(L), reinterpret_cast<const float*>(Zt), part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
-    } else if (vec) contract_simt<TL, T, KS, KD, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
-    else contract_simt<TL, T, KS, KD, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split); \
+      kern<<<g2, 256, smem, st>>>(reinterpret_cast<const float*>(L), reinterpret_cast<const float*>(Zt), part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split, d->circular); \
+    } else if (vec) contract_simt<TL, T, KS, KD, DYS, true><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split, d->circular); \
+    else contract_simt<TL, T, KS, KD, DYS, false><<<g2, 256, 0, st>>>(L, Zt, part, d->r, depth(d), d->H, d->W, d->Cin, d->Cout, p.items_per_split, d->circular); \
   } while (0)
   if (volumetric(d)) XC_CONTRACT(3, 3, 3);
   else if (d->KH == 3) XC_CONTRACT(3, 1, 3);
@@ -373,8 +375,8 @@ static xconv_status run_conv_simt(const xconv_desc* d, bool dgrad, const void* i
   const T* w_ = static_cast<const T*>(Wt);
   T* o_ = static_cast<T*>(out);
 #define XC_CONV(KS, KD) do { \
-    if (dgrad) conv_simt<T, KS, KD, true><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin); \
-    else       conv_simt<T, KS, KD, false><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin); \
+    if (dgrad) conv_simt<T, KS, KD, true><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin, d->circular); \
+    else       conv_simt<T, KS, KD, false><<<grid, 256, 0, st>>>(i_, w_, o_, planes, D, d->H, d->W, Ci, Co, d->Cin, d->circular); \
   } while (0)
   if (volumetric(d)) XC_CONV(3, 3);
   else if (d->KH == 3) XC_CONV(3, 1);

@@ -7,6 +7,9 @@
 
 namespace xconv {
 
+// v modulo n for v that may be negative: the pixel a circular shift reads (the paper's T_k; Section 3).
+__device__ __forceinline__ int wrap_index(int v, int n) { v %= n; return v < 0 ? v + n : v; }
+
 // ---------------------------------------------------------------------------------------------
 // Sketch, S = Z^T X (Algorithm 1 forward step 3): D[m][n] = sum_k A[m,k] * Bm[n,k], both operands
 // contiguous along k (k runs over pixel-major, channel-minor positions of one sample / one probe).
@@ -263,7 +266,7 @@ __global__ void __launch_bounds__(256) backprobe_simt(const float* __restrict__ 
 template <typename TL, typename TZ, int KS, int KD, int DYS, bool VEC>
 __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, const TZ* __restrict__ Z,
                                                      float* __restrict__ part, int r, int D, int H, int W, int Cin,
-                                                     int Cout, long items_per_split) {
+                                                     int Cout, long items_per_split, int circ) {
   constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = DYS * KS, TALL = KD * KS * KS;
   __shared__ __align__(16) float Ls[XC][32];
   __shared__ __align__(16) float Zs[DYS][XC + KS - 1][64];
@@ -306,7 +309,8 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
         const int px = (idx >> 4) % (XC + KS - 1);
         const int dy = (idx >> 4) / (XC + KS - 1);
         const int rho = dy0 + dy, dz = rho / KS - PD;
-        const int yy = y + rho % KS - P, xx = x0 + px - P;
+        int yy = y + rho % KS - P, xx = x0 + px - P;
+        if (circ) { yy = wrap_index(yy, H); xx = wrap_index(xx, W); }   // circular shift instead of zero fill
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
           v = ld4(Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn);
@@ -324,7 +328,8 @@ __global__ void __launch_bounds__(256) contract_simt(const TL* __restrict__ L, c
       const int px = (idx >> 6) % (XC + KS - 1);
       const int dy = (idx >> 6) / (XC + KS - 1);
       const int rho = dy0 + dy, dz = rho / KS - PD;
-      const int yy = y + rho % KS - P, xx = x0 + px - P;
+      int yy = y + rho % KS - P, xx = x0 + px - P;
+      if (circ) { yy = wrap_index(yy, H); xx = wrap_index(xx, W); }
       float v = 0.f;
       if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin)
         v = to_f(Z[(((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn]);
@@ -376,7 +381,7 @@ __host__ __device__ constexpr int contract_async_tile_floats() { return 32 * 32 
 template <int KS, int KD, int DYS>
 __global__ void __launch_bounds__(256) contract_simt_async(const float* __restrict__ L, const float* __restrict__ Z,
                                                            float* __restrict__ part, int r, int D, int H, int W, int Cin,
-                                                           int Cout, long items_per_split) {
+                                                           int Cout, long items_per_split, int circ) {
   constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = DYS * KS, TALL = KD * KS * KS, ZW = XC + KS - 1;
   constexpr int TILE = contract_async_tile_floats<KS, DYS>();
   extern __shared__ __align__(16) float tiles[];          // [2][ Ls[XC][32] | Zs[DYS][ZW][64] ]
@@ -416,7 +421,8 @@ __global__ void __launch_bounds__(256) contract_simt_async(const float* __restri
       const int px = (idx >> 4) % ZW;
       const int dy = (idx >> 4) / ZW;
       const int rho = dy0 + dy, dz = rho / KS - PD;
-      const int yy = y + rho % KS - P, xx = x0 + px - P;
+      int yy = y + rho % KS - P, xx = x0 + px - P;
+      if (circ) { yy = wrap_index(yy, H); xx = wrap_index(xx, W); }
       const bool ok = z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && n0 + nn < Cin;
       cp_async16_f(Zs + (dy * ZW + px) * 64 + nn, ok ? Z + (((jz + dz) * H + yy) * W + xx) * Cin + n0 + nn : Z, ok);
     }
@@ -483,7 +489,7 @@ __global__ void __launch_bounds__(256) contract_simt_async(const float* __restri
 template <typename T_, int KS, int KD, bool DGRAD>
 __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, const T_* __restrict__ Wt,
                                                  T_* __restrict__ out, int B, int D, int H, int W, int Ci, int Co,
-                                                 int Cin_w) {
+                                                 int Cin_w, int circ) {
   constexpr int P = (KS - 1) / 2, PD = (KD - 1) / 2, XC = 32, T = KD * KS * KS, CK = T >= 25 ? 4 : 16, R = KD * KS;
   __shared__ __align__(16) float Xs[R][XC + KS - 1][CK];
   __shared__ __align__(16) float Ws[T][CK][64];
@@ -504,7 +510,8 @@ __global__ void __launch_bounds__(256) conv_simt(const T_* __restrict__ in, cons
       const int cc = idx % CK;
       const int px = (idx / CK) % (XC + KS - 1);
       const int rho = idx / (CK * (XC + KS - 1)), dz = rho / KS - PD;
-      const int yy = y + rho % KS - P, xx = x0 + px - P;
+      int yy = y + rho % KS - P, xx = x0 + px - P;
+      if (circ) { yy = wrap_index(yy, H); xx = wrap_index(xx, W); }
       float v = 0.f;
       if (z + dz >= 0 && z + dz < D && yy >= 0 && yy < H && xx >= 0 && xx < W && ci0 + cc < Ci)
         v = to_f(in[(((long)(b + dz) * H + yy) * W + xx) * Ci + ci0 + cc]);

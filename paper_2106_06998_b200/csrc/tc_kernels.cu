@@ -1582,7 +1582,8 @@ int tc_plan_wgrad(const xconv_desc* d, TcWgradPlan* p) {
   // contraction: rows = Cout, cols = Cin per offset, k = (probe, patch); volumes: d->r counts planes
   const int T = d->KH * d->KW * (d->KD > 1 ? d->KD : 1);
   p->ct_cw = (d->Cout % 64 == 0 && d->Cin % 64 == 0) ? 64 : ((d->Cout % 32 == 0 && d->Cin % 32 == 0) ? 32 : 0);
-  if (p->ct_cw && (long)d->H * d->W >= 16) {
+  // a circular shift wraps around the image, which a copy-engine box cannot (it fills with zeros): FP32-FMA kernels
+  if (p->ct_cw && (long)d->H * d->W >= 16 && !d->circular) {
     mask |= 2;
     pick_patch(d->H, d->W, &p->patch_w, &p->patch_h);
     p->patches_x = (int)cdivl(d->W, p->patch_w);
@@ -1932,7 +1933,7 @@ static void pick_patch_conv(int H, int W, int* pw, int* ph) {
 bool tc_plan_conv(const xconv_desc* d, bool dgrad, TcConvPlan* p) {
   if (d->dtype != XCONV_BF16 && d->dtype != XCONV_F16) return false;
   const int Ci = dgrad ? d->Cout : d->Cin, Co = dgrad ? d->Cin : d->Cout;
-  if (Ci % 32 != 0 || Co % 8 != 0 || Co < 16) return false;
+  if (Ci % 32 != 0 || Co % 8 != 0 || Co < 16 || d->circular) return false;   // circular padding: FP32-FMA kernels
   p->tile_n = std::min(256, round_up(Co, 16));
   p->tiles_n = (int)cdivl(Co, p->tile_n);
   pick_patch_conv(d->H, d->W, &p->patch_w, &p->patch_h);

@@ -45,9 +45,17 @@ def test_workspace_sizes_are_positive_and_monotone_in_r(lib):
 def test_invalid_descriptors_are_rejected(lib):
     assert xb.workspace_bytes(_desc(B=0), xb.OP_SKETCH) == 0
     assert xb.engine_for(_desc(r=-1), xb.OP_SKETCH) == "none"
-    d = _desc()
-    d.circular = 1                       # the paper's circular shift has no kernel
+    d = _desc(Cin=64, Cout=64, dtype=xb.XCONV_BF16)
+    assert xb.engine_for(d, xb.OP_CONTRACT) == "tcgen05_bf16" and xb.engine_for(d, xb.OP_FORWARD) == "tcgen05_bf16"
+    d.circular = 1                       # circular shifts are served for planar layers, by the FP32-FMA kernels ...
+    assert xb.workspace_bytes(d, xb.OP_WGRAD) > 0
+    assert xb.engine_for(d, xb.OP_CONTRACT) == "simt_f32" and xb.engine_for(d, xb.OP_FORWARD) == "simt_f32"
+    assert xb.engine_for(d, xb.OP_SKETCH) == "tcgen05_bf16"       # the sketch shifts nothing
+    d.D, d.KD, d.pad_d = 4, 3, 1         # ... not for volumes
     assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
+    d = _desc()
+    d.circular = 2                       # a flag, not a count
+    assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 1
     d = _desc(K=7)                       # kernel sizes beyond 5 x 5 have no kernel
     assert lib.xconv_sketch(ctypes.byref(d), 16, 16, 16, 16, 1 << 20, None) == 2
     d = _desc()
