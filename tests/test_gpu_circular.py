@@ -96,3 +96,50 @@ def test_circular_shifts_over_volumes_are_refused():
     desc = xb.make_desc(2, 4, 4, 6, 6, 4, torch.float32, D=3, KD=3, circular=True)
     assert xb.workspace_bytes(desc, xb.OP_WGRAD) == 0
     assert xb.engine_for(desc, xb.OP_CONTRACT) == "none"
+
+
+def _draw_case(seed):
+    g = np.random.Generator(np.random.PCG64(seed))
+    dtype = ["f32", "bf16", "f16"][int(g.integers(0, 3))]
+    K = [1, 3, 3, 5][int(g.integers(0, 4))]
+    chans = [1, 3, 8, 16, 24, 32, 40, 64, 96, 128]
+    Cin, Cout = int(g.choice(chans)), int(g.choice(chans))
+    H, W = int(g.integers(1, 15)), int(g.integers(1, 41))
+    B, r = int(g.integers(1, 25)), int(g.integers(1, 41))
+    return dict(dtype=dtype, K=K, Cin=Cin, Cout=Cout, H=H, W=W, B=B, r=r)
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_circular_layer(seed):
+    """Seeded random planar layers with circular shifts: every storage type and kernel size, channel counts on and off
+    the tensor-core tiles (the flag must take those layers off them), batch above and below the probe count, images
+    narrower than the kernel and wider than a 32-pixel chunk; stored and redrawn probes."""
+    c = _draw_case(31000 + seed)
+    dtype, K = c["dtype"], c["K"]
+    B, Cin, Cout, H, W, r = c["B"], c["Cin"], c["Cout"], c["H"], c["W"], c["r"]
+    note = str(c)
+    lay = dict(X=inputs.draw("relu", (B, Cin, H, W), seed * 10 + 40, dtype),
+               W=inputs.draw("normal", (Cout, Cin, K, K), seed * 10 + 41, dtype, (2.0 / (Cin * K * K)) ** 0.5),
+               dY=inputs.draw("normal", (B, Cout, H, W), seed * 10 + 42, dtype, 0.1 if dtype == "f16" else 1.0),
+               Z=inputs.draw(["rademacher", "gaussian"][seed % 2], (r, Cin, H, W), seed * 10 + 43, dtype))
+    d = {k: xb.to_device(v, dtype) for k, v in lay.items()}
+    tol = TOL[dtype]
+    Y, S = xb.xconv_forward(d["X"], d["W"], d["Z"], circular=True)
+    dW = xb.xconv_wgrad(S, d["dY"], d["Z"], kernel_size=K, circular=True)
+    dX = xb.xconv_dgrad(d["dY"], d["W"], circular=True)
+    torch.cuda.synchronize()
+    So = O.sketch(lay["X"], lay["Z"])
+    check("sketch " + note, host(S), So, TOL_SKETCH)
+    check("Y " + note, host(Y), O.conv_forward(lay["X"], lay["W"], circular=True), tol)
+    check("dX " + note, host(dX), O.dx_exact(lay["dY"], lay["W"], circular=True), tol)
+    dWo = O.wgrad_estimate(So, lay["dY"], lay["Z"], K, K, circular=True)
+    check("dW " + note, host(dW), dWo, tol)
+    # the paper's order through the two halves, whatever order xconv_wgrad took
+    L = xb.xconv_backprobe(torch.from_numpy(So.astype(np.float32)).cuda(), d["dY"])
+    check("dW (halves) " + note, host(xb.xconv_contract(L, d["Z"], kernel_size=K, circular=True)), dWo, tol)
+    # probes redrawn from a seed
+    zseed = 910000 + seed
+    Zo = O.rademacher_probes(zseed, r, Cin, H, W)
+    Ss = xb.xconv_sketch_seeded(d["X"], zseed, r)
+    dWs = xb.xconv_wgrad_seeded(Ss, d["dY"], zseed, Cin, kernel_size=K, circular=True)
+    check("seeded dW " + note, host(dWs), O.wgrad_estimate(host(Ss), lay["dY"], Zo, K, K, circular=True), tol)
