@@ -36,6 +36,10 @@ literal block-matrix estimator of Eq. (6) (sketch, backprobe, wgrad_estimate).
 philox4x32_10 and rademacher_probes (probing vectors redrawn from a stored seed, Algorithm 1) are pinned
 by the generator's published known-answer vectors (tests/golden/philox4x32_10_kat.txt), by the
 balance and independence of the signs, and by the unbiasedness of the estimator run on them.
+gaussian_probes (standard normal probing vectors from a stored seed: Box-Muller on Philox words, with float32 series
+for the logarithm, sine and cosine that a GPU can repeat bit for bit) is pinned by numpy's float64 functions on the
+same arguments, by a float64 recomputation of single entries from the stated definition, by its moments, a
+Kolmogorov-Smirnov test, E[z z^T] = I, and the unbiasedness of the estimator run on it.
 sketch_independent and wgrad_estimate_independent (the estimator applied to each channel pair on its own) are
 pinned by exact recovery with one orthogonal basis per channel, by unbiasedness with the crosstalk-free
 Hutchinson variance, and by their reduction to the multi-channel functions for a single input channel.
@@ -393,6 +397,84 @@ def rademacher_probes(seed: int, r: int, Cin: int, H: int, W: int) -> np.ndarray
     bits = np.stack([(w[:, None] >> shifts[None, :]) & np.uint64(1) for w in words], axis=1)   # [block, word, bit]
     signs = 1.0 - 2.0 * bits.reshape(-1)[:total].astype(F64)
     return np.ascontiguousarray(signs.reshape(r, H, W, Cin).transpose(0, 3, 1, 2))
+
+
+def _ln_f32(t):
+    """Natural logarithm of (t * 2^-24) for odd integers 0 < t < 2^24, in float32 arithmetic whose every step is a
+    single correctly rounded IEEE operation (+, -, *, /), so that a GPU can repeat it bit for bit.
+    t = 2^k * f with f in [1, 2); if f > sqrt(2) halve it; then ln f = 2 artanh(s), s = (f - 1) / (f + 1),
+    |s| <= 0.1716, by the odd series up to s^11 (the next term is below 1e-11)."""
+    f32 = np.float32
+    t = np.asarray(t, dtype=np.int64)
+    k = np.floor(np.log2(t.astype(np.float64))).astype(np.int64)          # position of the leading bit (exact: t < 2^24)
+    f = (t.astype(np.float64) / np.exp2(k)).astype(f32)                   # exact: a 24-bit integer scaled by a power of two
+    big = f > f32(1.41421354)
+    f = np.where(big, f * f32(0.5), f).astype(f32)
+    e = (k - 24 + big.astype(np.int64)).astype(f32)
+    s = ((f - f32(1.0)) / (f + f32(1.0))).astype(f32)
+    s2 = (s * s).astype(f32)
+    p = f32(1.0 / 11.0)
+    for c in (1.0 / 9.0, 1.0 / 7.0, 1.0 / 5.0, 1.0 / 3.0, 1.0):
+        p = ((p * s2).astype(f32) + f32(c)).astype(f32)
+    lnf = ((f32(2.0) * s).astype(f32) * p).astype(f32)
+    return ((e * f32(0.693147182)).astype(f32) + lnf).astype(f32)
+
+
+def _sincos_2pi_f32(t):
+    """(cos, sin) of 2 pi t / 2^24 for odd integers 0 < t < 2^24, in float32 arithmetic of single IEEE operations.
+    The top three bits of t pick the octant, the rest is an angle x in (0, pi/4) (taken from the nearer end of the
+    octant), where sin and cos are their Taylor polynomials up to x^9 and x^10 (next terms below 2e-9)."""
+    f32 = np.float32
+    t = np.asarray(t, dtype=np.int64)
+    octant = t >> 21
+    frac = t & ((1 << 21) - 1)                              # odd, below 2^21: angle frac * 2 pi / 2^24 within the octant
+    frac = np.where(octant & 1, (1 << 21) - frac, frac)     # odd octants measure the angle back from their upper end
+    x = (frac.astype(f32) * f32(3.74507039e-07)).astype(f32)        # 2 pi / 2^24
+    x2 = (x * x).astype(f32)
+    ps = f32(1.0 / 362880.0)
+    for c in (-1.0 / 5040.0, 1.0 / 120.0, -1.0 / 6.0, 1.0):
+        ps = ((ps * x2).astype(f32) + f32(c)).astype(f32)
+    sn = (ps * x).astype(f32)
+    pc = f32(-1.0 / 3628800.0)
+    for c in (1.0 / 40320.0, -1.0 / 720.0, 1.0 / 24.0, -0.5, 1.0):
+        pc = ((pc * x2).astype(f32) + f32(c)).astype(f32)
+    cs = pc
+    # octants 0..7: (cos, sin) of the full angle from (cs, sn) of the reduced one
+    swap = ((octant + 1) >> 1) & 1                          # octants 1, 2, 5, 6: the roles of sin and cos trade places
+    c_abs = np.where(swap, sn, cs)
+    s_abs = np.where(swap, cs, sn)
+    c_neg = ((octant + 2) >> 2) & 1                         # cos < 0 in octants 2..5
+    s_neg = octant >> 2                                     # sin < 0 in octants 4..7
+    return np.where(c_neg, -c_abs, c_abs).astype(f32), np.where(s_neg, -s_abs, s_abs).astype(f32)
+
+
+def gaussian_probes(seed: int, r: int, Cin: int, H: int, W: int) -> np.ndarray:
+    """Probing vectors with standard normal entries redrawn from the stored seed (Algorithm 1, backward step 2:
+    "Z = randn(N, r)" from the seed drawn in forward step 2; Section 3 takes z ~ N(0, I)).
+
+    Definition (fixed by this library): number the entries of Z by e = ((j*H + y)*W + x)*Cin + n as for the
+    Rademacher probes.  Philox block b = e div 4 has counter (b as 64 bits in words 0-1, word 2 = 1, word 3 = 0) --
+    word 2 keeps it apart from the Rademacher stream of the same seed -- and the seed as key.  Its four words
+    w0..w3 give two pairs (w0, w1), (w2, w3) of uniforms u = (2 (w >> 9) + 1) / 2^24 in (0, 1), and each pair two
+    normals by the Box-Muller transform: sqrt(-2 ln u_a) cos(2 pi u_b) for the even entry, ... sin(...) for the odd
+    one.  Logarithm, sine and cosine are the float32 series of _ln_f32 and _sincos_2pi_f32, the square root and the
+    products single float32 operations.  Returns Z [r, Cin, H, W] (float32 values in a float64 array)."""
+    f32 = np.float32
+    total = r * Cin * H * W
+    blocks = np.arange((total + 3) // 4, dtype=np.uint64)
+    one, zero = np.ones_like(blocks), np.zeros_like(blocks)
+    w = philox4x32_10((blocks & np.uint64(0xFFFFFFFF), blocks >> np.uint64(32), one, zero),
+                      (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    out = np.empty((blocks.size, 4), dtype=f32)
+    for pair in range(2):
+        ta = ((w[2 * pair] >> np.uint64(9)).astype(np.int64) << 1) | 1
+        tb = ((w[2 * pair + 1] >> np.uint64(9)).astype(np.int64) << 1) | 1
+        rad = np.sqrt(((f32(-2.0) * _ln_f32(ta)).astype(f32))).astype(f32)
+        cs, sn = _sincos_2pi_f32(tb)
+        out[:, 2 * pair] = (rad * cs).astype(f32)
+        out[:, 2 * pair + 1] = (rad * sn).astype(f32)
+    z = out.reshape(-1)[:total].astype(F64)
+    return np.ascontiguousarray(z.reshape(r, H, W, Cin).transpose(0, 3, 1, 2))
 
 
 def memory_factor(Cin, H, W, r):

@@ -662,3 +662,77 @@ def test_c_and_numpy_oracles_agree_on_random_layers(seed):
                       (C.backprobe(S, dY), O.backprobe(S, dY)),
                       (C.wgrad_estimate(S, dY, Z, K, K, scale=sc), O.wgrad_estimate(S, dY, Z, K, K, scale=sc))):
         np.testing.assert_allclose(got, want, rtol=0, atol=1e-11)
+
+
+# ------------------------------------------------------------------ Gaussian probes redrawn from a seed
+
+def test_gaussian_probe_series_against_float64_functions():
+    """The float32 series the generator is built from, against numpy's float64 log, cos and sin on the same arguments."""
+    t = np.arange(1, 1 << 24, 2, dtype=np.int64)[::53]
+    t = np.concatenate([t, [1, 3, (1 << 24) - 1, (1 << 23) - 1, (1 << 23) + 1, 11863283, 11863285]])   # ends, sqrt(2) cut
+    ref = np.log(t / 2.0 ** 24)
+    assert np.max(np.abs(O._ln_f32(t) - ref) / np.maximum(np.abs(ref), 1e-3)) < 5e-7
+    c, s = O._sincos_2pi_f32(t)
+    a = 2.0 * np.pi * t / 2.0 ** 24
+    assert np.max(np.abs(c - np.cos(a))) < 2.5e-7 and np.max(np.abs(s - np.sin(a))) < 2.5e-7
+    # every octant boundary from both sides
+    tb = np.array([k * (1 << 21) + d for k in range(8) for d in (1, (1 << 21) - 1)], dtype=np.int64)
+    c, s = O._sincos_2pi_f32(tb)
+    a = 2.0 * np.pi * tb / 2.0 ** 24
+    assert np.max(np.abs(c - np.cos(a))) < 2.5e-7 and np.max(np.abs(s - np.sin(a))) < 2.5e-7
+
+
+def test_gaussian_probes_follow_the_stated_definition():
+    """Entries recomputed one by one from the definition in float64 (Philox block e div 4 with counter word 2 = 1,
+    uniforms from the top 23 bits, Box-Muller: cosine for even entries, sine for odd ones), in memory order."""
+    import math
+    seed, r, Cin, H, W = 0x0123456789ABCDEF, 3, 5, 4, 6
+    Z = O.gaussian_probes(seed, r, Cin, H, W)
+    flat = Z.transpose(0, 2, 3, 1).reshape(-1)               # entry e = ((j*H + y)*W + x)*Cin + n
+    for e in list(range(0, 24)) + [101, 102, 103, 357, 358, 359]:
+        b = e // 4
+        w = [int(v[0]) for v in O.philox4x32_10(([b & 0xFFFFFFFF], [b >> 32], [1], [0]),
+                                             (seed & 0xFFFFFFFF, seed >> 32))]
+        pair, odd = (e % 4) // 2, e % 2
+        ua = (2 * (w[2 * pair] >> 9) + 1) / 2.0 ** 24
+        ub = (2 * (w[2 * pair + 1] >> 9) + 1) / 2.0 ** 24
+        rad = math.sqrt(-2.0 * math.log(ua))
+        want = rad * (math.sin(2 * math.pi * ub) if odd else math.cos(2 * math.pi * ub))
+        assert abs(flat[e] - want) < 2e-6 * max(1.0, abs(want)), (e, flat[e], want)
+    assert np.array_equal(Z.astype(np.float32).astype(np.float64), Z)          # float32 values
+
+
+def test_gaussian_probes_are_standard_normal_independent_and_apart_from_the_rademacher_stream():
+    from scipy import stats
+    r, Cin, H, W = 64, 8, 20, 20
+    Z = O.gaussian_probes(99, r, Cin, H, W)
+    z = Z.ravel()
+    n = z.size
+    assert abs(z.mean()) < 5.0 / np.sqrt(n) and abs(z.var() - 1.0) < 5.0 * np.sqrt(2.0 / n)
+    assert abs(np.mean(z ** 3)) < 5.0 * np.sqrt(15.0 / n) and abs(np.mean(z ** 4) - 3.0) < 5.0 * np.sqrt(96.0 / n)
+    assert stats.kstest(z[::3], "norm").pvalue > 1e-3
+    # E[z z^T] = I (Section 3, "E(z z^T) = I"): Gram matrix of the probes over their entries, off-diagonal ~ 1/sqrt(len)
+    G = Z.reshape(r, -1) @ Z.reshape(r, -1).T / (Cin * H * W)
+    assert np.abs(G - np.eye(r)).max() < 6.0 / np.sqrt(Cin * H * W) * np.sqrt(2.0)
+    # neighbours in memory (the cosine and the sine of one pair, and the two pairs of a block) are uncorrelated
+    f = Z.transpose(0, 2, 3, 1).reshape(-1)
+    for lag in (1, 2, 3, 4):
+        assert abs(np.mean(f[:-lag] * f[lag:])) < 5.0 / np.sqrt(n)
+    # another seed, and the Rademacher stream of the same seed, are unrelated to it
+    assert abs(np.mean(z * O.gaussian_probes(100, r, Cin, H, W).ravel())) < 5.0 / np.sqrt(n)
+    assert abs(np.mean(np.sign(z) * O.rademacher_probes(99, r, Cin, H, W).ravel())) < 5.0 / np.sqrt(n)
+
+
+def test_estimator_on_gaussian_probes_from_seeds_is_unbiased_with_the_gaussian_variance():
+    """Mean over seeds -> exact gradient, and the spread is the closed-form Hutchinson variance with c = 0 (Gaussian)."""
+    X, Wt, dY = _tiny(seed=44, B=3, Cin=2, Cout=2, H=4, W=4)
+    r, T = 4, 1500
+    est = np.stack([O.wgrad_estimate(O.sketch(X, Z), dY, Z) for Z in
+                    (O.gaussian_probes(5000 + t, r, 2, 4, 4) for t in range(T))])
+    exact = O.dw_exact(X, dY)
+    sd = est.std(axis=0)
+    assert np.all(np.abs(est.mean(axis=0) - exact) < 4.5 * sd / np.sqrt(T))
+    # against Rademacher probes the Gaussian estimator has the larger own-block variance (the -2 sum A_ii^2 term is absent)
+    est_r = np.stack([O.wgrad_estimate(O.sketch(X, Z), dY, Z) for Z in
+                      (O.rademacher_probes(5000 + t, r, 2, 4, 4) for t in range(T))])
+    assert est.var(axis=0).sum() > est_r.var(axis=0).sum()
