@@ -80,7 +80,8 @@ typedef enum {
 
 typedef enum { XCONV_OP_FORWARD = 0, XCONV_OP_WGRAD = 1, XCONV_OP_DGRAD = 2, XCONV_OP_SKETCH = 3,
                XCONV_OP_BACKPROBE = 4, XCONV_OP_CONTRACT = 5, XCONV_OP_SKETCH_SEEDED = 6,
-               XCONV_OP_WGRAD_SEEDED = 7, XCONV_OP_WGRAD_INDEPENDENT = 8 } xconv_op;
+               XCONV_OP_WGRAD_SEEDED = 7, XCONV_OP_WGRAD_INDEPENDENT = 8,
+               XCONV_OP_SKETCH_SEEDED_GAUSSIAN = 9, XCONV_OP_WGRAD_SEEDED_GAUSSIAN = 10 } xconv_op;
 
 /* Which arithmetic engine a call will use for its dominant kernel. */
 typedef enum { XCONV_ENGINE_NONE = 0, XCONV_ENGINE_SIMT_F32 = 1, XCONV_ENGINE_TCGEN05_BF16 = 2,
@@ -165,6 +166,29 @@ xconv_status xconv_sketch_seeded(const xconv_desc* desc, const void* X, unsigned
                                  void* ws, size_t ws_bytes, void* cuda_stream);
 xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, const void* dY, unsigned long long seed,
                                 float* dW, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* The same with standard normal probing vectors, the distribution of the paper's theory (Section 3: z ~ N(0, I);
+ * Algorithm 1 backward step 2: "Z = randn(N, r)" redrawn from the stored seed).  Definition: entries numbered in
+ * memory order as above; Philox-4x32-10 block b = e div 4 has counter (b in words 0-1, word 2 = 1, word 3 = 0) --
+ * word 2 keeps it apart from the Rademacher stream of the same seed -- and the seed as key; its words w0..w3 give
+ * two pairs (w0, w1), (w2, w3) of uniforms u = (2 (w >> 9) + 1) / 2^24, and each pair (u_a, u_b) two normals by the
+ * Box-Muller transform: sqrt(-2 ln u_a) cos(2 pi u_b) for the even entry, sqrt(-2 ln u_a) sin(2 pi u_b) for the
+ * odd one, rounded to desc.dtype.  Logarithm, sine and cosine are short float series of single IEEE operations
+ * (relative error 2e-7, absolute 1e-7), so that a host program can reproduce every entry bit for bit.
+ *
+ * xconv_gaussian_probes_from_seed writes Z [r,H,W,Cin] (volumes [r,D,H,W,Cin]) in desc.dtype; no scratch.
+ * Drawing a normal costs more than reading it back from memory (one Philox block per four entries against one per
+ * 128 signs, plus the series), so these probes are not redrawn inside the sketch and estimator kernels:
+ * xconv_sketch_seeded_gaussian and xconv_wgrad_seeded_gaussian write Z[seed] into `ws` (behind the regular scratch:
+ * xconv_workspace_bytes(desc, XCONV_OP_SKETCH_SEEDED_GAUSSIAN / XCONV_OP_WGRAD_SEEDED_GAUSSIAN) bytes) and run
+ * xconv_sketch / xconv_wgrad on it -- Algorithm 1 taken literally.  Between the passes a layer keeps S and the seed. */
+xconv_status xconv_gaussian_probes_from_seed(const xconv_desc* desc, unsigned long long seed, void* Z,
+                                             void* cuda_stream);
+xconv_status xconv_sketch_seeded_gaussian(const xconv_desc* desc, const void* X, unsigned long long seed,
+                                          float* sketch, void* ws, size_t ws_bytes, void* cuda_stream);
+xconv_status xconv_wgrad_seeded_gaussian(const xconv_desc* desc, const float* sketch, const void* dY,
+                                         unsigned long long seed, float* dW, void* ws, size_t ws_bytes,
+                                         void* cuda_stream);
 
 /* Algorithm 1, backward steps 3-4: L = S dY^T, then dW[m,n,k] = scale[n] * tr(L^m T_{-k} Z_n) for
  * every offset (Eq. 6; three-step procedure of Section 3).  sketch [r,B] float as written by

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libxconv.so")
 
 XCONV_F32, XCONV_BF16, XCONV_F16 = 0, 1, 2
 OP_FORWARD, OP_WGRAD, OP_DGRAD, OP_SKETCH, OP_BACKPROBE, OP_CONTRACT, OP_SKETCH_SEEDED, OP_WGRAD_SEEDED, OP_WGRAD_INDEPENDENT = 0, 1, 2, 3, 4, 5, 6, 7, 8
+OP_SKETCH_SEEDED_GAUSSIAN, OP_WGRAD_SEEDED_GAUSSIAN = 9, 10
 ENGINE_NAMES = {0: "none", 1: "simt_f32", 2: "tcgen05_bf16", 3: "tcgen05_f16"}
 STATUS_OK = 0
 
@@ -26,6 +27,7 @@ EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_
            "xconv_dgrad", "xconv_probes_from_seed", "xconv_sketch_seeded", "xconv_wgrad_seeded", "xconv_backprobe_bytes", "xconv_backprobe", "xconv_contract", "xconv_host_arena_bytes", "xconv_sketch_wgrad_host", "xconv_sketch_static",
            "xconv_workspace_status", "xconv_selftest_wait_limit", "xconv_measure_fma_rate",
            "xconv_sketch_independent", "xconv_wgrad_independent", "xconv_zero_blocks", "xconv_zero_blocks_used",
+           "xconv_gaussian_probes_from_seed", "xconv_sketch_seeded_gaussian", "xconv_wgrad_seeded_gaussian",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -69,6 +71,12 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_seeded.restype = c_int
     L.xconv_wgrad_seeded.argtypes = [P, c_void_p, c_void_p, ctypes.c_ulonglong, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad_seeded.restype = c_int
+    L.xconv_gaussian_probes_from_seed.argtypes = L.xconv_probes_from_seed.argtypes
+    L.xconv_gaussian_probes_from_seed.restype = c_int
+    L.xconv_sketch_seeded_gaussian.argtypes = L.xconv_sketch_seeded.argtypes
+    L.xconv_sketch_seeded_gaussian.restype = c_int
+    L.xconv_wgrad_seeded_gaussian.argtypes = L.xconv_wgrad_seeded.argtypes
+    L.xconv_wgrad_seeded_gaussian.restype = c_int
     L.xconv_wgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad.restype = c_int
     L.xconv_sketch_independent.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -278,31 +286,39 @@ def xconv_sketch(X: torch.Tensor, Z: torch.Tensor) -> torch.Tensor:
 
 
 def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=torch.bfloat16, device="cuda",
-                           D: int = 1) -> torch.Tensor:
-    """Z[seed]: Rademacher probing vectors (r, Cin, H, W) (volumes, D > 1: (r, Cin, D, H, W)), channels-last, from the
-    library's Philox stream."""
+                           D: int = 1, gaussian: bool = False) -> torch.Tensor:
+    """Z[seed]: Rademacher (or, with ``gaussian``, standard normal) probing vectors (r, Cin, H, W) (volumes, D > 1:
+    (r, Cin, D, H, W)), channels-last, from the library's Philox streams."""
     desc = make_desc(1, Cin, 1, H, W, r, dtype, D=D)
     Z = _like((r, Cin), (D, H, W), 5 if D > 1 else 4, dtype=dtype, device=device)
-    _check(lib().xconv_probes_from_seed(ctypes.byref(desc), seed, Z.data_ptr(), _stream()), "xconv_probes_from_seed")
+    fn = lib().xconv_gaussian_probes_from_seed if gaussian else lib().xconv_probes_from_seed
+    _check(fn(ctypes.byref(desc), seed, Z.data_ptr(), _stream()), "xconv_probes_from_seed")
     return Z
 
 
-def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int) -> torch.Tensor:
-    """S = Z[seed]^T X without a stored Z (Algorithm 1 keeps the seed): float32 tensor [r, B]."""
+def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int, gaussian: bool = False) -> torch.Tensor:
+    """S = Z[seed]^T X without a stored Z (Algorithm 1 keeps the seed): float32 tensor [r, B].  ``gaussian``: standard
+    normal probing vectors (drawn into the workspace) instead of Rademacher ones."""
     _cl(X, "X")
     B, Cin = X.shape[:2]
     D, H, W = _geo(X)
     desc = make_desc(B, Cin, 1, H, W, r, X.dtype, D=D)
     S = torch.empty((r, B), dtype=torch.float32, device=X.device)
+    if gaussian:
+        ws = workspace(workspace_bytes(desc, OP_SKETCH_SEEDED_GAUSSIAN), X.device)
+        _check(lib().xconv_sketch_seeded_gaussian(ctypes.byref(desc), X.data_ptr(), seed, S.data_ptr(), ws.data_ptr(),
+                                                  ws.numel(), _stream()), "xconv_sketch_seeded_gaussian")
+        return S
     ws = workspace(workspace_bytes(desc, OP_SKETCH_SEEDED), X.device)
     sketch_seeded_into(desc, X, seed, S, ws)
     return S
 
 
 def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: int, kernel_size: int = 3,
-                       kernel_depth: int = 1, circular: bool = False) -> torch.Tensor:
+                       kernel_depth: int = 1, circular: bool = False, gaussian: bool = False) -> torch.Tensor:
     """dW estimate from the sketch and the seed (Algorithm 1 backward steps 2-4): Z[seed] is redrawn on chip or into
-    the workspace, never passed in.  float32 (Cout, Cin, [KD,] K, K), channels-last."""
+    the workspace, never passed in.  float32 (Cout, Cin, [KD,] K, K), channels-last.  ``gaussian``: standard normal
+    probing vectors instead of Rademacher ones."""
     _cl(dY, "dY")
     B, Cout = dY.shape[:2]
     D, H, Wd = _geo(dY)
@@ -312,9 +328,10 @@ def xconv_wgrad_seeded(sketch: torch.Tensor, dY: torch.Tensor, seed: int, Cin: i
     K = kernel_size
     desc = make_desc(B, Cin, Cout, H, Wd, r, dY.dtype, K, D=D, KD=kernel_depth, circular=circular)
     dW = _like((Cout, Cin), (kernel_depth, K, K), dY.dim(), dtype=torch.float32, device=dY.device)
-    ws = workspace(workspace_bytes(desc, OP_WGRAD_SEEDED), dY.device)
-    _check(lib().xconv_wgrad_seeded(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
-                                    ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_seeded")
+    fn = lib().xconv_wgrad_seeded_gaussian if gaussian else lib().xconv_wgrad_seeded
+    ws = workspace(workspace_bytes(desc, OP_WGRAD_SEEDED_GAUSSIAN if gaussian else OP_WGRAD_SEEDED), dY.device)
+    _check(fn(ctypes.byref(desc), sketch.data_ptr(), dY.data_ptr(), seed, dW.data_ptr(),
+              ws.data_ptr(), ws.numel(), _stream()), "xconv_wgrad_seeded")
     return dW
 
 

@@ -256,6 +256,38 @@ static xconv_status run_probes_from_seed(const xconv_desc* d, unsigned long long
   return XCONV_OK;
 }
 
+// Z with standard normal entries from a seed: Philox block b (counter word 2 = 1, which keeps the stream apart from
+// the Rademacher one) gives entries 4b .. 4b+3, two Box-Muller pairs.  One thread per block.
+template <typename T>
+__global__ void __launch_bounds__(256) gaussian_probes_kernel(T* __restrict__ Z, long total, uint32_t k0, uint32_t k1) {
+  pdl_trigger();
+  pdl_wait();
+  const long b = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long e0 = b * 4;
+  if (e0 >= total) return;
+  const uint4 w = philox4x32_10((uint32_t)b, (uint32_t)((unsigned long long)b >> 32), k0, k1, 1u);
+  const float2 p0 = box_muller_u24(w.x, w.y), p1 = box_muller_u24(w.z, w.w);
+  if (e0 + 4 <= total) { st4(Z + e0, make_float4(p0.x, p0.y, p1.x, p1.y)); return; }
+  const float v[4] = {p0.x, p0.y, p1.x, p1.y};
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (e0 + i < total) Z[e0 + i] = from_f<T>(v[i]);
+}
+
+static xconv_status run_gaussian_probes(const xconv_desc* d, unsigned long long seed, void* Z, cudaStream_t st) {
+  const long total = (long)d->r * depth(d) * d->H * d->W * d->Cin;
+  const unsigned grid = (unsigned)cdiv(cdiv(total, 4), 256);
+  const uint32_t k0 = (uint32_t)(seed & 0xFFFFFFFFull), k1 = (uint32_t)(seed >> 32);
+  cudaError_t e = d->dtype == XCONV_F32
+      ? launch_pdl(gaussian_probes_kernel<float>, dim3(grid), dim3(256), 0, st, static_cast<float*>(Z), total, k0, k1)
+      : d->dtype == XCONV_F16
+      ? launch_pdl(gaussian_probes_kernel<f16>, dim3(grid), dim3(256), 0, st, static_cast<f16*>(Z), total, k0, k1)
+      : launch_pdl(gaussian_probes_kernel<bf16>, dim3(grid), dim3(256), 0, st, static_cast<bf16*>(Z), total, k0, k1);
+  ++g_launches;
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
+  return XCONV_OK;
+}
+
 static size_t probes_bytes(const xconv_desc* d) {
   return align_up((size_t)d->r * depth(d) * d->H * d->W * d->Cin * (d->dtype == XCONV_F32 ? 4 : 2), 256);
 }
@@ -572,6 +604,8 @@ size_t xconv_workspace_bytes(const xconv_desc* desc, int op) {
       const SketchPlan p = plan_sketch(desc, true);
       return p.bytes + (sketch_redraws(desc, p) ? 0 : probes_bytes(desc));
     }
+    case XCONV_OP_SKETCH_SEEDED_GAUSSIAN: return plan_sketch(desc).bytes + probes_bytes(desc);
+    case XCONV_OP_WGRAD_SEEDED_GAUSSIAN: return plan_wgrad(desc).bytes + probes_bytes(desc);
     case XCONV_OP_WGRAD:
     case XCONV_OP_BACKPROBE:
     case XCONV_OP_CONTRACT: return plan_wgrad(desc).bytes;
@@ -645,6 +679,51 @@ xconv_status xconv_wgrad_seeded(const xconv_desc* desc, const float* sketch, con
   // Algorithm 1 backward step 2: redraw Z from the seed (behind the regular scratch), then steps 3-4
   char* Z = static_cast<char*>(ws) + base;
   s = run_probes_from_seed(desc, seed, Z, st);
+  if (s != XCONV_OK) return s;
+  return run_wgrad(desc, sketch, dY, Z, dW, ws, base, st);
+}
+
+xconv_status xconv_gaussian_probes_from_seed(const xconv_desc* desc, unsigned long long seed, void* Z,
+                                             void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!Z) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(Z)) return XCONV_ERR_ALIGNMENT;
+  new_call();
+  return run_gaussian_probes(desc, seed, Z, static_cast<cudaStream_t>(cuda_stream));
+}
+
+xconv_status xconv_sketch_seeded_gaussian(const xconv_desc* desc, const void* X, unsigned long long seed,
+                                          float* sketch, void* ws, size_t ws_bytes, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!X || !sketch) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(sketch)) return XCONV_ERR_ALIGNMENT;
+  const size_t base = plan_sketch(desc).bytes;
+  s = check_ws(ws, ws_bytes, base + probes_bytes(desc));
+  if (s != XCONV_OK) return s;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* Z = static_cast<char*>(ws) + base;             // Z[seed] behind the regular scratch, then the regular kernels
+  s = run_gaussian_probes(desc, seed, Z, st);
+  if (s != XCONV_OK) return s;
+  return run_sketch(desc, X, Z, sketch, ws, base, st);
+}
+
+xconv_status xconv_wgrad_seeded_gaussian(const xconv_desc* desc, const float* sketch, const void* dY,
+                                         unsigned long long seed, float* dW, void* ws, size_t ws_bytes,
+                                         void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!sketch || !dY || !dW) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(sketch) || !aligned16(dY) || !aligned16(dW)) return XCONV_ERR_ALIGNMENT;
+  const size_t base = plan_wgrad(desc).bytes;
+  s = check_ws(ws, ws_bytes, base + probes_bytes(desc));
+  if (s != XCONV_OK) return s;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* Z = static_cast<char*>(ws) + base;             // Algorithm 1 backward step 2, then steps 3-4
+  s = run_gaussian_probes(desc, seed, Z, st);
   if (s != XCONV_OK) return s;
   return run_wgrad(desc, sketch, dY, Z, dW, ws, base, st);
 }

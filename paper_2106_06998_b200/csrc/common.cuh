@@ -101,11 +101,11 @@ __device__ __forceinline__ void st4_guard(T* p, long idx, long limit, bool vec, 
   if (idx + 3 < limit) p[idx + 3] = from_f<T>(v.w);
 }
 
-// Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11): counter (c0, c1, 0, 0), key = the seed.
+// Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11): counter (c0, c1, c2, 0), key = the seed.
 // One round: (hi0, lo0) = M0 * c0, (hi1, lo1) = M1 * c2, c <- (hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0), then
 // the key moves on by the Weyl constants.
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1) {
-  uint32_t c2 = 0u, c3 = 0u;
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1, uint32_t c2 = 0u) {
+  uint32_t c3 = 0u;
 #pragma unroll
   for (int i = 0; i < 10; ++i) {
     const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
@@ -114,6 +114,64 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
   }
   return make_uint4(c0, c1, c2, c3);
+}
+
+// Standard normal probing vectors from Philox words (xconv_gaussian_probes_from_seed).  Every step below is one
+// correctly rounded IEEE float operation (the _rn intrinsics are never contracted into fused multiply-adds), in a
+// fixed order, so that a host program following the same steps in float gets the same bits.
+
+// ln(t * 2^-24) for an odd t below 2^24: t = 2^k f, f in [1, 2), halved when above sqrt(2); ln f = 2 artanh(s),
+// s = (f - 1) / (f + 1), by the odd series up to s^11.
+__device__ __forceinline__ float ln_u24(uint32_t t) {
+  const int k = 31 - __clz((int)t);
+  float f = __uint_as_float(((t << (23 - k)) & 0x007FFFFFu) | 0x3F800000u);
+  const int big = f > 1.41421354f ? 1 : 0;
+  if (big) f = __fmul_rn(f, 0.5f);
+  const float e = (float)(k - 24 + big);
+  const float s = __fdiv_rn(__fsub_rn(f, 1.0f), __fadd_rn(f, 1.0f));
+  const float s2 = __fmul_rn(s, s);
+  float p = (float)(1.0 / 11.0);
+  p = __fadd_rn(__fmul_rn(p, s2), (float)(1.0 / 9.0));
+  p = __fadd_rn(__fmul_rn(p, s2), (float)(1.0 / 7.0));
+  p = __fadd_rn(__fmul_rn(p, s2), (float)(1.0 / 5.0));
+  p = __fadd_rn(__fmul_rn(p, s2), (float)(1.0 / 3.0));
+  p = __fadd_rn(__fmul_rn(p, s2), 1.0f);
+  const float lnf = __fmul_rn(__fmul_rn(2.0f, s), p);
+  return __fadd_rn(__fmul_rn(e, (float)0.693147182), lnf);
+}
+
+// (cos, sin) of 2 pi t / 2^24 for an odd t below 2^24: the top three bits are the octant, the rest an angle in
+// (0, pi/4) measured from the nearer end of the octant, where the Taylor polynomials up to x^9 and x^10 serve.
+__device__ __forceinline__ float2 sincos_u24(uint32_t t) {
+  const uint32_t octant = t >> 21;
+  uint32_t frac = t & 0x1FFFFFu;
+  if (octant & 1u) frac = 0x200000u - frac;
+  const float x = __fmul_rn((float)frac, (float)3.74507039e-07);      // 2 pi / 2^24
+  const float x2 = __fmul_rn(x, x);
+  float ps = (float)(1.0 / 362880.0);
+  ps = __fadd_rn(__fmul_rn(ps, x2), (float)(-1.0 / 5040.0));
+  ps = __fadd_rn(__fmul_rn(ps, x2), (float)(1.0 / 120.0));
+  ps = __fadd_rn(__fmul_rn(ps, x2), (float)(-1.0 / 6.0));
+  ps = __fadd_rn(__fmul_rn(ps, x2), 1.0f);
+  const float sn = __fmul_rn(ps, x);
+  float pc = (float)(-1.0 / 3628800.0);
+  pc = __fadd_rn(__fmul_rn(pc, x2), (float)(1.0 / 40320.0));
+  pc = __fadd_rn(__fmul_rn(pc, x2), (float)(-1.0 / 720.0));
+  pc = __fadd_rn(__fmul_rn(pc, x2), (float)(1.0 / 24.0));
+  pc = __fadd_rn(__fmul_rn(pc, x2), -0.5f);
+  pc = __fadd_rn(__fmul_rn(pc, x2), 1.0f);
+  const bool swap = ((octant + 1u) >> 1) & 1u;           // octants 1, 2, 5, 6: sine and cosine trade places
+  float c = swap ? sn : pc, s = swap ? pc : sn;
+  if (((octant + 2u) >> 2) & 1u) c = -c;                 // cos < 0 in octants 2..5
+  if (octant >> 2) s = -s;                               // sin < 0 in octants 4..7
+  return make_float2(c, s);
+}
+
+// The two normals of one pair of Philox words: uniforms (2 (w >> 9) + 1) / 2^24, Box-Muller.
+__device__ __forceinline__ float2 box_muller_u24(uint32_t wa, uint32_t wb) {
+  const float rad = __fsqrt_rn(__fmul_rn(-2.0f, ln_u24(((wa >> 9) << 1) | 1u)));
+  const float2 cs = sincos_u24(((wb >> 9) << 1) | 1u);
+  return make_float2(__fmul_rn(rad, cs.x), __fmul_rn(rad, cs.y));
 }
 
 }  // namespace xconv

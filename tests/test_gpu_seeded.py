@@ -127,3 +127,73 @@ def test_seeded_estimator_back_to_back_calls_give_the_same_bits():
     assert all(torch.equal(outs[0], o) for o in outs[1:])
     Zo = O.rademacher_probes(5, r, Cin, H, W)
     check("dW", host(outs[-1]), O.wgrad_estimate(host(S), lay["dY"], Zo), TOL["bf16"])
+
+
+# ------------------------------------------------------------------ standard normal probing vectors from a seed
+
+_NP_DT = {torch.float32: "f32", torch.bfloat16: "bf16", torch.float16: "f16"}
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("shape", [(1, 1, 1, 1), (3, 5, 4, 7), (8, 16, 9, 9), (5, 64, 6, 12), (130, 8, 5, 13), (64, 32, 40, 40)])
+def test_gaussian_probes_from_seed_match_the_oracle_generator_bit_for_bit(shape, dtype):
+    """Every float operation of the generator is a single IEEE operation in a fixed order, on both sides: the float
+    values agree bit for bit, and so do their roundings to the 16-bit storage types."""
+    r, Cin, H, W = shape
+    for seed in (0, 0x1234567890ABCDEF, 2**64 - 1):
+        Z = xb.xconv_probes_from_seed(seed, r, Cin, H, W, dtype, gaussian=True)
+        torch.cuda.synchronize()
+        want = inputs.round_to_storage(O.gaussian_probes(seed, r, Cin, H, W).astype(np.float32), _NP_DT[dtype])
+        assert np.array_equal(host(Z), want.astype(np.float64))
+
+
+def test_gaussian_probes_over_a_volume_are_numbered_in_memory_order():
+    r, Cin, D, H, W = 3, 4, 3, 5, 6
+    Z = xb.xconv_probes_from_seed(77, r, Cin, H, W, torch.float32, D=D, gaussian=True)
+    torch.cuda.synchronize()
+    want = O.gaussian_probes(77, r, Cin, D * H, W).reshape(r, Cin, D, H, W)
+    assert np.array_equal(host(Z), want)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16", "f16"])
+@pytest.mark.parametrize("shape", [
+    # B, Cin, Cout, H, W, r, K
+    (4, 3, 5, 7, 9, 6, 3),           # FP32-FMA kernels, odd sizes
+    (16, 64, 64, 12, 12, 24, 3),     # tensor-core kernels for 16-bit storage
+    (8, 32, 32, 20, 24, 40, 3),      # r > B
+    (6, 16, 32, 16, 16, 8, 5),
+])
+def test_algorithm_one_with_gaussian_probes_kept_as_a_seed(shape, dtype):
+    """Forward: S = Z[seed]^T X; backward: dW from S, dY and the seed -- nothing but S and the seed kept between them.
+    Against the oracle run on the oracle's own Z[seed] (rounded to the storage type), and bit for bit against the
+    library's stored-Z calls on the library's Z[seed]."""
+    B, Cin, Cout, H, W, r, K = shape
+    seed = 4242 + sum(shape)
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype=dtype, seed=sum(shape) + 9, KH=K, KW=K, x="relu")
+    X, dY = xb.to_device(lay["X"], dtype), xb.to_device(lay["dY"], dtype)
+    Zo = inputs.round_to_storage(O.gaussian_probes(seed, r, Cin, H, W).astype(np.float32), dtype)
+    S = xb.xconv_sketch_seeded(X, seed, r, gaussian=True)
+    dW = xb.xconv_wgrad_seeded(S, dY, seed, Cin, kernel_size=K, gaussian=True)
+    torch.cuda.synchronize()
+    check("seeded sketch", host(S), O.sketch(lay["X"], Zo), TOL_SKETCH)
+    check("seeded dW", host(dW), O.wgrad_estimate(host(S), lay["dY"], Zo, K, K), TOL[dtype])
+    Zg = xb.xconv_probes_from_seed(seed, r, Cin, H, W, X.dtype, gaussian=True)
+    assert torch.equal(S, xb.xconv_sketch(X, Zg))
+    assert torch.equal(dW, xb.xconv_wgrad(S, dY, Zg, kernel_size=K))
+    # twice in a row: the same bits
+    assert torch.equal(dW, xb.xconv_wgrad_seeded(S, dY, seed, Cin, kernel_size=K, gaussian=True))
+
+
+def test_gaussian_seeded_calls_refuse_a_short_workspace():
+    import ctypes
+    desc = xb.make_desc(8, 16, 16, 8, 8, 8, torch.float32)
+    need = xb.workspace_bytes(desc, xb.OP_WGRAD_SEEDED_GAUSSIAN)
+    assert need >= xb.workspace_bytes(desc, xb.OP_WGRAD) + 8 * 16 * 8 * 8 * 4
+    ws = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    S = torch.zeros((8, 8), device="cuda")
+    dY = torch.zeros((8, 16, 8, 8), device="cuda").contiguous(memory_format=torch.channels_last)
+    dW = torch.full((16, 16, 3, 3), 5.0, device="cuda").contiguous(memory_format=torch.channels_last)
+    st = xb.lib().xconv_wgrad_seeded_gaussian(ctypes.byref(desc), S.data_ptr(), dY.data_ptr(), 1, dW.data_ptr(),
+                                              ws.data_ptr(), ws.numel(), None)
+    torch.cuda.synchronize()
+    assert st == 4 and float(dW.min()) == 5.0
