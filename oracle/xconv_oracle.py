@@ -40,6 +40,9 @@ gaussian_probes (standard normal probing vectors from a stored seed: Box-Muller 
 for the logarithm, sine and cosine that a GPU can repeat bit for bit) is pinned by numpy's float64 functions on the
 same arguments, by a float64 recomputation of single entries from the stated definition, by its moments, a
 Kolmogorov-Smirnov test, E[z z^T] = I, and the unbiasedness of the estimator run on it.
+block_keep_mask and block_sparse_probes (the block-sparse probing vectors of Eq. 7 from a seed) are pinned by a
+word-by-word recomputation of the mask from the stated definition, by the kept share and the independence of the
+mask bits, by the limits p = 0 and p = 1, and by the unbiasedness of the estimator with the Eq. 8 scale on them.
 sketch_independent and wgrad_estimate_independent (the estimator applied to each channel pair on its own) are
 pinned by exact recovery with one orthogonal basis per channel, by unbiasedness with the crosstalk-free
 Hutchinson variance, and by their reduction to the multi-channel functions for a single input channel.
@@ -475,6 +478,31 @@ def gaussian_probes(seed: int, r: int, Cin: int, H: int, W: int) -> np.ndarray:
         out[:, 2 * pair + 1] = (rad * sn).astype(f32)
     z = out.reshape(-1)[:total].astype(F64)
     return np.ascontiguousarray(z.reshape(r, H, W, Cin).transpose(0, 3, 1, 2))
+
+
+def block_keep_mask(seed: int, r: int, Cin: int, p: float) -> np.ndarray:
+    """Which blocks z_{n,j} of Eq. (7) are non-zero, redrawn from the stored seed: block n of probing vector j is kept
+    with probability p, independently for every (n, j).
+
+    Definition (fixed by this library): number the blocks by g = j*Cin + n.  Philox block g div 4 has counter (g div 4
+    in words 0-1, word 2 = 2, word 3 = 0) -- word 2 keeps it apart from the two value streams -- and the seed as key;
+    block g is kept iff its output word (g mod 4) is below floor(p * 2^32).  Returns a boolean array [r, Cin]."""
+    total = r * Cin
+    blocks = np.arange((total + 3) // 4, dtype=np.uint64)
+    two, zero = np.full_like(blocks, 2), np.zeros_like(blocks)
+    w = philox4x32_10((blocks & np.uint64(0xFFFFFFFF), blocks >> np.uint64(32), two, zero),
+                      (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    words = np.stack(w, axis=1).reshape(-1)[:total]
+    threshold = np.uint64(min(max(int(np.floor(float(p) * 4294967296.0)), 0), 1 << 32))
+    return (words < threshold).reshape(r, Cin)
+
+
+def block_sparse_probes(seed: int, r: int, Cin: int, H: int, W: int, p: float, gaussian: bool = False) -> np.ndarray:
+    """Probing vectors of Eq. (7) from a seed: the dense probes of the same seed (Rademacher, or standard normal as the
+    equation prints them) with the blocks block_keep_mask drops set to zero.  Returns Z [r, Cin, H, W]; the scale of
+    Eq. (8) for it is channel_scale(Z)."""
+    dense = gaussian_probes(seed, r, Cin, H, W) if gaussian else rademacher_probes(seed, r, Cin, H, W)
+    return dense * block_keep_mask(seed, r, Cin, p)[:, :, None, None]
 
 
 def memory_factor(Cin, H, W, r):

@@ -736,3 +736,49 @@ def test_estimator_on_gaussian_probes_from_seeds_is_unbiased_with_the_gaussian_v
     est_r = np.stack([O.wgrad_estimate(O.sketch(X, Z), dY, Z) for Z in
                       (O.rademacher_probes(5000 + t, r, 2, 4, 4) for t in range(T))])
     assert est.var(axis=0).sum() > est_r.var(axis=0).sum()
+
+
+# ------------------------------------------------------------------ block-sparse probes (Eq. 7) redrawn from a seed
+
+def test_block_keep_mask_follows_the_stated_definition():
+    seed, r, Cin, p = 0xFEDCBA9876543210, 7, 5, 0.3
+    keep = O.block_keep_mask(seed, r, Cin, p)
+    thr = int(np.floor(p * 2.0 ** 32))
+    for g in range(r * Cin):
+        b = g // 4
+        w = [int(v[0]) for v in O.philox4x32_10(([b & 0xFFFFFFFF], [b >> 32], [2], [0]), (seed & 0xFFFFFFFF, seed >> 32))]
+        assert bool(keep[g // Cin, g % Cin]) == (w[g % 4] < thr)
+    assert O.block_keep_mask(seed, r, Cin, 1.0).all() and not O.block_keep_mask(seed, r, Cin, 0.0).any()
+
+
+def test_block_keep_mask_keeps_a_share_p_of_independent_blocks():
+    r, Cin = 400, 300
+    n = r * Cin
+    for p in (0.125, 0.5, 0.9):
+        k = O.block_keep_mask(11, r, Cin, p).astype(np.float64)
+        assert abs(k.mean() - p) < 5.0 * np.sqrt(p * (1 - p) / n)
+        c = k - p
+        for a, b in ((c[:, :-1], c[:, 1:]), (c[:-1], c[1:])):        # neighbours along the channels, along the probes
+            assert abs(np.mean(a * b)) < 5.0 * p * (1 - p) / np.sqrt(a.size)
+    # another seed gives another mask; the mask is unrelated to the signs of the same seed
+    k1, k2 = O.block_keep_mask(11, r, Cin, 0.5), O.block_keep_mask(12, r, Cin, 0.5)
+    assert 0.4 < np.mean(k1 != k2) < 0.6
+
+
+@pytest.mark.parametrize("gaussian", [False, True])
+def test_block_sparse_probes_are_the_dense_ones_with_blocks_dropped_and_keep_the_estimator_unbiased(gaussian):
+    r, Cin, H, W, p = 12, 3, 4, 4, 0.5
+    Z = O.block_sparse_probes(21, r, Cin, H, W, p, gaussian)
+    dense = (O.gaussian_probes if gaussian else O.rademacher_probes)(21, r, Cin, H, W)
+    keep = O.block_keep_mask(21, r, Cin, p)
+    assert np.array_equal(Z[keep], dense[keep]) and not Z[~keep].any() and 0 < keep.sum() < keep.size
+    # Eq. 8: with the 1/nnz(Z_n) scale the mean over seeds is the exact gradient
+    X, Wt, dY = _tiny(seed=45, B=3, Cin=Cin, Cout=2, H=H, W=W)
+    T = 1200
+    est = []
+    for t in range(T):
+        Zt = O.block_sparse_probes(7000 + t, r, Cin, H, W, p, gaussian)
+        est.append(O.wgrad_estimate(O.sketch(X, Zt), dY, Zt, scale=O.channel_scale(Zt)))
+    est = np.stack(est)
+    # a channel whose r blocks are all dropped (probability 2^-12 per channel and seed) estimates 0: negligible bias
+    assert np.all(np.abs(est.mean(axis=0) - O.dw_exact(X, dY)) < 4.5 * est.std(axis=0) / np.sqrt(T) + 1e-3 * np.abs(O.dw_exact(X, dY)).max())
