@@ -190,6 +190,19 @@ xconv_status xconv_wgrad_seeded_gaussian(const xconv_desc* desc, const float* sk
                                          unsigned long long seed, float* dW, void* ws, size_t ws_bytes,
                                          void* cuda_stream);
 
+/* The block-sparse probing vectors of Eq. 7 from a seed: block n of probing vector j (the H*W entries of input
+ * channel n) is kept with probability p and is zero otherwise, independently for every (n, j); the kept blocks are
+ * those of the dense probes of the same seed (gaussian = 0: xconv_probes_from_seed, 1: xconv_gaussian_probes_from_seed;
+ * Eq. 7 prints the normal ones).  Definition of the mask: blocks numbered g = j*Cin + n; Philox-4x32-10 block g div 4
+ * with counter (g div 4 in words 0-1, word 2 = 2, word 3 = 0) and the seed as key; block g is kept iff output word
+ * (g mod 4) is below floor(p * 2^32).  Outputs, all device pointers: Z [r,H,W,Cin] (volumes [r,D,H,W,Cin]) in
+ * desc.dtype, 16-byte aligned; keep, r*Cin bytes (1 = kept); chan_scale, Cin floats, 1/nnz(Z_n) of Eq. 8 (0 for a
+ * channel none of the r vectors probes) -- what desc.chan_scale takes.  p outside [0, 1]: XCONV_ERR_INVALID_ARG.
+ * Four small launches (dense probes, mask, scale, zeroing); no scratch.  A caller that keeps the seed and p between the
+ * passes redraws the same Z, keep and chan_scale in the backward pass. */
+xconv_status xconv_block_sparse_probes_from_seed(const xconv_desc* desc, unsigned long long seed, int gaussian, double p,
+                                                 void* Z, unsigned char* keep, float* chan_scale, void* cuda_stream);
+
 /* Algorithm 1, backward steps 3-4: L = S dY^T, then dW[m,n,k] = scale[n] * tr(L^m T_{-k} Z_n) for
  * every offset (Eq. 6; three-step procedure of Section 3).  sketch [r,B] float as written by
  * xconv_forward; dY [B,H,W,Cout], Z [r,H,W,Cin] in desc.dtype; dW [Cout,KH,KW,Cin] float.

@@ -28,6 +28,7 @@ EXPORTS = ("xconv_workspace_bytes", "xconv_engine_for", "xconv_forward", "xconv_
            "xconv_workspace_status", "xconv_selftest_wait_limit", "xconv_measure_fma_rate",
            "xconv_sketch_independent", "xconv_wgrad_independent", "xconv_zero_blocks", "xconv_zero_blocks_used",
            "xconv_gaussian_probes_from_seed", "xconv_sketch_seeded_gaussian", "xconv_wgrad_seeded_gaussian",
+           "xconv_block_sparse_probes_from_seed",
            "xconv_last_launch_count", "xconv_last_cuda_error", "xconv_status_string")
 
 
@@ -77,6 +78,9 @@ def lib() -> ctypes.CDLL:
     L.xconv_sketch_seeded_gaussian.restype = c_int
     L.xconv_wgrad_seeded_gaussian.argtypes = L.xconv_wgrad_seeded.argtypes
     L.xconv_wgrad_seeded_gaussian.restype = c_int
+    L.xconv_block_sparse_probes_from_seed.argtypes = [P, ctypes.c_ulonglong, c_int, ctypes.c_double, c_void_p, c_void_p,
+                                                      c_void_p, c_void_p]
+    L.xconv_block_sparse_probes_from_seed.restype = c_int
     L.xconv_wgrad.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     L.xconv_wgrad.restype = c_int
     L.xconv_sketch_independent.argtypes = [P, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -294,6 +298,20 @@ def xconv_probes_from_seed(seed: int, r: int, Cin: int, H: int, W: int, dtype=to
     fn = lib().xconv_gaussian_probes_from_seed if gaussian else lib().xconv_probes_from_seed
     _check(fn(ctypes.byref(desc), seed, Z.data_ptr(), _stream()), "xconv_probes_from_seed")
     return Z
+
+
+def xconv_block_sparse_probes_from_seed(seed: int, p: float, r: int, Cin: int, H: int, W: int, dtype=torch.bfloat16,
+                                        device="cuda", D: int = 1, gaussian: bool = False):
+    """The block-sparse probing vectors of Eq. 7 from a seed: (Z, keep [r, Cin] uint8, chan_scale [Cin] float32 =
+    1/nnz(Z_n) of Eq. 8).  Blocks are kept with probability p; the kept ones are those of the dense probes of the seed."""
+    desc = make_desc(1, Cin, 1, H, W, r, dtype, D=D)
+    Z = _like((r, Cin), (D, H, W), 5 if D > 1 else 4, dtype=dtype, device=device)
+    keep = torch.empty((r, Cin), dtype=torch.uint8, device=device)
+    scale = torch.empty((Cin,), dtype=torch.float32, device=device)
+    _check(lib().xconv_block_sparse_probes_from_seed(ctypes.byref(desc), seed, 1 if gaussian else 0, float(p), Z.data_ptr(),
+                                                     keep.data_ptr(), scale.data_ptr(), _stream()),
+           "xconv_block_sparse_probes_from_seed")
+    return Z, keep, scale
 
 
 def xconv_sketch_seeded(X: torch.Tensor, seed: int, r: int, gaussian: bool = False) -> torch.Tensor:

@@ -1,4 +1,5 @@
 // libxconv C ABI: argument checks, workspace planning and kernel dispatch.
+#include <cmath>
 #include "../../include/xconv.h"
 
 #include <algorithm>
@@ -286,6 +287,40 @@ static xconv_status run_gaussian_probes(const xconv_desc* d, unsigned long long 
   ++g_launches;
   if (e != cudaSuccess) { g_last_cuda_error = (int)e; return XCONV_ERR_CUDA; }
   return XCONV_OK;
+}
+
+// Block-sparse probing vectors (Eq. 7) from a seed.  keep[g], g = j * Cin + n: block n of probing vector j is non-zero
+// iff word (g mod 4) of Philox block (g div 4) -- counter word 2 = 2, apart from the two value streams -- is below the
+// threshold floor(p * 2^32).
+__global__ void __launch_bounds__(256) block_keep_kernel(unsigned char* __restrict__ keep, long total, uint32_t k0,
+                                                         uint32_t k1, unsigned long long threshold) {
+  const long b = (long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (b * 4 >= total) return;
+  const uint4 w = philox4x32_10((uint32_t)b, (uint32_t)((unsigned long long)b >> 32), k0, k1, 2u);
+  const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    if (b * 4 + i < total) keep[b * 4 + i] = (unsigned long long)v[i] < threshold ? 1 : 0;
+}
+// scale[n] = 1 / nnz(Z_n), the number of probing vectors whose block n is kept (Eq. 8); 0 for a channel no vector probes.
+__global__ void __launch_bounds__(256) keep_scale_kernel(const unsigned char* __restrict__ keep, int r, int Cin,
+                                                         float* __restrict__ scale) {
+  const int n = blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= Cin) return;
+  int nnz = 0;
+  for (int j = 0; j < r; ++j) nnz += keep[(long)j * Cin + n];
+  scale[n] = nnz > 0 ? __fdiv_rn(1.0f, (float)nnz) : 0.0f;
+}
+// The dropped blocks of a dense Z set to +0.  Entry e belongs to probe e / per_probe and channel e % Cin.
+template <typename T>
+__global__ void __launch_bounds__(256) drop_blocks_kernel(T* __restrict__ Z, const unsigned char* __restrict__ keep,
+                                                          long total, long per_probe, int Cin) {
+  const long e0 = ((long)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long e = e0 + i;
+    if (e < total && !keep[(e / per_probe) * Cin + e % Cin]) Z[e] = from_f<T>(0.0f);
+  }
 }
 
 static size_t probes_bytes(const xconv_desc* d) {
@@ -691,6 +726,31 @@ xconv_status xconv_gaussian_probes_from_seed(const xconv_desc* desc, unsigned lo
   if (!aligned16(Z)) return XCONV_ERR_ALIGNMENT;
   new_call();
   return run_gaussian_probes(desc, seed, Z, static_cast<cudaStream_t>(cuda_stream));
+}
+
+xconv_status xconv_block_sparse_probes_from_seed(const xconv_desc* desc, unsigned long long seed, int gaussian, double p,
+                                                 void* Z, unsigned char* keep, float* chan_scale, void* cuda_stream) {
+  xconv_status s = validate(desc);
+  if (s != XCONV_OK) return s;
+  if (!Z || !keep || !chan_scale || !(p >= 0.0 && p <= 1.0) || (gaussian != 0 && gaussian != 1)) return XCONV_ERR_INVALID_ARG;
+  if (!aligned16(Z)) return XCONV_ERR_ALIGNMENT;
+  new_call();
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  s = gaussian ? run_gaussian_probes(desc, seed, Z, st) : run_probes_from_seed(desc, seed, Z, st);
+  if (s != XCONV_OK) return s;
+  const long blocks = (long)desc->r * desc->Cin;
+  const unsigned long long threshold = (unsigned long long)std::floor(p * 4294967296.0);
+  block_keep_kernel<<<(unsigned)cdiv(cdiv(blocks, 4), 256), 256, 0, st>>>(keep, blocks, (uint32_t)(seed & 0xFFFFFFFFull),
+                                                                          (uint32_t)(seed >> 32), threshold);
+  if ((s = check_launch()) != XCONV_OK) return s;
+  keep_scale_kernel<<<(unsigned)cdiv(desc->Cin, 256), 256, 0, st>>>(keep, desc->r, desc->Cin, chan_scale);
+  if ((s = check_launch()) != XCONV_OK) return s;
+  const long per_probe = (long)depth(desc) * desc->H * desc->W * desc->Cin, total = per_probe * desc->r;
+  const unsigned grid = (unsigned)cdiv(cdiv(total, 4), 256);
+  if (desc->dtype == XCONV_F32) drop_blocks_kernel<float><<<grid, 256, 0, st>>>(static_cast<float*>(Z), keep, total, per_probe, desc->Cin);
+  else if (desc->dtype == XCONV_F16) drop_blocks_kernel<f16><<<grid, 256, 0, st>>>(static_cast<f16*>(Z), keep, total, per_probe, desc->Cin);
+  else drop_blocks_kernel<bf16><<<grid, 256, 0, st>>>(static_cast<bf16*>(Z), keep, total, per_probe, desc->Cin);
+  return check_launch();
 }
 
 xconv_status xconv_sketch_seeded_gaussian(const xconv_desc* desc, const void* X, unsigned long long seed,

@@ -197,3 +197,56 @@ def test_gaussian_seeded_calls_refuse_a_short_workspace():
                                               ws.data_ptr(), ws.numel(), None)
     torch.cuda.synchronize()
     assert st == 4 and float(dW.min()) == 5.0
+
+
+# ------------------------------------------------------------------ block-sparse probing vectors (Eq. 7) from a seed
+
+@pytest.mark.parametrize("gaussian", [False, True])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("shape,p", [((1, 1, 1, 1), 0.5), ((7, 5, 4, 6), 0.3), ((40, 64, 6, 6), 0.5), ((33, 130, 3, 5), 0.125),
+                                     ((6, 8, 5, 5), 1.0), ((6, 8, 5, 5), 0.0)])
+def test_block_sparse_probes_from_seed_match_the_oracle_bit_for_bit(shape, p, dtype, gaussian):
+    r, Cin, H, W = shape
+    seed = 0xA5A5A5A5DEADBEEF ^ (r * 1000 + Cin)
+    Z, keep, scale = xb.xconv_block_sparse_probes_from_seed(seed, p, r, Cin, H, W, dtype, gaussian=gaussian)
+    torch.cuda.synchronize()
+    Zo = inputs.round_to_storage(O.block_sparse_probes(seed, r, Cin, H, W, p, gaussian).astype(np.float32), _NP_DT[dtype])
+    assert np.array_equal(host(Z), Zo.astype(np.float64))
+    assert np.array_equal(keep.cpu().numpy().astype(bool), O.block_keep_mask(seed, r, Cin, p))
+    np.testing.assert_allclose(scale.cpu().numpy(), O.channel_scale(O.block_sparse_probes(seed, r, Cin, H, W, p, False)),
+                               rtol=1e-7, atol=0)
+
+
+def test_block_sparse_probes_from_seed_through_the_layer_with_the_equation_8_scale():
+    """Forward sketch and backward estimate on the probes of Eq. 7 redrawn from (seed, p) in each pass; the estimate
+    against the oracle on the oracle's own redraw, with the 1/nnz scale the call returns; the mask the contraction
+    takes (xconv_zero_blocks) agrees with the keep mask on 64-channel blocks."""
+    B, Cin, Cout, H, W, r, p, seed = 16, 64, 64, 12, 12, 24, 0.5, 31337
+    lay = inputs.make_custom(B, Cin, Cout, H, W, r, dtype="bf16", seed=5150, x="relu")
+    X, dY = xb.to_device(lay["X"], "bf16"), xb.to_device(lay["dY"], "bf16")
+    Z, keep, scale = xb.xconv_block_sparse_probes_from_seed(seed, p, r, Cin, H, W, torch.bfloat16)
+    S = xb.xconv_sketch(X, Z)
+    del Z
+    Z2, keep2, scale2 = xb.xconv_block_sparse_probes_from_seed(seed, p, r, Cin, H, W, torch.bfloat16)     # backward pass
+    dW = xb.xconv_wgrad(S, dY, Z2, chan_scale=scale2)
+    torch.cuda.synchronize()
+    assert torch.equal(keep, keep2) and torch.equal(scale, scale2)
+    Zo = O.block_sparse_probes(seed, r, Cin, H, W, p)
+    check("sketch", host(S), O.sketch(lay["X"], Zo), TOL_SKETCH)
+    check("dW", host(dW), O.wgrad_estimate(host(S), lay["dY"], Zo, scale=O.channel_scale(Zo)), TOL["bf16"])
+    zb = xb.xconv_zero_blocks(Z2).cpu().numpy().astype(bool)                  # [r, Cin/64]: all 64 channels dropped
+    assert np.array_equal(zb[:, 0], ~O.block_keep_mask(seed, r, Cin, p).any(axis=1))
+
+
+def test_block_sparse_probes_refuse_a_probability_outside_the_unit_interval():
+    import ctypes
+    desc = xb.make_desc(1, 8, 1, 4, 4, 4, torch.float32)
+    Z = torch.full((4, 8, 4, 4), 7.0, device="cuda").contiguous(memory_format=torch.channels_last)
+    keep = torch.zeros((4, 8), dtype=torch.uint8, device="cuda")
+    scale = torch.zeros(8, device="cuda")
+    for p in (-0.1, 1.5, float("nan")):
+        st = xb.lib().xconv_block_sparse_probes_from_seed(ctypes.byref(desc), 1, 0, p, Z.data_ptr(), keep.data_ptr(),
+                                                          scale.data_ptr(), None)
+        assert st == 1
+    torch.cuda.synchronize()
+    assert float(Z.min()) == 7.0
